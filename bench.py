@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark of the Anakin hot path: env frames/s (acting + learning) on the "throughput" workload.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
+
+One step = one pass of the whole hot path: a T-step rollout of all B envs followed by one A2C/Adam update
+(B*T frames).  Prints ONE JSON line.  With N > 1 (torchrun) every rank runs an independent replica of the
+workload with its own seed ("replicas only": the library has no cross-device exchange step yet).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2104_06272_b200.workloads import WORKLOADS  # noqa: E402
+
+METRIC = "env_frames_per_sec_act_plus_learn"
+UNIT = "frames/s"
+# FP32 FMA peak of a B200: 148 SMs x 128 FMA lanes x 2 FLOP x max SM clock.
+FP32_ALU_TFLOPS_PER_MHZ = 148 * 128 * 2 / 1e6
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    sm_max_mhz=float(p.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=5)
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def workload_label(w):
+    return (f"throughput: B={w.B} envs, {w.N}x{w.N} gridworld (obs {w.D}), MLP {w.D}-{w.H}-{w.H}+5, "
+            f"{'fp32' if w.precision == 0 else 'bf16'}, T={w.T}")
+
+
+# ------------------------------------------------------------------------------------------------------
+# Kernel work model (algorithmic FLOPs / bytes per launch) for the roofline entry
+# ------------------------------------------------------------------------------------------------------
+def kernel_work(w):
+    B, T, H, C = w.B, w.T, w.H, w.C
+    R = B * T
+    return {
+        # name: (bound, flops per launch, bytes per launch)
+        "rollout": ("alu", 2.0 * B * (T + 1) * (H + H * H + 5 * H), R * 15.0 + B * 4),
+        "fwd2": ("alu", 2.0 * R * H * H, 2.0 * R * H * 4),
+        "dh1": ("alu", 2.0 * R * H * H, 3.0 * R * H * 4),
+        "dw2": ("alu", 2.0 * R * H * H, 2.0 * R * H * 4),
+        "dw1_agent": ("alu", 2.0 * R * C * H, R * H * 4.0 + R),
+        "dw1_walls": ("alu", 2.0 * B * C * H, B * H * 4.0),
+        "dw1_goal": ("alu", 2.0 * B * C * H, B * H * 4.0),
+        "h1": ("hbm", R * H * 2.0, R * H * 4.0 + R),
+        "heads_loss": ("hbm", R * H * 20.0, 2.0 * R * H * 4 + R * 45.0),
+        "colsums": ("hbm", R * H * 12.0, 3.0 * R * H * 4 + R * 32.0),
+        "sum_over_t": ("hbm", R * H * 1.0, R * H * 4.0 + B * H * 4.0),
+        "gae": ("hbm", R * 6.0, R * 17.0),
+        "env_base": ("hbm", B * H * 0.2 * C, B * H * 4.0),
+        "reduce_adam": ("hbm", w.P * 12.0, w.P * 28.0),
+    }
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2104_06272_b200 import binding as bnd
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("launch with torchrun --nproc-per-node N for --gpus N")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    w = WORKLOADS["throughput"]
+    peaks = load_peaks()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        an = bnd.Anakin(bnd.cfg_from_workload(w, device=local_rank), stream=stream)
+    seed = 1 + rank
+    an.reset(seed)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K, W = args.steps, args.warmup
+    # ---- warm-up
+    an.run(W)
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps, each bracketed by events on the library's stream; L2 flushed between steps
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    n0 = an.launch_count()
+    barrier()
+    t_wall0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        for a, b in ev:
+            flush.fill_(0)
+            a.record(stream)
+            an.run(1)
+            b.record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    launches = an.launch_count() - n0
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(step_ms))
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    frames = float(w.B) * w.T * K * world
+    value = frames / (total_ms * 1e-3)
+
+    # ---- per-kernel pass (events around every launch), same K steps, for the roofline entry
+    an.profile_enable(True)
+    with torch.cuda.stream(stream):
+        for _ in range(K):
+            flush.fill_(0)
+            an.run(1)
+    prof = an.profile_read()
+    an.profile_enable(False)
+
+    # ---- end to end through the C ABI with host buffers: per step, parameters and env state go host->device
+    # from pinned memory, one act+learn pass runs, statistics and parameters come back
+    P = an.P
+    h_theta = torch.from_numpy(an.get(bnd.PARAMS)).pin_memory()
+    h_pos = torch.from_numpy(an.get(bnd.ENV_POS)).pin_memory()
+    h_tep = torch.from_numpy(an.get(bnd.ENV_TEP)).pin_memory()
+    h_out = torch.empty(P, dtype=torch.float32).pin_memory()
+    Ke = max(3, min(K, 20))
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(Ke):
+        an.set(bnd.PARAMS, h_theta)
+        an.set(bnd.ENV_POS, h_pos)
+        an.set(bnd.ENV_TEP, h_tep)
+        an.run(1)
+        st = an.stats()
+        an.get_into(bnd.PARAMS, h_out)
+        an.get_into(bnd.ENV_POS, h_pos)
+        an.get_into(bnd.ENV_TEP, h_tep)
+        h_theta.copy_(h_out)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = float(w.B) * w.T * Ke * world / e2e_s
+    assert np.isfinite(st.loss_total) and an.status() == 0
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel
+    work = kernel_work(w)
+    tot = sum(ms for ms, _ in prof.values())
+    top = max(prof, key=lambda k: prof[k][0])
+    top_ms, top_n = prof[top]
+    bound, flops, nbytes = work.get(top, ("hbm", 0.0, 0.0))
+    per_launch_s = top_ms / top_n * 1e-3
+    sm_mhz = (clocks or {}).get("sm_max_mhz") or peaks["sm_max_mhz"]
+    if bound == "alu":
+        achieved, peak, unit = flops / per_launch_s / 1e12, FP32_ALU_TFLOPS_PER_MHZ * sm_mhz, "TFLOP/s"
+        peak_note = f"fp32 FMA peak = 148 SMs x 128 lanes x 2 x {sm_mhz:.0f} MHz (derived)"
+    else:
+        achieved, peak, unit = nbytes / per_launch_s / 1e9, peaks["hbm_gbs"], "GB/s"
+        peak_note = f"HBM copy bandwidth, {peaks['source']}"
+    roofline = {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                "traffic": None, "peak_source": peak_note, "us_per_launch": per_launch_s * 1e6,
+                "share_of_step": top_ms / tot,
+                "kernels": {k: {"us_per_launch": ms / n * 1e3, "launches_per_step": n / K, "share": ms / tot} for k, (ms, n) in
+                            sorted(prof.items(), key=lambda kv: -kv[1][0])}}
+
+    # ---- the oracle on the host cores, bounded sample of the same workload
+    cpu = cpu_baseline(w, iters=2)
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_label(w), "frames_per_step": w.B * w.T, "seed": seed,
+                   "l2": "flushed between timed steps (256 MiB write outside the event brackets)",
+                   "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": P * 4 + 2 * w.B, "d2h_bytes_per_step": P * 4 + 2 * w.B + 48,
+                "steps": Ke, "what": "set(PARAMS, ENV_POS, ENV_TEP) from pinned host, run(1), get(STATS, PARAMS, ENV_POS, ENV_TEP)"},
+        "gpu_launches": int(launches),
+        "wall_s_timed_region": t_wall,
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(w, iters: int, B: int | None = None):
+    """Times the oracle, as it stands, on `iters` act+learn passes of the workload (optionally on a reduced batch)."""
+    from oracle import binding as orc
+
+    Bs = w.B if B is None else B
+    ag = orc.Agent(Bs, w.N, w.H, w.T, w.precision, w.episode_cap, w.wall_density, w.gamma, w.gae_lambda, w.entropy_coef,
+                   w.value_coef, w.lr, w.adam_b1, w.adam_b2, w.adam_eps)
+    ag.reset(1)
+    t0 = time.perf_counter()
+    ag.run(iters)
+    dt = time.perf_counter() - t0
+    return {"value": Bs * w.T * iters / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{iters} full act+learn passes of B={Bs}, T={w.T} ({Bs * w.T * iters} frames, {dt:.1f} s)"}
+
+
+def run_reference(args):
+    """The reference arm is the CPU oracle: each step is one act+learn pass on a quarter of the batch."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import binding as orc
+
+    w = WORKLOADS["throughput"]
+    Bs = w.B // 4
+    ag = orc.Agent(Bs, w.N, w.H, w.T, w.precision, w.episode_cap, w.wall_density, w.gamma, w.gae_lambda, w.entropy_coef,
+                   w.value_coef, w.lr, w.adam_b1, w.adam_b2, w.adam_eps)
+    ag.reset(1)
+    K, W = args.steps, args.warmup
+    ag.run(W)
+    t0 = time.perf_counter()
+    ag.run(K)
+    dt = time.perf_counter() - t0
+    value = Bs * w.T * K / dt
+    sample = f"each step = one act+learn pass on B={Bs} of the workload's {w.B} envs, T={w.T}"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K, "warmup": W,
+        "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": workload_label(w), "frames_per_step": Bs * w.T, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,205 @@
+/*
+ * anakin.h -- C ABI of the Anakin hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The library runs the co-located loop of the Anakin architecture (Podracer paper, Section 3.1 "Online
+ * Learning with Anakin"; Figure 2, top): a batch of environments written as array code is stepped on the
+ * accelerator next to the agent for T interactions, then one parameter update is computed from those
+ * interactions and averaged over the batch.  Nothing crosses the host/device boundary inside the loop
+ * (Section 3.1: the host only schedules); the workload is self-contained and deterministic given a seed
+ * (Section 3.1).
+ *
+ * Workload (the paper says only "small neural networks and grid-world environments", Section 4.1; the
+ * concrete rules are this library's):
+ *   env      N x N integer gridworld per env, C = N*N cells; per-env wall mask, start and goal cell drawn from the
+ *            seed; actions 0 up (row-1), 1 right (col+1), 2 down (row+1), 3 left (col-1); a move into a wall or
+ *            off the grid leaves the agent in place; reaching the goal pays +1 and ends the episode, the step cap
+ *            ends it with 0; an ended episode restarts from the seeded start cell inside the same step.
+ *   obs      three one-hot planes (walls, agent, goal) flattened to D = 3C values; never stored, rebuilt from state.
+ *   agent    MLP D-H-H with ReLU, a head of 4 action logits and 1 value; categorical sampling by inverse CDF
+ *            with a Philox4x32-10 uniform keyed by (seed) and counted by (env, global step).
+ *   update   GAE(gamma, lambda) advantages, A2C loss  -mean(A log pi) + value_coef mean((V-ret)^2)
+ *            - entropy_coef mean(entropy), gradient = mean over all B*T rows, one Adam step.
+ *
+ * Conventions
+ *   - Every call returns int: ANAKIN_OK (0) or a negative ANAKIN_E_* code.  Nothing throws or aborts.
+ *   - The caller owns ALL device memory: one workspace of anakin_workspace_bytes() bytes, 256-byte aligned,
+ *     allocated by the caller (e.g. a torch uint8 tensor) and alive until anakin_destroy().  The library
+ *     allocates no device memory.  The handle itself is host memory owned by the library.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work is
+ *     enqueued on it.  reset/rollout/learn/run are asynchronous; get/set with a HOST pointer and
+ *     anakin_status synchronise the stream before returning.
+ *   - A handle is not thread-safe.  Different handles (different workspaces) are independent.
+ *   - Unsupported shapes are refused with ANAKIN_E_UNSUPPORTED_CFG; there is no CPU fallback.
+ *
+ * Flat parameter order (PARAMS, GRADS, ADAM_M, ADAM_V; fp32):
+ *   W1[D][H], b1[H], W2[H][H], b2[H], Wh[H][5] (columns 0..3 logits, 4 value), bh[5];
+ *   P = D*H + H + H*H + H + 5*H + 5.
+ * Trajectory arrays are time-major: element (t, b) at index t*B + b.
+ */
+#ifndef ANAKIN_H_
+#define ANAKIN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct anakin_handle anakin_t;
+
+enum {
+    ANAKIN_OK = 0,
+    ANAKIN_E_INVALID_ARG = -1,
+    ANAKIN_E_BAD_STATE = -2,           /* e.g. learn() with no rollout pending, rollout() before reset() */
+    ANAKIN_E_WORKSPACE_TOO_SMALL = -3,
+    ANAKIN_E_UNSUPPORTED_CFG = -4,
+    ANAKIN_E_CUDA = -5,                /* a CUDA runtime call failed; see anakin_last_cuda_error() */
+    ANAKIN_E_DEVICE_STATUS = -6        /* the sticky device status word is non-zero */
+};
+
+enum { ANAKIN_PRECISION_FP32 = 0, ANAKIN_PRECISION_BF16 = 1 };
+
+/* Plain-old-data configuration.  struct_size must be sizeof(anakin_cfg) (ABI versioning). */
+typedef struct anakin_cfg {
+    uint32_t struct_size;
+    int32_t B;            /* environments, >= 1 */
+    int32_t N;            /* grid side, 2..16 (cells fit a uint8) */
+    int32_t H;            /* hidden width, multiple of 32, 32..1024 */
+    int32_t T_max;        /* largest rollout length, >= 1 */
+    int32_t episode_cap;  /* 1..255 */
+    double wall_density;  /* [0, 1); a cell is a wall when its 32-bit draw is below floor(wall_density * 2^32) */
+    float gamma, gae_lambda, entropy_coef, value_coef;
+    float lr, adam_b1, adam_b2, adam_eps;
+    int32_t precision;    /* ANAKIN_PRECISION_*: BF16 = bf16 weights/activations as GEMM inputs, fp32 accumulate,
+                             fp32 master parameters in Adam */
+    int32_t device;       /* CUDA device ordinal the workspace lives on */
+    int32_t debug_logits; /* non-zero: rollouts also record the 4 logits of every (t, b) */
+    int32_t reserved;     /* must be 0 */
+} anakin_cfg;
+
+/* Blob selectors for anakin_get / anakin_set.  Sizes in bytes for the LAST rollout length T (or T_max where noted). */
+enum {
+    ANAKIN_PARAMS = 0,       /* f32[P]                       get/set */
+    ANAKIN_GRADS = 1,        /* f32[P]   last batch-mean gradient      get */
+    ANAKIN_ADAM_M = 2,       /* f32[P]                       get/set */
+    ANAKIN_ADAM_V = 3,       /* f32[P]                       get/set */
+    ANAKIN_ADAM_STEP = 4,    /* i64[1]  host-side counter; pointer must be HOST   get/set */
+    ANAKIN_ENV_WALLS = 5,    /* u32[B][ceil(C/32)] bit c of an env = cell c is a wall   get/set */
+    ANAKIN_ENV_START = 6,    /* u8[B]                        get/set */
+    ANAKIN_ENV_GOAL = 7,     /* u8[B]                        get/set */
+    ANAKIN_ENV_POS = 8,      /* u8[B]   agent cell            get/set */
+    ANAKIN_ENV_TEP = 9,      /* u8[B]   steps into the episode get/set */
+    ANAKIN_GLOBAL_STEP = 10, /* i64[1]  env steps since reset (the Philox step counter); HOST pointer   get/set */
+    ANAKIN_TRAJ_POS = 11,    /* u8[T][B]  state the action was taken in   get/set */
+    ANAKIN_TRAJ_ACTION = 12, /* i8[T][B]                     get/set */
+    ANAKIN_TRAJ_DONE = 13,   /* u8[T][B]                     get/set */
+    ANAKIN_TRAJ_REWARD = 14, /* f32[T][B]                    get/set */
+    ANAKIN_TRAJ_VALUE = 15,  /* f32[T+1][B]  row T = bootstrap value of the state after the last step   get/set */
+    ANAKIN_TRAJ_LOGP = 16,   /* f32[T][B]  log pi(a_t|s_t)   get/set */
+    ANAKIN_ADV = 17,         /* f32[T][B]                    get/set */
+    ANAKIN_RET = 18,         /* f32[T][B]                    get/set */
+    ANAKIN_STATS = 19,       /* anakin_stats                 get */
+    ANAKIN_DEBUG_LOGITS = 20 /* f32[T][B][4], only with cfg.debug_logits   get */
+};
+
+/* Counters since reset plus the loss terms of the last update. */
+typedef struct anakin_stats {
+    uint64_t frames;         /* env steps taken (B per step) */
+    uint64_t episodes;       /* episodes finished (goal or cap) */
+    uint64_t goals;          /* episodes that ended at the goal = sum of rewards */
+    uint64_t episode_steps;  /* sum of the lengths of finished episodes */
+    float loss_total, loss_pg, loss_value, entropy;
+} anakin_stats;
+
+/* Size of the device workspace a configuration needs.  Validates cfg. */
+int anakin_workspace_bytes(const anakin_cfg* cfg, size_t* bytes);
+
+/*
+ * Creates a handle over a caller-provided DEVICE workspace (256-byte aligned, >= anakin_workspace_bytes()).
+ * No device memory is allocated and nothing is enqueued.  The state is undefined until anakin_reset().
+ * Errors: INVALID_ARG (null / misaligned / bad struct_size), UNSUPPORTED_CFG, WORKSPACE_TOO_SMALL, CUDA.
+ */
+int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void* cuda_stream, anakin_t** out);
+
+/* Frees the host handle.  The workspace stays the caller's.  Does not synchronise. */
+int anakin_destroy(anakin_t* h);
+
+/*
+ * The paper's `initial_state` for all B envs (Section 3.1) plus agent initialisation: draws walls, start and
+ * goal of every env from the seed, puts every agent on its start cell, draws Xavier-uniform weights (zero
+ * biases), zeroes the Adam moments, the step counters and the statistics.  Enqueued on the stream.
+ */
+int anakin_reset(anakin_t* h, uint64_t seed);
+
+/*
+ * T interactions of every env with the current policy (Figure 2, top: "a sequence of interactions"), 1 <= T <= T_max,
+ * continuing from the current env state: per step, observation from state -> MLP -> sample -> env `step`; records
+ * pos, action, done, reward, value, logp (time-major) and the bootstrap value row T.  Advances GLOBAL_STEP by T.
+ * Errors: BAD_STATE before reset, INVALID_ARG for T out of range.
+ */
+int anakin_rollout(anakin_t* h, int T);
+
+/*
+ * Same kernel path with sampling overridden by dev_actions (DEVICE pointer, i8[T][B], values 0..3): the env is
+ * "driven by the same action sequence" for transition parity tests.  logp is that of the forced action.
+ */
+int anakin_rollout_forced(anakin_t* h, int T, const int8_t* dev_actions);
+
+/*
+ * The parameter update of the minimal unit (Section 3.1; Figure 2, top): GAE over the last rollout, A2C loss,
+ * backward through the MLP on all B*T rows (the env and the sampled actions carry no gradient), batch mean of
+ * the gradient (the single-device form of the cross-core average), one Adam step.  Consumes the pending
+ * rollout.  Errors: BAD_STATE if no rollout is pending.
+ */
+int anakin_learn(anakin_t* h);
+
+/* Only the update's first half: fills ADV and RET from the pending rollout (for stage-wise parity tests). */
+int anakin_gae(anakin_t* h);
+
+/* Only the update's second half: loss, backward, batch mean and Adam from the ADV and RET blobs as they stand
+ * (anakin_learn == anakin_gae followed by anakin_update).  Consumes the pending rollout. */
+int anakin_update(anakin_t* h);
+
+/* iters x ( anakin_rollout(T_max); anakin_learn() ), enqueue-only: no copy and no synchronisation. */
+int anakin_run(anakin_t* h, int iters);
+
+/*
+ * Copy a blob out of / into the workspace.  `ptr` is a host pointer (ptr_is_device = 0; the call synchronises the
+ * stream) or a device pointer (ptr_is_device = 1; asynchronous on the stream).  `bytes` must equal the blob's
+ * size.  Setting any TRAJ_* / ADV / RET blob marks a rollout of the last used length as pending, so the stages
+ * can be driven with the other side's data.  Errors: INVALID_ARG (unknown blob, wrong size, read-only blob).
+ */
+int anakin_get(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is_device);
+int anakin_set(anakin_t* h, int which, const void* ptr, size_t bytes, int ptr_is_device);
+
+/* Size in bytes of a blob for the current rollout length (0 if unknown). */
+size_t anakin_blob_bytes(anakin_t* h, int which);
+
+/* Synchronises the stream and returns the sticky device status word (0 = clean) in *device_status. */
+int anakin_status(anakin_t* h, int* device_status);
+
+/* Number of kernel launches enqueued by this handle since creation (host-side counter). */
+uint64_t anakin_launch_count(anakin_t* h);
+
+/*
+ * Per-kernel timing with CUDA events recorded on the handle's stream around every launch (off by default; the
+ * events add a little launch overhead while on).  anakin_profile_read synchronises the stream, writes the summed
+ * duration in milliseconds and the number of launches of each kernel id (0 .. anakin_kernel_count()-1) since the
+ * last read into total_ms[] / counts[] (both of n_ids >= anakin_kernel_count() entries), and clears the records.
+ */
+int anakin_profile_enable(anakin_t* h, int on);
+int anakin_profile_read(anakin_t* h, int n_ids, double* total_ms, uint64_t* counts);
+int anakin_kernel_count(void);
+const char* anakin_kernel_name(int id);
+
+/* Static description of an error code. */
+const char* anakin_strerror(int code);
+
+/* Text of the last CUDA runtime error seen by this handle ("" if none). */
+const char* anakin_last_cuda_error(anakin_t* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ANAKIN_H_ */

@@ -1,0 +1,422 @@
+// Host side of the C ABI declared in include/anakin.h: configuration checks, workspace carving, state
+// tracking and kernel enqueueing.  The host only schedules (Podracer paper, Section 3.1): no call in the
+// rollout/learn/run path copies data or synchronises.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+using namespace anakin;
+
+struct anakin_handle {
+    anakin_cfg cfg;
+    Dims d;
+    Buffers b;
+    unsigned char* ws;
+    size_t ws_bytes;
+    cudaStream_t stream;
+    bool is_reset;
+    bool rollout_pending;
+    bool base_valid;  // `base` matches the current parameters
+    int last_T;
+    int NS;
+    uint64_t seed;
+    int64_t gstep;
+    int64_t adam_k;
+    uint64_t launches;
+    Profiler prof;
+    char cuda_err[256];
+    Ctx ctx() { return Ctx{stream, &launches, &prof}; }
+};
+
+namespace {
+
+int validate(const anakin_cfg* c) {
+    if (!c) return ANAKIN_E_INVALID_ARG;
+    if (c->struct_size != sizeof(anakin_cfg)) return ANAKIN_E_INVALID_ARG;
+    if (c->B < 1 || c->T_max < 1 || c->episode_cap < 1 || c->episode_cap > 255) return ANAKIN_E_INVALID_ARG;
+    if (!(c->wall_density >= 0.0 && c->wall_density < 1.0)) return ANAKIN_E_INVALID_ARG;
+    if (c->precision != ANAKIN_PRECISION_FP32 && c->precision != ANAKIN_PRECISION_BF16) return ANAKIN_E_INVALID_ARG;
+    if (c->reserved != 0) return ANAKIN_E_INVALID_ARG;
+    if (c->N < 2 || c->N > 16) return ANAKIN_E_UNSUPPORTED_CFG;
+    const int hj = c->H / 32;
+    if (c->H % 32 != 0) return ANAKIN_E_UNSUPPORTED_CFG;
+    switch (hj) {
+        case 1: case 2: case 3: case 4: case 6: case 8: case 12: case 16: case 24: case 32: break;
+        default: return ANAKIN_E_UNSUPPORTED_CFG;
+    }
+    if ((double)c->B * (double)c->T_max > 2.0e9) return ANAKIN_E_UNSUPPORTED_CFG;
+    return ANAKIN_OK;
+}
+
+int choose_splits(const Dims& d) {
+    const int tiles = ((d.H + 63) / 64) * ((d.H + 63) / 64);
+    int ns = (4 * 148 + tiles - 1) / tiles;
+    if (ns > 64) ns = 64;
+    const size_t R = (size_t)d.B * d.Tmax;
+    const size_t cap = R / 64 > 0 ? R / 64 : 1;
+    if ((size_t)ns > cap) ns = (int)cap;
+    if (ns < 1) ns = 1;
+    return ns;
+}
+
+// Carves the workspace; with base == nullptr only sizes it.
+size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Buffers* out) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> void* {
+        void* p = base ? base + off : nullptr;
+        off += (bytes + 255) / 256 * 256;
+        return p;
+    };
+    Buffers b;
+    memset(&b, 0, sizeof(b));
+    const size_t P = d.P, B = d.B, T = d.Tmax, R = B * T, H = d.H;
+    b.theta = (float*)take(P * 4);
+    b.theta_c = c.precision == ANAKIN_PRECISION_BF16 ? (float*)take(P * 4) : b.theta;
+    b.grads = (float*)take(P * 4);
+    b.adam_m = (float*)take(P * 4);
+    b.adam_v = (float*)take(P * 4);
+    b.walls = (uint32_t*)take(B * d.W * 4);
+    b.start = (uint8_t*)take(B);
+    b.goal = (uint8_t*)take(B);
+    b.pos = (uint8_t*)take(B);
+    b.tep = (uint8_t*)take(B);
+    b.tpos = (uint8_t*)take(R);
+    b.tact = (int8_t*)take(R);
+    b.tdone = (uint8_t*)take(R);
+    b.trew = (float*)take(R * 4);
+    b.tval = (float*)take((R + B) * 4);
+    b.tlogp = (float*)take(R * 4);
+    b.adv = (float*)take(R * 4);
+    b.ret = (float*)take(R * 4);
+    b.dbg_logits = c.debug_logits ? (float*)take(R * 16) : nullptr;
+    b.base = (float*)take(B * H * 4);
+    b.h1 = (float*)take(R * H * 4);
+    b.h2 = (float*)take(R * H * 4);
+    b.dh2 = (float*)take(R * H * 4);
+    b.dh1 = (float*)take(R * H * 4);
+    b.dout = (float*)take(R * 8 * 4);
+    b.S = (float*)take(B * H * 4);
+    b.part = (float*)take((size_t)NS * P * 4);
+    b.loss_part = (float*)take((size_t)LOSS_BLOCKS * 4 * 4);
+    b.stats = (anakin_stats*)take(sizeof(anakin_stats));
+    b.status = (int*)take(sizeof(int));
+    if (out) *out = b;
+    return off;
+}
+
+int fail_cuda(anakin_t* h, cudaError_t e) {
+    snprintf(h->cuda_err, sizeof(h->cuda_err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return ANAKIN_E_CUDA;
+}
+
+struct Blob {
+    void* ptr;
+    size_t bytes;
+    bool writable;
+    bool host_only;
+    bool is_traj;
+};
+
+Blob blob_of(anakin_t* h, int which) {
+    const Dims& d = h->d;
+    const Buffers& b = h->b;
+    const size_t B = d.B, T = h->last_T > 0 ? h->last_T : d.Tmax, R = B * T, P = d.P;
+    switch (which) {
+        case ANAKIN_PARAMS: return {b.theta, P * 4, true, false, false};
+        case ANAKIN_GRADS: return {b.grads, P * 4, false, false, false};
+        case ANAKIN_ADAM_M: return {b.adam_m, P * 4, true, false, false};
+        case ANAKIN_ADAM_V: return {b.adam_v, P * 4, true, false, false};
+        case ANAKIN_ADAM_STEP: return {&h->adam_k, 8, true, true, false};
+        case ANAKIN_ENV_WALLS: return {b.walls, B * d.W * 4, true, false, false};
+        case ANAKIN_ENV_START: return {b.start, B, true, false, false};
+        case ANAKIN_ENV_GOAL: return {b.goal, B, true, false, false};
+        case ANAKIN_ENV_POS: return {b.pos, B, true, false, false};
+        case ANAKIN_ENV_TEP: return {b.tep, B, true, false, false};
+        case ANAKIN_GLOBAL_STEP: return {&h->gstep, 8, true, true, false};
+        case ANAKIN_TRAJ_POS: return {b.tpos, R, true, false, true};
+        case ANAKIN_TRAJ_ACTION: return {b.tact, R, true, false, true};
+        case ANAKIN_TRAJ_DONE: return {b.tdone, R, true, false, true};
+        case ANAKIN_TRAJ_REWARD: return {b.trew, R * 4, true, false, true};
+        case ANAKIN_TRAJ_VALUE: return {b.tval, (R + B) * 4, true, false, true};
+        case ANAKIN_TRAJ_LOGP: return {b.tlogp, R * 4, true, false, true};
+        case ANAKIN_ADV: return {b.adv, R * 4, true, false, true};
+        case ANAKIN_RET: return {b.ret, R * 4, true, false, true};
+        case ANAKIN_STATS: return {b.stats, sizeof(anakin_stats), false, false, false};
+        case ANAKIN_DEBUG_LOGITS: return {b.dbg_logits, b.dbg_logits ? R * 16 : 0, false, false, false};
+        default: return {nullptr, 0, false, false, false};
+    }
+}
+
+int do_rollout(anakin_t* h, int T, const int8_t* forced) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset) return ANAKIN_E_BAD_STATE;
+    if (T < 1 || T > h->cfg.T_max) return ANAKIN_E_INVALID_ARG;
+    cudaError_t e;
+    if (!h->base_valid) {
+        e = launch_env_base(h->d, h->b, h->ctx());
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->base_valid = true;
+    }
+    RolloutArgs a;
+    a.d = h->d;
+    a.b = h->b;
+    a.T = T;
+    a.cap = h->cfg.episode_cap;
+    a.gstep0 = (uint32_t)h->gstep;
+    a.key0 = (uint32_t)(h->seed & 0xFFFFFFFFu);
+    a.key1 = (uint32_t)(h->seed >> 32);
+    a.forced = forced;
+    e = launch_rollout(a, h->cfg.precision, h->ctx());
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->gstep += T;
+    h->last_T = T;
+    h->rollout_pending = true;
+    return ANAKIN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int anakin_workspace_bytes(const anakin_cfg* cfg, size_t* bytes) {
+    if (!bytes) return ANAKIN_E_INVALID_ARG;
+    const int rc = validate(cfg);
+    if (rc != ANAKIN_OK) return rc;
+    const Dims d = make_dims(cfg->B, cfg->N, cfg->H, cfg->T_max);
+    *bytes = carve(*cfg, d, choose_splits(d), nullptr, nullptr);
+    return ANAKIN_OK;
+}
+
+int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void* cuda_stream, anakin_t** out) {
+    if (!out) return ANAKIN_E_INVALID_ARG;
+    *out = nullptr;
+    const int rc = validate(cfg);
+    if (rc != ANAKIN_OK) return rc;
+    if (!dev_workspace || ((uintptr_t)dev_workspace & 255u)) return ANAKIN_E_INVALID_ARG;
+    const Dims d = make_dims(cfg->B, cfg->N, cfg->H, cfg->T_max);
+    const int NS = choose_splits(d);
+    const size_t need = carve(*cfg, d, NS, nullptr, nullptr);
+    if (bytes < need) return ANAKIN_E_WORKSPACE_TOO_SMALL;
+    anakin_t* h = new (std::nothrow) anakin_t();
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    h->is_reset = h->rollout_pending = h->base_valid = false;
+    h->last_T = 0;
+    h->seed = 0;
+    h->gstep = h->adam_k = 0;
+    h->launches = 0;
+    h->cuda_err[0] = 0;
+    h->cfg = *cfg;
+    h->d = d;
+    h->NS = NS;
+    h->ws = (unsigned char*)dev_workspace;
+    h->ws_bytes = bytes;
+    h->stream = (cudaStream_t)cuda_stream;
+    carve(*cfg, d, NS, h->ws, &h->b);
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e == cudaSuccess && cur != cfg->device) e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) {
+        delete h;
+        return ANAKIN_E_CUDA;
+    }
+    *out = h;
+    return ANAKIN_OK;
+}
+
+int anakin_destroy(anakin_t* h) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    for (const Profiler::Rec& r : h->prof.recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    for (cudaEvent_t e : h->prof.pool) cudaEventDestroy(e);
+    delete h;
+    return ANAKIN_OK;
+}
+
+int anakin_reset(anakin_t* h, uint64_t seed) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    cudaError_t e = launch_reset(h->d, h->b, seed, h->cfg.wall_density, h->cfg.precision, h->ctx());
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->seed = seed;
+    h->gstep = 0;
+    h->adam_k = 0;
+    h->is_reset = true;
+    h->rollout_pending = false;
+    h->base_valid = false;
+    h->last_T = 0;
+    return ANAKIN_OK;
+}
+
+int anakin_rollout(anakin_t* h, int T) { return do_rollout(h, T, nullptr); }
+
+int anakin_rollout_forced(anakin_t* h, int T, const int8_t* dev_actions) {
+    if (!dev_actions) return ANAKIN_E_INVALID_ARG;
+    return do_rollout(h, T, dev_actions);
+}
+
+int anakin_gae(anakin_t* h) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
+    cudaError_t e = launch_gae(h->d, h->b, h->last_T, h->cfg.gamma, h->cfg.gae_lambda, h->ctx());
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    return ANAKIN_OK;
+}
+
+// The update proper, given ADV/RET already in place.
+static int learn_after_gae(anakin_t* h) {
+    cudaError_t e;
+    if (!h->base_valid) {
+        e = launch_env_base(h->d, h->b, h->ctx());
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->base_valid = true;
+    }
+    LearnArgs a;
+    a.d = h->d;
+    a.b = h->b;
+    a.T = h->last_T;
+    a.NS = h->NS;
+    a.c_v = h->cfg.value_coef;
+    a.c_e = h->cfg.entropy_coef;
+    a.lr = h->cfg.lr;
+    a.beta1 = h->cfg.adam_b1;
+    a.beta2 = h->cfg.adam_b2;
+    a.eps = h->cfg.adam_eps;
+    a.adam_k = (int)(h->adam_k + 1);
+    e = launch_learn(a, h->cfg.precision, h->ctx());
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->adam_k += 1;
+    h->base_valid = false;  // parameters changed
+    h->rollout_pending = false;
+    return ANAKIN_OK;
+}
+
+int anakin_learn(anakin_t* h) {
+    const int rc = anakin_gae(h);
+    if (rc != ANAKIN_OK) return rc;
+    return learn_after_gae(h);
+}
+
+int anakin_update(anakin_t* h) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
+    return learn_after_gae(h);
+}
+
+int anakin_run(anakin_t* h, int iters) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    if (iters < 0) return ANAKIN_E_INVALID_ARG;
+    for (int it = 0; it < iters; ++it) {
+        int rc = do_rollout(h, h->cfg.T_max, nullptr);
+        if (rc != ANAKIN_OK) return rc;
+        rc = anakin_learn(h);
+        if (rc != ANAKIN_OK) return rc;
+    }
+    return ANAKIN_OK;
+}
+
+size_t anakin_blob_bytes(anakin_t* h, int which) {
+    if (!h) return 0;
+    return blob_of(h, which).bytes;
+}
+
+static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is_device, bool to_lib) {
+    if (!h || !ptr) return ANAKIN_E_INVALID_ARG;
+    const Blob bl = blob_of(h, which);
+    if (!bl.ptr || bl.bytes == 0 || bytes != bl.bytes) return ANAKIN_E_INVALID_ARG;
+    if (to_lib && !bl.writable) return ANAKIN_E_INVALID_ARG;
+    if (bl.host_only) {
+        if (ptr_is_device) return ANAKIN_E_INVALID_ARG;
+        if (to_lib) memcpy(bl.ptr, ptr, bytes); else memcpy(ptr, bl.ptr, bytes);
+        return ANAKIN_OK;
+    }
+    const cudaMemcpyKind kind = ptr_is_device ? cudaMemcpyDeviceToDevice : (to_lib ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost);
+    cudaError_t e = to_lib ? cudaMemcpyAsync(bl.ptr, ptr, bytes, kind, h->stream) : cudaMemcpyAsync(ptr, bl.ptr, bytes, kind, h->stream);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    if (to_lib) {
+        if (which == ANAKIN_PARAMS) {
+            e = launch_refresh_compute_params(h->d, h->b, h->cfg.precision, h->ctx());
+            if (e != cudaSuccess) return fail_cuda(h, e);
+            h->base_valid = false;
+        }
+        if (which == ANAKIN_ENV_WALLS || which == ANAKIN_ENV_GOAL) h->base_valid = false;
+        if (bl.is_traj && h->is_reset) {
+            if (h->last_T == 0) h->last_T = h->cfg.T_max;
+            h->rollout_pending = true;
+        }
+    }
+    if (!ptr_is_device) {
+        e = cudaStreamSynchronize(h->stream);
+        if (e != cudaSuccess) return fail_cuda(h, e);
+    }
+    return ANAKIN_OK;
+}
+
+int anakin_get(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is_device) {
+    return copy_blob(h, which, ptr, bytes, ptr_is_device, false);
+}
+
+int anakin_set(anakin_t* h, int which, const void* ptr, size_t bytes, int ptr_is_device) {
+    return copy_blob(h, which, const_cast<void*>(ptr), bytes, ptr_is_device, true);
+}
+
+int anakin_status(anakin_t* h, int* device_status) {
+    if (!h || !device_status) return ANAKIN_E_INVALID_ARG;
+    int st = 0;
+    cudaError_t e = cudaMemcpyAsync(&st, h->b.status, sizeof(int), cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    *device_status = st;
+    return st == 0 ? ANAKIN_OK : ANAKIN_E_DEVICE_STATUS;
+}
+
+uint64_t anakin_launch_count(anakin_t* h) { return h ? h->launches : 0; }
+
+int anakin_kernel_count(void) { return K_COUNT; }
+
+const char* anakin_kernel_name(int id) {
+    static const char* names[K_COUNT] = {"reset_env", "reset_params", "refresh_params", "env_base", "rollout", "gae", "h1",
+                                         "fwd2", "heads_loss", "dh1", "dw2", "colsums", "sum_over_t", "dw1_agent",
+                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total"};
+    return (id >= 0 && id < K_COUNT) ? names[id] : "";
+}
+
+int anakin_profile_enable(anakin_t* h, int on) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    h->prof.on = on != 0;
+    return ANAKIN_OK;
+}
+
+int anakin_profile_read(anakin_t* h, int n_ids, double* total_ms, uint64_t* counts) {
+    if (!h || !total_ms || !counts || n_ids < K_COUNT) return ANAKIN_E_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    for (int i = 0; i < n_ids; ++i) { total_ms[i] = 0.0; counts[i] = 0; }
+    for (const Profiler::Rec& r : h->prof.recs) {
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, r.a, r.b);
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        total_ms[r.id] += ms;
+        counts[r.id] += 1;
+        h->prof.pool.push_back(r.a);
+        h->prof.pool.push_back(r.b);
+    }
+    h->prof.recs.clear();
+    return ANAKIN_OK;
+}
+
+const char* anakin_strerror(int code) {
+    switch (code) {
+        case ANAKIN_OK: return "ok";
+        case ANAKIN_E_INVALID_ARG: return "invalid argument";
+        case ANAKIN_E_BAD_STATE: return "call not valid in the handle's current state";
+        case ANAKIN_E_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case ANAKIN_E_UNSUPPORTED_CFG: return "unsupported configuration";
+        case ANAKIN_E_CUDA: return "CUDA runtime error";
+        case ANAKIN_E_DEVICE_STATUS: return "device status word is non-zero";
+        default: return "unknown error code";
+    }
+}
+
+const char* anakin_last_cuda_error(anakin_t* h) { return h ? h->cuda_err : ""; }
+
+}  // extern "C"

@@ -1,0 +1,175 @@
+// Shared device/host declarations of the Anakin library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "anakin.h"
+
+namespace anakin {
+
+// Sticky device status bits (anakin_status).
+enum : int {
+    DEV_OK = 0,
+    DEV_E_BAD_ACTION = 1,   // a forced action outside 0..3
+    DEV_E_BAD_STATE = 2,    // an env position outside the grid or on a wall
+    DEV_E_WAIT_TIMEOUT = 4  // a bounded wait gave up
+};
+
+struct Dims {
+    int B, N, C, D, H, W, Tmax;  // envs, grid side, cells, obs features, hidden, wall words per env, max T
+    size_t oW1, ob1, oW2, ob2, oWh, obh, P;
+};
+
+inline Dims make_dims(int B, int N, int H, int Tmax) {
+    Dims d;
+    d.B = B; d.N = N; d.C = N * N; d.D = 3 * d.C; d.H = H; d.W = (d.C + 31) / 32; d.Tmax = Tmax;
+    d.oW1 = 0;
+    d.ob1 = d.oW1 + (size_t)d.D * H;
+    d.oW2 = d.ob1 + H;
+    d.ob2 = d.oW2 + (size_t)H * H;
+    d.oWh = d.ob2 + H;
+    d.obh = d.oWh + (size_t)H * 5;
+    d.P = d.obh + 5;
+    return d;
+}
+
+// Every sub-buffer of the caller's workspace.
+struct Buffers {
+    float* theta;    // fp32 master parameters [P]
+    float* theta_c;  // parameters the network computes with: == theta (fp32) or bf16-rounded weights (bf16 mode)
+    float* grads;    // [P]
+    float* adam_m;   // [P]
+    float* adam_v;   // [P]
+    uint32_t* walls; // [B][W]
+    uint8_t* start;  // [B]
+    uint8_t* goal;   // [B]
+    uint8_t* pos;    // [B]
+    uint8_t* tep;    // [B]
+    uint8_t* tpos;   // [Tmax][B]
+    int8_t* tact;    // [Tmax][B]
+    uint8_t* tdone;  // [Tmax][B]
+    float* trew;     // [Tmax][B]
+    float* tval;     // [Tmax+1][B]
+    float* tlogp;    // [Tmax][B]
+    float* adv;      // [Tmax][B]
+    float* ret;      // [Tmax][B]
+    float* dbg_logits;  // [Tmax][B][4] or null
+    float* base;     // [B][H]  b1 + sum of W1 rows of the wall cells + W1 row of the goal cell
+    float* h1;       // [R][H]
+    float* h2;       // [R][H]
+    float* dh2;      // [R][H]
+    float* dh1;      // [R][H]
+    float* dout;     // [R][8]  (5 used)
+    float* S;        // [B][H]  sum over t of dh1
+    float* part;     // [NS][P] split-K partial gradients
+    float* loss_part;  // [LOSS_BLOCKS][4]
+    anakin_stats* stats;
+    int* status;
+};
+
+constexpr int LOSS_BLOCKS = 592;
+
+// ---- Philox4x32-10 (Salmon et al., SC'11) ----
+struct U4 { uint32_t x, y, z, w; };
+
+__host__ __device__ inline U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t pa = (uint64_t)0xD2511F53u * c0;
+        const uint64_t pb = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(pb >> 32) ^ c1 ^ k0;
+        const uint32_t n2 = (uint32_t)(pa >> 32) ^ c3 ^ k1;
+        c1 = (uint32_t)pb;
+        c3 = (uint32_t)pa;
+        c0 = n0;
+        c2 = n2;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return U4{c0, c1, c2, c3};
+}
+
+enum : uint32_t { STREAM_ENV = 1, STREAM_PARAM = 2, STREAM_ACT = 3 };
+
+__device__ inline float uniform24(uint32_t x) { return (float)(x >> 8) * (1.0f / 16777216.0f); }
+
+__device__ inline float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+template <int PREC> __device__ inline float rnd(float x) { return PREC == 1 ? round_bf16(x) : x; }
+
+// launch parameter blocks --------------------------------------------------------------------------
+struct RolloutArgs {
+    Dims d;
+    Buffers b;
+    int T;
+    int cap;
+    uint32_t gstep0;
+    uint32_t key0, key1;
+    const int8_t* forced;  // nullable
+};
+
+struct LearnArgs {
+    Dims d;
+    Buffers b;
+    int T;
+    int NS;  // split-K factor of the weight-gradient GEMMs
+    float c_v, c_e;
+    float lr, beta1, beta2, eps;
+    int adam_k;  // step index after the increment
+};
+
+// Kernel identifiers (anakin_kernel_name / anakin_profile_read index by these).
+enum KernelId : int {
+    K_RESET_ENV = 0, K_RESET_PARAMS, K_REFRESH_PARAMS, K_ENV_BASE, K_ROLLOUT, K_GAE, K_H1, K_FWD2, K_HEADS_LOSS, K_DH1,
+    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_COUNT
+};
+
+// Optional per-kernel timing with CUDA events on the launching stream (off by default).
+struct Profiler {
+    struct Rec { int id; cudaEvent_t a, b; };
+    bool on = false;
+    std::vector<Rec> recs;
+    std::vector<cudaEvent_t> pool;
+    cudaEvent_t take() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+};
+
+// What a launch site needs: the stream, the launch counter and the profiler.
+struct Ctx {
+    cudaStream_t s;
+    uint64_t* launches;
+    Profiler* prof;
+};
+
+// Counts one kernel launch and, when profiling, brackets it with two events.
+struct Scope {
+    const Ctx& c;
+    cudaEvent_t b = nullptr;
+    Scope(const Ctx& ctx, int id) : c(ctx) {
+        ++*c.launches;
+        if (c.prof && c.prof->on) {
+            Profiler::Rec r{id, c.prof->take(), c.prof->take()};
+            cudaEventRecord(r.a, c.s);
+            b = r.b;
+            c.prof->recs.push_back(r);
+        }
+    }
+    ~Scope() { if (b) cudaEventRecord(b, c.s); }
+};
+
+// kernels (defined in the .cu files) ----------------------------------------------------------------
+cudaError_t launch_reset(const Dims& d, const Buffers& b, uint64_t seed, double density, int prec, const Ctx& c);
+cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c);
+cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c);
+cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
+cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
+cudaError_t launch_refresh_compute_params(const Dims& d, const Buffers& b, int prec, const Ctx& c);
+
+}  // namespace anakin

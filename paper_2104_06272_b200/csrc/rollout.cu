@@ -1,0 +1,284 @@
+// Acting half of the Anakin minimal unit (Podracer paper, Section 3.1; Figure 2, top): T interactions of
+// every env with the policy, fused into one persistent kernel.  A CTA owns ME envs for the whole rollout,
+// so there is no inter-CTA dependency and no grid-wide wait anywhere.
+#include "common.cuh"
+
+namespace anakin {
+
+// base[b][j] = b1[j] + sum over wall cells c (ascending) of W1[c][j] + W1[2C+goal_b][j].
+// The wall and goal planes of the observation do not change during an env's life, so their contribution
+// to the first layer is computed once per parameter version instead of once per step.
+__global__ void __launch_bounds__(256) k_env_base(Dims d, Buffers b) {
+    const int e = blockIdx.x;
+    const uint32_t* w = b.walls + (size_t)e * d.W;
+    const float* W1 = b.theta_c + d.oW1;
+    const int goal = b.goal[e];
+    for (int j = threadIdx.x; j < d.H; j += blockDim.x) {
+        float acc = b.theta_c[d.ob1 + j];
+        for (int wi = 0; wi < d.W; ++wi) {
+            uint32_t bits = w[wi];
+            while (bits) {
+                const int c = wi * 32 + (__ffs(bits) - 1);
+                bits &= bits - 1;
+                acc += W1[(size_t)c * d.H + j];
+            }
+        }
+        acc += W1[(size_t)(2 * d.C + goal) * d.H + j];
+        b.base[(size_t)e * d.H + j] = acc;
+    }
+}
+
+cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c) {
+    Scope sc(c, K_ENV_BASE);
+    k_env_base<<<d.B, d.H < 256 ? d.H : 256, 0, c.s>>>(d, b);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------------------------
+// Persistent rollout.  256 threads = 8 warps; H = 32*HJ hidden units; ME = 8*RR envs per CTA.
+// Per step: h1 = relu(base + W1[agent row]) -> h2 = relu(h1 W2 + b2) (register-tiled FFMA, W2 streamed through
+// L1/L2) -> 5 head outputs by warp reduction -> one thread per env: softmax, inverse-CDF sample with the
+// Philox uniform of (env, global step), env step, coalesced time-major stores.
+// ----------------------------------------------------------------------------------------------------
+template <int HJ, int RR, int PREC>
+__global__ void __launch_bounds__(256) k_rollout(RolloutArgs a) {
+    constexpr int H = 32 * HJ, ME = 8 * RR;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* s_base = reinterpret_cast<float*>(smem_raw);  // [ME][H]
+    float* s_h1 = s_base + ME * H;                       // [ME][H]
+    float* s_h2 = s_h1 + ME * H;                         // [ME][H]
+    float* s_out = s_h2 + ME * H;                        // [ME][8]
+    uint32_t* s_walls = reinterpret_cast<uint32_t*>(s_out + ME * 8);  // [ME][8]
+    int* s_pos = reinterpret_cast<int*>(s_walls + ME * 8);            // [ME]
+
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int e0 = blockIdx.x * ME;
+    const int B = d.B, C = d.C, N = d.N;
+    const float* W1 = b.theta_c + d.oW1;
+    const float* W2 = b.theta_c + d.oW2;
+    const float* b2 = b.theta_c + d.ob2;
+    const float* Wh = b.theta_c + d.oWh;
+    const float* bh = b.theta_c + d.obh;
+
+    for (int idx = tid; idx < ME * H; idx += 256) {
+        const int e = idx / H, j = idx - e * H;
+        s_base[idx] = (e0 + e < B) ? b.base[(size_t)(e0 + e) * H + j] : 0.f;
+    }
+    // per-env state lives in the registers of thread `tid` (tid < ME)
+    int my_pos = 0, my_tep = 0, my_start = 0, my_goal = 0;
+    const bool owner = tid < ME && e0 + tid < B;
+    if (tid < ME) {
+        if (owner) {
+            my_pos = b.pos[e0 + tid];
+            my_tep = b.tep[e0 + tid];
+            my_start = b.start[e0 + tid];
+            my_goal = b.goal[e0 + tid];
+            for (int wi = 0; wi < 8; ++wi) s_walls[tid * 8 + wi] = wi < d.W ? b.walls[(size_t)(e0 + tid) * d.W + wi] : 0u;
+        }
+        s_pos[tid] = my_pos;
+    }
+    unsigned long long n_episodes = 0, n_goals = 0, n_epsteps = 0;
+    int bad = 0;
+    __syncthreads();
+
+    for (int t = 0; t <= a.T; ++t) {
+        // ---- layer 1: only the agent plane changes from step to step
+        for (int idx = tid; idx < ME * H; idx += 256) {
+            const int e = idx / H, j = idx - e * H;
+            const float z = s_base[idx] + W1[(size_t)(C + s_pos[e]) * H + j];
+            s_h1[idx] = rnd<PREC>(fmaxf(z, 0.f));
+        }
+        __syncthreads();
+        // ---- layer 2: thread (wid, lane) owns rows wid+8*rr and columns lane+32*jj
+        {
+            float acc[RR][HJ];
+#pragma unroll
+            for (int rr = 0; rr < RR; ++rr)
+#pragma unroll
+                for (int jj = 0; jj < HJ; ++jj) acc[rr][jj] = 0.f;
+#pragma unroll 2
+            for (int k = 0; k < H; ++k) {
+                float w[HJ];
+#pragma unroll
+                for (int jj = 0; jj < HJ; ++jj) w[jj] = __ldg(W2 + (size_t)k * H + lane + 32 * jj);
+#pragma unroll
+                for (int rr = 0; rr < RR; ++rr) {
+                    const float x = s_h1[(wid + 8 * rr) * H + k];
+#pragma unroll
+                    for (int jj = 0; jj < HJ; ++jj) acc[rr][jj] = fmaf(x, w[jj], acc[rr][jj]);
+                }
+            }
+#pragma unroll
+            for (int jj = 0; jj < HJ; ++jj) {
+                const float bias = __ldg(b2 + lane + 32 * jj);
+#pragma unroll
+                for (int rr = 0; rr < RR; ++rr)
+                    s_h2[(wid + 8 * rr) * H + lane + 32 * jj] = rnd<PREC>(fmaxf(acc[rr][jj] + bias, 0.f));
+            }
+        }
+        __syncthreads();
+        // ---- heads: warp `wid` reduces its RR envs
+#pragma unroll
+        for (int rr = 0; rr < RR; ++rr) {
+            const int e = wid + 8 * rr;
+            float o[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int k = lane; k < H; k += 32) {
+                const float x = s_h2[e * H + k];
+#pragma unroll
+                for (int c = 0; c < 5; ++c) o[c] = fmaf(x, __ldg(Wh + k * 5 + c), o[c]);
+            }
+#pragma unroll
+            for (int c = 0; c < 5; ++c) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) o[c] += __shfl_xor_sync(0xFFFFFFFFu, o[c], off);
+            }
+            if (lane < 5) s_out[e * 8 + lane] = o[lane] + __ldg(bh + lane);
+        }
+        __syncthreads();
+        // ---- one thread per env: value, sample, env step, records
+        if (owner) {
+            const int env = e0 + tid;
+            const float l0 = s_out[tid * 8 + 0], l1 = s_out[tid * 8 + 1], l2 = s_out[tid * 8 + 2], l3 = s_out[tid * 8 + 3];
+            b.tval[(size_t)t * B + env] = s_out[tid * 8 + 4];
+            if (t < a.T) {
+                const size_t i = (size_t)t * B + env;
+                const float mx = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
+                const float x0 = expf(l0 - mx), x1 = expf(l1 - mx), x2 = expf(l2 - mx), x3 = expf(l3 - mx);
+                const float Z = ((x0 + x1) + x2) + x3;
+                const float c0 = x0 / Z, c1 = c0 + x1 / Z, c2 = c1 + x2 / Z;
+                const U4 r = philox4x32_10((uint32_t)env, a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
+                const float u = uniform24(r.x);
+                int act = (u >= c0) + (u >= c1) + (u >= c2);
+                if (a.forced) {
+                    act = a.forced[i];
+                    if (act < 0 || act > 3) { bad |= DEV_E_BAD_ACTION; act &= 3; }
+                }
+                const float la = act == 0 ? l0 : act == 1 ? l1 : act == 2 ? l2 : l3;
+                b.tlogp[i] = (la - mx) - logf(Z);
+                b.tpos[i] = (uint8_t)my_pos;
+                b.tact[i] = (int8_t)act;
+                if (b.dbg_logits) reinterpret_cast<float4*>(b.dbg_logits)[i] = make_float4(l0, l1, l2, l3);
+                // env step
+                const int row = my_pos / N, col = my_pos - row * N;
+                int nr = row, nc = col;
+                if (act == 0) nr = row - 1;
+                else if (act == 1) nc = col + 1;
+                else if (act == 2) nr = row + 1;
+                else nc = col - 1;
+                int np = my_pos;
+                if (nr >= 0 && nr < N && nc >= 0 && nc < N) {
+                    const int cand = nr * N + nc;
+                    if (!((s_walls[tid * 8 + (cand >> 5)] >> (cand & 31)) & 1u)) np = cand;
+                }
+                const int te = my_tep + 1;
+                float rew = 0.f;
+                int done = 0;
+                if (np == my_goal) { rew = 1.f; done = 1; }
+                else if (te >= a.cap) { done = 1; }
+                if (done) {
+                    n_episodes += 1;
+                    n_goals += (np == my_goal);
+                    n_epsteps += te;
+                    my_pos = my_start;
+                    my_tep = 0;
+                } else {
+                    my_pos = np;
+                    my_tep = te;
+                }
+                b.trew[i] = rew;
+                b.tdone[i] = (uint8_t)done;
+                s_pos[tid] = my_pos;
+            }
+        }
+        __syncthreads();
+    }
+    if (owner) {
+        b.pos[e0 + tid] = (uint8_t)my_pos;
+        b.tep[e0 + tid] = (uint8_t)my_tep;
+    }
+    // statistics: integer atomics only, so totals do not depend on arrival order
+    if (tid < 32) {
+        // ME <= 32: all owners are in warp 0
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            n_episodes += __shfl_xor_sync(0xFFFFFFFFu, n_episodes, off);
+            n_goals += __shfl_xor_sync(0xFFFFFFFFu, n_goals, off);
+            n_epsteps += __shfl_xor_sync(0xFFFFFFFFu, n_epsteps, off);
+            bad |= __shfl_xor_sync(0xFFFFFFFFu, bad, off);
+        }
+        if (tid == 0) {
+            if (n_episodes) atomicAdd((unsigned long long*)&b.stats->episodes, n_episodes);
+            if (n_goals) atomicAdd((unsigned long long*)&b.stats->goals, n_goals);
+            if (n_epsteps) atomicAdd((unsigned long long*)&b.stats->episode_steps, n_epsteps);
+            if (blockIdx.x == 0) atomicAdd((unsigned long long*)&b.stats->frames, (unsigned long long)B * a.T);
+            if (bad) atomicOr(b.status, bad);
+        }
+    }
+}
+
+template <int HJ, int RR, int PREC>
+static cudaError_t launch_rollout_t(const RolloutArgs& a, cudaStream_t s) {
+    constexpr int H = 32 * HJ, ME = 8 * RR;
+    const size_t smem = (size_t)(3 * ME * H + ME * 8) * sizeof(float) + ME * 8 * sizeof(uint32_t) + ME * sizeof(int);
+    cudaError_t e = cudaFuncSetAttribute(k_rollout<HJ, RR, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_rollout<HJ, RR, PREC><<<(a.d.B + ME - 1) / ME, 256, smem, s>>>(a);
+    return cudaGetLastError();
+}
+
+template <int PREC>
+static cudaError_t launch_rollout_p(const RolloutArgs& a, cudaStream_t s) {
+    switch (a.d.H / 32) {
+        case 1: return launch_rollout_t<1, 4, PREC>(a, s);
+        case 2: return launch_rollout_t<2, 4, PREC>(a, s);
+        case 3: return launch_rollout_t<3, 4, PREC>(a, s);
+        case 4: return launch_rollout_t<4, 4, PREC>(a, s);
+        case 6: return launch_rollout_t<6, 4, PREC>(a, s);
+        case 8: return launch_rollout_t<8, 4, PREC>(a, s);
+        case 12: return launch_rollout_t<12, 4, PREC>(a, s);
+        case 16: return launch_rollout_t<16, 2, PREC>(a, s);
+        case 24: return launch_rollout_t<24, 2, PREC>(a, s);
+        case 32: return launch_rollout_t<32, 2, PREC>(a, s);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c) {
+    Scope sc(c, K_ROLLOUT);
+    return prec == 1 ? launch_rollout_p<1>(a, c.s) : launch_rollout_p<0>(a, c.s);
+}
+
+// ----------------------------------------------------------------------------------------------------
+// GAE reverse scan: lane = env, so every load and store of a warp is one contiguous segment per t.
+//   d_t = 1 - done_t; delta_t = r_t + gamma d_t V_{t+1} - V_t; A_t = delta_t + gamma lambda d_t A_{t+1}; ret = A + V
+// ----------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_gae(Dims d, Buffers b, int T, float gamma, float lambda) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= d.B) return;
+    const size_t B = (size_t)d.B;
+    float A = 0.f;
+    float vnext = b.tval[(size_t)T * B + e];
+    const float gl = gamma * lambda;
+#pragma unroll 4
+    for (int t = T - 1; t >= 0; --t) {
+        const size_t i = (size_t)t * B + e;
+        const float v = b.tval[i];
+        const float r = b.trew[i];
+        const float nd = b.tdone[i] ? 0.f : 1.f;
+        const float delta = r + gamma * nd * vnext - v;
+        A = delta + gl * nd * A;
+        b.adv[i] = A;
+        b.ret[i] = A + v;
+        vnext = v;
+    }
+}
+
+cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c) {
+    Scope sc(c, K_GAE);
+    k_gae<<<(d.B + 127) / 128, 128, 0, c.s>>>(d, b, T, gamma, lambda);
+    return cudaGetLastError();
+}
+
+}  // namespace anakin

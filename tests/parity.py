@@ -1,0 +1,145 @@
+"""Helpers for the GPU-vs-oracle parity tests: the tolerance metric and the staged, teacher-forced
+comparison of one act+learn iteration."""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import binding as orc
+
+RTOL_FP32 = 1e-4
+RTOL_BF16 = 2e-2
+
+
+def rtol_of(prec: int) -> float:
+    return RTOL_BF16 if prec == 1 else RTOL_FP32
+
+
+def assert_close(got, want, rtol, name):
+    """Per tensor: |g - o| <= rtol * (|o| + rms(o)) for every element (a purely element-wise relative
+    error is meaningless at zero crossings)."""
+    got = np.asarray(got, dtype=np.float64).ravel()
+    want = np.asarray(want, dtype=np.float64).ravel()
+    assert got.shape == want.shape, (name, got.shape, want.shape)
+    assert np.isfinite(got).all(), f"{name}: non-finite values"
+    rms = np.sqrt((want**2).mean()) if want.size else 0.0
+    err = np.abs(got - want)
+    bound = rtol * (np.abs(want) + rms)
+    bad = err > bound
+    if bad.any():
+        i = int(np.argmax(err - bound))
+        raise AssertionError(f"{name}: {int(bad.sum())}/{got.size} outside rtol={rtol}; worst at {i}: got {got[i]!r} "
+                             f"want {want[i]!r} (rms {rms:.3e})")
+
+
+def gpu_state(an, bnd):
+    """Host copies of everything the oracle needs to shadow the library."""
+    return dict(theta=an.get(bnd.PARAMS), m=an.get(bnd.ADAM_M), v=an.get(bnd.ADAM_V), k=int(an.get(bnd.ADAM_STEP)),
+                walls=an.get(bnd.ENV_WALLS).reshape(an.B, -1), start=an.get(bnd.ENV_START), goal=an.get(bnd.ENV_GOAL),
+                pos=an.get(bnd.ENV_POS), tep=an.get(bnd.ENV_TEP), gstep=int(an.get(bnd.GLOBAL_STEP)))
+
+
+def gpu_traj(an, bnd, T):
+    B = an.B
+    return dict(pos=an.get(bnd.TRAJ_POS).reshape(T, B), action=an.get(bnd.TRAJ_ACTION).reshape(T, B),
+                done=an.get(bnd.TRAJ_DONE).reshape(T, B), reward=an.get(bnd.TRAJ_REWARD).reshape(T, B),
+                value=an.get(bnd.TRAJ_VALUE).reshape(T + 1, B), logp=an.get(bnd.TRAJ_LOGP).reshape(T, B),
+                logits=an.get(bnd.DEBUG_LOGITS).reshape(T, B, 4))
+
+
+def check_rollout(an, bnd, w, seed, st, T, forced=None, envs=None):
+    """Stage 1+2: acts on the GPU, then the oracle replays the GPU's action sequence from the same
+    state.  Transitions are bit-exact; logits/values/logp within tolerance; the GPU's actions equal the
+    oracle's samples from the GPU's own logits except where the uniform is within 1e-5 of a CDF
+    boundary.  `envs` restricts the oracle's replay to a subset of env indices (full-size workloads)."""
+    rtol = rtol_of(w.precision)
+    if forced is None:
+        an.rollout(T)
+    else:
+        import torch
+
+        an.rollout_forced(torch.from_numpy(forced).cuda())
+    g = gpu_traj(an, bnd, T)
+    assert an.status() == 0
+    sel = np.arange(an.B) if envs is None else np.asarray(envs)
+    pos, tep = st["pos"][sel].copy(), st["tep"][sel].copy()
+    tr = orc.rollout(w.N, w.H, w.precision, T, w.episode_cap, st["theta"], np.ascontiguousarray(st["walls"][sel]),
+                     st["start"][sel].copy(), st["goal"][sel].copy(), pos, tep, seed, st["gstep"],
+                     forced=np.ascontiguousarray(g["action"][:, sel]))
+    if forced is not None:
+        assert (g["action"] == forced).all()
+    assert (g["pos"][:, sel] == tr.pos).all(), "recorded positions differ"
+    assert (g["reward"][:, sel] == tr.reward).all(), "rewards differ"
+    assert (g["done"][:, sel] == tr.done).all(), "done flags differ"
+    assert (an.get(bnd.ENV_POS)[sel] == pos).all() and (an.get(bnd.ENV_TEP)[sel] == tep).all(), "final env state differs"
+    assert int(an.get(bnd.GLOBAL_STEP)) == st["gstep"] + T
+    assert_close(g["logits"][:, sel], tr.logits, rtol, "logits")
+    assert_close(g["value"][:, sel], tr.value, rtol, "values")
+    assert_close(g["logp"][:, sel], tr.logp, rtol, "logp")
+    n_near = n_mis = 0
+    if forced is None:
+        # sample from the GPU's own logits with the same uniforms
+        if envs is None:
+            act, logp, near = orc.sample_from_logits(seed, st["gstep"], g["logits"])
+        else:
+            act = np.zeros((T, len(sel)), np.int8)
+            logp = np.zeros((T, len(sel)), np.float32)
+            near = np.zeros((T, len(sel)), np.uint8)
+            for t in range(T):
+                for j, b in enumerate(sel):
+                    a, lp, nr = orc.sample_one(g["logits"][t, b], orc.act_uniform(seed, int(b), st["gstep"] + t))
+                    act[t, j], logp[t, j], near[t, j] = a, lp, nr
+        mism = act != g["action"][:, sel]
+        n_near, n_mis = int(near.sum()), int(mism.sum())
+        assert not (mism & (near == 0)).any(), "an action differs away from any CDF boundary"
+        assert n_mis <= max(1, int(1e-4 * mism.size)), f"{n_mis} action mismatches in {mism.size} samples"
+        ok = ~mism
+        assert_close(g["logp"][:, sel][ok], logp[ok], 1e-4 if w.precision == 0 else 1e-4, "logp of sampled action")
+    return g, dict(near=n_near, mismatched=n_mis)
+
+
+def check_gae(an, bnd, w, g, T):
+    an.gae()
+    adv, ret = orc.gae(np.float32(w.gamma), np.float32(w.gae_lambda), g["reward"], g["value"], g["done"])
+    gadv, gret = an.get(bnd.ADV).reshape(T, an.B), an.get(bnd.RET).reshape(T, an.B)
+    assert_close(gadv, adv, RTOL_FP32, "advantages")
+    assert_close(gret, ret, RTOL_FP32, "returns")
+    return gadv, gret
+
+
+def check_learn(an, bnd, w, st, g, gadv, gret):
+    """Stage 4: the oracle learns from the GPU's trajectory, advantages/returns and pre-update
+    parameters.  Gradients and loss terms are compared directly; Adam is compared on the GPU's own
+    gradient (its early steps are close to lr*sign(g), which would otherwise turn a 1e-7 gradient
+    difference on a near-zero element into a full-size parameter difference)."""
+    rtol = rtol_of(w.precision)
+    an.learn()
+    ograds, oloss = orc.learn(w.N, w.H, w.precision, st["theta"], st["walls"], st["goal"], g["pos"], g["action"], gadv,
+                              gret, np.float32(w.value_coef), np.float32(w.entropy_coef))
+    ggrads = an.get(bnd.GRADS)
+    d = orc.Dims(w.N, w.H)
+    for name, sl in d.slices().items():
+        assert_close(ggrads[sl], ograds[sl], rtol, f"grad {name}")
+    s = an.stats()
+    gl = np.array([s.loss_total, s.loss_pg, s.loss_value, s.entropy], dtype=np.float64)
+    lt = max(rtol, 1e-4)
+    scale = np.abs(oloss).max()
+    assert (np.abs(gl - oloss) <= lt * (np.abs(oloss) + 1e-3 * scale) + 1e-7).all(), (gl, oloss)
+    theta, m, v = st["theta"].copy(), st["m"].copy(), st["v"].copy()
+    orc.adam(theta, ggrads, m, v, st["k"] + 1, np.float32(w.lr), np.float32(w.adam_b1), np.float32(w.adam_b2),
+             np.float32(w.adam_eps))
+    assert int(an.get(bnd.ADAM_STEP)) == st["k"] + 1
+    assert_close(an.get(bnd.ADAM_M), m, RTOL_FP32, "adam m")
+    assert_close(an.get(bnd.ADAM_V), v, RTOL_FP32, "adam v")
+    gtheta = an.get(bnd.PARAMS)
+    assert_close(gtheta, theta, RTOL_FP32, "updated params")
+    assert_close(gtheta.astype(np.float64) - st["theta"], theta.astype(np.float64) - st["theta"], RTOL_FP32, "param step")
+    return ograds, oloss
+
+
+def check_iteration(an, bnd, w, seed, T=None):
+    T = w.T if T is None else T
+    st = gpu_state(an, bnd)
+    g, counts = check_rollout(an, bnd, w, seed, st, T)
+    gadv, gret = check_gae(an, bnd, w, g, T)
+    check_learn(an, bnd, w, st, g, gadv, gret)
+    return counts

@@ -1,0 +1,265 @@
+"""GPU-vs-oracle parity through the C ABI (needs a B200).
+
+Stages are teacher-forced: one flipped action would send a free-running comparison down a different
+trajectory, so each stage of the library is fed to the oracle and compared there.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import binding as orc
+from paper_2104_06272_b200.workloads import WORKLOADS, Workload, forced_actions, random_params
+from tests import parity as par
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bnd():
+    from paper_2104_06272_b200 import binding
+
+    return binding
+
+
+def make(bnd, w, T_max=None, debug=1):
+    return bnd.Anakin(bnd.cfg_from_workload(w, debug_logits=debug, T_max=T_max))
+
+
+# Reduced-batch versions of the large workloads (same grid, network, T and precision) whose oracle run takes
+# seconds; they still span several CTA tiles and a ragged tail.
+SMALL = {
+    "tiny": WORKLOADS["tiny"],
+    "memory_bound_s": WORKLOADS["memory_bound"].scaled(name="memory_bound_s", B=2048 + 37),
+    "large_batch_s": WORKLOADS["large_batch"].scaled(name="large_batch_s", B=1024 + 19),
+    "tensor_core_s": WORKLOADS["tensor_core"].scaled(name="tensor_core_s", B=256 + 5),
+    "ragged": Workload("ragged", B=77, N=7, H=96, T=5, iters=1, episode_cap=6),
+    "one_env": Workload("one_env", B=1, N=2, H=32, T=1, iters=1, episode_cap=1, wall_density=0.0),
+    "dense_walls": Workload("dense_walls", B=130, N=16, H=32, T=9, iters=1, episode_cap=255, wall_density=0.9),
+    "ragged_bf16": Workload("ragged_bf16", B=45, N=6, H=192, T=7, iters=1, precision=1, episode_cap=4),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_reset_is_bit_exact(bnd, name):
+    w = SMALL[name]
+    seed = (7 << 32) | 12345
+    an = make(bnd, w)
+    an.reset(seed)
+    walls, start, goal = orc.env_init(seed, w.B, w.N, w.wall_density)
+    assert (an.get(bnd.ENV_WALLS).reshape(w.B, -1) == walls).all()
+    assert (an.get(bnd.ENV_START) == start).all() and (an.get(bnd.ENV_GOAL) == goal).all()
+    assert (an.get(bnd.ENV_POS) == start).all() and not an.get(bnd.ENV_TEP).any()
+    theta = orc.param_init(seed, w.N, w.H)
+    assert (an.get(bnd.PARAMS).view(np.uint32) == theta.view(np.uint32)).all()
+    assert not an.get(bnd.ADAM_M).any() and not an.get(bnd.ADAM_V).any()
+    assert int(an.get(bnd.ADAM_STEP)) == 0 and int(an.get(bnd.GLOBAL_STEP)) == 0
+    s = an.stats()
+    assert (s.frames, s.episodes, s.goals, s.episode_steps) == (0, 0, 0, 0)
+    assert an.status() == 0
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_env_transitions_bit_exact_under_forced_actions(bnd, name):
+    w = SMALL[name]
+    an = make(bnd, w)
+    an.reset(3)
+    for it in range(2):  # the second pass continues from the first pass's env state
+        st = par.gpu_state(an, bnd)
+        f = forced_actions(100 + it, w.T, w.B)
+        g, _ = par.check_rollout(an, bnd, w, 3, st, w.T, forced=f)
+    s = an.stats()
+    assert s.frames == 2 * w.T * w.B
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_one_iteration_stage_by_stage(bnd, name):
+    w = SMALL[name]
+    an = make(bnd, w)
+    an.reset(11)
+    # start from parameters with non-zero biases so every term of the network is exercised
+    an.set(bnd.PARAMS, random_params(5, w.P, 0.15))
+    counts = par.check_iteration(an, bnd, w, 11)
+    # and a second iteration from the updated parameters and Adam state
+    counts2 = par.check_iteration(an, bnd, w, 11)
+    print(name, "near-boundary samples:", counts, counts2)
+
+
+def test_tiny_free_running_end_to_end(bnd):
+    """The tiny workload, both sides run freely for its 2 iterations from one seed: same actions, same
+    trajectories, parameters within tolerance."""
+    w = WORKLOADS["tiny"]
+    an = make(bnd, w)
+    ag = orc.Agent(w.B, w.N, w.H, w.T, w.precision, w.episode_cap, w.wall_density, np.float32(w.gamma),
+                   np.float32(w.gae_lambda), np.float32(w.entropy_coef), np.float32(w.value_coef), np.float32(w.lr),
+                   np.float32(w.adam_b1), np.float32(w.adam_b2), np.float32(w.adam_eps))
+    an.reset(1)
+    ag.reset(1)
+    for it in range(w.iters):
+        an.rollout()
+        tr = ag.rollout()
+        g = par.gpu_traj(an, bnd, w.T)
+        mism = g["action"] != tr.action
+        assert not (mism & (tr.near == 0)).any()
+        if mism.any():
+            pytest.skip("a near-boundary sample diverged the free-running comparison")
+        assert (g["pos"] == tr.pos).all() and (g["reward"] == tr.reward).all() and (g["done"] == tr.done).all()
+        par.assert_close(g["value"], tr.value, 1e-4, "values")
+        an.learn()
+        ag.learn()
+        par.assert_close(an.get(bnd.ADV), ag.adv, 1e-4, "adv")
+        par.assert_close(an.get(bnd.GRADS), ag.grads, 1e-4, "grads")
+    # Adam's first steps are ~lr*sign(g): compare parameters where the gradient is not within rounding of zero
+    gt, ot = an.get(bnd.PARAMS), ag.theta
+    assert np.abs(gt - ot).max() <= 2.1 * w.iters * w.lr
+    big = np.abs(ag.grads) > 1e-3 * np.sqrt((ag.grads.astype(np.float64) ** 2).mean())
+    par.assert_close(gt[big], ot[big], 1e-4, "params")
+    s = an.stats()
+    assert s.frames == w.B * w.T * w.iters and abs(s.loss_total - ag.loss[0]) < 1e-4 * (abs(ag.loss[0]) + 1e-2)
+
+
+def test_throughput_workload_full_size(bnd):
+    """The benchmarked configuration at full size (B=4096, 10x10, 300-256-256, T=32), two iterations."""
+    w = WORKLOADS["throughput"]
+    an = make(bnd, w)
+    an.reset(1)
+    for _ in range(2):
+        print("throughput near-boundary:", par.check_iteration(an, bnd, w, 1))
+
+
+@pytest.mark.parametrize("name", ["memory_bound", "large_batch", "tensor_core"])
+def test_full_size_workloads_on_sampled_envs(bnd, name):
+    """Full-size launches of the three large workloads.  The oracle replays a sample of envs for the acting
+    stage and for GAE; the learner's full-batch gradient is checked through properties that hold at any size
+    (it is compared element by element on the reduced-batch versions above)."""
+    w = WORKLOADS[name]
+    an = make(bnd, w)
+    an.reset(2)
+    rng = np.random.default_rng(0)
+    sel = np.unique(np.concatenate([[0, 1, 31, 32, w.B - 1], rng.integers(0, w.B, 59)]))
+    st = par.gpu_state(an, bnd)
+    g, counts = par.check_rollout(an, bnd, w, 2, st, w.T, envs=sel)
+    an.gae()
+    adv, ret = orc.gae(np.float32(w.gamma), np.float32(w.gae_lambda), np.ascontiguousarray(g["reward"][:, sel]),
+                       np.ascontiguousarray(g["value"][:, sel]), np.ascontiguousarray(g["done"][:, sel]))
+    gadv = an.get(bnd.ADV).reshape(w.T, w.B)
+    par.assert_close(gadv[:, sel], adv, 1e-4, "advantages")
+    par.assert_close(an.get(bnd.RET).reshape(w.T, w.B)[:, sel], ret, 1e-4, "returns")
+    an.learn()
+    grads = an.get(bnd.GRADS)
+    assert np.isfinite(grads).all() and np.abs(grads).max() > 0
+    sl = orc.Dims(w.N, w.H).slices()
+    bh = grads[sl["bh"]]
+    assert abs(bh[:4].sum()) <= 1e-3 * np.abs(bh[:4]).max() + 1e-9  # softmax gradients sum to zero in every row
+    # loss terms from the recorded data alone: policy term = -mean(A * logp), entropy <= ln 4
+    s = an.stats()
+    rt = par.rtol_of(w.precision)
+    want_pg = -(gadv.astype(np.float64) * g["logp"]).mean()
+    assert abs(s.loss_pg - want_pg) <= max(rt, 1e-3) * (abs(want_pg) + np.abs(gadv).mean() * 1e-2)
+    assert 0 < s.entropy <= np.log(4) + 1e-5
+    assert abs(s.loss_total - (s.loss_pg + w.value_coef * s.loss_value - w.entropy_coef * s.entropy)) < 1e-5
+    assert s.frames == w.B * w.T
+    # first Adam step moves every parameter with a non-zero gradient by at most lr (plus rounding)
+    step = an.get(bnd.PARAMS).astype(np.float64) - st["theta"]
+    assert np.abs(step).max() <= w.lr * 1.01 and (step[grads == 0] == 0).all()
+    assert an.status() == 0
+    print(name, counts)
+
+
+def test_runs_are_bitwise_deterministic(bnd):
+    w = WORKLOADS["throughput"].scaled(B=1500, iters=3)
+    outs = []
+    for _ in range(2):
+        an = make(bnd, w, debug=0)
+        an.reset(9)
+        an.run(3)
+        outs.append((an.get(bnd.PARAMS), an.get(bnd.TRAJ_ACTION), an.get(bnd.TRAJ_VALUE), an.get(bnd.ENV_POS),
+                     an.get(bnd.GRADS)))
+    for a, b in zip(*outs):
+        assert (a.view(np.uint8) == b.view(np.uint8)).all()
+    an2 = make(bnd, w, debug=0)
+    an2.reset(10)
+    an2.run(3)
+    assert (an2.get(bnd.PARAMS) != outs[0][0]).any()
+
+
+def test_checkpoint_resume_is_bitwise(bnd):
+    w = SMALL["large_batch_s"].scaled(B=300, T=8)
+    a = make(bnd, w, debug=0)
+    a.reset(4)
+    a.run(4)
+    b = make(bnd, w, debug=0)
+    b.reset(4)
+    b.run(2)
+    # the Philox key is the seed: a resumed handle needs the same one, so resume = reset(seed) + state
+    d = make(bnd, w, debug=0)
+    d.reset(4)
+    for blob in (bnd.PARAMS, bnd.ADAM_M, bnd.ADAM_V, bnd.ENV_POS, bnd.ENV_TEP):
+        d.set(blob, b.get(blob))
+    d.set(bnd.ADAM_STEP, b.get(bnd.ADAM_STEP))
+    d.set(bnd.GLOBAL_STEP, b.get(bnd.GLOBAL_STEP))
+    d.run(2)
+    assert (d.get(bnd.PARAMS).view(np.uint32) == a.get(bnd.PARAMS).view(np.uint32)).all()
+    assert (d.get(bnd.ENV_POS) == a.get(bnd.ENV_POS)).all()
+    assert (d.get(bnd.ADAM_V).view(np.uint32) == a.get(bnd.ADAM_V).view(np.uint32)).all()
+
+
+def test_run_equals_rollout_then_learn_and_enqueues_only(bnd):
+    w = SMALL["ragged"]
+    a = make(bnd, w, debug=0)
+    b = make(bnd, w, debug=0)
+    a.reset(6)
+    b.reset(6)
+    n0 = a.launch_count()
+    a.run(3)
+    per_iter = (a.launch_count() - n0) / 3
+    assert per_iter == int(per_iter) and per_iter >= 3
+    for _ in range(3):
+        b.rollout()
+        b.learn()
+    assert (a.get(bnd.PARAMS) == b.get(bnd.PARAMS)).all() and (a.get(bnd.ENV_POS) == b.get(bnd.ENV_POS)).all()
+    s = a.stats()
+    assert s.frames == 3 * w.B * w.T and s.episodes > 0 and s.episode_steps >= s.episodes
+    assert s.goals <= s.episodes
+
+
+def test_state_errors(bnd):
+    w = SMALL["ragged"]
+    an = make(bnd, w)
+    with pytest.raises(bnd.AnakinError) as e:
+        an.rollout()
+    assert e.value.code == bnd.E_BAD_STATE
+    an.reset(1)
+    with pytest.raises(bnd.AnakinError) as e:
+        an.learn()
+    assert e.value.code == bnd.E_BAD_STATE
+    for T in (0, w.T + 1):
+        with pytest.raises(bnd.AnakinError) as e:
+            an.rollout(T)
+        assert e.value.code == bnd.E_INVALID_ARG
+    an.rollout(2)  # shorter than T_max is fine
+    assert an.blob_bytes(bnd.TRAJ_REWARD) == 2 * w.B * 4
+    an.learn()
+    with pytest.raises(bnd.AnakinError):
+        an.learn()  # the rollout was consumed
+    with pytest.raises(bnd.AnakinError):
+        an.set(bnd.GRADS, np.zeros(an.P, np.float32))  # read-only blob
+    with pytest.raises(bnd.AnakinError):
+        an.set(bnd.PARAMS, np.zeros(an.P - 1, np.float32))  # wrong size
+    # a forced action outside 0..3 sets the sticky device status instead of faulting
+    bad = torch.full((w.T, w.B), 7, dtype=torch.int8, device="cuda")
+    an.rollout_forced(bad)
+    assert an.status() == 1
+
+
+def test_on_policy_forward_reuse(bnd):
+    """The update may reuse the policy's forward pass (Section 3.1): with unchanged parameters the learner's
+    policy term -mean(A log pi) computed from ITS recomputed forward equals the one from the recorded logp."""
+    w = SMALL["large_batch_s"]
+    an = make(bnd, w)
+    an.reset(8)
+    an.rollout()
+    logp = an.get(bnd.TRAJ_LOGP).astype(np.float64)
+    an.learn()
+    adv = an.get(bnd.ADV).astype(np.float64)
+    s = an.stats()
+    assert abs(s.loss_pg + (adv * logp).mean()) <= 1e-4 * (np.abs(adv * logp).mean() + 1e-6)
