@@ -74,7 +74,8 @@ typedef struct anakin_cfg {
     int32_t precision;    /* ANAKIN_PRECISION_*: BF16 = bf16 weights/activations as GEMM inputs, fp32 accumulate,
                              fp32 master parameters in Adam */
     int32_t device;       /* CUDA device ordinal the workspace lives on */
-    int32_t debug_logits; /* non-zero: rollouts also record the 4 logits of every (t, b) */
+    int32_t debug_logits; /* non-zero: debug records -- rollouts also store the 4 logits of every (t, b), updates
+                             also store the ReLU gates of every row (DEBUG_LOGITS / DEBUG_GATES blobs) */
     int32_t reserved;     /* must be 0 */
 } anakin_cfg;
 
@@ -100,7 +101,9 @@ enum {
     ANAKIN_ADV = 17,         /* f32[T][B]                    get/set */
     ANAKIN_RET = 18,         /* f32[T][B]                    get/set */
     ANAKIN_STATS = 19,       /* anakin_stats                 get */
-    ANAKIN_DEBUG_LOGITS = 20 /* f32[T][B][4], only with cfg.debug_logits   get */
+    ANAKIN_DEBUG_LOGITS = 20, /* f32[T][B][4], only with cfg.debug_logits   get */
+    ANAKIN_DEBUG_GATES = 21   /* u32[2][T*B][H/32], only with cfg.debug_logits: bit j%32 of word [layer][row][j/32] is
+                                 set when hidden unit j of that layer was active (h > 0) in the last update   get */
 };
 
 /* Counters since reset plus the loss terms of the last update. */

@@ -222,7 +222,7 @@ std::vector<S> compute_params(const Dims& d, const S* theta, int prec) {
 // In the bf16 workload h1 and h2 are rounded to bf16 after the ReLU; out stays in S.
 template <typename S>
 void forward_row(const Dims& d, const S* cp, int prec, const S* x, S* h1, S* h2, S* out5,
-                 std::vector<double>& acc) {
+                 std::vector<double>& acc, S* z1 = nullptr, S* z2 = nullptr) {
     const int H = d.H, D = d.D;
     acc.assign((size_t)H, 0.0);
     for (int k = 0; k < D; ++k) {
@@ -232,6 +232,7 @@ void forward_row(const Dims& d, const S* cp, int prec, const S* x, S* h1, S* h2,
     }
     for (int j = 0; j < H; ++j) {
         S z = (S)(acc[j] + (double)cp[d.ob1 + j]);
+        if (z1) z1[j] = z;
         z = z > (S)0 ? z : (S)0;
         h1[j] = maybe_bf16(z, prec);
     }
@@ -243,6 +244,7 @@ void forward_row(const Dims& d, const S* cp, int prec, const S* x, S* h1, S* h2,
     }
     for (int j = 0; j < H; ++j) {
         S z = (S)(acc[j] + (double)cp[d.ob2 + j]);
+        if (z2) z2[j] = z;
         z = z > (S)0 ? z : (S)0;
         h2[j] = maybe_bf16(z, prec);
     }
@@ -298,12 +300,22 @@ double act_uniform(uint64_t seed, uint32_t b, uint32_t gstep) {
 //   L = -(1/R) sum A_i log pi(a_i|s_i) + c_v (1/R) sum (V_i - ret_i)^2 - c_e (1/R) sum H_i
 // Advantages and returns are constants.  Gradients are the mean over all rows: this batch mean is the
 // single-device form of the paper's cross-core average of updates (Section 3.1).
+//
+// ReLU gates.  The derivative of ReLU is a floating-point comparison that decides a bit.  When the
+// caller passes gate bitmaps (bit j%32 of word [row][j/32]; recorded by the implementation under test),
+// the BACKWARD pass uses those gates instead of the oracle's own h > 0, so that both sides take the
+// decision in the same (the kernel's) precision; the forward pass is unchanged.  gate_info reports, per
+// layer, how many given gates differ from the oracle's own, the largest |pre-activation| among those,
+// and the rms pre-activation: a differing gate is legitimate only where the pre-activation is within
+// rounding of zero, which the caller checks.
 // ----------------------------------------------------------------------------------------------
 template <typename S>
 void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const uint32_t* walls,
                    const uint8_t* goal, const uint8_t* tpos, const int8_t* tact, const S* adv,
-                   const S* ret, double c_v, double c_e, S* grads /*nullable*/, double loss4[4]) {
+                   const S* ret, double c_v, double c_e, S* grads /*nullable*/, double loss4[4],
+                   const uint32_t* gate1 = nullptr, const uint32_t* gate2 = nullptr, double* gate_info /*[6]*/ = nullptr) {
     const size_t R = (size_t)B * T;
+    const int GW = (d.H + 31) / 32;
     const std::vector<S> cp = compute_params(d, theta, prec);
     const int H = d.H, D = d.D;
     int nthreads = 1;
@@ -312,6 +324,7 @@ void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const 
 #endif
     std::vector<std::vector<double>> gpart(nthreads);
     std::vector<double> lpart((size_t)nthreads * 3, 0.0);
+    std::vector<double> kpart((size_t)nthreads * 6, 0.0);
 #pragma omp parallel num_threads(nthreads)
     {
         int tid = 0;
@@ -320,16 +333,26 @@ void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const 
 #endif
         std::vector<double>& g = gpart[tid];
         if (grads) g.assign(d.P, 0.0);
-        std::vector<S> x(D), h1(H), h2(H), dh2(H), dh1(H);
+        std::vector<S> x(D), h1(H), h2(H), dh2(H), dh1(H), z1(H), z2(H);
         std::vector<double> acc;
         S out[5];
         double l_pg = 0.0, l_v = 0.0, l_ent = 0.0;
+        double* kp = kpart.data() + (size_t)tid * 6;  // mismatches, max|z| among them, sum z^2 (per layer)
         // static contiguous split of the rows over threads
         const size_t lo = R * (size_t)tid / nthreads, hi = R * (size_t)(tid + 1) / nthreads;
         for (size_t i = lo; i < hi; ++i) {
             const size_t b = i % (size_t)B;
             observe(d, walls + b * d.W, tpos[i], goal[b], x.data());
-            forward_row(d, cp.data(), prec, x.data(), h1.data(), h2.data(), out, acc);
+            forward_row(d, cp.data(), prec, x.data(), h1.data(), h2.data(), out, acc, z1.data(), z2.data());
+            // gate of unit j in each layer: the caller's bit if given, else the oracle's own h > 0
+            auto gate = [&](const uint32_t* g, const std::vector<S>& h, const std::vector<S>& z, int j, double* k3) -> bool {
+                const bool own = h[j] > (S)0;
+                k3[2] += (double)z[j] * (double)z[j];
+                if (!g) return own;
+                const bool given = (g[i * GW + (j >> 5)] >> (j & 31)) & 1u;
+                if (given != own) { k3[0] += 1.0; k3[1] = std::max(k3[1], std::fabs((double)z[j])); }
+                return given;
+            };
             const Soft s = softmax4(out);
             const int a = (int)tact[i];
             const double A = (double)adv[i];
@@ -354,7 +377,7 @@ void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const 
                     g[d.oWh + (size_t)j * 5 + k] += hj * (double)dOut[k];
                     back += (double)dOut[k] * (double)cp[d.oWh + (size_t)j * 5 + k];
                 }
-                S v = h2[j] > (S)0 ? (S)back : (S)0;
+                S v = gate(gate2, h2, z2, j, kp + 3) ? (S)back : (S)0;
                 dh2[j] = maybe_bf16(v, prec);
             }
             for (int k = 0; k < 5; ++k) g[d.obh + k] += (double)dOut[k];
@@ -368,7 +391,7 @@ void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const 
                     grow[j] += hi1 * (double)dh2[j];
                     back += (double)dh2[j] * (double)wrow[j];
                 }
-                S v = h1[i1] > (S)0 ? (S)back : (S)0;
+                S v = gate(gate1, h1, z1, i1, kp) ? (S)back : (S)0;
                 dh1[i1] = maybe_bf16(v, prec);
             }
             for (int j = 0; j < H; ++j) g[d.ob2 + j] += (double)dh2[j];
@@ -395,6 +418,19 @@ void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const 
     loss4[1] = l_pg;
     loss4[2] = l_v;
     loss4[3] = l_ent;
+    if (gate_info) {
+        for (int l = 0; l < 2; ++l) {
+            double n = 0.0, mx = 0.0, ss = 0.0;
+            for (int t = 0; t < nthreads; ++t) {
+                n += kpart[(size_t)t * 6 + 3 * l + 0];
+                mx = std::max(mx, kpart[(size_t)t * 6 + 3 * l + 1]);
+                ss += kpart[(size_t)t * 6 + 3 * l + 2];
+            }
+            gate_info[3 * l + 0] = n;
+            gate_info[3 * l + 1] = mx;
+            gate_info[3 * l + 2] = std::sqrt(ss / ((double)R * H));
+        }
+    }
     if (grads) {
         for (size_t i = 0; i < d.P; ++i) {
             double s = 0.0;
@@ -560,8 +596,10 @@ void orc_gae(int T, int B, double gamma, double lambda, const float* rew, const 
 
 void orc_learn_f32(int N, int H, int prec, int B, int T, const float* theta, const uint32_t* walls,
                    const uint8_t* goal, const uint8_t* tpos, const int8_t* tact, const float* adv,
-                   const float* ret, double c_v, double c_e, float* grads, double* loss4) {
-    loss_and_grad<float>(make_dims(N, H), prec, B, T, theta, walls, goal, tpos, tact, adv, ret, c_v, c_e, grads, loss4);
+                   const float* ret, double c_v, double c_e, float* grads, double* loss4,
+                   const uint32_t* gate1 /*nullable*/, const uint32_t* gate2 /*nullable*/, double* gate_info /*nullable [6]*/) {
+    loss_and_grad<float>(make_dims(N, H), prec, B, T, theta, walls, goal, tpos, tact, adv, ret, c_v, c_e, grads, loss4,
+                         gate1, gate2, gate_info);
 }
 
 // fp64 instantiation (storage in double): used only to pin the gradient against finite differences.

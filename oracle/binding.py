@@ -233,15 +233,27 @@ def gae(gamma: float, lam: float, reward: np.ndarray, value: np.ndarray, done: n
     return adv, ret
 
 
-def learn(N, H, prec, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, want_grads=True):
-    """fp32-storage loss and batch-mean gradient.  Returns (grads f32 [P] or None, loss[4] f64)."""
+def learn(N, H, prec, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, want_grads=True, gates=None):
+    """fp32-storage loss and batch-mean gradient.  Returns (grads f32 [P] or None, loss[4] f64), plus a
+    gate report when `gates` = (gate1, gate2) uint32 bitmaps [R][ceil(H/32)] recorded by the implementation
+    under test are given: the backward pass then takes the ReLU gate decisions from them."""
     T, B = tpos.shape
     grads = np.zeros(Dims(N, H).P, np.float32) if want_grads else None
     loss = np.zeros(4, np.float64)
+    g1 = g2 = info = None
+    if gates is not None:
+        g1 = np.ascontiguousarray(gates[0], np.uint32)
+        g2 = np.ascontiguousarray(gates[1], np.uint32)
+        assert g1.size == g2.size == T * B * ((H + 31) // 32)
+        info = np.zeros(6, np.float64)
     lib().orc_learn_f32(C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), _p(theta), _p(walls), _p(goal),
                         _p(np.ascontiguousarray(tpos, np.uint8)), _p(np.ascontiguousarray(tact, np.int8)),
                         _p(np.ascontiguousarray(adv, np.float32)), _p(np.ascontiguousarray(ret, np.float32)),
-                        C.c_double(c_v), C.c_double(c_e), _p(grads), _p(loss))
+                        C.c_double(c_v), C.c_double(c_e), _p(grads), _p(loss), _p(g1), _p(g2), _p(info))
+    if gates is not None:
+        report = {"layer1": dict(mismatched=int(info[0]), max_abs_z=float(info[1]), rms_z=float(info[2])),
+                  "layer2": dict(mismatched=int(info[3]), max_abs_z=float(info[4]), rms_z=float(info[5]))}
+        return grads, loss, report
     return grads, loss
 
 

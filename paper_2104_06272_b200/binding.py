@@ -41,7 +41,7 @@ class AnakinStats(C.Structure):
 # error codes / blob selectors (mirrors of the header's enums)
 OK, E_INVALID_ARG, E_BAD_STATE, E_WORKSPACE_TOO_SMALL, E_UNSUPPORTED_CFG, E_CUDA, E_DEVICE_STATUS = 0, -1, -2, -3, -4, -5, -6
 (PARAMS, GRADS, ADAM_M, ADAM_V, ADAM_STEP, ENV_WALLS, ENV_START, ENV_GOAL, ENV_POS, ENV_TEP, GLOBAL_STEP, TRAJ_POS,
- TRAJ_ACTION, TRAJ_DONE, TRAJ_REWARD, TRAJ_VALUE, TRAJ_LOGP, ADV, RET, STATS, DEBUG_LOGITS) = range(21)
+ TRAJ_ACTION, TRAJ_DONE, TRAJ_REWARD, TRAJ_VALUE, TRAJ_LOGP, ADV, RET, STATS, DEBUG_LOGITS, DEBUG_GATES) = range(22)
 
 EXPORTS = [
     "anakin_workspace_bytes", "anakin_create", "anakin_destroy", "anakin_reset", "anakin_rollout",
@@ -82,7 +82,7 @@ _BLOB_DTYPE = {
     PARAMS: np.float32, GRADS: np.float32, ADAM_M: np.float32, ADAM_V: np.float32, ENV_WALLS: np.uint32,
     ENV_START: np.uint8, ENV_GOAL: np.uint8, ENV_POS: np.uint8, ENV_TEP: np.uint8, TRAJ_POS: np.uint8,
     TRAJ_ACTION: np.int8, TRAJ_DONE: np.uint8, TRAJ_REWARD: np.float32, TRAJ_VALUE: np.float32, TRAJ_LOGP: np.float32,
-    ADV: np.float32, RET: np.float32, DEBUG_LOGITS: np.float32,
+    ADV: np.float32, RET: np.float32, DEBUG_LOGITS: np.float32, DEBUG_GATES: np.uint32,
 }
 
 

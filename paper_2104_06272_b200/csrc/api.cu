@@ -91,6 +91,7 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.adv = (float*)take(R * 4);
     b.ret = (float*)take(R * 4);
     b.dbg_logits = c.debug_logits ? (float*)take(R * 16) : nullptr;
+    b.dbg_gates = c.debug_logits ? (uint32_t*)take(2 * R * (H / 32) * 4) : nullptr;
     b.base = (float*)take(B * H * 4);
     b.h1 = (float*)take(R * H * 4);
     b.h2 = (float*)take(R * H * 4);
@@ -145,6 +146,7 @@ Blob blob_of(anakin_t* h, int which) {
         case ANAKIN_RET: return {b.ret, R * 4, true, false, true};
         case ANAKIN_STATS: return {b.stats, sizeof(anakin_stats), false, false, false};
         case ANAKIN_DEBUG_LOGITS: return {b.dbg_logits, b.dbg_logits ? R * 16 : 0, false, false, false};
+        case ANAKIN_DEBUG_GATES: return {b.dbg_gates, b.dbg_gates ? 2 * R * (size_t)(d.H / 32) * 4 : 0, false, false, false};
         default: return {nullptr, 0, false, false, false};
     }
 }
@@ -376,7 +378,7 @@ int anakin_kernel_count(void) { return K_COUNT; }
 const char* anakin_kernel_name(int id) {
     static const char* names[K_COUNT] = {"reset_env", "reset_params", "refresh_params", "env_base", "rollout", "gae", "h1",
                                          "fwd2", "heads_loss", "dh1", "dw2", "colsums", "sum_over_t", "dw1_agent",
-                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total"};
+                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "";
 }
 

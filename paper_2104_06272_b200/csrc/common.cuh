@@ -58,6 +58,7 @@ struct Buffers {
     float* adv;      // [Tmax][B]
     float* ret;      // [Tmax][B]
     float* dbg_logits;  // [Tmax][B][4] or null
+    uint32_t* dbg_gates;  // [2][R][H/32] or null: ReLU gates of the last update
     float* base;     // [B][H]  b1 + sum of W1 rows of the wall cells + W1 row of the goal cell
     float* h1;       // [R][H]
     float* h2;       // [R][H]
@@ -124,7 +125,7 @@ struct LearnArgs {
 // Kernel identifiers (anakin_kernel_name / anakin_profile_read index by these).
 enum KernelId : int {
     K_RESET_ENV = 0, K_RESET_PARAMS, K_REFRESH_PARAMS, K_ENV_BASE, K_ROLLOUT, K_GAE, K_H1, K_FWD2, K_HEADS_LOSS, K_DH1,
-    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_COUNT
+    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_COUNT
 };
 
 // Optional per-kernel timing with CUDA events on the launching stream (off by default).

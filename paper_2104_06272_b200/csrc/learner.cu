@@ -306,6 +306,18 @@ __global__ void __launch_bounds__(256) k_reduce_adam(LearnArgs a, size_t R, int 
     }
 }
 
+// Debug record: one warp packs the gates (h > 0) of 32 consecutive units of one row into a word.
+__global__ void __launch_bounds__(256) k_pack_gates(Dims d, Buffers b, size_t R) {
+    const int lane = threadIdx.x & 31;
+    const size_t words = R * (size_t)(d.H / 32);
+    for (size_t w = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5); w < 2 * words; w += (size_t)gridDim.x * 8) {
+        const float* h = w < words ? b.h1 : b.h2;
+        const size_t wi = w < words ? w : w - words;
+        const uint32_t bits = __ballot_sync(0xFFFFFFFFu, h[wi * 32 + lane] > 0.f);
+        if (lane == 0) b.dbg_gates[w] = bits;
+    }
+}
+
 __global__ void k_loss_total(Buffers b, float c_v, float c_e) {
     b.stats->loss_total = b.stats->loss_pg + c_v * b.stats->loss_value - c_e * b.stats->entropy;
 }
@@ -370,6 +382,11 @@ static cudaError_t launch_learn_p(const LearnArgs& a, const Ctx& c) {
     {
         Scope sc(c, K_REDUCE_ADAM);
         k_reduce_adam<PREC><<<(unsigned)((d.P + 255) / 256), 256, 0, s>>>(a, R, lb);
+        CK(cudaGetLastError());
+    }
+    if (b.dbg_gates) {
+        Scope sc(c, K_PACK_GATES);
+        k_pack_gates<<<148 * 8, 256, 0, s>>>(d, b, R);
         CK(cudaGetLastError());
     }
     Scope sc(c, K_LOSS_TOTAL);

@@ -113,8 +113,16 @@ def check_learn(an, bnd, w, st, g, gadv, gret):
     difference on a near-zero element into a full-size parameter difference)."""
     rtol = rtol_of(w.precision)
     an.learn()
-    ograds, oloss = orc.learn(w.N, w.H, w.precision, st["theta"], st["walls"], st["goal"], g["pos"], g["action"], gadv,
-                              gret, np.float32(w.value_coef), np.float32(w.entropy_coef))
+    # ReLU gates are floating-point decisions: the oracle's backward pass takes them as the library recorded
+    # them (the kernel's precision), and reports where they differ from its own
+    R = g["pos"].size
+    gates = an.get(bnd.DEBUG_GATES).reshape(2, R, w.H // 32)
+    ograds, oloss, rep = orc.learn(w.N, w.H, w.precision, st["theta"], st["walls"], st["goal"], g["pos"], g["action"], gadv,
+                                   gret, np.float32(w.value_coef), np.float32(w.entropy_coef), gates=(gates[0], gates[1]))
+    for layer, r in rep.items():
+        # a gate may differ only where the pre-activation is within rounding of zero, and only rarely
+        assert r["max_abs_z"] <= 10 * rtol * r["rms_z"], (layer, r)
+        assert r["mismatched"] <= 5 + 20 * rtol * R * w.H, (layer, r)
     ggrads = an.get(bnd.GRADS)
     d = orc.Dims(w.N, w.H)
     for name, sl in d.slices().items():
@@ -133,7 +141,7 @@ def check_learn(an, bnd, w, st, g, gadv, gret):
     gtheta = an.get(bnd.PARAMS)
     assert_close(gtheta, theta, RTOL_FP32, "updated params")
     assert_close(gtheta.astype(np.float64) - st["theta"], theta.astype(np.float64) - st["theta"], RTOL_FP32, "param step")
-    return ograds, oloss
+    return ograds, oloss, rep
 
 
 def check_iteration(an, bnd, w, seed, T=None):
@@ -141,5 +149,6 @@ def check_iteration(an, bnd, w, seed, T=None):
     st = gpu_state(an, bnd)
     g, counts = check_rollout(an, bnd, w, seed, st, T)
     gadv, gret = check_gae(an, bnd, w, g, T)
-    check_learn(an, bnd, w, st, g, gadv, gret)
+    rep = check_learn(an, bnd, w, st, g, gadv, gret)[2]
+    counts["gate_mismatches"] = (rep["layer1"]["mismatched"], rep["layer2"]["mismatched"])
     return counts

@@ -443,3 +443,34 @@ def test_agent_loop_is_deterministic_and_learns_from_its_own_rollout():
     c.reset(2)
     c.run(2)
     assert (a.theta != c.theta).any()
+
+
+def test_recorded_relu_gates_override_only_the_backward_decision():
+    """Passing the oracle its own gates changes nothing and reports no mismatch; flipping one gate of a unit
+    whose pre-activation is far from zero is reported and changes exactly the gradients that unit feeds."""
+    N, H = 5, 32
+    d = orc.Dims(N, H)
+    ag = orc.Agent(16, N, H, 6)
+    ag.reset(4)
+    ag.theta = random_params(3, d.P, 0.3)
+    tr = ag.rollout()
+    adv, ret = orc.gae(0.99, 0.95, tr.reward, tr.value, tr.done)
+    g0, l0 = orc.learn(N, H, 0, ag.theta, ag.walls, ag.goal, tr.pos, tr.action, adv, ret)
+    T, B = tr.pos.shape
+    x = np.stack([orc.observe(N, ag.walls[b], int(tr.pos[t, b]), int(ag.goal[b])) for t in range(T) for b in range(B)])
+    _, h1, h2 = orc.forward(N, H, 0, ag.theta, x, want_hidden=True)
+    pack = lambda h: np.packbits(h > 0, axis=1, bitorder="little").view(np.uint32)
+    g1, l1, rep = orc.learn(N, H, 0, ag.theta, ag.walls, ag.goal, tr.pos, tr.action, adv, ret, gates=(pack(h1), pack(h2)))
+    assert (g1 == g0).all() and (l1 == l0).all()
+    assert rep["layer1"]["mismatched"] == 0 and rep["layer2"]["mismatched"] == 0 and rep["layer2"]["rms_z"] > 0
+    # flip the layer-2 gate of (row 7, unit 5)
+    gates2 = pack(h2).copy()
+    gates2[7, 0] ^= np.uint32(1 << 5)
+    g2, l2, rep2 = orc.learn(N, H, 0, ag.theta, ag.walls, ag.goal, tr.pos, tr.action, adv, ret, gates=(pack(h1), gates2))
+    assert rep2["layer2"]["mismatched"] == 1 and rep2["layer1"]["mismatched"] == 0 and rep2["layer2"]["max_abs_z"] > 0
+    assert (l2 == l0).all()  # the forward pass and the loss do not depend on the gates
+    s = d.slices()
+    changed = g2 != g0
+    W2c = changed[s["W2"]].reshape(H, H)
+    assert W2c[:, 5].any() and not np.delete(W2c, 5, axis=1).any()  # only column 5 of dW2
+    assert not changed[s["Wh"]].any() and not changed[s["bh"]].any()  # heads see h2, not its gate
