@@ -196,6 +196,45 @@ int anakin_profile_read(anakin_t* h, int n_ids, double* total_ms, uint64_t* coun
 int anakin_kernel_count(void);
 const char* anakin_kernel_name(int id);
 
+/*
+ * anakin_rollout_noalloc -- a rollout for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of this library.)
+ *
+ * Some callers cannot call cudaMalloc, and so cannot size and provide the workspace the handle-based calls need:
+ * a control loop whose memory budget is fixed at start-up, a plug-in inside an application that owns the
+ * allocator, a process that must never synchronise the device (cudaMalloc and cudaFree may).  This call needs no
+ * handle and no workspace.  The caller passes the rollout's inputs and outputs as DEVICE pointers; the only
+ * scratch the rollout uses (B*H floats) is a fixed array compiled into the library, so
+ *     B * H  <=  ANAKIN_NOALLOC_MAX_BH  (1,048,576 floats = 4 MiB),
+ * which every GPU that loads the library holds until the process exits.  Larger sizes return
+ * ANAKIN_E_WORKSPACE_TOO_SMALL (with a message on stderr); precision must be ANAKIN_PRECISION_FP32
+ * (ANAKIN_E_UNSUPPORTED_CFG otherwise).  The call itself calls no cudaMalloc / cudaFree and no allocating library
+ * routine; it enqueues one small memset and two kernels on `cuda_stream` and returns without synchronising.
+ *
+ * It computes exactly what anakin_rollout(h, T) computes on a handle with the same cfg, seed, GLOBAL_STEP, PARAMS
+ * and env blobs: same kernels, same results.
+ *   in      dev_params f32[P]; dev_walls u32[B][ceil(C/32)]; dev_start, dev_goal u8[B]   (read only)
+ *   in/out  dev_pos, dev_tep u8[B]   (env dynamic state, advanced by T steps)
+ *   out     dev_traj_pos u8[T][B]; dev_traj_action i8[T][B]; dev_traj_done u8[T][B]; dev_traj_reward f32[T][B];
+ *           dev_traj_value f32[T+1][B]; dev_traj_logp f32[T][B]
+ *   global_step   env steps taken since the seed's reset (the caller adds T after each call); 1 <= T <= cfg->T_max
+ * All buffers are the caller's and must stay alive until the stream has run the call.
+ *
+ * Set-up: the FIRST call on each device looks up the array's device address (cudaGetSymbolAddress) with that
+ * device current; make that first call outside any stream capture.  The device that is current at the call must be
+ * the one the pointers and the stream belong to.
+ * Sharing: every call on a device uses the same array, which keeps the previous call's contents; the call
+ * overwrites or clears all of it that it reads, so sequential calls are independent, but two calls that overlap
+ * on the GPU (different streams, or different threads) race on it.  Not thread-safe.
+ */
+#define ANAKIN_NOALLOC_MAX_BH 1048576
+int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int64_t global_step, int T,
+                           const float* dev_params, const uint32_t* dev_walls, const uint8_t* dev_start,
+                           const uint8_t* dev_goal, uint8_t* dev_pos, uint8_t* dev_tep,
+                           uint8_t* dev_traj_pos, int8_t* dev_traj_action, uint8_t* dev_traj_done,
+                           float* dev_traj_reward, float* dev_traj_value, float* dev_traj_logp,
+                           void* cuda_stream);
+
 /* Static description of an error code. */
 const char* anakin_strerror(int code);
 

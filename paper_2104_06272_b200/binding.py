@@ -48,6 +48,7 @@ EXPORTS = [
     "anakin_rollout_forced", "anakin_learn", "anakin_gae", "anakin_update", "anakin_run", "anakin_get", "anakin_set",
     "anakin_blob_bytes", "anakin_status", "anakin_launch_count", "anakin_strerror", "anakin_last_cuda_error",
     "anakin_profile_enable", "anakin_profile_read", "anakin_kernel_count", "anakin_kernel_name",
+    "anakin_rollout_noalloc",
 ]
 
 _vp = C.c_void_p
@@ -77,6 +78,8 @@ _lib.anakin_profile_read.argtypes = [_vp, C.c_int, C.POINTER(C.c_double), C.POIN
 _lib.anakin_kernel_count.argtypes = []
 _lib.anakin_kernel_name.argtypes = [C.c_int]
 _lib.anakin_kernel_name.restype = C.c_char_p
+_lib.anakin_rollout_noalloc.argtypes = [C.POINTER(AnakinCfg), C.c_uint64, C.c_int64, C.c_int] + [_vp] * 13
+NOALLOC_MAX_BH = 1048576
 
 _BLOB_DTYPE = {
     PARAMS: np.float32, GRADS: np.float32, ADAM_M: np.float32, ADAM_V: np.float32, ENV_WALLS: np.uint32,
@@ -121,6 +124,18 @@ def workspace_bytes(cfg: AnakinCfg) -> int:
     if rc != OK:
         raise AnakinError(rc)
     return int(n.value)
+
+
+def rollout_noalloc(cfg: AnakinCfg, seed: int, global_step: int, T: int, params, walls, start, goal, pos, tep,
+                    traj_pos, traj_action, traj_done, traj_reward, traj_value, traj_logp, stream=None) -> int:
+    """anakin_rollout_noalloc: a rollout without handle or workspace, for callers that cannot allocate device
+    memory.  Every array argument is a CUDA tensor the caller owns (inputs, in/out env state, outputs); the call
+    allocates nothing.  Returns the library's status code (0 = ok) instead of raising, so a caller can test limits."""
+    ts = (params, walls, start, goal, pos, tep, traj_pos, traj_action, traj_done, traj_reward, traj_value, traj_logp)
+    assert all(t.is_cuda and t.is_contiguous() for t in ts)
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(_lib.anakin_rollout_noalloc(C.byref(cfg), C.c_uint64(seed), C.c_int64(global_step), C.c_int(T),
+                                           *[_vp(t.data_ptr()) for t in ts], _vp(s.cuda_stream)))
 
 
 class Anakin:
