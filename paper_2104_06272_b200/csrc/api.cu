@@ -93,6 +93,8 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.dbg_logits = c.debug_logits ? (float*)take(R * 16) : nullptr;
     b.dbg_gates = c.debug_logits ? (uint32_t*)take(2 * R * (H / 32) * 4) : nullptr;
     b.base = (float*)take(B * H * 4);
+    b.w2f_hi = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2f_lo = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
     b.h1 = (float*)take(R * H * 4);
     b.h2 = (float*)take(R * H * 4);
     b.dh2 = (float*)take(R * H * 4);
@@ -158,6 +160,7 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
+        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->ctx());
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->base_valid = true;
     }
@@ -269,6 +272,7 @@ static int learn_after_gae(anakin_t* h) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
+        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->ctx());
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->base_valid = true;
     }
@@ -378,7 +382,7 @@ int anakin_kernel_count(void) { return K_COUNT; }
 const char* anakin_kernel_name(int id) {
     static const char* names[K_COUNT] = {"reset_env", "reset_params", "refresh_params", "env_base", "rollout", "gae", "h1",
                                          "fwd2", "heads_loss", "dh1", "dw2", "colsums", "sum_over_t", "dw1_agent",
-                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates"};
+                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates", "pack_w2"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "";
 }
 

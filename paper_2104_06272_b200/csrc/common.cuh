@@ -60,6 +60,8 @@ struct Buffers {
     float* dbg_logits;  // [Tmax][B][4] or null
     uint32_t* dbg_gates;  // [2][R][H/32] or null: ReLU gates of the last update
     float* base;     // [B][H]  b1 + sum of W1 rows of the wall cells + W1 row of the goal cell
+    uint2* w2f_hi;   // [H*H/4] W2 as mma B fragments, bf16 high parts (null: tensor-pipe rollout not used)
+    uint2* w2f_lo;   // [H*H/4] bf16 low parts
     float* h1;       // [R][H]
     float* h2;       // [R][H]
     float* dh2;      // [R][H]
@@ -125,7 +127,7 @@ struct LearnArgs {
 // Kernel identifiers (anakin_kernel_name / anakin_profile_read index by these).
 enum KernelId : int {
     K_RESET_ENV = 0, K_RESET_PARAMS, K_REFRESH_PARAMS, K_ENV_BASE, K_ROLLOUT, K_GAE, K_H1, K_FWD2, K_HEADS_LOSS, K_DH1,
-    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_COUNT
+    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_PACK_W2, K_COUNT
 };
 
 // Optional per-kernel timing with CUDA events on the launching stream (off by default).
@@ -169,6 +171,9 @@ struct Scope {
 cudaError_t launch_reset(const Dims& d, const Buffers& b, uint64_t seed, double density, int prec, const Ctx& c);
 cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c);
 cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c);
+cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s);  // cudaErrorNotSupported if not covered
+bool rollout_mma_supported(int H);
+cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, const Ctx& c);
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_refresh_compute_params(const Dims& d, const Buffers& b, int prec, const Ctx& c);

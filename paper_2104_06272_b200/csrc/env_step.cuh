@@ -1,0 +1,113 @@
+// Per-env part of one interaction (Podracer paper, Section 3.1: `step` maps a state and an action to a new state
+// and a reward): categorical sampling from the 4 logits, the integer gridworld step, and the time-major records.
+// One thread owns one env for the whole rollout; its dynamic state lives in that thread's registers.
+#pragma once
+#include "common.cuh"
+
+namespace anakin {
+
+struct EnvLane {
+    int pos, tep, start, goal;
+    unsigned long long n_episodes, n_goals, n_epsteps;
+    int bad;
+};
+
+// walls: this env's wall words (shared memory), 8 words.
+__device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
+                                             float l3, const uint32_t* walls) {
+    const Buffers& b = a.b;
+    const int N = a.d.N;
+    const size_t i = (size_t)t * a.d.B + env;
+    // softmax and inverse CDF: c0 = p0, c1 = c0 + p1, c2 = c1 + p2; a = [u>=c0] + [u>=c1] + [u>=c2]
+    const float mx = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
+    const float x0 = expf(l0 - mx), x1 = expf(l1 - mx), x2 = expf(l2 - mx), x3 = expf(l3 - mx);
+    const float Z = ((x0 + x1) + x2) + x3;
+    const float c0 = x0 / Z, c1 = c0 + x1 / Z, c2 = c1 + x2 / Z;
+    const U4 r = philox4x32_10((uint32_t)env, a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
+    const float u = uniform24(r.x);
+    int act = (u >= c0) + (u >= c1) + (u >= c2);
+    if (a.forced) {
+        act = a.forced[i];
+        if (act < 0 || act > 3) { s.bad |= DEV_E_BAD_ACTION; act &= 3; }
+    }
+    const float la = act == 0 ? l0 : act == 1 ? l1 : act == 2 ? l2 : l3;
+    b.tlogp[i] = (la - mx) - logf(Z);
+    b.tpos[i] = (uint8_t)s.pos;
+    b.tact[i] = (int8_t)act;
+    if (b.dbg_logits) reinterpret_cast<float4*>(b.dbg_logits)[i] = make_float4(l0, l1, l2, l3);
+    // gridworld: 0 up, 1 right, 2 down, 3 left; blocked moves stay in place
+    const int row = s.pos / N, col = s.pos - row * N;
+    int nr = row, nc = col;
+    if (act == 0) nr = row - 1;
+    else if (act == 1) nc = col + 1;
+    else if (act == 2) nr = row + 1;
+    else nc = col - 1;
+    int np = s.pos;
+    if (nr >= 0 && nr < N && nc >= 0 && nc < N) {
+        const int cand = nr * N + nc;
+        if (!((walls[cand >> 5] >> (cand & 31)) & 1u)) np = cand;
+    }
+    const int te = s.tep + 1;
+    float rew = 0.f;
+    int done = 0;
+    if (np == s.goal) { rew = 1.f; done = 1; }
+    else if (te >= a.cap) { done = 1; }
+    if (done) {
+        s.n_episodes += 1;
+        s.n_goals += (np == s.goal);
+        s.n_epsteps += te;
+        s.pos = s.start;
+        s.tep = 0;
+    } else {
+        s.pos = np;
+        s.tep = te;
+    }
+    b.trew[i] = rew;
+    b.tdone[i] = (uint8_t)done;
+}
+
+// Warp 0 holds every owner thread: fold the per-env counters and add them with integer atomics (order-free totals).
+__device__ __forceinline__ void flush_env_stats(EnvLane& s, const RolloutArgs& a) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        s.n_episodes += __shfl_xor_sync(0xFFFFFFFFu, s.n_episodes, off);
+        s.n_goals += __shfl_xor_sync(0xFFFFFFFFu, s.n_goals, off);
+        s.n_epsteps += __shfl_xor_sync(0xFFFFFFFFu, s.n_epsteps, off);
+        s.bad |= __shfl_xor_sync(0xFFFFFFFFu, s.bad, off);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        const Buffers& b = a.b;
+        if (s.n_episodes) atomicAdd((unsigned long long*)&b.stats->episodes, s.n_episodes);
+        if (s.n_goals) atomicAdd((unsigned long long*)&b.stats->goals, s.n_goals);
+        if (s.n_epsteps) atomicAdd((unsigned long long*)&b.stats->episode_steps, s.n_epsteps);
+        if (blockIdx.x == 0) atomicAdd((unsigned long long*)&b.stats->frames, (unsigned long long)a.d.B * a.T);
+        if (s.bad) atomicOr(b.status, s.bad);
+    }
+}
+
+// ---- warp-level tensor-core helpers (mma.sync m16n8k16, bf16 inputs, fp32 accumulate) ----
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* smem_ptr) {
+    const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* smem_ptr) {
+    const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_ptr);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+// Two-term bf16 split of an fp32 value: x ~= hi + lo with hi = bf16(x), lo = bf16(x - hi) (about 16 mantissa bits).
+// Three bf16 products hi*hi + lo*hi + hi*lo accumulated in fp32 then reproduce an fp32 product to ~1e-5 relative.
+__device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+__device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 lo_elem, __nv_bfloat16 hi_elem) {
+    return (uint32_t)__bfloat16_as_ushort(lo_elem) | ((uint32_t)__bfloat16_as_ushort(hi_elem) << 16);
+}
+
+}  // namespace anakin

@@ -4,8 +4,8 @@
 // fixed memory budget handed out at start-up, a plug-in inside a host application that owns the allocator, a
 // process that must not synchronise the device (cudaMalloc and cudaFree may) -- and that therefore cannot size
 // and provide the library's workspace either.  Such a caller passes only the rollout's inputs and outputs; the
-// one scratch buffer the rollout needs (the per-env first-layer constant `base`, B*H floats) lives in a
-// file-scope device array of fixed size inside this library.
+// scratch the rollout needs (the per-env first-layer constant `base`, B*H floats, and a repacked copy of the
+// second-layer weights) lives in a file-scope device array of fixed size inside this library.
 //
 // The array below is device memory reserved in every CUDA context that loads the library, from load to exit,
 // whether or not this entry point is ever called.  Its name is a host-side stand-in in host code: the device
@@ -20,11 +20,12 @@ using namespace anakin;
 namespace {
 
 constexpr size_t kMaxBaseFloats = ANAKIN_NOALLOC_MAX_BH;  // B*H limit (floats)
+constexpr size_t kW2FragBytes = 2 * 256 * 256 * 2;          // W2 as tensor-pipe fragments, hi and lo planes (H <= 256)
 constexpr size_t kTailBytes = 256;                          // statistics block + status word
 constexpr int kMaxDevices = 64;
 
-// [ base: kMaxBaseFloats floats | anakin_stats | status word ]
-static __device__ __align__(256) unsigned char g_noalloc_scratch[kMaxBaseFloats * sizeof(float) + kTailBytes];
+// [ base: kMaxBaseFloats floats | W2 fragments hi, lo | anakin_stats | status word ]
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kMaxBaseFloats * sizeof(float) + kW2FragBytes + kTailBytes];
 
 unsigned char* g_scratch_ptr[kMaxDevices] = {nullptr};  // device address of the array, per device ordinal
 
@@ -86,10 +87,16 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     b.tval = dev_traj_value;
     b.tlogp = dev_traj_logp;
     b.base = reinterpret_cast<float*>(scratch);
-    b.stats = reinterpret_cast<anakin_stats*>(scratch + kMaxBaseFloats * sizeof(float));
-    b.status = reinterpret_cast<int*>(scratch + kMaxBaseFloats * sizeof(float) + 128);
+    unsigned char* frag = scratch + kMaxBaseFloats * sizeof(float);
+    if (rollout_mma_supported(cfg->H)) {  // same kernel choice as the handle-based rollout
+        b.w2f_hi = reinterpret_cast<uint2*>(frag);
+        b.w2f_lo = reinterpret_cast<uint2*>(frag + kW2FragBytes / 2);
+    }
+    unsigned char* tail = frag + kW2FragBytes;
+    b.stats = reinterpret_cast<anakin_stats*>(tail);
+    b.status = reinterpret_cast<int*>(tail + 128);
     // the tail holds accumulators and a sticky status word left by the previous call: start them at zero
-    if (cudaMemsetAsync(scratch + kMaxBaseFloats * sizeof(float), 0, kTailBytes, s) != cudaSuccess) return ANAKIN_E_CUDA;
+    if (cudaMemsetAsync(tail, 0, kTailBytes, s) != cudaSuccess) return ANAKIN_E_CUDA;
     a.T = T;
     a.cap = cfg->episode_cap;
     a.gstep0 = (uint32_t)global_step;
@@ -99,6 +106,7 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     uint64_t launches = 0;
     const Ctx ctx{s, &launches, nullptr};
     if (launch_env_base(a.d, b, ctx) != cudaSuccess) return ANAKIN_E_CUDA;  // fills `base`: nothing of the last call survives
+    if (launch_pack_w2(a.d, b, ctx) != cudaSuccess) return ANAKIN_E_CUDA;   // likewise the weight fragments
     if (launch_rollout(a, cfg->precision, ctx) != cudaSuccess) return ANAKIN_E_CUDA;
     return ANAKIN_OK;
 }

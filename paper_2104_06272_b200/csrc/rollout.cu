@@ -247,6 +247,8 @@ static cudaError_t launch_rollout_p(const RolloutArgs& a, cudaStream_t s) {
 
 cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c) {
     Scope sc(c, K_ROLLOUT);
+    const cudaError_t e = launch_rollout_mma(a, prec, c.s);  // tensor-pipe kernel where the shape is covered
+    if (e != cudaErrorNotSupported) return e;
     return prec == 1 ? launch_rollout_p<1>(a, c.s) : launch_rollout_p<0>(a, c.s);
 }
 

@@ -1,0 +1,271 @@
+// Persistent rollout on the tensor pipe (warp-level mma.sync), second-layer weights resident on chip.
+//
+// Acting half of the Anakin minimal unit (Podracer paper, Section 3.1; Figure 2, top).  A CTA owns 32 envs for all
+// T+1 forward passes of a rollout; nothing is exchanged between CTAs.  Per step:
+//   layer 1   h1 = relu(base + W1[agent row])            gather-add, written to smem as bf16 (hi, lo) planes
+//   layer 2   h2 = relu(h1 W2 + b2)                      mma.sync m16n8k16; warp w owns output columns [NC*w, NC*w+NC)
+//   heads     out = h2 Wh + bh                           fp32 FMA on the accumulator fragments, fixed-order reduction
+//   env       softmax, Philox inverse-CDF sample, gridworld step, time-major records   (one thread per env)
+// fp32 workloads use a two-term bf16 split of both operands and three MMAs per product (hi*hi + lo*hi + hi*lo,
+// fp32 accumulate).  W2's "hi" B-fragments stay in shared memory and its "lo" B-fragments in registers for the
+// whole kernel (H = 256: 128 KB + 128 KB), so after the prologue the loop touches no weight bytes beyond the
+// agent's W1 row.  The bf16 workload needs one MMA per product and no lo planes.
+#include "env_step.cuh"
+
+namespace anakin {
+
+// B fragments of W2 for mma.m16n8k16 (.col B): entry [(ks*(H/8) + nt)*32 + lane] holds, for g = lane/4, t = lane%4,
+// n = 8*nt + g:  x = {W2[16ks+2t][n], W2[16ks+2t+1][n]},  y = {W2[16ks+2t+8][n], W2[16ks+2t+9][n]}  (low half first).
+__global__ void __launch_bounds__(256) k_pack_w2(Dims d, Buffers b) {
+    const int H = d.H;
+    const int total = H * H / 4;
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int lane = idx & 31, nt = (idx >> 5) % (H / 8), ks = (idx >> 5) / (H / 8);
+    const int g = lane >> 2, t = lane & 3;
+    const int n = nt * 8 + g, k0 = ks * 16 + 2 * t;
+    const float* W2 = b.theta_c + d.oW2;
+    __nv_bfloat16 hi[4], lo[4];
+    const int ks4[4] = {k0, k0 + 1, k0 + 8, k0 + 9};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) split_bf16(W2[(size_t)ks4[i] * H + n], hi[i], lo[i]);
+    b.w2f_hi[idx] = make_uint2(pack_bf16(hi[0], hi[1]), pack_bf16(hi[2], hi[3]));
+    b.w2f_lo[idx] = make_uint2(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]));
+}
+
+cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, const Ctx& c) {
+    if (!b.w2f_hi) return cudaSuccess;
+    Scope sc(c, K_PACK_W2);
+    k_pack_w2<<<(d.H * d.H / 4 + 255) / 256, 256, 0, c.s>>>(d, b);
+    return cudaGetLastError();
+}
+
+template <int H, int NW, int PREC>
+struct RolloutMmaCfg {
+    static constexpr int ME = 32;            // envs per CTA (two m16 tiles)
+    static constexpr int NC = H / NW;        // output columns per warp
+    static constexpr int NT = NC / 8;        // n8 tiles per warp
+    static constexpr int KS = H / 16;        // k16 steps
+    static constexpr int LD = H + 8;         // bf16 row pitch of the h1 planes (16-byte skew: conflict-free ldmatrix)
+    static constexpr int PLANES = PREC == 1 ? 1 : 2;
+    static constexpr size_t smem_bytes =
+        (size_t)H * H * 2                    // W2 hi fragments
+        + (size_t)ME * H * 4                 // base
+        + (size_t)PLANES * ME * LD * 2       // h1 hi (and lo)
+        + (size_t)NW * ME * 5 * 4            // per-warp head partials
+        + (size_t)(H * 5 + H + 8) * 4        // Wh, b2, bh
+        + (size_t)ME * 8 * 4 + ME * 4;       // walls, pos
+};
+
+template <int H, int NW, int PREC>
+__global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(RolloutArgs a) {
+    using Cfg = RolloutMmaCfg<H, NW, PREC>;
+    constexpr int ME = Cfg::ME, NT = Cfg::NT, KS = Cfg::KS, LD = Cfg::LD, NTHREADS = NW * 32;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint2* s_w2hi = reinterpret_cast<uint2*>(smem_raw);                        // [KS][H/8][32]
+    float* s_base = reinterpret_cast<float*>(smem_raw + (size_t)H * H * 2);    // [ME][H]
+    __nv_bfloat16* s_h1hi = reinterpret_cast<__nv_bfloat16*>(s_base + ME * H); // [ME][LD]
+    __nv_bfloat16* s_h1lo = s_h1hi + (PREC == 1 ? 0 : ME * LD);               // [ME][LD] (fp32 workloads only)
+    float* s_red = reinterpret_cast<float*>(s_h1hi + Cfg::PLANES * ME * LD);   // [NW][ME][5]
+    float* s_wh = s_red + NW * ME * 5;                                         // [H][5]
+    float* s_b2 = s_wh + H * 5;                                                // [H]
+    float* s_bh = s_b2 + H;                                                    // [8]
+    uint32_t* s_walls = reinterpret_cast<uint32_t*>(s_bh + 8);                 // [ME][8]
+    int* s_pos = reinterpret_cast<int*>(s_walls + ME * 8);                     // [ME]
+
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int g = lane >> 2, t4 = lane & 3;
+    const int e0 = blockIdx.x * ME;
+    const int B = d.B, C = d.C;
+    const float* W1 = b.theta_c + d.oW1;
+
+    // ---- prologue: weights and per-env constants on chip
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(b.w2f_hi);
+        uint4* dst = reinterpret_cast<uint4*>(s_w2hi);
+        for (int i = tid; i < H * H * 2 / 16; i += NTHREADS) dst[i] = src[i];
+    }
+    for (int i = tid; i < ME * H; i += NTHREADS) {
+        const int e = i / H, j = i - e * H;
+        s_base[i] = (e0 + e < B) ? b.base[(size_t)(e0 + e) * H + j] : 0.f;
+    }
+    for (int i = tid; i < H * 5; i += NTHREADS) s_wh[i] = b.theta_c[d.oWh + i];
+    for (int i = tid; i < H; i += NTHREADS) s_b2[i] = b.theta_c[d.ob2 + i];
+    if (tid < 5) s_bh[tid] = b.theta_c[d.obh + tid];
+    uint2 blo[PREC == 1 ? 1 : KS][NT];
+    if (PREC == 0) {
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int j = 0; j < NT; ++j) blo[ks][j] = b.w2f_lo[(ks * (H / 8) + wid * NT + j) * 32 + lane];
+    }
+    EnvLane s;
+    s.pos = s.tep = s.start = s.goal = 0;
+    s.n_episodes = s.n_goals = s.n_epsteps = 0;
+    s.bad = 0;
+    const bool owner = tid < ME && e0 + tid < B;
+    if (tid < ME) {
+        for (int wi = 0; wi < 8; ++wi) s_walls[tid * 8 + wi] = (owner && wi < d.W) ? b.walls[(size_t)(e0 + tid) * d.W + wi] : 0u;
+        if (owner) {
+            s.pos = b.pos[e0 + tid];
+            s.tep = b.tep[e0 + tid];
+            s.start = b.start[e0 + tid];
+            s.goal = b.goal[e0 + tid];
+        }
+        s_pos[tid] = s.pos;
+    }
+    __syncthreads();
+
+    for (int t = 0; t <= a.T; ++t) {
+        // ---- layer 1: pairs of consecutive hidden units per thread
+        for (int p = tid; p < ME * H / 2; p += NTHREADS) {
+            const int e = p / (H / 2), k = 2 * (p - e * (H / 2));
+            const float2 bs = *reinterpret_cast<const float2*>(s_base + e * H + k);
+            const float2 w = __ldg(reinterpret_cast<const float2*>(W1 + (size_t)(C + s_pos[e]) * H + k));
+            const float z0 = fmaxf(bs.x + w.x, 0.f), z1 = fmaxf(bs.y + w.y, 0.f);
+            __nv_bfloat16 h0, h1v, l0, l1;
+            if (PREC == 1) {
+                h0 = __float2bfloat16_rn(z0);
+                h1v = __float2bfloat16_rn(z1);
+            } else {
+                split_bf16(z0, h0, l0);
+                split_bf16(z1, h1v, l1);
+                *reinterpret_cast<uint32_t*>(s_h1lo + e * LD + k) = pack_bf16(l0, l1);
+            }
+            *reinterpret_cast<uint32_t*>(s_h1hi + e * LD + k) = pack_bf16(h0, h1v);
+        }
+        __syncthreads();
+        // ---- layer 2 on the tensor pipe: acc[mt][j] = rows 16mt.. x columns 8(wid*NT+j)..
+        float acc[2][NT][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[mt][j][q] = 0.f;
+        {
+            const int arow = (lane & 7) + ((lane >> 3) & 1) * 8, acol = (lane >> 4) * 8;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t ahi[2][4], alo[2][4];
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    ldmatrix_x4(ahi[mt], s_h1hi + (16 * mt + arow) * LD + 16 * ks + acol);
+                    if (PREC == 0) ldmatrix_x4(alo[mt], s_h1lo + (16 * mt + arow) * LD + 16 * ks + acol);
+                }
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                    const uint2 bhi = s_w2hi[(ks * (H / 8) + wid * NT + j) * 32 + lane];
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt) {
+                        if (PREC == 0) {
+                            mma_bf16(acc[mt][j], alo[mt], bhi.x, bhi.y);
+                            mma_bf16(acc[mt][j], ahi[mt], blo[ks][j].x, blo[ks][j].y);
+                        }
+                        mma_bf16(acc[mt][j], ahi[mt], bhi.x, bhi.y);
+                    }
+                }
+            }
+        }
+        // ---- epilogue: bias, ReLU, head partials over this warp's columns
+        {
+            float ps[4][5];  // rows g, g+8, 16+g, 24+g
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < 5; ++c) ps[r][c] = 0.f;
+#pragma unroll
+            for (int j = 0; j < NT; ++j) {
+#pragma unroll
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int col = (wid * NT + j) * 8 + 2 * t4 + cc;
+                    const float bias = s_b2[col];
+                    float wh[5];
+#pragma unroll
+                    for (int c = 0; c < 5; ++c) wh[c] = s_wh[col * 5 + c];
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const float h2 = rnd<PREC>(fmaxf(acc[mt][j][2 * hh + cc] + bias, 0.f));
+#pragma unroll
+                            for (int c = 0; c < 5; ++c) ps[2 * mt + hh][c] = fmaf(h2, wh[c], ps[2 * mt + hh][c]);
+                        }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int c = 0; c < 5; ++c) {
+                    ps[r][c] += __shfl_xor_sync(0xFFFFFFFFu, ps[r][c], 1);
+                    ps[r][c] += __shfl_xor_sync(0xFFFFFFFFu, ps[r][c], 2);
+                }
+            if (t4 == 0) {
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int row = 16 * (r >> 1) + 8 * (r & 1) + g;
+#pragma unroll
+                    for (int c = 0; c < 5; ++c) s_red[(wid * ME + row) * 5 + c] = ps[r][c];
+                }
+            }
+        }
+        __syncthreads();
+        // ---- one thread per env: fixed-order sum of the warps' partials, then act and step
+        if (owner) {
+            float o[5];
+#pragma unroll
+            for (int c = 0; c < 5; ++c) o[c] = 0.f;
+            for (int w = 0; w < NW; ++w)
+#pragma unroll
+                for (int c = 0; c < 5; ++c) o[c] += s_red[(w * ME + tid) * 5 + c];
+#pragma unroll
+            for (int c = 0; c < 5; ++c) o[c] += s_bh[c];
+            const int env = e0 + tid;
+            b.tval[(size_t)t * B + env] = o[4];
+            if (t < a.T) {
+                act_and_step(s, a, env, t, o[0], o[1], o[2], o[3], s_walls + tid * 8);
+                s_pos[tid] = s.pos;
+            }
+        }
+        __syncthreads();
+    }
+    if (owner) {
+        b.pos[e0 + tid] = (uint8_t)s.pos;
+        b.tep[e0 + tid] = (uint8_t)s.tep;
+    }
+    if (tid < 32) flush_env_stats(s, a);
+}
+
+template <int H, int NW, int PREC>
+static cudaError_t launch_t(const RolloutArgs& a, cudaStream_t s) {
+    using Cfg = RolloutMmaCfg<H, NW, PREC>;
+    cudaError_t e = cudaFuncSetAttribute(k_rollout_mma<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
+    if (e != cudaSuccess) return e;
+    k_rollout_mma<H, NW, PREC><<<(a.d.B + Cfg::ME - 1) / Cfg::ME, NW * 32, Cfg::smem_bytes, s>>>(a);
+    return cudaGetLastError();
+}
+
+bool rollout_mma_supported(int H) { return H == 64 || H == 128 || H == 256; }
+
+// Returns cudaErrorNotSupported when the shape is not covered by the tensor-pipe kernel.
+cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
+    if (!a.b.w2f_hi || !rollout_mma_supported(a.d.H)) return cudaErrorNotSupported;
+    if (prec == 1) {
+        switch (a.d.H) {
+            case 64: return launch_t<64, 4, 1>(a, s);
+            case 128: return launch_t<128, 8, 1>(a, s);
+            case 256: return launch_t<256, 16, 1>(a, s);
+        }
+    } else {
+        switch (a.d.H) {
+            case 64: return launch_t<64, 4, 0>(a, s);
+            case 128: return launch_t<128, 8, 0>(a, s);
+            case 256: return launch_t<256, 16, 0>(a, s);
+        }
+    }
+    return cudaErrorNotSupported;
+}
+
+}  // namespace anakin
