@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/anakin.h: configuration checks, workspace carving, state
 // tracking and kernel enqueueing.  The host only schedules (Podracer paper, Section 3.1): no call in the
 // rollout/learn/run path copies data or synchronises.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -19,6 +20,7 @@ struct anakin_handle {
     bool is_reset;
     bool rollout_pending;
     bool base_valid;  // `base` matches the current parameters
+    bool acts_valid;  // the saved h1/h2 belong to the pending trajectory and the current parameters
     int last_T;
     int NS;
     uint64_t seed;
@@ -95,14 +97,23 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.base = (float*)take(B * H * 4);
     b.w2f_hi = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
     b.w2f_lo = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2tf_hi = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2tf_lo = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
     b.h1 = (float*)take(R * H * 4);
     b.h2 = (float*)take(R * H * 4);
     b.dh2 = (float*)take(R * H * 4);
     b.dh1 = (float*)take(R * H * 4);
     b.dout = (float*)take(R * 8 * 4);
     b.S = (float*)take(B * H * 4);
-    b.part = (float*)take((size_t)NS * P * 4);
-    b.loss_part = (float*)take((size_t)LOSS_BLOCKS * 4 * 4);
+    size_t part_floats = (size_t)NS * P, loss_blocks = LOSS_BLOCKS;
+    if (rollout_mma_supported(d.H)) {
+        LearnPlan pl;
+        learn_mma_plan(d, &pl);
+        if (pl.part_floats > part_floats) part_floats = pl.part_floats;
+        if ((size_t)pl.loss_blocks > loss_blocks) loss_blocks = pl.loss_blocks;
+    }
+    b.part = (float*)take(part_floats * 4);
+    b.loss_part = (float*)take(loss_blocks * 4 * 4);
     b.stats = (anakin_stats*)take(sizeof(anakin_stats));
     b.status = (int*)take(sizeof(int));
     if (out) *out = b;
@@ -160,7 +171,7 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
-        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->ctx());
+        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->base_valid = true;
     }
@@ -173,11 +184,40 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     a.key0 = (uint32_t)(h->seed & 0xFFFFFFFFu);
     a.key1 = (uint32_t)(h->seed >> 32);
     a.forced = forced;
+    a.replay = 0;
     e = launch_rollout(a, h->cfg.precision, h->ctx());
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->gstep += T;
     h->last_T = T;
     h->rollout_pending = true;
+    h->acts_valid = rollout_mma_supported(h->d.H);  // the tensor-pipe rollout saved h1 and h2 of every row
+    return ANAKIN_OK;
+}
+
+// Recomputes and saves the activations of the pending trajectory's rows (positions from TRAJ_POS).
+int replay_activations(anakin_t* h) {
+    cudaError_t e;
+    if (!h->base_valid) {
+        e = launch_env_base(h->d, h->b, h->ctx());
+        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->base_valid = true;
+    }
+    RolloutArgs a;
+    a.d = h->d;
+    a.b = h->b;
+    a.T = h->last_T;
+    a.cap = h->cfg.episode_cap;
+    a.gstep0 = 0;
+    a.key0 = a.key1 = 0;
+    a.forced = nullptr;
+    a.replay = 1;
+    {
+        Scope sc(h->ctx(), K_REPLAY);
+        e = launch_rollout_mma(a, h->cfg.precision, h->stream);
+    }
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->acts_valid = true;
     return ANAKIN_OK;
 }
 
@@ -206,7 +246,7 @@ int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void
     if (bytes < need) return ANAKIN_E_WORKSPACE_TOO_SMALL;
     anakin_t* h = new (std::nothrow) anakin_t();
     if (!h) return ANAKIN_E_INVALID_ARG;
-    h->is_reset = h->rollout_pending = h->base_valid = false;
+    h->is_reset = h->rollout_pending = h->base_valid = h->acts_valid = false;
     h->last_T = 0;
     h->seed = 0;
     h->gstep = h->adam_k = 0;
@@ -248,6 +288,7 @@ int anakin_reset(anakin_t* h, uint64_t seed) {
     h->is_reset = true;
     h->rollout_pending = false;
     h->base_valid = false;
+    h->acts_valid = false;
     h->last_T = 0;
     return ANAKIN_OK;
 }
@@ -272,7 +313,7 @@ static int learn_after_gae(anakin_t* h) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
-        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->ctx());
+        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->base_valid = true;
     }
@@ -288,10 +329,26 @@ static int learn_after_gae(anakin_t* h) {
     a.beta2 = h->cfg.adam_b2;
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
-    e = launch_learn(a, h->cfg.precision, h->ctx());
+    {   // smallest power of two >= R: keeps the scaled output gradients O(1) for the fp16 operand format
+        const double Rrows = (double)h->d.B * (double)h->last_T;
+        int ex = 0;
+        while (ldexp(1.0, ex) < Rrows) ++ex;
+        a.gscale = (float)ldexp(1.0, ex);
+        a.inv_gscale = (float)ldexp(1.0, -ex);
+    }
+    if (rollout_mma_supported(h->d.H)) {
+        if (!h->acts_valid) {
+            const int rc = replay_activations(h);
+            if (rc != ANAKIN_OK) return rc;
+        }
+        e = launch_learn_mma(a, h->cfg.precision, h->ctx());
+    } else {
+        e = launch_learn(a, h->cfg.precision, h->ctx());
+    }
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->adam_k += 1;
     h->base_valid = false;  // parameters changed
+    h->acts_valid = false;
     h->rollout_pending = false;
     return ANAKIN_OK;
 }
@@ -343,8 +400,10 @@ static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is
             e = launch_refresh_compute_params(h->d, h->b, h->cfg.precision, h->ctx());
             if (e != cudaSuccess) return fail_cuda(h, e);
             h->base_valid = false;
+            h->acts_valid = false;
         }
-        if (which == ANAKIN_ENV_WALLS || which == ANAKIN_ENV_GOAL) h->base_valid = false;
+        if (which == ANAKIN_ENV_WALLS || which == ANAKIN_ENV_GOAL) h->base_valid = h->acts_valid = false;
+        if (which == ANAKIN_TRAJ_POS) h->acts_valid = false;
         if (bl.is_traj && h->is_reset) {
             if (h->last_T == 0) h->last_T = h->cfg.T_max;
             h->rollout_pending = true;
@@ -382,7 +441,7 @@ int anakin_kernel_count(void) { return K_COUNT; }
 const char* anakin_kernel_name(int id) {
     static const char* names[K_COUNT] = {"reset_env", "reset_params", "refresh_params", "env_base", "rollout", "gae", "h1",
                                          "fwd2", "heads_loss", "dh1", "dw2", "colsums", "sum_over_t", "dw1_agent",
-                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates", "pack_w2"};
+                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates", "pack_w2", "learn_bwd", "replay"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "";
 }
 

@@ -62,6 +62,8 @@ struct Buffers {
     float* base;     // [B][H]  b1 + sum of W1 rows of the wall cells + W1 row of the goal cell
     uint2* w2f_hi;   // [H*H/4] W2 as mma B fragments, bf16 high parts (null: tensor-pipe rollout not used)
     uint2* w2f_lo;   // [H*H/4] bf16 low parts
+    uint2* w2tf_hi;  // the same for W2 transposed (backward pass)
+    uint2* w2tf_lo;
     float* h1;       // [R][H]
     float* h2;       // [R][H]
     float* dh2;      // [R][H]
@@ -112,22 +114,44 @@ struct RolloutArgs {
     uint32_t gstep0;
     uint32_t key0, key1;
     const int8_t* forced;  // nullable
+    int replay;            // 1: recompute and save the activations of the recorded rows only (no sampling, no env step)
+};
+
+// One parameter range and where its split-K partial sums live: partial s of parameter i is part[s*stride + (i - start)].
+struct PartRegion {
+    const float* part;
+    int ns;
+    size_t stride;
+    size_t start;
 };
 
 struct LearnArgs {
+    static constexpr int NREG = 8;
     Dims d;
     Buffers b;
     int T;
-    int NS;  // split-K factor of the weight-gradient GEMMs
+    int NS;  // split-K factor of the weight-gradient GEMMs (FFMA path)
     float c_v, c_e;
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
+    // tensor-pipe path
+    float gscale, inv_gscale;  // power of two carried by every gradient-side tensor, divided out in the reduction
+    float* part_small;    // per (CTA, row group) partials of dWh | db2 | dbh
+    size_t small_stride;
+    PartRegion reg[NREG];
 };
+
+// Split counts and partial-buffer layout of the tensor-pipe learner (a pure function of the sizes).
+struct LearnPlan {
+    int ns_w2, ns_agent, ns_env, ns_small, loss_blocks;
+    size_t small_stride, off_w2, off_agent, off_walls, off_goal, off_small, part_floats;
+};
+void learn_mma_plan(const Dims& d, LearnPlan* p);
 
 // Kernel identifiers (anakin_kernel_name / anakin_profile_read index by these).
 enum KernelId : int {
     K_RESET_ENV = 0, K_RESET_PARAMS, K_REFRESH_PARAMS, K_ENV_BASE, K_ROLLOUT, K_GAE, K_H1, K_FWD2, K_HEADS_LOSS, K_DH1,
-    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_PACK_W2, K_COUNT
+    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_PACK_W2, K_LEARN_BWD, K_REPLAY, K_COUNT
 };
 
 // Optional per-kernel timing with CUDA events on the launching stream (off by default).
@@ -173,9 +197,10 @@ cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c);
 cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c);
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s);  // cudaErrorNotSupported if not covered
 bool rollout_mma_supported(int H);
-cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, const Ctx& c);
+cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
+cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c);  // needs the activations the rollout saved
 cudaError_t launch_refresh_compute_params(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 
 }  // namespace anakin

@@ -2,6 +2,8 @@
 // and a reward): categorical sampling from the 4 logits, the integer gridworld step, and the time-major records.
 // One thread owns one env for the whole rollout; its dynamic state lives in that thread's registers.
 #pragma once
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace anakin {
@@ -100,8 +102,49 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
 
-// Two-term bf16 split of an fp32 value: x ~= hi + lo with hi = bf16(x), lo = bf16(x - hi) (about 16 mantissa bits).
-// Three bf16 products hi*hi + lo*hi + hi*lo accumulated in fp32 then reproduce an fp32 product to ~1e-5 relative.
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Operand formats of the tensor-pipe kernels.
+//   PREC 0 (fp32 workloads): every fp32 operand is split into two fp16 terms, x ~= hi + lo with hi = fp16(x),
+//     lo = fp16(x - hi): 22 significand bits.  Three fp16 products hi*hi + lo*hi + hi*lo accumulated in fp32 reproduce
+//     the fp32 product to about 2^-21.  (A bf16 split keeps only 16 bits, which is not enough for the 1e-4 parity
+//     bound on the weight gradients.)  fp16 has a narrow exponent range, so gradient-side tensors are carried
+//     multiplied by a power of two (LearnArgs::gscale) that is divided out exactly when the partials are reduced.
+//   PREC 1 (bf16 workload): operands are bf16 values already; one bf16 product, no lo term.
+// pack2<PREC> rounds two consecutive elements to the 16-bit format: the lower-index element goes to the low half.
+template <int PREC>
+__device__ __forceinline__ void split2(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+    if (PREC == 1) {
+        hi = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x0)) | ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x1)) << 16);
+        lo = 0u;
+    } else {
+        const __half h0 = __float2half_rn(x0), h1 = __float2half_rn(x1);
+        const __half l0 = __float2half_rn(x0 - __half2float(h0)), l1 = __float2half_rn(x1 - __half2float(h1));
+        hi = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
+        lo = (uint32_t)__half_as_ushort(l0) | ((uint32_t)__half_as_ushort(l1) << 16);
+    }
+}
+template <int PREC>
+__device__ __forceinline__ void split1(float x, uint16_t& hi, uint16_t& lo) {
+    if (PREC == 1) {
+        hi = __bfloat16_as_ushort(__float2bfloat16_rn(x));
+        lo = 0;
+    } else {
+        const __half h = __float2half_rn(x);
+        hi = __half_as_ushort(h);
+        lo = __half_as_ushort(__float2half_rn(x - __half2float(h)));
+    }
+}
+template <int PREC>
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    if (PREC == 1) mma_bf16(d, a, b0, b1);
+    else mma_f16(d, a, b0, b1);
+}
+// Two-term bf16 split (used for fp32 sums that feed a bf16 product in the bf16 workload).
 __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bfloat16& lo) {
     hi = __float2bfloat16_rn(x);
     lo = __float2bfloat16_rn(x - __bfloat162float(hi));
@@ -109,5 +152,7 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 __device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 lo_elem, __nv_bfloat16 hi_elem) {
     return (uint32_t)__bfloat16_as_ushort(lo_elem) | ((uint32_t)__bfloat16_as_ushort(hi_elem) << 16);
 }
+// 1.0 in the 16-bit operand format
+template <int PREC> __device__ __forceinline__ uint32_t one16() { return PREC == 1 ? 0x3F80u : 0x3C00u; }
 
 }  // namespace anakin

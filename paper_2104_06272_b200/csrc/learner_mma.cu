@@ -1,0 +1,705 @@
+// Learning half of the Anakin minimal unit on the tensor pipe (Podracer paper, Section 3.1; Figure 2, top), for the
+// hidden sizes the tensor-pipe rollout covers.  The update reuses the policy's forward pass (Section 3.1): the rollout
+// kernel saved h1 (as bf16 hi/lo planes) and h2 for every recorded row, so the learner starts at the heads.
+//
+//   k_learn_bwd   one CTA per 32 envs, looping over t like the rollout: heads -> softmax / loss terms -> dOut -> dh2
+//                 (fp32 FMA), then dh1 = (dh2 W2^T) gated by h1 > 0 with mma.sync (W2^T resident on chip: hi fragments
+//                 in shared memory, lo fragments in registers).  Emits dh2 and dh1 as bf16 hi/lo planes, S = sum_t dh1
+//                 per env, and per-CTA partial sums of dWh, dbh, db2 and the loss terms.
+//   k_gemm_tn     C[m][n] = sum_k A[k][m] B[k][n] with split-K partial outputs, bf16 hi/lo planes as operands and
+//                 three MMAs per product (two when A is an exact 0/1 plane, one in the bf16 workload):
+//                 dW2 = h1^T dh2 (K = B*T), dW1[agent plane] = X^T dh1 (K = B*T), dW1[wall, goal planes] = X^T S
+//                 (K = B; an extra all-ones row of A yields db1 = sum_b S[b]).
+//   k_reduce_adam2  fixed-order sum of every region's partials (= the batch-mean gradient, the single-device form of
+//                 the paper's cross-core average), Adam, loss statistics.
+// No floating-point atomics: every sum has a fixed order, so runs are bitwise reproducible.
+#include "env_step.cuh"
+
+namespace anakin {
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(gsrc), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+// ----------------------------------------------------------------------------------------------------
+// k_learn_bwd
+// ----------------------------------------------------------------------------------------------------
+template <int H, int NW, int PREC>
+struct LearnBwdCfg {
+    static constexpr int ME = 32;
+    static constexpr int NT = H / NW / 8;
+    static constexpr int KS = H / 16;
+    static constexpr int LD = H + 8;            // bf16 pitch of the dh2/dh1 planes in smem
+    static constexpr int PARTS = NW;            // threads per row in the heads phase (NW*32 / 32 rows)
+    static constexpr int HP = H + PARTS;        // fp32 pitch of the h2 tile (bank skew between rows)
+    static constexpr int PLANES = PREC == 1 ? 1 : 2;
+    static constexpr size_t smem_bytes = (size_t)H * H * 2 + (size_t)ME * HP * 4 + (size_t)PLANES * ME * LD * 2 +
+                                         (size_t)ME * 8 * 4 + (size_t)(H * 5 + 8) * 4 + (size_t)ME * 4 * 4;
+};
+
+template <int H, int NW, int PREC>
+__global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_learn_bwd(LearnArgs a) {
+    using Cfg = LearnBwdCfg<H, NW, PREC>;
+    constexpr int ME = Cfg::ME, NT = Cfg::NT, KS = Cfg::KS, LD = Cfg::LD, HP = Cfg::HP, PARTS = Cfg::PARTS;
+    constexpr int NTHREADS = NW * 32, QN = H / PARTS;  // QN = 16 hidden units per thread in the heads phase
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint2* s_wt_hi = reinterpret_cast<uint2*>(smem_raw);                          // W2^T hi fragments
+    float* s_h2 = reinterpret_cast<float*>(smem_raw + (size_t)H * H * 2);         // [ME][HP]
+    __nv_bfloat16* s_phi = reinterpret_cast<__nv_bfloat16*>(s_h2 + ME * HP);      // [ME][LD] dh2 (then dh1) hi plane
+    __nv_bfloat16* s_plo = s_phi + (PREC == 1 ? 0 : ME * LD);                    // lo plane
+    float* s_dout = reinterpret_cast<float*>(s_phi + Cfg::PLANES * ME * LD);      // [ME][8]
+    float* s_wh = s_dout + ME * 8;                                                // [H][5]
+    float* s_bh = s_wh + H * 5;                                                   // [8]
+    float* s_loss = s_bh + 8;                                                     // [ME][4]
+
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int g = lane >> 2, t4 = lane & 3;
+    const int e0 = blockIdx.x * ME;
+    const int B = d.B, T = a.T;
+    const size_t RH = (size_t)B * d.Tmax * H;
+    const __nv_bfloat16* g_h1hi = reinterpret_cast<const __nv_bfloat16*>(b.h1);
+    __nv_bfloat16* g_dh2hi = reinterpret_cast<__nv_bfloat16*>(b.dh2);
+    __nv_bfloat16* g_dh2lo = g_dh2hi + RH;
+    __nv_bfloat16* g_dh1hi = reinterpret_cast<__nv_bfloat16*>(b.dh1);
+    __nv_bfloat16* g_dh1lo = g_dh1hi + RH;
+    const float invR = a.gscale / (float)((size_t)B * T);  // output gradients are carried times gscale
+
+    // ---- prologue
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(b.w2tf_hi);
+        uint4* dst = reinterpret_cast<uint4*>(s_wt_hi);
+        for (int i = tid; i < H * H * 2 / 16; i += NTHREADS) dst[i] = src[i];
+    }
+    for (int i = tid; i < H * 5; i += NTHREADS) s_wh[i] = b.theta_c[d.oWh + i];
+    if (tid < 5) s_bh[tid] = b.theta_c[d.obh + tid];
+    uint2 blo[PREC == 1 ? 1 : KS][NT];
+    if (PREC == 0) {
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks)
+#pragma unroll
+            for (int j = 0; j < NT; ++j) blo[ks][j] = b.w2tf_lo[(ks * (H / 8) + wid * NT + j) * 32 + lane];
+    }
+    // heads phase: thread = (row hr, part hp); column phase: thread = (column cj, row group cg of 16 rows)
+    const int hr = tid / PARTS, hp = tid % PARTS;
+    const int cj = tid % H, cg = tid / H;
+    float wh_c[5];  // Wh row of this thread's column
+#pragma unroll
+    for (int c = 0; c < 5; ++c) wh_c[c] = b.theta_c[d.oWh + cj * 5 + c];
+    float a_wh[5] = {0.f, 0.f, 0.f, 0.f, 0.f}, a_b2 = 0.f, a_bh = 0.f;  // running sums over t of this thread's rows
+    float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
+    float s_acc[2][NT][4];  // S = sum over t of dh1, in accumulator-fragment layout
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) s_acc[mt][j][q] = 0.f;
+
+    auto load_h2_tile = [&](int t) {  // 16-byte chunks, zero-filled past the batch end
+        for (int c = tid; c < ME * (H / 4); c += NTHREADS) {
+            const int e = c / (H / 4), k = 4 * (c - e * (H / 4));
+            const bool ok = e0 + e < B;
+            const float* src = b.h2 + ((size_t)t * B + (ok ? e0 + e : 0)) * H + k;
+            cp_async16(s_h2 + e * HP + k, src, ok ? 16 : 0);
+        }
+        cp_async_commit();
+    };
+    load_h2_tile(0);
+
+    for (int t = 0; t < T; ++t) {
+        cp_async_wait<0>();
+        __syncthreads();
+        // ---- heads, softmax, loss terms, output gradients (PARTS threads per row, shuffle reduction)
+        {
+            float o[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int q = 0; q < QN; ++q) {
+                const int j = hp + PARTS * q;
+                const float x = s_h2[hr * HP + j];
+#pragma unroll
+                for (int c = 0; c < 5; ++c) o[c] = fmaf(x, s_wh[j * 5 + c], o[c]);
+            }
+#pragma unroll
+            for (int c = 0; c < 5; ++c) {
+#pragma unroll
+                for (int off = PARTS / 2; off > 0; off >>= 1) o[c] += __shfl_xor_sync(0xFFFFFFFFu, o[c], off);
+                o[c] += s_bh[c];
+            }
+            const int env = e0 + hr;
+            if (hp == 0) {
+                float dO[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+                if (env < B) {
+                    const size_t i = (size_t)t * B + env;
+                    const float mx = fmaxf(fmaxf(o[0], o[1]), fmaxf(o[2], o[3]));
+                    float ex[4], Z = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) { ex[c] = expf(o[c] - mx); Z += ex[c]; }
+                    const float logZ = logf(Z);
+                    float p[4], lp[4], ent = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
+                    const int act = b.tact[i];
+                    const float A = b.adv[i];
+                    const float err = o[4] - b.ret[i];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        dO[c] = rnd<PREC>((-A * ((c == act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
+                    dO[4] = rnd<PREC>(2.f * a.c_v * err * invR);
+                    l_pg += -A * (act == 0 ? lp[0] : act == 1 ? lp[1] : act == 2 ? lp[2] : lp[3]);
+                    l_v += err * err;
+                    l_ent += ent;
+                }
+                float4* o4 = reinterpret_cast<float4*>(s_dout + hr * 8);
+                o4[0] = make_float4(dO[0], dO[1], dO[2], dO[3]);
+                o4[1] = make_float4(dO[4], 0.f, 0.f, 0.f);
+            }
+        }
+        __syncthreads();
+        // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0; running sums of dWh, db2, dbh
+        {
+#pragma unroll 4
+            for (int r = 0; r < 16; ++r) {
+                const int e = cg * 16 + r;
+                const float4 d0 = *reinterpret_cast<const float4*>(s_dout + e * 8);
+                const float d4 = s_dout[e * 8 + 4];
+                const float h2 = s_h2[e * HP + cj];
+                float back = d0.x * wh_c[0];
+                back = fmaf(d0.y, wh_c[1], back);
+                back = fmaf(d0.z, wh_c[2], back);
+                back = fmaf(d0.w, wh_c[3], back);
+                back = fmaf(d4, wh_c[4], back);
+                const float dh2 = rnd<PREC>(h2 > 0.f ? back : 0.f);
+                a_wh[0] = fmaf(h2, d0.x, a_wh[0]);
+                a_wh[1] = fmaf(h2, d0.y, a_wh[1]);
+                a_wh[2] = fmaf(h2, d0.z, a_wh[2]);
+                a_wh[3] = fmaf(h2, d0.w, a_wh[3]);
+                a_wh[4] = fmaf(h2, d4, a_wh[4]);
+                a_b2 += dh2;
+                if (cj < 5) a_bh += cj == 0 ? d0.x : cj == 1 ? d0.y : cj == 2 ? d0.z : cj == 3 ? d0.w : d4;
+                uint16_t hi16, lo16;
+                split1<PREC>(dh2, hi16, lo16);
+                reinterpret_cast<uint16_t*>(s_phi)[e * LD + cj] = hi16;
+                if (PREC == 0) reinterpret_cast<uint16_t*>(s_plo)[e * LD + cj] = lo16;
+            }
+        }
+        __syncthreads();
+        // ---- h2 is dead: start fetching the next tile; fetch this tile's layer-1 gates; write dh2 planes out
+        if (t + 1 < T) load_h2_tile(t + 1);
+        uint32_t gate1[2][NT][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int row = 16 * mt + 8 * hh + g, col0 = (wid * NT + j) * 8 + 2 * t4;
+                    gate1[mt][j][hh] = (e0 + row < B)
+                                           ? __ldg(reinterpret_cast<const uint32_t*>(g_h1hi + ((size_t)t * B + e0 + row) * H + col0))
+                                           : 0u;
+                }
+        for (int c = tid; c < ME * (H / 8); c += NTHREADS) {
+            const int e = c / (H / 8), k = 8 * (c - e * (H / 8));
+            if (e0 + e < B) {
+                const size_t gi = ((size_t)t * B + e0 + e) * H + k;
+                *reinterpret_cast<uint4*>(g_dh2hi + gi) = *reinterpret_cast<const uint4*>(s_phi + e * LD + k);
+                if (PREC == 0) *reinterpret_cast<uint4*>(g_dh2lo + gi) = *reinterpret_cast<const uint4*>(s_plo + e * LD + k);
+            }
+        }
+        // ---- dh1 = dh2 W2^T on the tensor pipe
+        float acc[2][NT][4];
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[mt][j][q] = 0.f;
+        {
+            const int arow = (lane & 7) + ((lane >> 3) & 1) * 8, acol = (lane >> 4) * 8;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t ahi[2][4], alo[2][4];
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                    ldmatrix_x4(ahi[mt], s_phi + (16 * mt + arow) * LD + 16 * ks + acol);
+                    if (PREC == 0) ldmatrix_x4(alo[mt], s_plo + (16 * mt + arow) * LD + 16 * ks + acol);
+                }
+#pragma unroll
+                for (int j = 0; j < NT; ++j) {
+                    const uint2 bhi = s_wt_hi[(ks * (H / 8) + wid * NT + j) * 32 + lane];
+#pragma unroll
+                    for (int mt = 0; mt < 2; ++mt) {
+                        if (PREC == 0) {
+                            mma16816<PREC>(acc[mt][j], alo[mt], bhi.x, bhi.y);
+                            mma16816<PREC>(acc[mt][j], ahi[mt], blo[ks][j].x, blo[ks][j].y);
+                        }
+                        mma16816<PREC>(acc[mt][j], ahi[mt], bhi.x, bhi.y);
+                    }
+                }
+            }
+        }
+        __syncthreads();  // every warp is done reading the dh2 planes
+        // ---- gate by h1 > 0, accumulate S, stage dh1 planes
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int row = 16 * mt + 8 * hh + g, col0 = (wid * NT + j) * 8 + 2 * t4;
+                    const uint32_t gt = gate1[mt][j][hh];
+                    // h1 >= 0 always, so "h1 > 0" is "any bit of the 16-bit high part set"
+                    const float v0 = rnd<PREC>((gt & 0x0000FFFFu) ? acc[mt][j][2 * hh] : 0.f);
+                    const float v1 = rnd<PREC>((gt & 0xFFFF0000u) ? acc[mt][j][2 * hh + 1] : 0.f);
+                    s_acc[mt][j][2 * hh] += v0;
+                    s_acc[mt][j][2 * hh + 1] += v1;
+                    uint32_t phi, plo;
+                    split2<PREC>(v0, v1, phi, plo);
+                    *reinterpret_cast<uint32_t*>(s_phi + row * LD + col0) = phi;
+                    if (PREC == 0) *reinterpret_cast<uint32_t*>(s_plo + row * LD + col0) = plo;
+                }
+        __syncthreads();
+        for (int c = tid; c < ME * (H / 8); c += NTHREADS) {
+            const int e = c / (H / 8), k = 8 * (c - e * (H / 8));
+            if (e0 + e < B) {
+                const size_t gi = ((size_t)t * B + e0 + e) * H + k;
+                *reinterpret_cast<uint4*>(g_dh1hi + gi) = *reinterpret_cast<const uint4*>(s_phi + e * LD + k);
+                if (PREC == 0) *reinterpret_cast<uint4*>(g_dh1lo + gi) = *reinterpret_cast<const uint4*>(s_plo + e * LD + k);
+            }
+        }
+        // the loop-top barrier orders these plane reads before the next column phase overwrites them
+    }
+
+    // ---- per-CTA results
+    // S (sum over t of dh1) as hi/lo planes [B][H]: always two planes, S is an fp32 sum even in the bf16 workload
+    {
+        __nv_bfloat16* S_hi = reinterpret_cast<__nv_bfloat16*>(b.S);
+        __nv_bfloat16* S_lo = S_hi + (size_t)B * H;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int row = 16 * mt + 8 * hh + g, col0 = (wid * NT + j) * 8 + 2 * t4;
+                    if (e0 + row < B) {
+                        // two terms in either workload: PREC 1 keeps bf16 hi + bf16 lo of the fp32 sum
+                        uint32_t phi, plo;
+                        if (PREC == 1) {
+                            __nv_bfloat16 h0, l0, h1v, l1;
+                            split_bf16(s_acc[mt][j][2 * hh], h0, l0);
+                            split_bf16(s_acc[mt][j][2 * hh + 1], h1v, l1);
+                            phi = pack_bf16(h0, h1v);
+                            plo = pack_bf16(l0, l1);
+                        } else {
+                            split2<0>(s_acc[mt][j][2 * hh], s_acc[mt][j][2 * hh + 1], phi, plo);
+                        }
+                        const size_t gi = (size_t)(e0 + row) * H + col0;
+                        *reinterpret_cast<uint32_t*>(S_hi + gi) = phi;
+                        *reinterpret_cast<uint32_t*>(S_lo + gi) = plo;
+                    }
+                }
+    }
+    // dWh, db2, dbh partials: split index = 2*CTA + row group
+    {
+        float* part = a.part_small + (size_t)(2 * blockIdx.x + cg) * a.small_stride;
+#pragma unroll
+        for (int c = 0; c < 5; ++c) part[(size_t)cj * 5 + c] = a_wh[c];  // Wh region first
+        part[(size_t)H * 5 + cj] = a_b2;                                 // then b2
+        if (cj < 5) part[(size_t)H * 6 + cj] = a_bh;                     // then bh
+    }
+    // loss partials, rows in index order
+    if (hp == 0) { s_loss[hr * 4 + 0] = l_pg; s_loss[hr * 4 + 1] = l_v; s_loss[hr * 4 + 2] = l_ent; }
+    __syncthreads();
+    if (tid < 3) {
+        float s = 0.f;
+        for (int e = 0; e < ME; ++e) s += s_loss[e * 4 + tid];
+        b.loss_part[(size_t)blockIdx.x * 4 + tid] = s;
+    }
+}
+
+// ----------------------------------------------------------------------------------------------------
+// k_gemm_tn: C[m][n] = sum_k A[k][m] B[k][n], split-K partial outputs.
+// ----------------------------------------------------------------------------------------------------
+enum : int { A_PLANES = 0, A_ONEHOT = 1, A_WALLS = 2 };
+
+struct GemmTnArgs {
+    int M, N, K, klen;
+    const __nv_bfloat16 *Ahi, *Alo;  // A_PLANES: [K][lda]
+    int lda;
+    const uint8_t* idx;              // A_ONEHOT: A[k][m] = (idx[k] == m)
+    const uint32_t* walls;           // A_WALLS: A[k][m] = bit m of env k (m < ones_row), 1 for m == ones_row
+    int W, ones_row;
+    const __nv_bfloat16 *Bhi, *Blo;  // [K][ldb]
+    int ldb;
+    float* part;                     // out: part[split*stride + off + m*ldc + n]; row ones_row goes to off_ones + n
+    size_t stride, off, off_ones;
+    int ldc;
+};
+
+template <int BM, int BN, int AMODE, int APL, int BPL, int PREC>
+struct GemmTnCfg {
+    static constexpr int BK = 32, STAGES = 3, THREADS = 256;
+    static constexpr int LDA = BM + 8, LDB = BN + 8;  // bf16 pitches
+    static constexpr int A_STAGE = APL * BK * LDA, B_STAGE = BPL * BK * LDB;  // elements
+    static constexpr size_t smem_bytes = (size_t)STAGES * (A_STAGE + B_STAGE) * 2;
+    static constexpr int WM = BM / 2, WN = BN / 4;   // warp tile (2 x 4 warps)
+    static constexpr int MT = WM / 16, NT = WN / 8;
+};
+
+template <int BM, int BN, int AMODE, int APL, int BPL, int PREC>
+__global__ void __launch_bounds__(256) k_gemm_tn(GemmTnArgs g) {
+    using Cfg = GemmTnCfg<BM, BN, AMODE, APL, BPL, PREC>;
+    constexpr int BK = Cfg::BK, STAGES = Cfg::STAGES, LDA = Cfg::LDA, LDB = Cfg::LDB, MT = Cfg::MT, NT = Cfg::NT;
+    static_assert(NT % 2 == 0, "B fragments are loaded two n-tiles at a time");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __nv_bfloat16* sA = reinterpret_cast<__nv_bfloat16*>(smem_raw);
+    __nv_bfloat16* sB = sA + STAGES * Cfg::A_STAGE;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int wm = wid >> 2, wn = wid & 3;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, split = blockIdx.z;
+    const int kbeg = split * g.klen, kend = min(g.K, kbeg + g.klen);
+    const int ntiles = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
+
+    auto issue = [&](int tile, int stage) {
+        const int k0 = kbeg + tile * BK;
+        __nv_bfloat16* a_s = sA + stage * Cfg::A_STAGE;
+        __nv_bfloat16* b_s = sB + stage * Cfg::B_STAGE;
+        // B planes: BK rows of BN bf16 -> 16-byte chunks
+        for (int c = tid; c < BK * (BN / 8); c += 256) {
+            const int kk = c / (BN / 8), nn = 8 * (c - kk * (BN / 8));
+            const bool ok = k0 + kk < kend && n0 + nn < g.N;
+            const size_t gi = (size_t)(ok ? k0 + kk : 0) * g.ldb + (ok ? n0 + nn : 0);
+            cp_async16(b_s + kk * LDB + nn, g.Bhi + gi, ok ? 16 : 0);
+            if (BPL == 2) cp_async16(b_s + BK * LDB + kk * LDB + nn, g.Blo + gi, ok ? 16 : 0);
+        }
+        if (AMODE == A_PLANES) {
+            for (int c = tid; c < BK * (BM / 8); c += 256) {
+                const int kk = c / (BM / 8), mm = 8 * (c - kk * (BM / 8));
+                const bool ok = k0 + kk < kend && m0 + mm < g.M;
+                const size_t gi = (size_t)(ok ? k0 + kk : 0) * g.lda + (ok ? m0 + mm : 0);
+                cp_async16(a_s + kk * LDA + mm, g.Ahi + gi, ok ? 16 : 0);
+                if (APL == 2) cp_async16(a_s + BK * LDA + kk * LDA + mm, g.Alo + gi, ok ? 16 : 0);
+            }
+        } else if (AMODE == A_ONEHOT) {
+            // one 16-byte chunk per thread: zeros, except the chunk that holds this k's single 1.0
+            for (int c = tid; c < BK * (BM / 8); c += 256) {
+                const int kk = c / (BM / 8), mm = 8 * (c - kk * (BM / 8));
+                const int k = k0 + kk;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (k < kend) {
+                    const int rel = (int)g.idx[k] - (m0 + mm);
+                    if (rel >= 0 && rel < 8) {
+                        const uint32_t one = (rel & 1) ? (one16<PREC>() << 16) : one16<PREC>();
+                        if ((rel >> 1) == 0) v.x = one; else if ((rel >> 1) == 1) v.y = one; else if ((rel >> 1) == 2) v.z = one; else v.w = one;
+                    }
+                }
+                *reinterpret_cast<uint4*>(a_s + kk * LDA + mm) = v;
+            }
+        } else {  // A_WALLS
+            for (int c = tid; c < BK * (BM / 8); c += 256) {
+                const int kk = c / (BM / 8), mm = 8 * (c - kk * (BM / 8));
+                const int k = k0 + kk;
+                uint32_t w[4] = {0u, 0u, 0u, 0u};
+                if (k < kend) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const int m = m0 + mm + q;
+                        bool on = false;
+                        if (m < g.ones_row) on = (g.walls[(size_t)k * g.W + (m >> 5)] >> (m & 31)) & 1u;
+                        else if (m == g.ones_row) on = true;
+                        if (on) w[q >> 1] |= (q & 1) ? (one16<PREC>() << 16) : one16<PREC>();
+                    }
+                }
+                *reinterpret_cast<uint4*>(a_s + kk * LDA + mm) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+    };
+
+    float acc[MT][NT][4];
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[i][j][q] = 0.f;
+
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        if (s < ntiles) issue(s, s);
+        cp_async_commit();
+    }
+    const int jm = lane >> 3, r8 = lane & 7;
+    for (int tile = 0; tile < ntiles; ++tile) {
+        cp_async_wait<STAGES - 2>();
+        __syncthreads();
+        {   // refill the stage consumed in the previous iteration
+            const int nxt = tile + STAGES - 1;
+            if (nxt < ntiles) issue(nxt, nxt % STAGES);
+            cp_async_commit();
+        }
+        const int stage = tile % STAGES;
+        const __nv_bfloat16* a_s = sA + stage * Cfg::A_STAGE;
+        const __nv_bfloat16* b_s = sB + stage * Cfg::B_STAGE;
+#pragma unroll
+        for (int k16 = 0; k16 < BK / 16; ++k16) {
+            uint32_t ahi[MT][4], alo[MT][4];
+#pragma unroll
+            for (int i = 0; i < MT; ++i) {
+                const __nv_bfloat16* p = a_s + (16 * k16 + 8 * (jm >> 1) + r8) * LDA + wm * Cfg::WM + 16 * i + 8 * (jm & 1);
+                ldmatrix_x4_trans(ahi[i], p);
+                if (APL == 2) ldmatrix_x4_trans(alo[i], p + BK * LDA);
+            }
+#pragma unroll
+            for (int j2 = 0; j2 < NT / 2; ++j2) {
+                uint32_t bhi[4], blo[4];
+                const __nv_bfloat16* p = b_s + (16 * k16 + 8 * (jm & 1) + r8) * LDB + wn * Cfg::WN + 16 * j2 + 8 * (jm >> 1);
+                ldmatrix_x4_trans(bhi, p);
+                if (BPL == 2) ldmatrix_x4_trans(blo, p + BK * LDB);
+#pragma unroll
+                for (int i = 0; i < MT; ++i)
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        if (APL == 2) mma16816<PREC>(acc[i][2 * j2 + q], alo[i], bhi[2 * q], bhi[2 * q + 1]);
+                        if (BPL == 2) mma16816<PREC>(acc[i][2 * j2 + q], ahi[i], blo[2 * q], blo[2 * q + 1]);
+                        mma16816<PREC>(acc[i][2 * j2 + q], ahi[i], bhi[2 * q], bhi[2 * q + 1]);
+                    }
+            }
+        }
+    }
+    cp_async_wait<0>();
+    // ---- split-K partial out
+    const int gq = lane >> 2, t4 = lane & 3;
+    float* part = g.part + (size_t)split * g.stride;
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int m = m0 + wm * Cfg::WM + 16 * i + 8 * hh + gq;
+                const int n = n0 + wn * Cfg::WN + 8 * j + 2 * t4;
+                if (n < g.N) {
+                    const float2 v = make_float2(acc[i][j][2 * hh], acc[i][j][2 * hh + 1]);
+                    if (AMODE == A_WALLS && m == g.ones_row) *reinterpret_cast<float2*>(part + g.off_ones + n) = v;
+                    else if (m < g.M && !(AMODE == A_WALLS && m > g.ones_row)) *reinterpret_cast<float2*>(part + g.off + (size_t)m * g.ldc + n) = v;
+                }
+            }
+}
+
+template <int BM, int BN, int AMODE, int APL, int BPL, int PREC>
+static cudaError_t launch_gemm_tn(const GemmTnArgs& g, int rows_m, int splits, cudaStream_t s) {
+    using Cfg = GemmTnCfg<BM, BN, AMODE, APL, BPL, PREC>;
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_tn<BM, BN, AMODE, APL, BPL, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
+    if (e != cudaSuccess) return e;
+    dim3 grid((rows_m + BM - 1) / BM, (g.N + BN - 1) / BN, splits);
+    k_gemm_tn<BM, BN, AMODE, APL, BPL, PREC><<<grid, 256, Cfg::smem_bytes, s>>>(g);
+    return cudaGetLastError();
+}
+
+// ----------------------------------------------------------------------------------------------------
+// k_reduce_adam2: fixed-order sums of each parameter region's partials, then Adam (Kingma & Ba, Algorithm 1).
+// ----------------------------------------------------------------------------------------------------
+template <int PREC>
+__global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int loss_blocks) {
+    __shared__ float s_c[2];
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    if (threadIdx.x == 0) {
+        s_c[0] = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
+        s_c[1] = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
+    }
+    __syncthreads();
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < d.P) {
+        int r = 0;
+#pragma unroll
+        for (int q = 1; q < LearnArgs::NREG; ++q)
+            if (i >= a.reg[q].start) r = q;
+        const PartRegion& rg = a.reg[r];
+        const float* p = rg.part + (i - rg.start);
+        float gsum = 0.f;
+        for (int s = 0; s < rg.ns; ++s) gsum += p[(size_t)s * rg.stride];
+        gsum *= a.inv_gscale;  // exact: a power of two
+        b.grads[i] = gsum;
+        const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * gsum;
+        const float v = a.beta2 * b.adam_v[i] + (1.f - a.beta2) * gsum * gsum;
+        b.adam_m[i] = m;
+        b.adam_v[i] = v;
+        const float mhat = m / s_c[0], vhat = v / s_c[1];
+        const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
+        b.theta[i] = th;
+        if (PREC == 1) {
+            const bool is_bias = (i >= d.ob1 && i < d.oW2) || (i >= d.ob2 && i < d.oWh) || i >= d.obh;
+            b.theta_c[i] = is_bias ? th : round_bf16(th);
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 3) {
+        float s = 0.f;
+        for (int q = 0; q < loss_blocks; ++q) s += b.loss_part[(size_t)q * 4 + threadIdx.x];
+        s /= (float)R;
+        float* dst = threadIdx.x == 0 ? &b.stats->loss_pg : threadIdx.x == 1 ? &b.stats->loss_value : &b.stats->entropy;
+        *dst = s;
+    }
+}
+
+__global__ void k_loss_total2(Buffers b, float c_v, float c_e) {
+    b.stats->loss_total = b.stats->loss_pg + c_v * b.stats->loss_value - c_e * b.stats->entropy;
+}
+
+// Debug record of the ReLU gates from the saved activations (h1 hi plane, h2).
+__global__ void __launch_bounds__(256) k_pack_gates2(Dims d, Buffers b, size_t R) {
+    const int lane = threadIdx.x & 31;
+    const size_t words = R * (size_t)(d.H / 32);
+    const __nv_bfloat16* h1hi = reinterpret_cast<const __nv_bfloat16*>(b.h1);
+    for (size_t w = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5); w < 2 * words; w += (size_t)gridDim.x * 8) {
+        bool on;
+        if (w < words) on = (__bfloat16_as_ushort(h1hi[w * 32 + lane]) & 0x7FFFu) != 0;  // h1 >= 0: any magnitude bit
+        else on = b.h2[(w - words) * 32 + lane] > 0.f;
+        const uint32_t bits = __ballot_sync(0xFFFFFFFFu, on);
+        if (lane == 0) b.dbg_gates[w] = bits;
+    }
+}
+
+// ----------------------------------------------------------------------------------------------------
+// host side
+// ----------------------------------------------------------------------------------------------------
+static int splits_for(int K, int tiles, int min_k) {
+    int ns = (2 * 148 + tiles - 1) / tiles;
+    const int cap = K / min_k > 0 ? K / min_k : 1;
+    if (ns > cap) ns = cap;
+    if (ns > 128) ns = 128;
+    return ns < 1 ? 1 : ns;
+}
+
+void learn_mma_plan(const Dims& d, LearnPlan* p) {
+    const int H = d.H, C = d.C;
+    const size_t R = (size_t)d.B * d.Tmax;
+    const int bt = H >= 128 ? 128 : 64;  // gemm tile side
+    const int tiles_hh = ((H + bt - 1) / bt) * ((H + bt - 1) / bt);
+    const int tiles_ch = ((C + 1 + bt - 1) / bt) * ((H + bt - 1) / bt);
+    p->ns_w2 = splits_for((int)R, tiles_hh, 256);
+    p->ns_agent = splits_for((int)R, tiles_ch, 256);
+    p->ns_env = splits_for(d.B, tiles_ch, 128);
+    p->ns_small = 2 * ((d.B + 31) / 32);
+    p->small_stride = (size_t)6 * H + 8;
+    size_t off = 0;
+    p->off_w2 = off; off += (size_t)p->ns_w2 * H * H;
+    p->off_agent = off; off += (size_t)p->ns_agent * C * H;
+    p->off_walls = off; off += (size_t)p->ns_env * (C + 1) * H;
+    p->off_goal = off; off += (size_t)p->ns_env * C * H;
+    p->off_small = off; off += (size_t)p->ns_small * p->small_stride;
+    p->part_floats = off;
+    p->loss_blocks = (d.B + 31) / 32;
+}
+
+#define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
+
+template <int H, int NW, int PREC>
+static cudaError_t launch_bwd_t(const LearnArgs& a, cudaStream_t s) {
+    using Cfg = LearnBwdCfg<H, NW, PREC>;
+    CK(cudaFuncSetAttribute(k_learn_bwd<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
+    k_learn_bwd<H, NW, PREC><<<(a.d.B + 31) / 32, NW * 32, Cfg::smem_bytes, s>>>(a);
+    return cudaGetLastError();
+}
+
+template <int PREC>
+static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    const int H = d.H, C = d.C, B = d.B, T = a.T;
+    const size_t R = (size_t)B * T, RH = (size_t)B * d.Tmax * H;
+    cudaStream_t s = c.s;
+    LearnPlan pl;
+    learn_mma_plan(d, &pl);
+    a.part_small = b.part + pl.off_small;
+    a.small_stride = pl.small_stride;
+    // parameter regions in flat order: W1 walls | W1 agent | W1 goal | b1 | W2 | b2 | Wh | bh
+    const size_t CH = (size_t)C * H;
+    a.reg[0] = PartRegion{b.part + pl.off_walls, pl.ns_env, (size_t)(C + 1) * H, d.oW1};
+    a.reg[1] = PartRegion{b.part + pl.off_agent, pl.ns_agent, CH, d.oW1 + CH};
+    a.reg[2] = PartRegion{b.part + pl.off_goal, pl.ns_env, CH, d.oW1 + 2 * CH};
+    a.reg[3] = PartRegion{b.part + pl.off_walls + CH, pl.ns_env, (size_t)(C + 1) * H, d.ob1};  // the all-ones row
+    a.reg[4] = PartRegion{b.part + pl.off_w2, pl.ns_w2, (size_t)H * H, d.oW2};
+    a.reg[5] = PartRegion{b.part + pl.off_small + (size_t)5 * H, pl.ns_small, pl.small_stride, d.ob2};
+    a.reg[6] = PartRegion{b.part + pl.off_small, pl.ns_small, pl.small_stride, d.oWh};
+    a.reg[7] = PartRegion{b.part + pl.off_small + (size_t)6 * H, pl.ns_small, pl.small_stride, d.obh};
+
+    {
+        Scope sc(c, K_LEARN_BWD);
+        switch (H) {
+            case 64: CK((launch_bwd_t<64, 4, PREC>(a, s))); break;
+            case 128: CK((launch_bwd_t<128, 8, PREC>(a, s))); break;
+            case 256: CK((launch_bwd_t<256, 16, PREC>(a, s))); break;
+            default: return cudaErrorNotSupported;
+        }
+    }
+    const __nv_bfloat16* h1hi = reinterpret_cast<const __nv_bfloat16*>(b.h1);
+    const __nv_bfloat16* dh2hi = reinterpret_cast<const __nv_bfloat16*>(b.dh2);
+    const __nv_bfloat16* dh1hi = reinterpret_cast<const __nv_bfloat16*>(b.dh1);
+    const __nv_bfloat16* Shi = reinterpret_cast<const __nv_bfloat16*>(b.S);
+    constexpr int PL = PREC == 1 ? 1 : 2;
+    auto klen_of = [](int K, int ns) { return ((K + ns - 1) / ns + 31) / 32 * 32; };
+    GemmTnArgs g;
+    memset(&g, 0, sizeof(g));
+    // dW2 = h1^T dh2
+    g.M = H; g.N = H; g.K = (int)R; g.klen = klen_of(g.K, pl.ns_w2);
+    g.Ahi = h1hi; g.Alo = h1hi + RH; g.lda = H;
+    g.Bhi = dh2hi; g.Blo = dh2hi + RH; g.ldb = H;
+    g.part = b.part + pl.off_w2; g.stride = (size_t)H * H; g.off = 0; g.ldc = H; g.ones_row = -1;
+    {
+        Scope sc(c, K_DW2);
+        if (H >= 128) CK((launch_gemm_tn<128, 128, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s)));
+        else CK((launch_gemm_tn<64, 64, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s)));
+    }
+    // dW1, agent plane = onehot(pos)^T dh1
+    g.M = C; g.K = (int)R; g.klen = klen_of(g.K, pl.ns_agent);
+    g.idx = b.tpos;
+    g.Bhi = dh1hi; g.Blo = dh1hi + RH;
+    g.part = b.part + pl.off_agent; g.stride = CH; g.off = 0;
+    {
+        Scope sc(c, K_DW1_AGENT);
+        if (H >= 128) CK((launch_gemm_tn<128, 128, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s)));
+        else CK((launch_gemm_tn<64, 64, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s)));
+    }
+    // dW1, wall plane (+ db1 through the all-ones row) = walls^T S; goal plane = onehot(goal)^T S
+    g.K = B; g.klen = klen_of(g.K, pl.ns_env);
+    g.Bhi = Shi; g.Blo = Shi + (size_t)B * H;
+    g.walls = b.walls; g.W = d.W; g.ones_row = C; g.M = C + 1;
+    g.part = b.part + pl.off_walls; g.stride = (size_t)(C + 1) * H; g.off = 0; g.off_ones = CH;
+    {
+        Scope sc(c, K_DW1_WALLS);
+        if (H >= 128) CK((launch_gemm_tn<128, 128, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s)));
+        else CK((launch_gemm_tn<64, 64, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s)));
+    }
+    g.M = C; g.ones_row = -1; g.idx = b.goal;
+    g.part = b.part + pl.off_goal; g.stride = CH;
+    {
+        Scope sc(c, K_DW1_GOAL);
+        if (H >= 128) CK((launch_gemm_tn<128, 128, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s)));
+        else CK((launch_gemm_tn<64, 64, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s)));
+    }
+    {
+        Scope sc(c, K_REDUCE_ADAM);
+        k_reduce_adam2<PREC><<<(unsigned)((d.P + 255) / 256), 256, 0, s>>>(a, R, pl.loss_blocks);
+        CK(cudaGetLastError());
+    }
+    if (b.dbg_gates) {
+        Scope sc(c, K_PACK_GATES);
+        k_pack_gates2<<<148 * 8, 256, 0, s>>>(d, b, R);
+        CK(cudaGetLastError());
+    }
+    Scope sc(c, K_LOSS_TOTAL);
+    k_loss_total2<<<1, 1, 0, s>>>(b, a.c_v, a.c_e);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c) {
+    return prec == 1 ? launch_learn_mma_p<1>(a, c) : launch_learn_mma_p<0>(a, c);
+}
+
+}  // namespace anakin

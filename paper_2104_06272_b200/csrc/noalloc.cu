@@ -106,7 +106,7 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     uint64_t launches = 0;
     const Ctx ctx{s, &launches, nullptr};
     if (launch_env_base(a.d, b, ctx) != cudaSuccess) return ANAKIN_E_CUDA;  // fills `base`: nothing of the last call survives
-    if (launch_pack_w2(a.d, b, ctx) != cudaSuccess) return ANAKIN_E_CUDA;   // likewise the weight fragments
+    if (launch_pack_w2(a.d, b, cfg->precision, ctx) != cudaSuccess) return ANAKIN_E_CUDA;   // likewise the weight fragments
     if (launch_rollout(a, cfg->precision, ctx) != cudaSuccess) return ANAKIN_E_CUDA;
     return ANAKIN_OK;
 }

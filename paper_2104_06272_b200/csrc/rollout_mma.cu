@@ -2,11 +2,11 @@
 //
 // Acting half of the Anakin minimal unit (Podracer paper, Section 3.1; Figure 2, top).  A CTA owns 32 envs for all
 // T+1 forward passes of a rollout; nothing is exchanged between CTAs.  Per step:
-//   layer 1   h1 = relu(base + W1[agent row])            gather-add, written to smem as bf16 (hi, lo) planes
+//   layer 1   h1 = relu(base + W1[agent row])            gather-add, written to smem as 16-bit (hi, lo) planes
 //   layer 2   h2 = relu(h1 W2 + b2)                      mma.sync m16n8k16; warp w owns output columns [NC*w, NC*w+NC)
 //   heads     out = h2 Wh + bh                           fp32 FMA on the accumulator fragments, fixed-order reduction
 //   env       softmax, Philox inverse-CDF sample, gridworld step, time-major records   (one thread per env)
-// fp32 workloads use a two-term bf16 split of both operands and three MMAs per product (hi*hi + lo*hi + hi*lo,
+// fp32 workloads use a two-term fp16 split of both operands and three MMAs per product (hi*hi + lo*hi + hi*lo,
 // fp32 accumulate).  W2's "hi" B-fragments stay in shared memory and its "lo" B-fragments in registers for the
 // whole kernel (H = 256: 128 KB + 128 KB), so after the prologue the loop touches no weight bytes beyond the
 // agent's W1 row.  The bf16 workload needs one MMA per product and no lo planes.
@@ -16,6 +16,7 @@ namespace anakin {
 
 // B fragments of W2 for mma.m16n8k16 (.col B): entry [(ks*(H/8) + nt)*32 + lane] holds, for g = lane/4, t = lane%4,
 // n = 8*nt + g:  x = {W2[16ks+2t][n], W2[16ks+2t+1][n]},  y = {W2[16ks+2t+8][n], W2[16ks+2t+9][n]}  (low half first).
+template <int PREC>
 __global__ void __launch_bounds__(256) k_pack_w2(Dims d, Buffers b) {
     const int H = d.H;
     const int total = H * H / 4;
@@ -25,18 +26,25 @@ __global__ void __launch_bounds__(256) k_pack_w2(Dims d, Buffers b) {
     const int g = lane >> 2, t = lane & 3;
     const int n = nt * 8 + g, k0 = ks * 16 + 2 * t;
     const float* W2 = b.theta_c + d.oW2;
-    __nv_bfloat16 hi[4], lo[4];
     const int ks4[4] = {k0, k0 + 1, k0 + 8, k0 + 9};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) split_bf16(W2[(size_t)ks4[i] * H + n], hi[i], lo[i]);
-    b.w2f_hi[idx] = make_uint2(pack_bf16(hi[0], hi[1]), pack_bf16(hi[2], hi[3]));
-    b.w2f_lo[idx] = make_uint2(pack_bf16(lo[0], lo[1]), pack_bf16(lo[2], lo[3]));
+    uint2 hi, lo;
+    split2<PREC>(W2[(size_t)ks4[0] * H + n], W2[(size_t)ks4[1] * H + n], hi.x, lo.x);
+    split2<PREC>(W2[(size_t)ks4[2] * H + n], W2[(size_t)ks4[3] * H + n], hi.y, lo.y);
+    b.w2f_hi[idx] = hi;
+    b.w2f_lo[idx] = lo;
+    // the same for W2^T (the backward pass contracts over W2's second index): B[k][n] = W2[n][k]
+    if (!b.w2tf_hi) return;
+    split2<PREC>(W2[(size_t)n * H + ks4[0]], W2[(size_t)n * H + ks4[1]], hi.x, lo.x);
+    split2<PREC>(W2[(size_t)n * H + ks4[2]], W2[(size_t)n * H + ks4[3]], hi.y, lo.y);
+    b.w2tf_hi[idx] = hi;
+    b.w2tf_lo[idx] = lo;
 }
 
-cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, const Ctx& c) {
+cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c) {
     if (!b.w2f_hi) return cudaSuccess;
     Scope sc(c, K_PACK_W2);
-    k_pack_w2<<<(d.H * d.H / 4 + 255) / 256, 256, 0, c.s>>>(d, b);
+    if (prec == 1) k_pack_w2<1><<<(d.H * d.H / 4 + 255) / 256, 256, 0, c.s>>>(d, b);
+    else k_pack_w2<0><<<(d.H * d.H / 4 + 255) / 256, 256, 0, c.s>>>(d, b);
     return cudaGetLastError();
 }
 
@@ -118,25 +126,37 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
     }
     __syncthreads();
 
-    for (int t = 0; t <= a.T; ++t) {
+    // Saved activations (the update reuses the policy's forward pass: Section 3.1): row i = t*B + env.
+    __nv_bfloat16* g_h1hi = reinterpret_cast<__nv_bfloat16*>(b.h1);
+    __nv_bfloat16* g_h1lo = g_h1hi + (size_t)B * d.Tmax * H;
+    const int t_end = a.replay ? a.T - 1 : a.T;  // replay recomputes the T recorded rows only (no bootstrap row)
+    for (int t = 0; t <= t_end; ++t) {
+        if (a.replay) {  // positions come from the recorded trajectory
+            if (tid < ME) s_pos[tid] = owner ? b.tpos[(size_t)t * B + e0 + tid] : 0;
+            __syncthreads();
+        }
         // ---- layer 1: pairs of consecutive hidden units per thread
         for (int p = tid; p < ME * H / 2; p += NTHREADS) {
             const int e = p / (H / 2), k = 2 * (p - e * (H / 2));
             const float2 bs = *reinterpret_cast<const float2*>(s_base + e * H + k);
             const float2 w = __ldg(reinterpret_cast<const float2*>(W1 + (size_t)(C + s_pos[e]) * H + k));
             const float z0 = fmaxf(bs.x + w.x, 0.f), z1 = fmaxf(bs.y + w.y, 0.f);
-            __nv_bfloat16 h0, h1v, l0, l1;
-            if (PREC == 1) {
-                h0 = __float2bfloat16_rn(z0);
-                h1v = __float2bfloat16_rn(z1);
-            } else {
-                split_bf16(z0, h0, l0);
-                split_bf16(z1, h1v, l1);
-                *reinterpret_cast<uint32_t*>(s_h1lo + e * LD + k) = pack_bf16(l0, l1);
-            }
-            *reinterpret_cast<uint32_t*>(s_h1hi + e * LD + k) = pack_bf16(h0, h1v);
+            uint32_t phi, plo;
+            split2<PREC>(z0, z1, phi, plo);
+            if (PREC == 0) *reinterpret_cast<uint32_t*>(s_h1lo + e * LD + k) = plo;
+            *reinterpret_cast<uint32_t*>(s_h1hi + e * LD + k) = phi;
         }
         __syncthreads();
+        if (b.h1 && t < a.T) {  // save the h1 planes, 16 bytes per thread per trip, coalesced
+            for (int c = tid; c < ME * (H / 8); c += NTHREADS) {
+                const int e = c / (H / 8), k = 8 * (c - e * (H / 8));
+                if (e0 + e < B) {
+                    const size_t gi = ((size_t)t * B + e0 + e) * H + k;
+                    *reinterpret_cast<uint4*>(g_h1hi + gi) = *reinterpret_cast<const uint4*>(s_h1hi + e * LD + k);
+                    if (PREC == 0) *reinterpret_cast<uint4*>(g_h1lo + gi) = *reinterpret_cast<const uint4*>(s_h1lo + e * LD + k);
+                }
+            }
+        }
         // ---- layer 2 on the tensor pipe: acc[mt][j] = rows 16mt.. x columns 8(wid*NT+j)..
         float acc[2][NT][4];
 #pragma unroll
@@ -161,10 +181,10 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
 #pragma unroll
                     for (int mt = 0; mt < 2; ++mt) {
                         if (PREC == 0) {
-                            mma_bf16(acc[mt][j], alo[mt], bhi.x, bhi.y);
-                            mma_bf16(acc[mt][j], ahi[mt], blo[ks][j].x, blo[ks][j].y);
+                            mma16816<PREC>(acc[mt][j], alo[mt], bhi.x, bhi.y);
+                            mma16816<PREC>(acc[mt][j], ahi[mt], blo[ks][j].x, blo[ks][j].y);
                         }
-                        mma_bf16(acc[mt][j], ahi[mt], bhi.x, bhi.y);
+                        mma16816<PREC>(acc[mt][j], ahi[mt], bhi.x, bhi.y);
                     }
                 }
             }
@@ -176,23 +196,42 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
             for (int r = 0; r < 4; ++r)
 #pragma unroll
                 for (int c = 0; c < 5; ++c) ps[r][c] = 0.f;
+            const bool save_h2 = b.h2 != nullptr && t < a.T;
 #pragma unroll
             for (int j = 0; j < NT; ++j) {
+                const int col0 = (wid * NT + j) * 8 + 2 * t4;
 #pragma unroll
                 for (int cc = 0; cc < 2; ++cc) {
-                    const int col = (wid * NT + j) * 8 + 2 * t4 + cc;
-                    const float bias = s_b2[col];
-                    float wh[5];
-#pragma unroll
-                    for (int c = 0; c < 5; ++c) wh[c] = s_wh[col * 5 + c];
+                    const float bias = s_b2[col0 + cc];
 #pragma unroll
                     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-                        for (int hh = 0; hh < 2; ++hh) {
-                            const float h2 = rnd<PREC>(fmaxf(acc[mt][j][2 * hh + cc] + bias, 0.f));
+                        for (int hh = 0; hh < 2; ++hh) acc[mt][j][2 * hh + cc] = rnd<PREC>(fmaxf(acc[mt][j][2 * hh + cc] + bias, 0.f));
+                }
 #pragma unroll
-                            for (int c = 0; c < 5; ++c) ps[2 * mt + hh][c] = fmaf(h2, wh[c], ps[2 * mt + hh][c]);
-                        }
+                for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int row = 16 * mt + 8 * hh + g;
+                        if (save_h2 && e0 + row < B)
+                            *reinterpret_cast<float2*>(b.h2 + ((size_t)t * B + e0 + row) * H + col0) =
+                                make_float2(acc[mt][j][2 * hh], acc[mt][j][2 * hh + 1]);
+                    }
+                if (!a.replay) {
+#pragma unroll
+                    for (int cc = 0; cc < 2; ++cc) {
+                        float wh[5];
+#pragma unroll
+                        for (int c = 0; c < 5; ++c) wh[c] = s_wh[(col0 + cc) * 5 + c];
+#pragma unroll
+                        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh) {
+                                const float h2 = acc[mt][j][2 * hh + cc];
+#pragma unroll
+                                for (int c = 0; c < 5; ++c) ps[2 * mt + hh][c] = fmaf(h2, wh[c], ps[2 * mt + hh][c]);
+                            }
+                    }
                 }
             }
 #pragma unroll
@@ -213,7 +252,7 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
         }
         __syncthreads();
         // ---- one thread per env: fixed-order sum of the warps' partials, then act and step
-        if (owner) {
+        if (owner && !a.replay) {
             float o[5];
 #pragma unroll
             for (int c = 0; c < 5; ++c) o[c] = 0.f;
@@ -231,6 +270,7 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
         }
         __syncthreads();
     }
+    if (a.replay) return;
     if (owner) {
         b.pos[e0 + tid] = (uint8_t)s.pos;
         b.tep[e0 + tid] = (uint8_t)s.tep;

@@ -263,3 +263,38 @@ def test_on_policy_forward_reuse(bnd):
     adv = an.get(bnd.ADV).astype(np.float64)
     s = an.stats()
     assert abs(s.loss_pg + (adv * logp).mean()) <= 1e-4 * (np.abs(adv * logp).mean() + 1e-6)
+
+
+def test_update_from_set_trajectory_recomputes_the_forward_pass(bnd):
+    """The learner reuses the activations the rollout saved (Section 3.1: the update may reuse the policy's forward
+    pass).  A trajectory written with anakin_set has no saved activations: the library must recompute them, and the
+    update must come out bitwise the same."""
+    w = SMALL["large_batch_s"].scaled(B=200, T=9)
+    a = make(bnd, w, debug=0)
+    b = make(bnd, w, debug=0)
+    for an in (a, b):
+        an.reset(12)
+        an.set(bnd.PARAMS, random_params(2, w.P, 0.15))
+        an.rollout()
+    b.set(bnd.TRAJ_POS, b.get(bnd.TRAJ_POS))  # same data, but it invalidates what the rollout saved
+    n0 = b.launch_count()
+    a.learn()
+    b.learn()
+    assert b.launch_count() - n0 > 0
+    for blob in (bnd.GRADS, bnd.PARAMS, bnd.ADAM_V):
+        assert (a.get(blob).view(np.uint32) == b.get(blob).view(np.uint32)).all()
+    # and a trajectory built entirely from another handle's blobs
+    c = make(bnd, w, debug=0)
+    c.reset(12)
+    c.set(bnd.PARAMS, random_params(2, w.P, 0.15))
+    d = make(bnd, w, debug=0)
+    d.reset(12)
+    d.set(bnd.PARAMS, random_params(2, w.P, 0.15))
+    c.rollout()
+    d.rollout(1)  # fixes nothing but the blob sizes; every trajectory blob is overwritten below
+    d.rollout()
+    for blob in (bnd.TRAJ_POS, bnd.TRAJ_ACTION, bnd.TRAJ_DONE, bnd.TRAJ_REWARD, bnd.TRAJ_VALUE, bnd.TRAJ_LOGP):
+        d.set(blob, c.get(blob))
+    c.learn()
+    d.learn()
+    assert (c.get(bnd.GRADS).view(np.uint32) == d.get(bnd.GRADS).view(np.uint32)).all()
