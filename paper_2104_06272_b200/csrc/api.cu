@@ -20,6 +20,7 @@ struct anakin_handle {
     bool is_reset;
     bool rollout_pending;
     bool base_valid;  // `base` matches the current parameters
+    bool frags_valid; // the tensor-pipe fragment copies of W2 match the current parameters
     bool acts_valid;  // the saved h1/h2 belong to the pending trajectory and the current parameters
     int last_T;
     int NS;
@@ -171,9 +172,13 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
-        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->base_valid = true;
+    }
+    if (!h->frags_valid) {
+        e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->frags_valid = true;
     }
     RolloutArgs a;
     a.d = h->d;
@@ -199,9 +204,13 @@ int replay_activations(anakin_t* h) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
-        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->base_valid = true;
+    }
+    if (!h->frags_valid) {
+        e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->frags_valid = true;
     }
     RolloutArgs a;
     a.d = h->d;
@@ -246,7 +255,7 @@ int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void
     if (bytes < need) return ANAKIN_E_WORKSPACE_TOO_SMALL;
     anakin_t* h = new (std::nothrow) anakin_t();
     if (!h) return ANAKIN_E_INVALID_ARG;
-    h->is_reset = h->rollout_pending = h->base_valid = h->acts_valid = false;
+    h->is_reset = h->rollout_pending = h->base_valid = h->frags_valid = h->acts_valid = false;
     h->last_T = 0;
     h->seed = 0;
     h->gstep = h->adam_k = 0;
@@ -288,6 +297,7 @@ int anakin_reset(anakin_t* h, uint64_t seed) {
     h->is_reset = true;
     h->rollout_pending = false;
     h->base_valid = false;
+    h->frags_valid = false;
     h->acts_valid = false;
     h->last_T = 0;
     return ANAKIN_OK;
@@ -308,14 +318,19 @@ int anakin_gae(anakin_t* h) {
     return ANAKIN_OK;
 }
 
-// The update proper, given ADV/RET already in place.
-static int learn_after_gae(anakin_t* h) {
+// The update proper.  fuse_gae: the tensor-pipe backward kernel computes ADV/RET itself; otherwise they are used as
+// they stand.
+static int learn_after_gae(anakin_t* h, bool fuse_gae) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
-        if (e == cudaSuccess) e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->base_valid = true;
+    }
+    if (!h->frags_valid) {
+        e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->frags_valid = true;
     }
     LearnArgs a;
     a.d = h->d;
@@ -329,6 +344,9 @@ static int learn_after_gae(anakin_t* h) {
     a.beta2 = h->cfg.adam_b2;
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
+    a.fuse_gae = fuse_gae ? 1 : 0;
+    a.gamma = h->cfg.gamma;
+    a.lambda = h->cfg.gae_lambda;
     {   // smallest power of two >= R: keeps the scaled output gradients O(1) for the fp16 operand format
         const double Rrows = (double)h->d.B * (double)h->last_T;
         int ex = 0;
@@ -348,21 +366,25 @@ static int learn_after_gae(anakin_t* h) {
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->adam_k += 1;
     h->base_valid = false;  // parameters changed
+    h->frags_valid = rollout_mma_supported(h->d.H);  // the tensor-pipe update refreshes the fragment copies itself
     h->acts_valid = false;
     h->rollout_pending = false;
     return ANAKIN_OK;
 }
 
 int anakin_learn(anakin_t* h) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
+    if (rollout_mma_supported(h->d.H)) return learn_after_gae(h, true);
     const int rc = anakin_gae(h);
     if (rc != ANAKIN_OK) return rc;
-    return learn_after_gae(h);
+    return learn_after_gae(h, false);
 }
 
 int anakin_update(anakin_t* h) {
     if (!h) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
-    return learn_after_gae(h);
+    return learn_after_gae(h, false);
 }
 
 int anakin_run(anakin_t* h, int iters) {
@@ -400,6 +422,7 @@ static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is
             e = launch_refresh_compute_params(h->d, h->b, h->cfg.precision, h->ctx());
             if (e != cudaSuccess) return fail_cuda(h, e);
             h->base_valid = false;
+            h->frags_valid = false;
             h->acts_valid = false;
         }
         if (which == ANAKIN_ENV_WALLS || which == ANAKIN_ENV_GOAL) h->base_valid = h->acts_valid = false;

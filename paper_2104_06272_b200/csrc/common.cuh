@@ -135,6 +135,8 @@ struct LearnArgs {
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
     // tensor-pipe path
+    int fuse_gae;         // 1: the backward kernel first computes ADV/RET of its envs (anakin_learn); 0: uses them as they stand
+    float gamma, lambda;
     float gscale, inv_gscale;  // power of two carried by every gradient-side tensor, divided out in the reduction
     float* part_small;    // per (CTA, row group) partials of dWh | db2 | dbh
     size_t small_stride;

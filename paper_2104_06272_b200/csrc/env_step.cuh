@@ -87,6 +87,26 @@ __device__ __forceinline__ void flush_env_stats(EnvLane& s, const RolloutArgs& a
     }
 }
 
+// GAE reverse scan of one env (explicit rounding intrinsics: the standalone kernel and the fused learner agree bitwise):
+//   d_t = 1 - done_t; delta_t = r_t + gamma d_t V_{t+1} - V_t; A_t = delta_t + gamma lambda d_t A_{t+1}; ret_t = A_t + V_t
+__device__ __forceinline__ void gae_scan_env(const Buffers& b, int B, int T, int env, float gamma, float lambda) {
+    float A = 0.f;
+    float vnext = b.tval[(size_t)T * B + env];
+    const float gl = __fmul_rn(gamma, lambda);
+#pragma unroll 4
+    for (int t = T - 1; t >= 0; --t) {
+        const size_t i = (size_t)t * B + env;
+        const float v = b.tval[i];
+        const float r = b.trew[i];
+        const float nd = b.tdone[i] ? 0.f : 1.f;
+        const float delta = __fsub_rn(__fmaf_rn(__fmul_rn(gamma, nd), vnext, r), v);
+        A = __fmaf_rn(__fmul_rn(gl, nd), A, delta);
+        b.adv[i] = A;
+        b.ret[i] = __fadd_rn(A, v);
+        vnext = v;
+    }
+}
+
 // ---- warp-level tensor-core helpers (mma.sync m16n8k16, bf16 inputs, fp32 accumulate) ----
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"

@@ -84,6 +84,8 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_learn_bwd(LearnA
 #pragma unroll
             for (int j = 0; j < NT; ++j) blo[ks][j] = b.w2tf_lo[(ks * (H / 8) + wid * NT + j) * 32 + lane];
     }
+    // advantages and returns of this CTA's envs (one thread per env; the other warps are still loading weights)
+    if (a.fuse_gae && tid < ME && e0 + tid < B) gae_scan_env(b, B, T, e0 + tid, a.gamma, a.lambda);
     // heads phase: thread = (row hr, part hp); column phase: thread = (column cj, row group cg of 16 rows)
     const int hr = tid / PARTS, hp = tid % PARTS;
     const int cj = tid % H, cg = tid / H;
@@ -522,8 +524,17 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             if (i >= a.reg[q].start) r = q;
         const PartRegion& rg = a.reg[r];
         const float* p = rg.part + (i - rg.start);
+        // fixed order: partial s is always added after partial s-1 (eight loads in flight at a time)
         float gsum = 0.f;
-        for (int s = 0; s < rg.ns; ++s) gsum += p[(size_t)s * rg.stride];
+        int s = 0;
+        for (; s + 8 <= rg.ns; s += 8) {
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) gsum += v[q];
+        }
+        for (; s < rg.ns; ++s) gsum += p[(size_t)s * rg.stride];
         gsum *= a.inv_gscale;  // exact: a power of two
         b.grads[i] = gsum;
         const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * gsum;
@@ -533,22 +544,38 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
         const float mhat = m / s_c[0], vhat = v / s_c[1];
         const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
         b.theta[i] = th;
+        float thc = th;
         if (PREC == 1) {
             const bool is_bias = (i >= d.ob1 && i < d.oW2) || (i >= d.ob2 && i < d.oWh) || i >= d.obh;
-            b.theta_c[i] = is_bias ? th : round_bf16(th);
+            thc = is_bias ? th : round_bf16(th);
+            b.theta_c[i] = thc;
+        }
+        // refresh the tensor-pipe fragment copies of W2 and W2^T in place (same layout as k_pack_w2)
+        if (i >= d.oW2 && i < d.ob2) {
+            const int H = d.H;
+            const int k = (int)((i - d.oW2) / H), n = (int)((i - d.oW2) % H);
+            uint16_t hi, lo;
+            split1<PREC>(thc, hi, lo);
+            const size_t ef = ((size_t)((k >> 4) * (H / 8) + (n >> 3)) * 32 + (n & 7) * 4 + ((k & 7) >> 1)) * 4 + ((k & 15) >> 3) * 2 + (k & 1);
+            const size_t et = ((size_t)((n >> 4) * (H / 8) + (k >> 3)) * 32 + (k & 7) * 4 + ((n & 7) >> 1)) * 4 + ((n & 15) >> 3) * 2 + (n & 1);
+            reinterpret_cast<uint16_t*>(b.w2f_hi)[ef] = hi;
+            reinterpret_cast<uint16_t*>(b.w2f_lo)[ef] = lo;
+            reinterpret_cast<uint16_t*>(b.w2tf_hi)[et] = hi;
+            reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
         }
     }
-    if (blockIdx.x == 0 && threadIdx.x < 3) {
-        float s = 0.f;
-        for (int q = 0; q < loss_blocks; ++q) s += b.loss_part[(size_t)q * 4 + threadIdx.x];
-        s /= (float)R;
-        float* dst = threadIdx.x == 0 ? &b.stats->loss_pg : threadIdx.x == 1 ? &b.stats->loss_value : &b.stats->entropy;
-        *dst = s;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        float l[3];
+        for (int c = 0; c < 3; ++c) {
+            float s = 0.f;
+            for (int q = 0; q < loss_blocks; ++q) s += b.loss_part[(size_t)q * 4 + c];
+            l[c] = s / (float)R;
+        }
+        b.stats->loss_pg = l[0];
+        b.stats->loss_value = l[1];
+        b.stats->entropy = l[2];
+        b.stats->loss_total = l[0] + a.c_v * l[1] - a.c_e * l[2];
     }
-}
-
-__global__ void k_loss_total2(Buffers b, float c_v, float c_e) {
-    b.stats->loss_total = b.stats->loss_pg + c_v * b.stats->loss_value - c_e * b.stats->entropy;
 }
 
 // Debug record of the ReLU gates from the saved activations (h1 hi plane, h2).
@@ -693,9 +720,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         k_pack_gates2<<<148 * 8, 256, 0, s>>>(d, b, R);
         CK(cudaGetLastError());
     }
-    Scope sc(c, K_LOSS_TOTAL);
-    k_loss_total2<<<1, 1, 0, s>>>(b, a.c_v, a.c_e);
-    return cudaGetLastError();
+    return cudaSuccess;
 }
 
 cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c) {

@@ -1,7 +1,7 @@
 // Acting half of the Anakin minimal unit (Podracer paper, Section 3.1; Figure 2, top): T interactions of
 // every env with the policy, fused into one persistent kernel.  A CTA owns ME envs for the whole rollout,
 // so there is no inter-CTA dependency and no grid-wide wait anywhere.
-#include "common.cuh"
+#include "env_step.cuh"
 
 namespace anakin {
 
@@ -259,22 +259,7 @@ cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c) {
 __global__ void __launch_bounds__(128) k_gae(Dims d, Buffers b, int T, float gamma, float lambda) {
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= d.B) return;
-    const size_t B = (size_t)d.B;
-    float A = 0.f;
-    float vnext = b.tval[(size_t)T * B + e];
-    const float gl = gamma * lambda;
-#pragma unroll 4
-    for (int t = T - 1; t >= 0; --t) {
-        const size_t i = (size_t)t * B + e;
-        const float v = b.tval[i];
-        const float r = b.trew[i];
-        const float nd = b.tdone[i] ? 0.f : 1.f;
-        const float delta = r + gamma * nd * vnext - v;
-        A = delta + gl * nd * A;
-        b.adv[i] = A;
-        b.ret[i] = A + v;
-        vnext = v;
-    }
+    gae_scan_env(b, d.B, T, e, gamma, lambda);
 }
 
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c) {
