@@ -21,6 +21,7 @@ struct anakin_handle {
     bool rollout_pending;
     bool base_valid;  // `base` matches the current parameters
     bool frags_valid; // the tensor-pipe fragment copies of W2 match the current parameters
+    bool adv_valid;   // ADV/RET were computed from the pending trajectory (by the rollout's fused GAE scan)
     bool acts_valid;  // the saved h1/h2 belong to the pending trajectory and the current parameters
     int last_T;
     int NS;
@@ -100,6 +101,8 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.w2f_lo = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
     b.w2tf_hi = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
     b.w2tf_lo = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2p_hi = rollout_mma_supported(d.H) ? (uint16_t*)take(H * H * 2) : nullptr;
+    b.w2p_lo = rollout_mma_supported(d.H) ? (uint16_t*)take(H * H * 2) : nullptr;
     b.h1 = (float*)take(R * H * 4);
     b.h2 = (float*)take(R * H * 4);
     b.dh2 = (float*)take(R * H * 4);
@@ -190,12 +193,16 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     a.key1 = (uint32_t)(h->seed >> 32);
     a.forced = forced;
     a.replay = 0;
+    a.fuse_gae = rollout_mma_supported(h->d.H) ? 1 : 0;
+    a.gamma = h->cfg.gamma;
+    a.lambda = h->cfg.gae_lambda;
     e = launch_rollout(a, h->cfg.precision, h->ctx());
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->gstep += T;
     h->last_T = T;
     h->rollout_pending = true;
     h->acts_valid = rollout_mma_supported(h->d.H);  // the tensor-pipe rollout saved h1 and h2 of every row
+    h->adv_valid = a.fuse_gae != 0;
     return ANAKIN_OK;
 }
 
@@ -221,6 +228,8 @@ int replay_activations(anakin_t* h) {
     a.key0 = a.key1 = 0;
     a.forced = nullptr;
     a.replay = 1;
+    a.fuse_gae = 0;
+    a.gamma = a.lambda = 0.f;
     {
         Scope sc(h->ctx(), K_REPLAY);
         e = launch_rollout_mma(a, h->cfg.precision, h->stream);
@@ -255,7 +264,7 @@ int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void
     if (bytes < need) return ANAKIN_E_WORKSPACE_TOO_SMALL;
     anakin_t* h = new (std::nothrow) anakin_t();
     if (!h) return ANAKIN_E_INVALID_ARG;
-    h->is_reset = h->rollout_pending = h->base_valid = h->frags_valid = h->acts_valid = false;
+    h->is_reset = h->rollout_pending = h->base_valid = h->frags_valid = h->acts_valid = h->adv_valid = false;
     h->last_T = 0;
     h->seed = 0;
     h->gstep = h->adam_k = 0;
@@ -299,6 +308,7 @@ int anakin_reset(anakin_t* h, uint64_t seed) {
     h->base_valid = false;
     h->frags_valid = false;
     h->acts_valid = false;
+    h->adv_valid = false;
     h->last_T = 0;
     return ANAKIN_OK;
 }
@@ -315,12 +325,12 @@ int anakin_gae(anakin_t* h) {
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
     cudaError_t e = launch_gae(h->d, h->b, h->last_T, h->cfg.gamma, h->cfg.gae_lambda, h->ctx());
     if (e != cudaSuccess) return fail_cuda(h, e);
+    h->adv_valid = true;
     return ANAKIN_OK;
 }
 
-// The update proper.  fuse_gae: the tensor-pipe backward kernel computes ADV/RET itself; otherwise they are used as
-// they stand.
-static int learn_after_gae(anakin_t* h, bool fuse_gae) {
+// The update proper, from ADV/RET as they stand.
+static int learn_after_gae(anakin_t* h) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
@@ -344,9 +354,6 @@ static int learn_after_gae(anakin_t* h, bool fuse_gae) {
     a.beta2 = h->cfg.adam_b2;
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
-    a.fuse_gae = fuse_gae ? 1 : 0;
-    a.gamma = h->cfg.gamma;
-    a.lambda = h->cfg.gae_lambda;
     {   // smallest power of two >= R: keeps the scaled output gradients O(1) for the fp16 operand format
         const double Rrows = (double)h->d.B * (double)h->last_T;
         int ex = 0;
@@ -365,6 +372,7 @@ static int learn_after_gae(anakin_t* h, bool fuse_gae) {
     }
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->adam_k += 1;
+    h->adv_valid = false;
     h->base_valid = false;  // parameters changed
     h->frags_valid = rollout_mma_supported(h->d.H);  // the tensor-pipe update refreshes the fragment copies itself
     h->acts_valid = false;
@@ -375,16 +383,17 @@ static int learn_after_gae(anakin_t* h, bool fuse_gae) {
 int anakin_learn(anakin_t* h) {
     if (!h) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
-    if (rollout_mma_supported(h->d.H)) return learn_after_gae(h, true);
-    const int rc = anakin_gae(h);
-    if (rc != ANAKIN_OK) return rc;
-    return learn_after_gae(h, false);
+    if (!h->adv_valid) {  // the tensor-pipe rollout already ran the GAE scan of a trajectory it produced
+        const int rc = anakin_gae(h);
+        if (rc != ANAKIN_OK) return rc;
+    }
+    return learn_after_gae(h);
 }
 
 int anakin_update(anakin_t* h) {
     if (!h) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
-    return learn_after_gae(h, false);
+    return learn_after_gae(h);
 }
 
 int anakin_run(anakin_t* h, int iters) {
@@ -427,6 +436,7 @@ static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is
         }
         if (which == ANAKIN_ENV_WALLS || which == ANAKIN_ENV_GOAL) h->base_valid = h->acts_valid = false;
         if (which == ANAKIN_TRAJ_POS) h->acts_valid = false;
+        if (bl.is_traj) h->adv_valid = false;  // includes ADV and RET: anakin_learn recomputes them, anakin_update uses them
         if (bl.is_traj && h->is_reset) {
             if (h->last_T == 0) h->last_T = h->cfg.T_max;
             h->rollout_pending = true;
@@ -464,7 +474,7 @@ int anakin_kernel_count(void) { return K_COUNT; }
 const char* anakin_kernel_name(int id) {
     static const char* names[K_COUNT] = {"reset_env", "reset_params", "refresh_params", "env_base", "rollout", "gae", "h1",
                                          "fwd2", "heads_loss", "dh1", "dw2", "colsums", "sum_over_t", "dw1_agent",
-                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates", "pack_w2", "learn_bwd", "replay"};
+                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates", "pack_w2", "heads_bwd", "replay"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "";
 }
 

@@ -64,6 +64,8 @@ struct Buffers {
     uint2* w2f_lo;   // [H*H/4] bf16 low parts
     uint2* w2tf_hi;  // the same for W2 transposed (backward pass)
     uint2* w2tf_lo;
+    uint16_t* w2p_hi;  // [H][H] W2 row-major as 16-bit hi / lo planes (B operand of the dh1 kernel)
+    uint16_t* w2p_lo;
     float* h1;       // [R][H]
     float* h2;       // [R][H]
     float* dh2;      // [R][H]
@@ -115,6 +117,8 @@ struct RolloutArgs {
     uint32_t key0, key1;
     const int8_t* forced;  // nullable
     int replay;            // 1: recompute and save the activations of the recorded rows only (no sampling, no env step)
+    int fuse_gae;          // 1: after the last step each env's owner thread also runs the GAE scan (fills ADV, RET)
+    float gamma, lambda;
 };
 
 // One parameter range and where its split-K partial sums live: partial s of parameter i is part[s*stride + (i - start)].
@@ -135,8 +139,6 @@ struct LearnArgs {
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
     // tensor-pipe path
-    int fuse_gae;         // 1: the backward kernel first computes ADV/RET of its envs (anakin_learn); 0: uses them as they stand
-    float gamma, lambda;
     float gscale, inv_gscale;  // power of two carried by every gradient-side tensor, divided out in the reduction
     float* part_small;    // per (CTA, row group) partials of dWh | db2 | dbh
     size_t small_stride;
@@ -145,7 +147,7 @@ struct LearnArgs {
 
 // Split counts and partial-buffer layout of the tensor-pipe learner (a pure function of the sizes).
 struct LearnPlan {
-    int ns_w2, ns_agent, ns_env, ns_small, loss_blocks;
+    int ns_w2, ns_agent, ns_env, ns_small, loss_blocks, heads_grid;
     size_t small_stride, off_w2, off_agent, off_walls, off_goal, off_small, part_floats;
 };
 void learn_mma_plan(const Dims& d, LearnPlan* p);
@@ -153,7 +155,7 @@ void learn_mma_plan(const Dims& d, LearnPlan* p);
 // Kernel identifiers (anakin_kernel_name / anakin_profile_read index by these).
 enum KernelId : int {
     K_RESET_ENV = 0, K_RESET_PARAMS, K_REFRESH_PARAMS, K_ENV_BASE, K_ROLLOUT, K_GAE, K_H1, K_FWD2, K_HEADS_LOSS, K_DH1,
-    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_PACK_W2, K_LEARN_BWD, K_REPLAY, K_COUNT
+    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_PACK_W2, K_HEADS_BWD, K_REPLAY, K_COUNT
 };
 
 // Optional per-kernel timing with CUDA events on the launching stream (off by default).

@@ -2,10 +2,10 @@
 // hidden sizes the tensor-pipe rollout covers.  The update reuses the policy's forward pass (Section 3.1): the rollout
 // kernel saved h1 (as bf16 hi/lo planes) and h2 for every recorded row, so the learner starts at the heads.
 //
-//   k_learn_bwd   one CTA per 32 envs, looping over t like the rollout: heads -> softmax / loss terms -> dOut -> dh2
-//                 (fp32 FMA), then dh1 = (dh2 W2^T) gated by h1 > 0 with mma.sync (W2^T resident on chip: hi fragments
-//                 in shared memory, lo fragments in registers).  Emits dh2 and dh1 as bf16 hi/lo planes, S = sum_t dh1
-//                 per env, and per-CTA partial sums of dWh, dbh, db2 and the loss terms.
+//   k_heads_bwd   flat 32-row tiles: heads -> softmax / loss terms -> dOut -> dh2 (fp32 FMA, HBM-bound).  Emits dh2 as
+//                 16-bit hi/lo planes and per-CTA partial sums of dWh, dbh, db2 and the loss terms.
+//   k_dh1         dh1 = (dh2 W2^T) gated by h1 > 0 with mma.sync; a CTA keeps its slice of W2 in shared memory and
+//                 walks t for 64 envs, so S = sum_t dh1 accumulates in registers.  Emits dh1 planes and S planes.
 //   k_gemm_tn     C[m][n] = sum_k A[k][m] B[k][n] with split-K partial outputs, bf16 hi/lo planes as operands and
 //                 three MMAs per product (two when A is an exact 0/1 plane, one in the bf16 workload):
 //                 dW2 = h1^T dh2 (K = B*T), dW1[agent plane] = X^T dh1 (K = B*T), dW1[wall, goal planes] = X^T S
@@ -25,104 +25,74 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
 
 // ----------------------------------------------------------------------------------------------------
-// k_learn_bwd
+// k_heads_bwd: heads, softmax, loss terms, output gradients and dh2 for flat 32-row tiles (row i = t*B + env).
+// Persistent CTAs walk the tiles with a double-buffered cp.async stream of h2; everything is fp32 FMA.
+// HBM-bound: reads h2 (4 B/elt) and writes the dh2 planes (2 x 2 B/elt).
 // ----------------------------------------------------------------------------------------------------
 template <int H, int NW, int PREC>
-struct LearnBwdCfg {
-    static constexpr int ME = 32;
-    static constexpr int NT = H / NW / 8;
-    static constexpr int KS = H / 16;
-    static constexpr int LD = H + 8;            // bf16 pitch of the dh2/dh1 planes in smem
-    static constexpr int PARTS = NW;            // threads per row in the heads phase (NW*32 / 32 rows)
+struct HeadsCfg {
+    static constexpr int TR = 32;               // rows per tile
+    static constexpr int PARTS = NW;            // threads per row in the heads phase
     static constexpr int HP = H + PARTS;        // fp32 pitch of the h2 tile (bank skew between rows)
-    static constexpr int PLANES = PREC == 1 ? 1 : 2;
-    static constexpr size_t smem_bytes = (size_t)H * H * 2 + (size_t)ME * HP * 4 + (size_t)PLANES * ME * LD * 2 +
-                                         (size_t)ME * 8 * 4 + (size_t)(H * 5 + 8) * 4 + (size_t)ME * 4 * 4;
+    static constexpr size_t smem_bytes = (size_t)2 * TR * HP * 4 + (size_t)TR * 8 * 4 + (size_t)(H * 5 + 8) * 4 + (size_t)TR * 4 * 4;
 };
 
 template <int H, int NW, int PREC>
-__global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_learn_bwd(LearnArgs a) {
-    using Cfg = LearnBwdCfg<H, NW, PREC>;
-    constexpr int ME = Cfg::ME, NT = Cfg::NT, KS = Cfg::KS, LD = Cfg::LD, HP = Cfg::HP, PARTS = Cfg::PARTS;
-    constexpr int NTHREADS = NW * 32, QN = H / PARTS;  // QN = 16 hidden units per thread in the heads phase
+__global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
+    using Cfg = HeadsCfg<H, NW, PREC>;
+    constexpr int TR = Cfg::TR, HP = Cfg::HP, PARTS = Cfg::PARTS, NTHREADS = NW * 32, QN = H / PARTS;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint2* s_wt_hi = reinterpret_cast<uint2*>(smem_raw);                          // W2^T hi fragments
-    float* s_h2 = reinterpret_cast<float*>(smem_raw + (size_t)H * H * 2);         // [ME][HP]
-    __nv_bfloat16* s_phi = reinterpret_cast<__nv_bfloat16*>(s_h2 + ME * HP);      // [ME][LD] dh2 (then dh1) hi plane
-    __nv_bfloat16* s_plo = s_phi + (PREC == 1 ? 0 : ME * LD);                    // lo plane
-    float* s_dout = reinterpret_cast<float*>(s_phi + Cfg::PLANES * ME * LD);      // [ME][8]
-    float* s_wh = s_dout + ME * 8;                                                // [H][5]
-    float* s_bh = s_wh + H * 5;                                                   // [8]
-    float* s_loss = s_bh + 8;                                                     // [ME][4]
-
+    float* s_h2 = reinterpret_cast<float*>(smem_raw);  // [2][TR][HP]
+    float* s_dout = s_h2 + 2 * TR * HP;                // [TR][8]
+    float* s_wh = s_dout + TR * 8;                     // [H][5]
+    float* s_bh = s_wh + H * 5;                        // [8]
+    float* s_loss = s_bh + 8;                          // [TR][4]
     const Dims& d = a.d;
     const Buffers& b = a.b;
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const int g = lane >> 2, t4 = lane & 3;
-    const int e0 = blockIdx.x * ME;
-    const int B = d.B, T = a.T;
-    const size_t RH = (size_t)B * d.Tmax * H;
-    const __nv_bfloat16* g_h1hi = reinterpret_cast<const __nv_bfloat16*>(b.h1);
-    __nv_bfloat16* g_dh2hi = reinterpret_cast<__nv_bfloat16*>(b.dh2);
-    __nv_bfloat16* g_dh2lo = g_dh2hi + RH;
-    __nv_bfloat16* g_dh1hi = reinterpret_cast<__nv_bfloat16*>(b.dh1);
-    __nv_bfloat16* g_dh1lo = g_dh1hi + RH;
-    const float invR = a.gscale / (float)((size_t)B * T);  // output gradients are carried times gscale
+    const int tid = threadIdx.x;
+    const size_t R = (size_t)d.B * a.T;
+    const size_t RH = (size_t)d.B * d.Tmax * H;
+    uint16_t* g_dh2hi = reinterpret_cast<uint16_t*>(b.dh2);
+    uint16_t* g_dh2lo = g_dh2hi + RH;
+    const float invR = a.gscale / (float)R;  // output gradients are carried times gscale
+    const int ntiles = (int)((R + TR - 1) / TR);
 
-    // ---- prologue
-    {
-        const uint4* src = reinterpret_cast<const uint4*>(b.w2tf_hi);
-        uint4* dst = reinterpret_cast<uint4*>(s_wt_hi);
-        for (int i = tid; i < H * H * 2 / 16; i += NTHREADS) dst[i] = src[i];
-    }
     for (int i = tid; i < H * 5; i += NTHREADS) s_wh[i] = b.theta_c[d.oWh + i];
     if (tid < 5) s_bh[tid] = b.theta_c[d.obh + tid];
-    uint2 blo[PREC == 1 ? 1 : KS][NT];
-    if (PREC == 0) {
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks)
-#pragma unroll
-            for (int j = 0; j < NT; ++j) blo[ks][j] = b.w2tf_lo[(ks * (H / 8) + wid * NT + j) * 32 + lane];
-    }
-    // advantages and returns of this CTA's envs (one thread per env; the other warps are still loading weights)
-    if (a.fuse_gae && tid < ME && e0 + tid < B) gae_scan_env(b, B, T, e0 + tid, a.gamma, a.lambda);
     // heads phase: thread = (row hr, part hp); column phase: thread = (column cj, row group cg of 16 rows)
     const int hr = tid / PARTS, hp = tid % PARTS;
     const int cj = tid % H, cg = tid / H;
-    float wh_c[5];  // Wh row of this thread's column
+    float wh_c[5];
 #pragma unroll
     for (int c = 0; c < 5; ++c) wh_c[c] = b.theta_c[d.oWh + cj * 5 + c];
-    float a_wh[5] = {0.f, 0.f, 0.f, 0.f, 0.f}, a_b2 = 0.f, a_bh = 0.f;  // running sums over t of this thread's rows
+    float a_wh[5] = {0.f, 0.f, 0.f, 0.f, 0.f}, a_b2 = 0.f, a_bh = 0.f;  // running sums over this thread's rows
     float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
-    float s_acc[2][NT][4];  // S = sum over t of dh1, in accumulator-fragment layout
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int j = 0; j < NT; ++j)
-#pragma unroll
-            for (int q = 0; q < 4; ++q) s_acc[mt][j][q] = 0.f;
 
-    auto load_h2_tile = [&](int t) {  // 16-byte chunks, zero-filled past the batch end
-        for (int c = tid; c < ME * (H / 4); c += NTHREADS) {
-            const int e = c / (H / 4), k = 4 * (c - e * (H / 4));
-            const bool ok = e0 + e < B;
-            const float* src = b.h2 + ((size_t)t * B + (ok ? e0 + e : 0)) * H + k;
-            cp_async16(s_h2 + e * HP + k, src, ok ? 16 : 0);
+    auto load_tile = [&](int tile, int buf) {  // 16-byte chunks, zero-filled past the last row
+        float* dst = s_h2 + buf * TR * HP;
+        for (int c = tid; c < TR * (H / 4); c += NTHREADS) {
+            const int r = c / (H / 4), k = 4 * (c - r * (H / 4));
+            const size_t row = (size_t)tile * TR + r;
+            const bool ok = row < R;
+            cp_async16(dst + r * HP + k, b.h2 + (ok ? row : 0) * H + k, ok ? 16 : 0);
         }
         cp_async_commit();
     };
-    load_h2_tile(0);
-
-    for (int t = 0; t < T; ++t) {
+    int it = 0;
+    if ((int)blockIdx.x < ntiles) load_tile(blockIdx.x, 0);
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
         cp_async_wait<0>();
-        __syncthreads();
-        // ---- heads, softmax, loss terms, output gradients (PARTS threads per row, shuffle reduction)
+        __syncthreads();  // tile `tile` has landed; everyone is done with the other buffer
+        if (tile + (int)gridDim.x < ntiles) load_tile(tile + gridDim.x, buf ^ 1);
+        const float* h2t = s_h2 + buf * TR * HP;
+        // ---- heads, softmax, loss terms, output gradients
         {
             float o[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int q = 0; q < QN; ++q) {
                 const int j = hp + PARTS * q;
-                const float x = s_h2[hr * HP + j];
+                const float x = h2t[hr * HP + j];
 #pragma unroll
                 for (int c = 0; c < 5; ++c) o[c] = fmaf(x, s_wh[j * 5 + c], o[c]);
             }
@@ -132,11 +102,10 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_learn_bwd(LearnA
                 for (int off = PARTS / 2; off > 0; off >>= 1) o[c] += __shfl_xor_sync(0xFFFFFFFFu, o[c], off);
                 o[c] += s_bh[c];
             }
-            const int env = e0 + hr;
             if (hp == 0) {
                 float dO[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-                if (env < B) {
-                    const size_t i = (size_t)t * B + env;
+                const size_t i = (size_t)tile * TR + hr;
+                if (i < R) {
                     const float mx = fmaxf(fmaxf(o[0], o[1]), fmaxf(o[2], o[3]));
                     float ex[4], Z = 0.f;
 #pragma unroll
@@ -162,166 +131,234 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_learn_bwd(LearnA
             }
         }
         __syncthreads();
-        // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0; running sums of dWh, db2, dbh
-        {
+        // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0, written as 16-bit planes; sums of dWh, db2, dbh
 #pragma unroll 4
-            for (int r = 0; r < 16; ++r) {
-                const int e = cg * 16 + r;
-                const float4 d0 = *reinterpret_cast<const float4*>(s_dout + e * 8);
-                const float d4 = s_dout[e * 8 + 4];
-                const float h2 = s_h2[e * HP + cj];
-                float back = d0.x * wh_c[0];
-                back = fmaf(d0.y, wh_c[1], back);
-                back = fmaf(d0.z, wh_c[2], back);
-                back = fmaf(d0.w, wh_c[3], back);
-                back = fmaf(d4, wh_c[4], back);
-                const float dh2 = rnd<PREC>(h2 > 0.f ? back : 0.f);
-                a_wh[0] = fmaf(h2, d0.x, a_wh[0]);
-                a_wh[1] = fmaf(h2, d0.y, a_wh[1]);
-                a_wh[2] = fmaf(h2, d0.z, a_wh[2]);
-                a_wh[3] = fmaf(h2, d0.w, a_wh[3]);
-                a_wh[4] = fmaf(h2, d4, a_wh[4]);
-                a_b2 += dh2;
-                if (cj < 5) a_bh += cj == 0 ? d0.x : cj == 1 ? d0.y : cj == 2 ? d0.z : cj == 3 ? d0.w : d4;
+        for (int r = 0; r < 16; ++r) {
+            const int e = cg * 16 + r;
+            const size_t i = (size_t)tile * TR + e;
+            const float4 d0 = *reinterpret_cast<const float4*>(s_dout + e * 8);
+            const float d4 = s_dout[e * 8 + 4];
+            const float h2 = h2t[e * HP + cj];
+            float back = d0.x * wh_c[0];
+            back = fmaf(d0.y, wh_c[1], back);
+            back = fmaf(d0.z, wh_c[2], back);
+            back = fmaf(d0.w, wh_c[3], back);
+            back = fmaf(d4, wh_c[4], back);
+            const float dh2 = rnd<PREC>(h2 > 0.f ? back : 0.f);
+            a_wh[0] = fmaf(h2, d0.x, a_wh[0]);
+            a_wh[1] = fmaf(h2, d0.y, a_wh[1]);
+            a_wh[2] = fmaf(h2, d0.z, a_wh[2]);
+            a_wh[3] = fmaf(h2, d0.w, a_wh[3]);
+            a_wh[4] = fmaf(h2, d4, a_wh[4]);
+            a_b2 += dh2;
+            if (cj < 5) a_bh += cj == 0 ? d0.x : cj == 1 ? d0.y : cj == 2 ? d0.z : cj == 3 ? d0.w : d4;
+            if (i < R) {
                 uint16_t hi16, lo16;
                 split1<PREC>(dh2, hi16, lo16);
-                reinterpret_cast<uint16_t*>(s_phi)[e * LD + cj] = hi16;
-                if (PREC == 0) reinterpret_cast<uint16_t*>(s_plo)[e * LD + cj] = lo16;
+                g_dh2hi[i * H + cj] = hi16;
+                if (PREC == 0) g_dh2lo[i * H + cj] = lo16;
             }
         }
-        __syncthreads();
-        // ---- h2 is dead: start fetching the next tile; fetch this tile's layer-1 gates; write dh2 planes out
-        if (t + 1 < T) load_h2_tile(t + 1);
-        uint32_t gate1[2][NT][2];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int j = 0; j < NT; ++j)
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int row = 16 * mt + 8 * hh + g, col0 = (wid * NT + j) * 8 + 2 * t4;
-                    gate1[mt][j][hh] = (e0 + row < B)
-                                           ? __ldg(reinterpret_cast<const uint32_t*>(g_h1hi + ((size_t)t * B + e0 + row) * H + col0))
-                                           : 0u;
-                }
-        for (int c = tid; c < ME * (H / 8); c += NTHREADS) {
-            const int e = c / (H / 8), k = 8 * (c - e * (H / 8));
-            if (e0 + e < B) {
-                const size_t gi = ((size_t)t * B + e0 + e) * H + k;
-                *reinterpret_cast<uint4*>(g_dh2hi + gi) = *reinterpret_cast<const uint4*>(s_phi + e * LD + k);
-                if (PREC == 0) *reinterpret_cast<uint4*>(g_dh2lo + gi) = *reinterpret_cast<const uint4*>(s_plo + e * LD + k);
-            }
-        }
-        // ---- dh1 = dh2 W2^T on the tensor pipe
-        float acc[2][NT][4];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int j = 0; j < NT; ++j)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) acc[mt][j][q] = 0.f;
-        {
-            const int arow = (lane & 7) + ((lane >> 3) & 1) * 8, acol = (lane >> 4) * 8;
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                uint32_t ahi[2][4], alo[2][4];
-#pragma unroll
-                for (int mt = 0; mt < 2; ++mt) {
-                    ldmatrix_x4(ahi[mt], s_phi + (16 * mt + arow) * LD + 16 * ks + acol);
-                    if (PREC == 0) ldmatrix_x4(alo[mt], s_plo + (16 * mt + arow) * LD + 16 * ks + acol);
-                }
-#pragma unroll
-                for (int j = 0; j < NT; ++j) {
-                    const uint2 bhi = s_wt_hi[(ks * (H / 8) + wid * NT + j) * 32 + lane];
-#pragma unroll
-                    for (int mt = 0; mt < 2; ++mt) {
-                        if (PREC == 0) {
-                            mma16816<PREC>(acc[mt][j], alo[mt], bhi.x, bhi.y);
-                            mma16816<PREC>(acc[mt][j], ahi[mt], blo[ks][j].x, blo[ks][j].y);
-                        }
-                        mma16816<PREC>(acc[mt][j], ahi[mt], bhi.x, bhi.y);
-                    }
-                }
-            }
-        }
-        __syncthreads();  // every warp is done reading the dh2 planes
-        // ---- gate by h1 > 0, accumulate S, stage dh1 planes
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int j = 0; j < NT; ++j)
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int row = 16 * mt + 8 * hh + g, col0 = (wid * NT + j) * 8 + 2 * t4;
-                    const uint32_t gt = gate1[mt][j][hh];
-                    // h1 >= 0 always, so "h1 > 0" is "any bit of the 16-bit high part set"
-                    const float v0 = rnd<PREC>((gt & 0x0000FFFFu) ? acc[mt][j][2 * hh] : 0.f);
-                    const float v1 = rnd<PREC>((gt & 0xFFFF0000u) ? acc[mt][j][2 * hh + 1] : 0.f);
-                    s_acc[mt][j][2 * hh] += v0;
-                    s_acc[mt][j][2 * hh + 1] += v1;
-                    uint32_t phi, plo;
-                    split2<PREC>(v0, v1, phi, plo);
-                    *reinterpret_cast<uint32_t*>(s_phi + row * LD + col0) = phi;
-                    if (PREC == 0) *reinterpret_cast<uint32_t*>(s_plo + row * LD + col0) = plo;
-                }
-        __syncthreads();
-        for (int c = tid; c < ME * (H / 8); c += NTHREADS) {
-            const int e = c / (H / 8), k = 8 * (c - e * (H / 8));
-            if (e0 + e < B) {
-                const size_t gi = ((size_t)t * B + e0 + e) * H + k;
-                *reinterpret_cast<uint4*>(g_dh1hi + gi) = *reinterpret_cast<const uint4*>(s_phi + e * LD + k);
-                if (PREC == 0) *reinterpret_cast<uint4*>(g_dh1lo + gi) = *reinterpret_cast<const uint4*>(s_plo + e * LD + k);
-            }
-        }
-        // the loop-top barrier orders these plane reads before the next column phase overwrites them
+        // the loop-top barrier orders these reads of the tile before the buffer is refilled
     }
-
-    // ---- per-CTA results
-    // S (sum over t of dh1) as hi/lo planes [B][H]: always two planes, S is an fp32 sum even in the bf16 workload
-    {
-        __nv_bfloat16* S_hi = reinterpret_cast<__nv_bfloat16*>(b.S);
-        __nv_bfloat16* S_lo = S_hi + (size_t)B * H;
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int j = 0; j < NT; ++j)
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int row = 16 * mt + 8 * hh + g, col0 = (wid * NT + j) * 8 + 2 * t4;
-                    if (e0 + row < B) {
-                        // two terms in either workload: PREC 1 keeps bf16 hi + bf16 lo of the fp32 sum
-                        uint32_t phi, plo;
-                        if (PREC == 1) {
-                            __nv_bfloat16 h0, l0, h1v, l1;
-                            split_bf16(s_acc[mt][j][2 * hh], h0, l0);
-                            split_bf16(s_acc[mt][j][2 * hh + 1], h1v, l1);
-                            phi = pack_bf16(h0, h1v);
-                            plo = pack_bf16(l0, l1);
-                        } else {
-                            split2<0>(s_acc[mt][j][2 * hh], s_acc[mt][j][2 * hh + 1], phi, plo);
-                        }
-                        const size_t gi = (size_t)(e0 + row) * H + col0;
-                        *reinterpret_cast<uint32_t*>(S_hi + gi) = phi;
-                        *reinterpret_cast<uint32_t*>(S_lo + gi) = plo;
-                    }
-                }
-    }
-    // dWh, db2, dbh partials: split index = 2*CTA + row group
+    cp_async_wait<0>();
+    // ---- per-CTA results: dWh, db2, dbh partials (split index = 2*CTA + row group) and loss partials
     {
         float* part = a.part_small + (size_t)(2 * blockIdx.x + cg) * a.small_stride;
 #pragma unroll
-        for (int c = 0; c < 5; ++c) part[(size_t)cj * 5 + c] = a_wh[c];  // Wh region first
-        part[(size_t)H * 5 + cj] = a_b2;                                 // then b2
-        if (cj < 5) part[(size_t)H * 6 + cj] = a_bh;                     // then bh
+        for (int c = 0; c < 5; ++c) part[(size_t)cj * 5 + c] = a_wh[c];
+        part[(size_t)H * 5 + cj] = a_b2;
+        if (cj < 5) part[(size_t)H * 6 + cj] = a_bh;
     }
-    // loss partials, rows in index order
+    __syncthreads();
     if (hp == 0) { s_loss[hr * 4 + 0] = l_pg; s_loss[hr * 4 + 1] = l_v; s_loss[hr * 4 + 2] = l_ent; }
     __syncthreads();
     if (tid < 3) {
         float s = 0.f;
-        for (int e = 0; e < ME; ++e) s += s_loss[e * 4 + tid];
+        for (int e = 0; e < TR; ++e) s += s_loss[e * 4 + tid];
         b.loss_part[(size_t)blockIdx.x * 4 + tid] = s;
     }
+}
+
+// ----------------------------------------------------------------------------------------------------
+// k_dh1: dh1 = (dh2 W2^T) gated by h1 > 0 on the tensor pipe, and S = sum over t of dh1.
+// A CTA owns 64 envs x BN output columns and walks t = 0..T-1.  Its slice of W2 (BN rows, all K, hi and lo planes)
+// stays in shared memory for the whole kernel; the dh2 planes stream through a cp.async ring in 64-wide k chunks
+// that runs across the t boundaries without draining.
+// ----------------------------------------------------------------------------------------------------
+template <int H, int BN, int PREC>
+struct Dh1Cfg {
+    static constexpr int BM = 64, KC = 64, STAGES = 4, THREADS = 256;
+    static constexpr int PL = PREC == 1 ? 1 : 2;
+    static constexpr int LDW = H + 8;     // 16-bit pitch of the resident W2 planes
+    static constexpr int LDA = KC + 8;    // 16-bit pitch of an A chunk
+    static constexpr int A_STAGE = PL * BM * LDA;
+    static constexpr int NCH = H / KC;    // chunks per t
+    static constexpr int WM = 32, WN = BN / 4;  // warp tile (2 x 4 warps)
+    static constexpr int MT = WM / 16, NT = WN / 8;
+    static constexpr size_t smem_bytes = ((size_t)PL * BN * LDW + (size_t)STAGES * A_STAGE) * 2;
+};
+
+template <int H, int BN, int PREC>
+__global__ void __launch_bounds__(256) k_dh1(LearnArgs a) {
+    using Cfg = Dh1Cfg<H, BN, PREC>;
+    constexpr int BM = Cfg::BM, KC = Cfg::KC, STAGES = Cfg::STAGES, PL = Cfg::PL, LDW = Cfg::LDW, LDA = Cfg::LDA;
+    constexpr int NCH = Cfg::NCH, MT = Cfg::MT, NT = Cfg::NT;
+    static_assert(NT % 2 == 0, "B fragments are loaded two n-tiles at a time");
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint16_t* sW = reinterpret_cast<uint16_t*>(smem_raw);  // [PL][BN][LDW]
+    uint16_t* sA = sW + PL * BN * LDW;                      // [STAGES][PL][BM][LDA]
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int wm = wid >> 2, wn = wid & 3;
+    const int g = lane >> 2, t4 = lane & 3;
+    const int B = d.B, T = a.T;
+    const int e0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const size_t RH = (size_t)B * d.Tmax * H;
+    const uint16_t* g_dh2hi = reinterpret_cast<const uint16_t*>(b.dh2);
+    const uint16_t* g_h1hi = reinterpret_cast<const uint16_t*>(b.h1);
+    uint16_t* g_dh1hi = reinterpret_cast<uint16_t*>(b.dh1);
+
+    // resident slice of W2: rows n0..n0+BN (output units), all k
+    for (int c = tid; c < BN * (H / 8); c += 256) {
+        const int n = c / (H / 8), k = 8 * (c - n * (H / 8));
+        cp_async16(sW + n * LDW + k, b.w2p_hi + (size_t)(n0 + n) * H + k, 16);
+        if (PL == 2) cp_async16(sW + BN * LDW + n * LDW + k, b.w2p_lo + (size_t)(n0 + n) * H + k, 16);
+    }
+    cp_async_commit();
+
+    const int nchunks = T * NCH;
+    auto issue = [&](int c, int stage) {
+        const int t = c / NCH, k0 = (c - t * NCH) * KC;
+        uint16_t* a_s = sA + stage * Cfg::A_STAGE;
+        for (int q = tid; q < BM * (KC / 8); q += 256) {
+            const int r = q / (KC / 8), k = 8 * (q - r * (KC / 8));
+            const bool ok = e0 + r < B;
+            const size_t gi = ((size_t)t * B + (ok ? e0 + r : 0)) * H + k0 + k;
+            cp_async16(a_s + r * LDA + k, g_dh2hi + gi, ok ? 16 : 0);
+            if (PL == 2) cp_async16(a_s + BM * LDA + r * LDA + k, g_dh2hi + RH + gi, ok ? 16 : 0);
+        }
+    };
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        if (s < nchunks) issue(s, s);
+        cp_async_commit();
+    }
+
+    float acc[MT][NT][4], s_acc[MT][NT][4];
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { acc[i][j][q] = 0.f; s_acc[i][j][q] = 0.f; }
+    uint32_t gate1[MT][NT][2];
+    const int jm = lane >> 3, r8 = lane & 7;
+
+    for (int c = 0; c < nchunks; ++c) {
+        const int t = c / NCH, kc = c - t * NCH;
+        cp_async_wait<STAGES - 2>();  // chunk c (and, the first time, the W2 slice) has landed
+        __syncthreads();
+        {
+            const int nxt = c + STAGES - 1;
+            if (nxt < nchunks) issue(nxt, nxt % STAGES);
+            cp_async_commit();
+        }
+        if (kc == 0) {  // this step's layer-1 gates, well ahead of the epilogue
+#pragma unroll
+            for (int i = 0; i < MT; ++i)
+#pragma unroll
+                for (int j = 0; j < NT; ++j)
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int row = wm * Cfg::WM + 16 * i + 8 * hh + g, col = n0 + wn * Cfg::WN + 8 * j + 2 * t4;
+                        gate1[i][j][hh] = (e0 + row < B)
+                                              ? __ldg(reinterpret_cast<const uint32_t*>(g_h1hi + ((size_t)t * B + e0 + row) * H + col))
+                                              : 0u;
+                    }
+        }
+        const uint16_t* a_s = sA + (c % STAGES) * Cfg::A_STAGE;
+#pragma unroll
+        for (int k16 = 0; k16 < KC / 16; ++k16) {
+            uint32_t ahi[MT][4], alo[MT][4];
+#pragma unroll
+            for (int i = 0; i < MT; ++i) {
+                const uint16_t* p = a_s + (wm * Cfg::WM + 16 * i + (lane & 7) + ((lane >> 3) & 1) * 8) * LDA + 16 * k16 + (lane >> 4) * 8;
+                ldmatrix_x4(ahi[i], p);
+                if (PL == 2) ldmatrix_x4(alo[i], p + BM * LDA);
+            }
+#pragma unroll
+            for (int j2 = 0; j2 < NT / 2; ++j2) {
+                uint32_t bhi[4], blo[4];
+                const uint16_t* p = sW + (wn * Cfg::WN + 16 * j2 + 8 * (jm >> 1) + r8) * LDW + kc * KC + 16 * k16 + 8 * (jm & 1);
+                ldmatrix_x4(bhi, p);
+                if (PL == 2) ldmatrix_x4(blo, p + BN * LDW);
+#pragma unroll
+                for (int i = 0; i < MT; ++i)
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        if (PL == 2) {
+                            mma16816<PREC>(acc[i][2 * j2 + q], alo[i], bhi[2 * q], bhi[2 * q + 1]);
+                            mma16816<PREC>(acc[i][2 * j2 + q], ahi[i], blo[2 * q], blo[2 * q + 1]);
+                        }
+                        mma16816<PREC>(acc[i][2 * j2 + q], ahi[i], bhi[2 * q], bhi[2 * q + 1]);
+                    }
+            }
+        }
+        if (kc == NCH - 1) {  // row tile of step t complete: gate, accumulate S, emit dh1 planes
+#pragma unroll
+            for (int i = 0; i < MT; ++i)
+#pragma unroll
+                for (int j = 0; j < NT; ++j)
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int row = wm * Cfg::WM + 16 * i + 8 * hh + g, col = n0 + wn * Cfg::WN + 8 * j + 2 * t4;
+                        const uint32_t gt = gate1[i][j][hh];
+                        // h1 >= 0 always, so "h1 > 0" is "any bit of the 16-bit high part set"
+                        const float v0 = rnd<PREC>((gt & 0x0000FFFFu) ? acc[i][j][2 * hh] : 0.f);
+                        const float v1 = rnd<PREC>((gt & 0xFFFF0000u) ? acc[i][j][2 * hh + 1] : 0.f);
+                        s_acc[i][j][2 * hh] += v0;
+                        s_acc[i][j][2 * hh + 1] += v1;
+                        acc[i][j][2 * hh] = 0.f;
+                        acc[i][j][2 * hh + 1] = 0.f;
+                        if (e0 + row < B) {
+                            uint32_t phi, plo;
+                            split2<PREC>(v0, v1, phi, plo);
+                            const size_t gi = ((size_t)t * B + e0 + row) * H + col;
+                            *reinterpret_cast<uint32_t*>(g_dh1hi + gi) = phi;
+                            if (PL == 2) *reinterpret_cast<uint32_t*>(g_dh1hi + RH + gi) = plo;
+                        }
+                    }
+        }
+    }
+    cp_async_wait<0>();
+    // S (sum over t of dh1) as two 16-bit planes [B][H]: S is an fp32 sum, so it keeps two terms in either workload
+    uint16_t* S_hi = reinterpret_cast<uint16_t*>(b.S);
+    uint16_t* S_lo = S_hi + (size_t)B * H;
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int row = wm * Cfg::WM + 16 * i + 8 * hh + g, col = n0 + wn * Cfg::WN + 8 * j + 2 * t4;
+                if (e0 + row < B) {
+                    uint32_t phi, plo;
+                    if (PREC == 1) {
+                        __nv_bfloat16 h0, l0, h1v, l1;
+                        split_bf16(s_acc[i][j][2 * hh], h0, l0);
+                        split_bf16(s_acc[i][j][2 * hh + 1], h1v, l1);
+                        phi = pack_bf16(h0, h1v);
+                        plo = pack_bf16(l0, l1);
+                    } else {
+                        split2<0>(s_acc[i][j][2 * hh], s_acc[i][j][2 * hh + 1], phi, plo);
+                    }
+                    const size_t gi = (size_t)(e0 + row) * H + col;
+                    *reinterpret_cast<uint32_t*>(S_hi + gi) = phi;
+                    *reinterpret_cast<uint32_t*>(S_lo + gi) = plo;
+                }
+            }
 }
 
 // ----------------------------------------------------------------------------------------------------
@@ -562,6 +599,8 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             reinterpret_cast<uint16_t*>(b.w2f_lo)[ef] = lo;
             reinterpret_cast<uint16_t*>(b.w2tf_hi)[et] = hi;
             reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
+            b.w2p_hi[i - d.oW2] = hi;
+            b.w2p_lo[i - d.oW2] = lo;
         }
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -595,6 +634,8 @@ __global__ void __launch_bounds__(256) k_pack_gates2(Dims d, Buffers b, size_t R
 // ----------------------------------------------------------------------------------------------------
 // host side
 // ----------------------------------------------------------------------------------------------------
+constexpr int HEADS_GRID = 2 * 148;  // persistent CTAs of k_heads_bwd (two per SM)
+
 static int splits_for(int K, int tiles, int min_k) {
     int ns = (2 * 148 + tiles - 1) / tiles;
     const int cap = K / min_k > 0 ? K / min_k : 1;
@@ -612,7 +653,9 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     p->ns_w2 = splits_for((int)R, tiles_hh, 256);
     p->ns_agent = splits_for((int)R, tiles_ch, 256);
     p->ns_env = splits_for(d.B, tiles_ch, 128);
-    p->ns_small = 2 * ((d.B + 31) / 32);
+    const size_t tiles32 = (R + 31) / 32;
+    p->heads_grid = (int)(tiles32 < (size_t)HEADS_GRID ? tiles32 : (size_t)HEADS_GRID);
+    p->ns_small = 2 * p->heads_grid;
     p->small_stride = (size_t)6 * H + 8;
     size_t off = 0;
     p->off_w2 = off; off += (size_t)p->ns_w2 * H * H;
@@ -621,16 +664,25 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     p->off_goal = off; off += (size_t)p->ns_env * C * H;
     p->off_small = off; off += (size_t)p->ns_small * p->small_stride;
     p->part_floats = off;
-    p->loss_blocks = (d.B + 31) / 32;
+    p->loss_blocks = p->heads_grid;
 }
 
 #define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
 
 template <int H, int NW, int PREC>
-static cudaError_t launch_bwd_t(const LearnArgs& a, cudaStream_t s) {
-    using Cfg = LearnBwdCfg<H, NW, PREC>;
-    CK(cudaFuncSetAttribute(k_learn_bwd<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
-    k_learn_bwd<H, NW, PREC><<<(a.d.B + 31) / 32, NW * 32, Cfg::smem_bytes, s>>>(a);
+static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s) {
+    using Cfg = HeadsCfg<H, NW, PREC>;
+    CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
+    k_heads_bwd<H, NW, PREC><<<grid, NW * 32, Cfg::smem_bytes, s>>>(a);
+    return cudaGetLastError();
+}
+
+template <int H, int BN, int PREC>
+static cudaError_t launch_dh1_t(const LearnArgs& a, cudaStream_t s) {
+    using Cfg = Dh1Cfg<H, BN, PREC>;
+    CK(cudaFuncSetAttribute(k_dh1<H, BN, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
+    dim3 grid((a.d.B + Cfg::BM - 1) / Cfg::BM, H / BN);
+    k_dh1<H, BN, PREC><<<grid, 256, Cfg::smem_bytes, s>>>(a);
     return cudaGetLastError();
 }
 
@@ -657,11 +709,20 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     a.reg[7] = PartRegion{b.part + pl.off_small + (size_t)6 * H, pl.ns_small, pl.small_stride, d.obh};
 
     {
-        Scope sc(c, K_LEARN_BWD);
+        Scope sc(c, K_HEADS_BWD);
         switch (H) {
-            case 64: CK((launch_bwd_t<64, 4, PREC>(a, s))); break;
-            case 128: CK((launch_bwd_t<128, 8, PREC>(a, s))); break;
-            case 256: CK((launch_bwd_t<256, 16, PREC>(a, s))); break;
+            case 64: CK((launch_heads_t<64, 4, PREC>(a, pl.heads_grid, s))); break;
+            case 128: CK((launch_heads_t<128, 8, PREC>(a, pl.heads_grid, s))); break;
+            case 256: CK((launch_heads_t<256, 16, PREC>(a, pl.heads_grid, s))); break;
+            default: return cudaErrorNotSupported;
+        }
+    }
+    {
+        Scope sc(c, K_DH1);
+        switch (H) {
+            case 64: CK((launch_dh1_t<64, 64, PREC>(a, s))); break;
+            case 128: CK((launch_dh1_t<128, 128, PREC>(a, s))); break;
+            case 256: CK((launch_dh1_t<256, 128, PREC>(a, s))); break;
             default: return cudaErrorNotSupported;
         }
     }

@@ -103,6 +103,8 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     a.key0 = (uint32_t)(seed & 0xFFFFFFFFu);
     a.key1 = (uint32_t)(seed >> 32);
     a.forced = nullptr;
+    a.replay = 0;
+    a.fuse_gae = 0;  // the caller gets the trajectory only
     uint64_t launches = 0;
     const Ctx ctx{s, &launches, nullptr};
     if (launch_env_base(a.d, b, ctx) != cudaSuccess) return ANAKIN_E_CUDA;  // fills `base`: nothing of the last call survives

@@ -38,6 +38,15 @@ __global__ void __launch_bounds__(256) k_pack_w2(Dims d, Buffers b) {
     split2<PREC>(W2[(size_t)n * H + ks4[2]], W2[(size_t)n * H + ks4[3]], hi.y, lo.y);
     b.w2tf_hi[idx] = hi;
     b.w2tf_lo[idx] = lo;
+    // and W2 itself as row-major hi / lo planes: this thread covers elements 4*idx .. 4*idx+3
+    if (!b.w2p_hi) return;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint16_t h16, l16;
+        split1<PREC>(W2[(size_t)4 * idx + q], h16, l16);
+        b.w2p_hi[(size_t)4 * idx + q] = h16;
+        b.w2p_lo[(size_t)4 * idx + q] = l16;
+    }
 }
 
 cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c) {
@@ -274,6 +283,8 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
     if (owner) {
         b.pos[e0 + tid] = (uint8_t)s.pos;
         b.tep[e0 + tid] = (uint8_t)s.tep;
+        // the owner thread wrote this env's rewards, values and done flags itself: it can scan them right away
+        if (a.fuse_gae) gae_scan_env(b, B, a.T, e0 + tid, a.gamma, a.lambda);
     }
     if (tid < 32) flush_env_stats(s, a);
 }
