@@ -188,20 +188,22 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
 // ----------------------------------------------------------------------------------------------------
 template <int H, int BN, int PREC>
 struct Dh1Cfg {
-    static constexpr int BM = 64, KC = 64, STAGES = 4, THREADS = 256;
+    static constexpr int BM = 64, KC = 64, STAGES = 4;
     static constexpr int PL = PREC == 1 ? 1 : 2;
     static constexpr int LDW = H + 8;     // 16-bit pitch of the resident W2 planes
     static constexpr int LDA = KC + 8;    // 16-bit pitch of an A chunk
     static constexpr int A_STAGE = PL * BM * LDA;
     static constexpr int NCH = H / KC;    // chunks per t
-    static constexpr int WM = 32, WN = BN / 4;  // warp tile (2 x 4 warps)
+    static constexpr int WM = 32, WN = 16;     // warp tile; 2 x (BN/16) warps
+    static constexpr int WARPS_N = BN / WN, THREADS = 2 * WARPS_N * 32;
     static constexpr int MT = WM / 16, NT = WN / 8;
     static constexpr size_t smem_bytes = ((size_t)PL * BN * LDW + (size_t)STAGES * A_STAGE) * 2;
 };
 
 template <int H, int BN, int PREC>
-__global__ void __launch_bounds__(256) k_dh1(LearnArgs a) {
+__global__ void __launch_bounds__(Dh1Cfg<H, BN, PREC>::THREADS, 1) k_dh1(LearnArgs a) {
     using Cfg = Dh1Cfg<H, BN, PREC>;
+    constexpr int NTH = Cfg::THREADS;
     constexpr int BM = Cfg::BM, KC = Cfg::KC, STAGES = Cfg::STAGES, PL = Cfg::PL, LDW = Cfg::LDW, LDA = Cfg::LDA;
     constexpr int NCH = Cfg::NCH, MT = Cfg::MT, NT = Cfg::NT;
     static_assert(NT % 2 == 0, "B fragments are loaded two n-tiles at a time");
@@ -211,7 +213,7 @@ __global__ void __launch_bounds__(256) k_dh1(LearnArgs a) {
     const Dims& d = a.d;
     const Buffers& b = a.b;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const int wm = wid >> 2, wn = wid & 3;
+    const int wm = wid / Cfg::WARPS_N, wn = wid % Cfg::WARPS_N;
     const int g = lane >> 2, t4 = lane & 3;
     const int B = d.B, T = a.T;
     const int e0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
@@ -221,7 +223,7 @@ __global__ void __launch_bounds__(256) k_dh1(LearnArgs a) {
     uint16_t* g_dh1hi = reinterpret_cast<uint16_t*>(b.dh1);
 
     // resident slice of W2: rows n0..n0+BN (output units), all k
-    for (int c = tid; c < BN * (H / 8); c += 256) {
+    for (int c = tid; c < BN * (H / 8); c += NTH) {
         const int n = c / (H / 8), k = 8 * (c - n * (H / 8));
         cp_async16(sW + n * LDW + k, b.w2p_hi + (size_t)(n0 + n) * H + k, 16);
         if (PL == 2) cp_async16(sW + BN * LDW + n * LDW + k, b.w2p_lo + (size_t)(n0 + n) * H + k, 16);
@@ -232,7 +234,7 @@ __global__ void __launch_bounds__(256) k_dh1(LearnArgs a) {
     auto issue = [&](int c, int stage) {
         const int t = c / NCH, k0 = (c - t * NCH) * KC;
         uint16_t* a_s = sA + stage * Cfg::A_STAGE;
-        for (int q = tid; q < BM * (KC / 8); q += 256) {
+        for (int q = tid; q < BM * (KC / 8); q += NTH) {
             const int r = q / (KC / 8), k = 8 * (q - r * (KC / 8));
             const bool ok = e0 + r < B;
             const size_t gi = ((size_t)t * B + (ok ? e0 + r : 0)) * H + k0 + k;
@@ -553,25 +555,8 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
         s_c[1] = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
     }
     __syncthreads();
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < d.P) {
-        int r = 0;
-#pragma unroll
-        for (int q = 1; q < LearnArgs::NREG; ++q)
-            if (i >= a.reg[q].start) r = q;
-        const PartRegion& rg = a.reg[r];
-        const float* p = rg.part + (i - rg.start);
-        // fixed order: partial s is always added after partial s-1 (eight loads in flight at a time)
-        float gsum = 0.f;
-        int s = 0;
-        for (; s + 8 <= rg.ns; s += 8) {
-            float v[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) gsum += v[q];
-        }
-        for (; s < rg.ns; ++s) gsum += p[(size_t)s * rg.stride];
+    // Applies the batch-mean gradient of parameter i: statistics, Adam, refreshed 16-bit copies.
+    auto apply = [&](size_t i, float gsum) {
         gsum *= a.inv_gscale;  // exact: a power of two
         b.grads[i] = gsum;
         const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * gsum;
@@ -587,7 +572,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             thc = is_bias ? th : round_bf16(th);
             b.theta_c[i] = thc;
         }
-        // refresh the tensor-pipe fragment copies of W2 and W2^T in place (same layout as k_pack_w2)
+        // refresh the tensor-pipe copies of W2 in place (fragment layouts as in k_pack_w2, and the row-major planes)
         if (i >= d.oW2 && i < d.ob2) {
             const int H = d.H;
             const int k = (int)((i - d.oW2) / H), n = (int)((i - d.oW2) % H);
@@ -601,6 +586,47 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
             b.w2p_hi[i - d.oW2] = hi;
             b.w2p_lo[i - d.oW2] = lo;
+        }
+    };
+    auto region_of = [&](size_t i) {
+        int r = 0;
+#pragma unroll
+        for (int q = 1; q < LearnArgs::NREG; ++q)
+            if (i >= a.reg[q].start) r = q;
+        return r;
+    };
+    // Parameters before b2 (W1, b1, W2) have at most ~128 partials: one thread each, partials added in index order,
+    // eight loads in flight.  The tail (b2 | Wh | bh) has two partials per CTA of the heads kernel: one warp per
+    // parameter, lane l adds partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
+    const int nb_main = (int)((d.ob2 + 255) / 256);
+    if ((int)blockIdx.x < nb_main) {
+        const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+        if (i < d.ob2) {
+            const PartRegion& rg = a.reg[region_of(i)];
+            const float* p = rg.part + (i - rg.start);
+            float gsum = 0.f;
+            int s = 0;
+            for (; s + 8 <= rg.ns; s += 8) {
+                float v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) gsum += v[q];
+            }
+            for (; s < rg.ns; ++s) gsum += p[(size_t)s * rg.stride];
+            apply(i, gsum);
+        }
+    } else {
+        const int lane = threadIdx.x & 31;
+        const size_t i = d.ob2 + (size_t)(blockIdx.x - nb_main) * 8 + (threadIdx.x >> 5);
+        if (i < d.P) {
+            const PartRegion& rg = a.reg[region_of(i)];
+            const float* p = rg.part + (i - rg.start);
+            float gsum = 0.f;
+            for (int s = lane; s < rg.ns; s += 32) gsum += p[(size_t)s * rg.stride];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, off);
+            if (lane == 0) apply(i, gsum);
         }
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -682,7 +708,7 @@ static cudaError_t launch_dh1_t(const LearnArgs& a, cudaStream_t s) {
     using Cfg = Dh1Cfg<H, BN, PREC>;
     CK(cudaFuncSetAttribute(k_dh1<H, BN, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
     dim3 grid((a.d.B + Cfg::BM - 1) / Cfg::BM, H / BN);
-    k_dh1<H, BN, PREC><<<grid, 256, Cfg::smem_bytes, s>>>(a);
+    k_dh1<H, BN, PREC><<<grid, Cfg::THREADS, Cfg::smem_bytes, s>>>(a);
     return cudaGetLastError();
 }
 
@@ -773,7 +799,8 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     }
     {
         Scope sc(c, K_REDUCE_ADAM);
-        k_reduce_adam2<PREC><<<(unsigned)((d.P + 255) / 256), 256, 0, s>>>(a, R, pl.loss_blocks);
+        const unsigned nb = (unsigned)((d.ob2 + 255) / 256 + (d.P - d.ob2 + 7) / 8);
+        k_reduce_adam2<PREC><<<nb, 256, 0, s>>>(a, R, pl.loss_blocks);
         CK(cudaGetLastError());
     }
     if (b.dbg_gates) {
