@@ -195,6 +195,26 @@ struct Scope {
     ~Scope() { if (b) cudaEventRecord(b, c.s); }
 };
 
+// Operands of the split-K "TN" GEMMs  C[m][n] = sum_k A[k][m] B[k][n]  (weight gradients).
+enum : int { A_PLANES = 0, A_ONEHOT = 1, A_WALLS = 2 };
+
+struct GemmTnArgs {
+    int M, N, K, klen;
+    const __nv_bfloat16 *Ahi, *Alo;  // A_PLANES: [K][lda]
+    int lda;
+    const uint8_t* idx;              // A_ONEHOT: A[k][m] = (idx[k] == m)
+    const uint32_t* walls;           // A_WALLS: A[k][m] = bit m of env k (m < ones_row), 1 for m == ones_row
+    int W, ones_row;
+    const __nv_bfloat16 *Bhi, *Blo;  // [K][ldb]
+    int ldb;
+    float* part;                     // out: part[split*stride + off + m*ldc + n]; row ones_row goes to off_ones + n
+    size_t stride, off, off_ones;
+    int ldc;
+};
+
+// tcgen05 version (tensor memory accumulators, TMA-fed); cudaErrorNotSupported when the shape is not covered.
+cudaError_t launch_gemm_tn_tc(const GemmTnArgs& g, int amode, int apl, int bpl, int prec, int splits, int* status, cudaStream_t s);
+
 // kernels (defined in the .cu files) ----------------------------------------------------------------
 cudaError_t launch_reset(const Dims& d, const Buffers& b, uint64_t seed, double density, int prec, const Ctx& c);
 cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c);

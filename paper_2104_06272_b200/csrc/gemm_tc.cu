@@ -1,0 +1,253 @@
+// Weight-gradient GEMMs on the 5th-generation tensor cores:  C[m][n] = sum_k A[k][m] B[k][n],  K = B*T rows.
+//
+// These are the batch-mean reductions of the update (the single-device form of the paper's cross-core gradient average,
+// Podracer paper, Section 3.1): dW2 = h1^T dh2 and the agent plane of dW1 = onehot(pos)^T dh1.  Both operands have the
+// contraction index as their slow (row) index, i.e. they are "MN-major" for the MMA.
+//
+// One CTA owns a 128 x BN output tile (BN = the hidden width, up to 256 accumulator columns in tensor memory) and a
+// K range (split-K; partials are summed later in a fixed order).  Per 64-row K chunk:
+//   warp 0 (one lane)  issues TMA loads of the operand planes (64 x 64 boxes, 128-byte swizzle) into a 2-stage ring,
+//   warps 2-5          for the one-hot A operand: write the 0/1 tile straight into the swizzled layout instead of loading it,
+//   warp 1 (one lane)  issues tcgen05.mma: for fp32 workloads three MMAs per k16 (lo*hi, hi*lo, hi*hi fp16 terms) into one
+//                      fp32 accumulator; commits free the stage,
+//   warps 2-5          after the last chunk: tcgen05.ld the accumulator and store the partial tile.
+// Every wait is bounded; a timeout raises DEV_E_WAIT_TIMEOUT in the status word and the CTA unwinds (tensor memory freed).
+#include <cstdio>
+#include <cstring>
+
+#include "tc_common.cuh"
+
+namespace anakin {
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+}  // namespace
+
+bool make_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool bf16) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int APL, int BPL>
+struct GemmTcCfg {
+    static constexpr int BM = 128, KC = 64, STAGES = 2, THREADS = 192;
+    static constexpr int BOX = 64 * 64 * 2;                  // one 64 x 64 box of 16-bit elements
+    static constexpr int A_PLANE = (BM / 64) * BOX;          // 16 KB
+    static constexpr int B_PLANE = (BN / 64) * BOX;
+    static constexpr int STAGE = APL * A_PLANE + BPL * B_PLANE;
+    static constexpr size_t smem_bytes = (size_t)STAGES * STAGE + 1024 /*alignment slack*/ + 128 /*barriers, tmem slot*/;
+};
+
+struct GemmTcMaps {
+    CUtensorMap a_hi, a_lo, b_hi, b_lo;
+};
+
+template <int BN, int AMODE, int APL, int BPL, int PREC>
+__global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ GemmTcMaps maps, GemmTnArgs g, int* status) {
+    using Cfg = GemmTcCfg<BN, APL, BPL>;
+    constexpr int BM = Cfg::BM, KC = Cfg::KC, STAGES = Cfg::STAGES;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // the swizzle needs 1024-byte alignment
+    uint64_t* bars = (uint64_t*)(base + STAGES * Cfg::STAGE);  // full[STAGES], empty[STAGES], done
+    uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 1);
+    const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.x * BM, split = blockIdx.z;
+    const int kbeg = split * g.klen, kend = min(g.K, kbeg + g.klen);
+    const int nchunks = kend > kbeg ? (kend - kbeg + KC - 1) / KC : 0;
+    constexpr uint32_t NBUILD = AMODE == A_PLANES ? 0u : 128u;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&bars[s], 1 + NBUILD); tc::mbar_init(&bars[STAGES + s], 1); }
+        tc::mbar_init(&bars[2 * STAGES], 1);
+        tc::mbar_fence_init();
+    }
+    if (wid == 2) tc::tmem_alloc(tmem_slot, BN);
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    bool ok = true;
+
+    if (wid == 0) {
+        if (lane == 0) {  // ---- TMA producer
+            for (int c = 0; c < nchunks && ok; ++c) {
+                const int s = c % STAGES, k0 = kbeg + c * KC;
+                if (c >= STAGES) ok = tc::mbar_wait(&bars[STAGES + s], ((c / STAGES) - 1) & 1);
+                if (!ok) break;
+                unsigned char* st = base + s * Cfg::STAGE;
+                constexpr uint32_t tx = (AMODE == A_PLANES ? APL * Cfg::A_PLANE : 0) + BPL * Cfg::B_PLANE;
+                tc::mbar_expect_tx(&bars[s], tx);
+                if (AMODE == A_PLANES) {
+#pragma unroll
+                    for (int bx = 0; bx < BM / 64; ++bx) {
+                        tc::tma_load_2d(st + bx * Cfg::BOX, &maps.a_hi, &bars[s], m0 + 64 * bx, k0);
+                        if (APL == 2) tc::tma_load_2d(st + Cfg::A_PLANE + bx * Cfg::BOX, &maps.a_lo, &bars[s], m0 + 64 * bx, k0);
+                    }
+                }
+                unsigned char* sb = st + APL * Cfg::A_PLANE;
+#pragma unroll
+                for (int bx = 0; bx < BN / 64; ++bx) {
+                    tc::tma_load_2d(sb + bx * Cfg::BOX, &maps.b_hi, &bars[s], 64 * bx, k0);
+                    if (BPL == 2) tc::tma_load_2d(sb + Cfg::B_PLANE + bx * Cfg::BOX, &maps.b_lo, &bars[s], 64 * bx, k0);
+                }
+            }
+            if (!ok) atomicOr(status, DEV_E_WAIT_TIMEOUT);
+        }
+    } else if (wid == 1) {
+        if (lane == 0) {  // ---- MMA issuer
+            const uint32_t idesc = tc::umma_idesc<PREC>(BM, BN, true, true);
+            for (int c = 0; c < nchunks && ok; ++c) {
+                const int s = c % STAGES;
+                ok = tc::mbar_wait(&bars[s], (c / STAGES) & 1);
+                if (!ok) break;
+                tc::tc_fence_after();
+                unsigned char* sa = base + s * Cfg::STAGE;
+                unsigned char* sb = sa + APL * Cfg::A_PLANE;
+#pragma unroll
+                for (int k16 = 0; k16 < KC / 16; ++k16) {
+                    // 16 k rows = two 8-row groups = 2048 bytes further into every box
+                    const uint64_t a_hi = tc::umma_desc(sa + k16 * 2048, Cfg::BOX, 1024);
+                    const uint64_t b_hi = tc::umma_desc(sb + k16 * 2048, Cfg::BOX, 1024);
+                    uint32_t accum = (c > 0 || k16 > 0) ? 1u : 0u;
+                    if (APL == 2) { tc::umma(tmem, tc::umma_desc(sa + Cfg::A_PLANE + k16 * 2048, Cfg::BOX, 1024), b_hi, idesc, accum); accum = 1u; }
+                    if (BPL == 2) { tc::umma(tmem, a_hi, tc::umma_desc(sb + Cfg::B_PLANE + k16 * 2048, Cfg::BOX, 1024), idesc, accum); accum = 1u; }
+                    tc::umma(tmem, a_hi, b_hi, idesc, accum);
+                }
+                tc::umma_commit(&bars[STAGES + s]);  // frees the stage when these MMAs are done
+            }
+            if (ok) tc::umma_commit(&bars[2 * STAGES]);
+            else atomicOr(status, DEV_E_WAIT_TIMEOUT);
+        }
+    } else {
+        // ---- warps 2-5: builders of a synthesized A tile, then the epilogue
+        const int bt = tid - 64;  // 0..127
+        if (AMODE != A_PLANES) {
+            // (after a timeout the loop keeps going without waiting, so that every thread still meets every bar.sync)
+            for (int c = 0; c < nchunks; ++c) {
+                const int s = c % STAGES, k0 = kbeg + c * KC;
+                if (ok && c >= STAGES) ok = tc::mbar_wait(&bars[STAGES + s], ((c / STAGES) - 1) & 1);
+                unsigned char* sa = base + s * Cfg::STAGE;
+                // element (k, m) of the tile lives in box m/64 at byte  k*128 + (((m%64)/8) ^ (k%8))*16 + (m%8)*2
+                uint4* z = reinterpret_cast<uint4*>(sa);
+                for (int i = bt; i < Cfg::A_PLANE / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
+                asm volatile("bar.sync 1, 128;" ::: "memory");  // zeros before ones
+                if (AMODE == A_ONEHOT) {
+                    if (bt < KC && k0 + bt < kend) {
+                        const int m = (int)g.idx[k0 + bt] - m0;
+                        if (m >= 0 && m < BM) {
+                            const int k = bt;
+                            const uint32_t off = (m >> 6) * Cfg::BOX + k * 128 + ((((m & 63) >> 3) ^ (k & 7)) << 4) + (m & 7) * 2;
+                            *reinterpret_cast<uint16_t*>(sa + off) = (uint16_t)one16<PREC>();
+                        }
+                    }
+                }
+                tc::fence_proxy_async();  // generic-proxy stores -> visible to the tensor core
+                tc::mbar_arrive(&bars[s]);
+            }
+            if (!ok && lane == 0) atomicOr(status, DEV_E_WAIT_TIMEOUT);
+        }
+        // epilogue: warp w reads accumulator lanes 32*(w%4)..+31 = output rows
+        bool got = true;
+        if (nchunks > 0) got = tc::mbar_wait(&bars[2 * STAGES], 0);
+        if (!got && lane == 0) atomicOr(status, DEV_E_WAIT_TIMEOUT);
+        tc::tc_fence_after();
+        __syncwarp();
+        const int q = wid & 3;
+        const int m = m0 + 32 * q + lane;
+        float* part = g.part + (size_t)split * g.stride + g.off;
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            if (nchunks > 0 && got) {
+                tc::tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, r);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;  // an empty K range contributes zeros
+            }
+            if (m < g.M && c0 < g.N) {
+                float4* dst = reinterpret_cast<float4*>(part + (size_t)m * g.ldc + c0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                                         __uint_as_float(r[4 * j + 3]));
+            }
+        }
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (wid == 2) tc::tmem_dealloc(tmem, BN);
+}
+
+template <int BN, int AMODE, int APL, int BPL, int PREC>
+static cudaError_t launch_t(const GemmTnArgs& g, int splits, int* status, cudaStream_t s) {
+    using Cfg = GemmTcCfg<BN, APL, BPL>;
+    GemmTcMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    const bool bf = PREC == 1;
+    if (AMODE == A_PLANES) {
+        if (!make_tensor_map_2d(&maps.a_hi, g.Ahi, (uint64_t)g.K, (uint64_t)g.lda, 64, bf)) return cudaErrorNotSupported;
+        if (APL == 2 && !make_tensor_map_2d(&maps.a_lo, g.Alo, (uint64_t)g.K, (uint64_t)g.lda, 64, bf)) return cudaErrorNotSupported;
+    }
+    if (!make_tensor_map_2d(&maps.b_hi, g.Bhi, (uint64_t)g.K, (uint64_t)g.ldb, 64, bf)) return cudaErrorNotSupported;
+    if (BPL == 2 && !make_tensor_map_2d(&maps.b_lo, g.Blo, (uint64_t)g.K, (uint64_t)g.ldb, 64, bf)) return cudaErrorNotSupported;
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_tn_tc<BN, AMODE, APL, BPL, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
+    if (e != cudaSuccess) return e;
+    dim3 grid((g.M + Cfg::BM - 1) / Cfg::BM, 1, splits);
+    k_gemm_tn_tc<BN, AMODE, APL, BPL, PREC><<<grid, Cfg::THREADS, Cfg::smem_bytes, s>>>(maps, g, status);
+    return cudaGetLastError();
+}
+
+template <int BN, int PREC>
+static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int splits, int* status, cudaStream_t s) {
+    constexpr int PL = PREC == 1 ? 1 : 2;
+    if (amode == A_PLANES) return launch_t<BN, A_PLANES, PL, PL, PREC>(g, splits, status, s);
+    if (amode == A_ONEHOT) return launch_t<BN, A_ONEHOT, 1, PL, PREC>(g, splits, status, s);
+    return cudaErrorNotSupported;
+}
+
+// Covered: N = ldb = 64, 128 or 256 (one CTA spans all output columns), klen a multiple of 64, A planes or one-hot A,
+// operand planes as the fp32 workloads (hi+lo fp16) or the bf16 workload (one plane) use them.
+cudaError_t launch_gemm_tn_tc(const GemmTnArgs& g, int amode, int apl, int bpl, int prec, int splits, int* status, cudaStream_t s) {
+    const int pl = prec == 1 ? 1 : 2;
+    if (g.N != g.ldb || g.klen % 64 != 0 || bpl != pl || (amode == A_PLANES && (apl != pl || g.lda % 64 != 0))) return cudaErrorNotSupported;
+    if (amode == A_ONEHOT && apl != 1) return cudaErrorNotSupported;
+    if (prec == 1) {
+        switch (g.N) {
+            case 64: return launch_bn<64, 1>(g, amode, splits, status, s);
+            case 128: return launch_bn<128, 1>(g, amode, splits, status, s);
+            case 256: return launch_bn<256, 1>(g, amode, splits, status, s);
+        }
+    } else {
+        switch (g.N) {
+            case 64: return launch_bn<64, 0>(g, amode, splits, status, s);
+            case 128: return launch_bn<128, 0>(g, amode, splits, status, s);
+            case 256: return launch_bn<256, 0>(g, amode, splits, status, s);
+        }
+    }
+    return cudaErrorNotSupported;
+}
+
+}  // namespace anakin

@@ -366,22 +366,6 @@ __global__ void __launch_bounds__(Dh1Cfg<H, BN, PREC>::THREADS, 1) k_dh1(LearnAr
 // ----------------------------------------------------------------------------------------------------
 // k_gemm_tn: C[m][n] = sum_k A[k][m] B[k][n], split-K partial outputs.
 // ----------------------------------------------------------------------------------------------------
-enum : int { A_PLANES = 0, A_ONEHOT = 1, A_WALLS = 2 };
-
-struct GemmTnArgs {
-    int M, N, K, klen;
-    const __nv_bfloat16 *Ahi, *Alo;  // A_PLANES: [K][lda]
-    int lda;
-    const uint8_t* idx;              // A_ONEHOT: A[k][m] = (idx[k] == m)
-    const uint32_t* walls;           // A_WALLS: A[k][m] = bit m of env k (m < ones_row), 1 for m == ones_row
-    int W, ones_row;
-    const __nv_bfloat16 *Bhi, *Blo;  // [K][ldb]
-    int ldb;
-    float* part;                     // out: part[split*stride + off + m*ldc + n]; row ones_row goes to off_ones + n
-    size_t stride, off, off_ones;
-    int ldc;
-};
-
 template <int BM, int BN, int AMODE, int APL, int BPL, int PREC>
 struct GemmTnCfg {
     static constexpr int BK = 32, STAGES = 3, THREADS = 256;
@@ -757,7 +741,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     const __nv_bfloat16* dh1hi = reinterpret_cast<const __nv_bfloat16*>(b.dh1);
     const __nv_bfloat16* Shi = reinterpret_cast<const __nv_bfloat16*>(b.S);
     constexpr int PL = PREC == 1 ? 1 : 2;
-    auto klen_of = [](int K, int ns) { return ((K + ns - 1) / ns + 31) / 32 * 32; };
+    auto klen_of = [](int K, int ns) { return ((K + ns - 1) / ns + 63) / 64 * 64; };
     GemmTnArgs g;
     memset(&g, 0, sizeof(g));
     // dW2 = h1^T dh2
@@ -767,8 +751,12 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     g.part = b.part + pl.off_w2; g.stride = (size_t)H * H; g.off = 0; g.ldc = H; g.ones_row = -1;
     {
         Scope sc(c, K_DW2);
-        if (H >= 128) CK((launch_gemm_tn<128, 128, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s)));
-        else CK((launch_gemm_tn<64, 64, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s)));
+        cudaError_t e = launch_gemm_tn_tc(g, A_PLANES, PL, PL, PREC, pl.ns_w2, b.status, s);  // tcgen05 where covered
+        if (e == cudaErrorNotSupported) {
+            if (H >= 128) e = launch_gemm_tn<128, 128, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s);
+            else e = launch_gemm_tn<64, 64, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s);
+        }
+        CK(e);
     }
     // dW1, agent plane = onehot(pos)^T dh1
     g.M = C; g.K = (int)R; g.klen = klen_of(g.K, pl.ns_agent);
@@ -777,8 +765,12 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     g.part = b.part + pl.off_agent; g.stride = CH; g.off = 0;
     {
         Scope sc(c, K_DW1_AGENT);
-        if (H >= 128) CK((launch_gemm_tn<128, 128, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s)));
-        else CK((launch_gemm_tn<64, 64, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s)));
+        cudaError_t e = launch_gemm_tn_tc(g, A_ONEHOT, 1, PL, PREC, pl.ns_agent, b.status, s);
+        if (e == cudaErrorNotSupported) {
+            if (H >= 128) e = launch_gemm_tn<128, 128, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s);
+            else e = launch_gemm_tn<64, 64, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s);
+        }
+        CK(e);
     }
     // dW1, wall plane (+ db1 through the all-ones row) = walls^T S; goal plane = onehot(goal)^T S
     g.K = B; g.klen = klen_of(g.K, pl.ns_env);
