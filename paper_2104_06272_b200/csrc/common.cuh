@@ -224,7 +224,8 @@ bool rollout_mma_supported(int H);
 cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
-cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c);  // needs the activations the rollout saved
+cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c);
+cudaError_t launch_dh1_tc(const LearnArgs& a, int prec, cudaStream_t s);  // tcgen05 dh1 kernel; cudaErrorNotSupported if not covered  // needs the activations the rollout saved
 cudaError_t launch_refresh_compute_params(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 
 }  // namespace anakin

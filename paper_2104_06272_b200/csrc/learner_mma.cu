@@ -729,7 +729,9 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     }
     {
         Scope sc(c, K_DH1);
-        switch (H) {
+        const cudaError_t etc = launch_dh1_tc(a, PREC, s);  // tcgen05 where covered, else the mma.sync kernel
+        if (etc != cudaErrorNotSupported) CK(etc);
+        else switch (H) {
             case 64: CK((launch_dh1_t<64, 64, PREC>(a, s))); break;
             case 128: CK((launch_dh1_t<128, 128, PREC>(a, s))); break;
             case 256: CK((launch_dh1_t<256, 128, PREC>(a, s))); break;
