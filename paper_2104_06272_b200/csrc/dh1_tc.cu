@@ -136,9 +136,17 @@ __global__ void __launch_bounds__(320, 1) k_dh1_tc(const __grid_constant__ Dh1Tc
         float s_acc[64];
 #pragma unroll
         for (int j = 0; j < 64; ++j) s_acc[j] = 0.f;
+        if (valid) {  // first two gate lines
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + (size_t)env * H + col0));
+            if (T > 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + ((size_t)B + env) * H + col0));
+        }
         for (int t = 0; t < T; ++t) {
             const int buf = t & 1;
             const size_t gi = ((size_t)t * B + (valid ? env : 0)) * H + col0;
+            // pull the gate line of step t+2 towards L2 now (one 128-byte line per thread), so that the load below
+            // costs an L2 hit by the time it is issued
+            if (valid && t + 2 < T)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + gi + (size_t)2 * B * H));
             // this row's layer-1 gates (64 units x 16 bit), fetched before the accumulator is waited for
             uint4 gate[8];
 #pragma unroll
