@@ -108,7 +108,7 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.dh2 = (float*)take(R * H * 4);
     b.dh1 = (float*)take(R * H * 4);
     b.dout = (float*)take(R * 8 * 4);
-    b.S = (float*)take(B * H * 4);
+    b.S = (float*)take(4 * B * H * 4);  // up to four t-slices of two 16-bit planes
     size_t part_floats = (size_t)NS * P, loss_blocks = LOSS_BLOCKS;
     if (rollout_mma_supported(d.H)) {
         LearnPlan pl;

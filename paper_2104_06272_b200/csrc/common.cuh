@@ -139,6 +139,7 @@ struct LearnArgs {
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
     // tensor-pipe path
+    int ts;               // t-slices of the dh1 kernel: S holds ts*B rows (slice z, env b at row z*B + b)
     float gscale, inv_gscale;  // power of two carried by every gradient-side tensor, divided out in the reduction
     float* part_small;    // per (CTA, row group) partials of dWh | db2 | dbh
     size_t small_stride;
@@ -202,8 +203,9 @@ struct GemmTnArgs {
     int M, N, K, klen;
     const __nv_bfloat16 *Ahi, *Alo;  // A_PLANES: [K][lda]
     int lda;
-    const uint8_t* idx;              // A_ONEHOT: A[k][m] = (idx[k] == m)
-    const uint32_t* walls;           // A_WALLS: A[k][m] = bit m of env k (m < ones_row), 1 for m == ones_row
+    const uint8_t* idx;              // A_ONEHOT: A[k][m] = (idx[k % kmod] == m)   (kmod = 0: idx[k])
+    int kmod;                        // rows of A repeat with this period (S holds several t-slices of B envs)
+    const uint32_t* walls;           // A_WALLS: A[k][m] = bit m of env k % kmod (m < ones_row), 1 for m == ones_row
     int W, ones_row;
     const __nv_bfloat16 *Bhi, *Blo;  // [K][ldb]
     int ldb;

@@ -55,6 +55,10 @@ __global__ void __launch_bounds__(320, 1) k_dh1_tc(const __grid_constant__ Dh1Tc
     const int e0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
     const size_t RH = (size_t)B * d.Tmax * H;
     int* status = b.status;
+    // this CTA's slice of the steps
+    const int tl = (T + a.ts - 1) / a.ts;
+    const int t0 = blockIdx.z * tl, t1 = min(T, t0 + tl);
+    const int nsteps = t1 > t0 ? t1 - t0 : 0;
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
@@ -67,7 +71,7 @@ __global__ void __launch_bounds__(320, 1) k_dh1_tc(const __grid_constant__ Dh1Tc
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const int nchunks = T * NCH;
+    const int nchunks = nsteps * NCH;
     bool ok = true;
 
     if (wid == 0) {
@@ -79,7 +83,7 @@ __global__ void __launch_bounds__(320, 1) k_dh1_tc(const __grid_constant__ Dh1Tc
                 if (PL == 2) tc::tma_load_2d(sW + (NCH + kc) * BOX, &maps.w_lo, wfull, kc * KC, n0);
             }
             for (int c = 0; c < nchunks && ok; ++c) {
-                const int s = c % STAGES, t = c / NCH, kc = c - t * NCH;
+                const int s = c % STAGES, u = c / NCH, kc = c - u * NCH, t = t0 + u;
                 if (c >= STAGES) ok = tc::mbar_wait(&empty[s], ((c / STAGES) - 1) & 1);
                 if (!ok) break;
                 tc::mbar_expect_tx(&full[s], Cfg::A_STAGE);
@@ -94,14 +98,14 @@ __global__ void __launch_bounds__(320, 1) k_dh1_tc(const __grid_constant__ Dh1Tc
         if (lane == 0) {  // ---- MMA issuer
             const uint32_t idesc = tc::umma_idesc<PREC>(BM, BN, false, false);
             ok = tc::mbar_wait(wfull, 0);
-            for (int t = 0; t < T && ok; ++t) {
-                const int buf = t & 1;
-                if (t >= 2) ok = tc::mbar_wait(&tempty[buf], ((t >> 1) - 1) & 1);  // epilogue of step t-2 has drained it
+            for (int u = 0; u < nsteps && ok; ++u) {
+                const int buf = u & 1;
+                if (u >= 2) ok = tc::mbar_wait(&tempty[buf], ((u >> 1) - 1) & 1);  // epilogue of step u-2 has drained it
                 if (!ok) break;
                 tc::tc_fence_after();
                 const uint32_t acc = tmem + (uint32_t)(buf * BN);
                 for (int kc = 0; kc < NCH && ok; ++kc) {
-                    const int c = t * NCH + kc, s = c % STAGES;
+                    const int c = u * NCH + kc, s = c % STAGES;
                     ok = tc::mbar_wait(&full[s], (c / STAGES) & 1);
                     if (!ok) break;
                     tc::tc_fence_after();
@@ -136,22 +140,22 @@ __global__ void __launch_bounds__(320, 1) k_dh1_tc(const __grid_constant__ Dh1Tc
         float s_acc[64];
 #pragma unroll
         for (int j = 0; j < 64; ++j) s_acc[j] = 0.f;
-        if (valid) {  // first two gate lines
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + (size_t)env * H + col0));
-            if (T > 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + ((size_t)B + env) * H + col0));
+        if (valid && nsteps > 0) {  // first two gate lines
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + ((size_t)t0 * B + env) * H + col0));
+            if (nsteps > 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + ((size_t)(t0 + 1) * B + env) * H + col0));
         }
-        for (int t = 0; t < T; ++t) {
-            const int buf = t & 1;
+        for (int t = t0; t < t1; ++t) {
+            const int u = t - t0, buf = u & 1;
             const size_t gi = ((size_t)t * B + (valid ? env : 0)) * H + col0;
             // pull the gate line of step t+2 towards L2 now (one 128-byte line per thread), so that the load below
             // costs an L2 hit by the time it is issued
-            if (valid && t + 2 < T)
+            if (valid && t + 2 < t1)
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(g_h1hi + gi + (size_t)2 * B * H));
             // this row's layer-1 gates (64 units x 16 bit), fetched before the accumulator is waited for
             uint4 gate[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) gate[j] = valid ? __ldg(reinterpret_cast<const uint4*>(g_h1hi + gi) + j) : make_uint4(0u, 0u, 0u, 0u);
-            if (ok) ok = tc::mbar_wait(&tfull[buf], (t >> 1) & 1);
+            if (ok) ok = tc::mbar_wait(&tfull[buf], (u >> 1) & 1);
             if (!ok) break;
             tc::tc_fence_after();
             uint32_t r0[32], r1[32];
@@ -191,8 +195,8 @@ __global__ void __launch_bounds__(320, 1) k_dh1_tc(const __grid_constant__ Dh1Tc
         // S (sum over t of dh1) as two 16-bit planes [B][H]: an fp32 sum keeps two terms in either workload
         if (valid) {
             uint16_t* S_hi = reinterpret_cast<uint16_t*>(b.S);
-            uint16_t* S_lo = S_hi + (size_t)B * H;
-            const size_t si = (size_t)env * H + col0;
+            uint16_t* S_lo = S_hi + (size_t)a.ts * B * H;
+            const size_t si = ((size_t)blockIdx.z * B + env) * H + col0;  // an empty slice writes zeros
             uint32_t phi[32], plo[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -236,7 +240,7 @@ static cudaError_t launch_t(const LearnArgs& a, cudaStream_t s) {
     }
     cudaError_t e = cudaFuncSetAttribute(k_dh1_tc<H, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
     if (e != cudaSuccess) return e;
-    dim3 grid((d.B + Cfg::BM - 1) / Cfg::BM, H / Cfg::BN);
+    dim3 grid((d.B + Cfg::BM - 1) / Cfg::BM, H / Cfg::BN, a.ts);
     k_dh1_tc<H, PREC><<<grid, Cfg::THREADS, Cfg::smem_bytes, s>>>(maps, a);
     return cudaGetLastError();
 }

@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
                 asm volatile("bar.sync 1, 128;" ::: "memory");  // zeros before ones
                 if (AMODE == A_ONEHOT) {
                     if (bt < KC && k0 + bt < kend) {
-                        const int m = (int)g.idx[k0 + bt] - m0;
+                        const int m = (int)g.idx[g.kmod ? (k0 + bt) % g.kmod : (k0 + bt)] - m0;
                         if (m >= 0 && m < BM) {
                             const int k = bt;
                             const uint32_t off = (m >> 6) * Cfg::BOX + k * 128 + ((((m & 63) >> 3) ^ (k & 7)) << 4) + (m & 7) * 2;

@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(256) k_gemm_tn(GemmTnArgs g) {
                 const int k = k0 + kk;
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
                 if (k < kend) {
-                    const int rel = (int)g.idx[k] - (m0 + mm);
+                    const int rel = (int)g.idx[g.kmod ? k % g.kmod : k] - (m0 + mm);
                     if (rel >= 0 && rel < 8) {
                         const uint32_t one = (rel & 1) ? (one16<PREC>() << 16) : one16<PREC>();
                         if ((rel >> 1) == 0) v.x = one; else if ((rel >> 1) == 1) v.y = one; else if ((rel >> 1) == 2) v.z = one; else v.w = one;
@@ -435,7 +435,7 @@ __global__ void __launch_bounds__(256) k_gemm_tn(GemmTnArgs g) {
                     for (int q = 0; q < 8; ++q) {
                         const int m = m0 + mm + q;
                         bool on = false;
-                        if (m < g.ones_row) on = (g.walls[(size_t)k * g.W + (m >> 5)] >> (m & 31)) & 1u;
+                        if (m < g.ones_row) on = (g.walls[(size_t)(g.kmod ? k % g.kmod : k) * g.W + (m >> 5)] >> (m & 31)) & 1u;
                         else if (m == g.ones_row) on = true;
                         if (on) w[q >> 1] |= (q & 1) ? (one16<PREC>() << 16) : one16<PREC>();
                     }
@@ -727,6 +727,16 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
             default: return cudaErrorNotSupported;
         }
     }
+    // t-slices: the tcgen05 dh1 kernel has ceil(B/128)*(H/128) CTAs per slice; slice the T steps so that one wave of
+    // CTAs covers the SMs.  The mma.sync fall-back keeps one slice.
+    a.ts = 1;
+    if (H == 128 || H == 256) {
+        const int per_slice = ((B + 127) / 128) * (H / 128);
+        int ts = 148 / per_slice;
+        if (ts > 4) ts = 4;
+        if (ts > T) ts = T;
+        if (ts >= 2) a.ts = ts;
+    }
     {
         Scope sc(c, K_DH1);
         const cudaError_t etc = launch_dh1_tc(a, PREC, s);  // tcgen05 where covered, else the mma.sync kernel
@@ -775,8 +785,8 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         CK(e);
     }
     // dW1, wall plane (+ db1 through the all-ones row) = walls^T S; goal plane = onehot(goal)^T S
-    g.K = B; g.klen = klen_of(g.K, pl.ns_env);
-    g.Bhi = Shi; g.Blo = Shi + (size_t)B * H;
+    g.K = a.ts * B; g.kmod = B; g.klen = klen_of(g.K, pl.ns_env);
+    g.Bhi = Shi; g.Blo = Shi + (size_t)a.ts * B * H;
     g.walls = b.walls; g.W = d.W; g.ones_row = C; g.M = C + 1;
     g.part = b.part + pl.off_walls; g.stride = (size_t)(C + 1) * H; g.off = 0; g.off_ones = CH;
     {
