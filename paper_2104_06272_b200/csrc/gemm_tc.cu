@@ -152,10 +152,10 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
                 if (ok && c >= STAGES) ok = tc::mbar_wait(&bars[STAGES + s], ((c / STAGES) - 1) & 1);
                 unsigned char* sa = base + s * Cfg::STAGE;
                 // element (k, m) of the tile lives in box m/64 at byte  k*128 + (((m%64)/8) ^ (k%8))*16 + (m%8)*2
-                uint4* z = reinterpret_cast<uint4*>(sa);
-                for (int i = bt; i < Cfg::A_PLANE / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
-                asm volatile("bar.sync 1, 128;" ::: "memory");  // zeros before ones
                 if (AMODE == A_ONEHOT) {
+                    uint4* z = reinterpret_cast<uint4*>(sa);
+                    for (int i = bt; i < Cfg::A_PLANE / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
+                    asm volatile("bar.sync 1, 128;" ::: "memory");  // zeros before ones
                     if (bt < KC && k0 + bt < kend) {
                         const int m = (int)g.idx[g.kmod ? (k0 + bt) % g.kmod : (k0 + bt)] - m0;
                         if (m >= 0 && m < BM) {
@@ -163,6 +163,25 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
                             const uint32_t off = (m >> 6) * Cfg::BOX + k * 128 + ((((m & 63) >> 3) ^ (k & 7)) << 4) + (m & 7) * 2;
                             *reinterpret_cast<uint16_t*>(sa + off) = (uint16_t)one16<PREC>();
                         }
+                    }
+                } else {  // A_WALLS: thread = (k row, 64-wide box); it writes all eight 16-byte chunks of its row segment
+                    const int k = bt >> 1, bx = bt & 1;
+                    const int kk = k0 + k;
+                    const uint32_t* wrow = g.walls + (size_t)(g.kmod ? kk % g.kmod : kk) * g.W;
+#pragma unroll
+                    for (int c8 = 0; c8 < 8; ++c8) {
+                        uint32_t w[4] = {0u, 0u, 0u, 0u};
+                        if (kk < kend) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                const int m = m0 + 64 * bx + 8 * c8 + q;
+                                bool on = false;
+                                if (m < g.ones_row) on = (wrow[m >> 5] >> (m & 31)) & 1u;
+                                else if (m == g.ones_row) on = true;
+                                if (on) w[q >> 1] |= (q & 1) ? (one16<PREC>() << 16) : one16<PREC>();
+                            }
+                        }
+                        *reinterpret_cast<uint4*>(sa + bx * Cfg::BOX + k * 128 + ((c8 ^ (k & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
                 tc::fence_proxy_async();  // generic-proxy stores -> visible to the tensor core
@@ -189,6 +208,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
             }
             if (m < g.M && c0 < g.N) {
                 float4* dst = reinterpret_cast<float4*>(part + (size_t)m * g.ldc + c0);
+                if (AMODE == A_WALLS && m == g.ones_row) dst = reinterpret_cast<float4*>(part - g.off + g.off_ones + c0);
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
@@ -225,6 +245,7 @@ static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int splits, int* st
     constexpr int PL = PREC == 1 ? 1 : 2;
     if (amode == A_PLANES) return launch_t<BN, A_PLANES, PL, PL, PREC>(g, splits, status, s);
     if (amode == A_ONEHOT) return launch_t<BN, A_ONEHOT, 1, PL, PREC>(g, splits, status, s);
+    if (amode == A_WALLS && g.M <= 128) return launch_t<BN, A_WALLS, 1, PL, PREC>(g, splits, status, s);
     return cudaErrorNotSupported;
 }
 
@@ -233,7 +254,7 @@ static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int splits, int* st
 cudaError_t launch_gemm_tn_tc(const GemmTnArgs& g, int amode, int apl, int bpl, int prec, int splits, int* status, cudaStream_t s) {
     const int pl = prec == 1 ? 1 : 2;
     if (g.N != g.ldb || g.klen % 64 != 0 || bpl != pl || (amode == A_PLANES && (apl != pl || g.lda % 64 != 0))) return cudaErrorNotSupported;
-    if (amode == A_ONEHOT && apl != 1) return cudaErrorNotSupported;
+    if (amode != A_PLANES && apl != 1) return cudaErrorNotSupported;
     if (prec == 1) {
         switch (g.N) {
             case 64: return launch_bn<64, 1>(g, amode, splits, status, s);

@@ -791,15 +791,23 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     g.part = b.part + pl.off_walls; g.stride = (size_t)(C + 1) * H; g.off = 0; g.off_ones = CH;
     {
         Scope sc(c, K_DW1_WALLS);
-        if (H >= 128) CK((launch_gemm_tn<128, 128, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s)));
-        else CK((launch_gemm_tn<64, 64, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s)));
+        cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_WALLS, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
+        if (e == cudaErrorNotSupported) {
+            if (H >= 128) e = launch_gemm_tn<128, 128, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
+            else e = launch_gemm_tn<64, 64, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
+        }
+        CK(e);
     }
     g.M = C; g.ones_row = -1; g.idx = b.goal;
     g.part = b.part + pl.off_goal; g.stride = CH;
     {
         Scope sc(c, K_DW1_GOAL);
-        if (H >= 128) CK((launch_gemm_tn<128, 128, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s)));
-        else CK((launch_gemm_tn<64, 64, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s)));
+        cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_ONEHOT, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
+        if (e == cudaErrorNotSupported) {
+            if (H >= 128) e = launch_gemm_tn<128, 128, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
+            else e = launch_gemm_tn<64, 64, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
+        }
+        CK(e);
     }
     {
         Scope sc(c, K_REDUCE_ADAM);
