@@ -105,6 +105,7 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.w2p_lo = rollout_mma_supported(d.H) ? (uint16_t*)take(H * H * 2) : nullptr;
     b.h1 = (float*)take(R * H * 4);
     b.h2 = (float*)take(R * H * 4);
+    b.out5 = rollout_mma_supported(d.H) ? (float*)take(R * 8 * 4) : nullptr;
     b.dh2 = (float*)take(R * H * 4);
     b.dh1 = (float*)take(R * H * 4);
     b.dout = (float*)take(R * 8 * 4);

@@ -68,6 +68,7 @@ struct Buffers {
     uint16_t* w2p_lo;
     float* h1;       // [R][H]
     float* h2;       // [R][H]
+    float* out5;     // [R][8] head outputs (4 logits, value) of every recorded row, saved by the tensor-pipe rollout
     float* dh2;      // [R][H]
     float* dh1;      // [R][H]
     float* dout;     // [R][8]  (5 used)

@@ -2,8 +2,8 @@
 // hidden sizes the tensor-pipe rollout covers.  The update reuses the policy's forward pass (Section 3.1): the rollout
 // kernel saved h1 (as bf16 hi/lo planes) and h2 for every recorded row, so the learner starts at the heads.
 //
-//   k_heads_bwd   flat 32-row tiles: heads -> softmax / loss terms -> dOut -> dh2 (fp32 FMA, HBM-bound).  Emits dh2 as
-//                 16-bit hi/lo planes and per-CTA partial sums of dWh, dbh, db2 and the loss terms.
+//   k_heads_bwd   flat 32-row tiles: saved head outputs -> softmax / loss terms -> dOut -> dh2 (fp32 FMA, HBM-bound).
+//                 Emits dh2 as 16-bit hi/lo planes and per-CTA partial sums of dWh, dbh, db2 and the loss terms.
 //   k_dh1         dh1 = (dh2 W2^T) gated by h1 > 0 with mma.sync; a CTA keeps its slice of W2 in shared memory and
 //                 walks t for 64 envs, so S = sum_t dh1 accumulates in registers.  Emits dh1 planes and S planes.
 //   k_gemm_tn     C[m][n] = sum_k A[k][m] B[k][n] with split-K partial outputs, bf16 hi/lo planes as operands and
@@ -25,158 +25,191 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
 
 // ----------------------------------------------------------------------------------------------------
-// k_heads_bwd: heads, softmax, loss terms, output gradients and dh2 for flat 32-row tiles (row i = t*B + env).
-// Persistent CTAs walk the tiles with a double-buffered cp.async stream of h2; everything is fp32 FMA.
-// HBM-bound: reads h2 (4 B/elt) and writes the dh2 planes (2 x 2 B/elt).
+// k_heads_bwd: softmax, loss terms, output gradients and dh2 for flat 32-row tiles (row i = t*B + env).
+// The head outputs (4 logits, value) of every row were saved by the rollout, so no h2 x Wh pass is needed here.
+// Persistent CTAs walk the tiles with a double-buffered cp.async stream of h2.  Per tile, every thread handles two
+// adjacent hidden units of 8 rows (dh2, running sums of dWh and db2) and then, for the NEXT tile, one thread per row
+// turns the saved head outputs into output gradients, so that the two phases of different warps overlap and one CTA
+// barrier per tile suffices.  HBM-bound in principle: reads h2 (4 B/elt), writes the dh2 planes (2 x 2 B/elt).
 // ----------------------------------------------------------------------------------------------------
 template <int H, int NW, int PREC>
 struct HeadsCfg {
-    static constexpr int TR = 32;               // rows per tile
-    static constexpr int PARTS = NW;            // threads per row in the heads phase
-    static constexpr int HP = H + PARTS;        // fp32 pitch of the h2 tile (bank skew between rows)
-    static constexpr size_t smem_bytes = (size_t)2 * TR * HP * 4 + (size_t)TR * 8 * 4 + (size_t)(H * 5 + 8) * 4 + (size_t)TR * 4 * 4;
+    static constexpr int TR = 32;  // rows per tile
+    static constexpr size_t smem_bytes = (size_t)2 * TR * H * 4 + (size_t)2 * TR * 8 * 4 + (size_t)TR * 8 * 4;
 };
 
 template <int H, int NW, int PREC>
 __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
     using Cfg = HeadsCfg<H, NW, PREC>;
-    constexpr int TR = Cfg::TR, HP = Cfg::HP, PARTS = Cfg::PARTS, NTHREADS = NW * 32, QN = H / PARTS;
+    constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = H / 2;
+    static_assert(NTHREADS / HP2 == 4, "four row groups of eight rows");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* s_h2 = reinterpret_cast<float*>(smem_raw);  // [2][TR][HP]
-    float* s_dout = s_h2 + 2 * TR * HP;                // [TR][8]
-    float* s_wh = s_dout + TR * 8;                     // [H][5]
-    float* s_bh = s_wh + H * 5;                        // [8]
-    float* s_loss = s_bh + 8;                          // [TR][4]
+    float* s_h2 = reinterpret_cast<float*>(smem_raw);  // [2][TR][H]
+    float* s_dout = s_h2 + 2 * TR * H;                 // [2][TR][8]
+    float* s_fin = s_dout + 2 * TR * 8;                // [TR][8] end-of-kernel reductions
     const Dims& d = a.d;
     const Buffers& b = a.b;
     const int tid = threadIdx.x;
     const size_t R = (size_t)d.B * a.T;
     const size_t RH = (size_t)d.B * d.Tmax * H;
-    uint16_t* g_dh2hi = reinterpret_cast<uint16_t*>(b.dh2);
-    uint16_t* g_dh2lo = g_dh2hi + RH;
+    uint32_t* g_dh2hi = reinterpret_cast<uint32_t*>(b.dh2);  // pairs of 16-bit elements
+    uint32_t* g_dh2lo = g_dh2hi + RH / 2;
     const float invR = a.gscale / (float)R;  // output gradients are carried times gscale
     const int ntiles = (int)((R + TR - 1) / TR);
 
-    for (int i = tid; i < H * 5; i += NTHREADS) s_wh[i] = b.theta_c[d.oWh + i];
-    if (tid < 5) s_bh[tid] = b.theta_c[d.obh + tid];
-    // heads phase: thread = (row hr, part hp); column phase: thread = (column cj, row group cg of 16 rows)
-    const int hr = tid / PARTS, hp = tid % PARTS;
-    const int cj = tid % H, cg = tid / H;
-    float wh_c[5];
+    // column phase: thread = (unit pair cp, row group rg of 8 rows); row phase: one thread per row
+    const int cp = tid % HP2, rg = tid / HP2;
+    const bool row_thread = (tid % NW) == 0;
+    const int rr = tid / NW;
+    float wh_c[2][5];
 #pragma unroll
-    for (int c = 0; c < 5; ++c) wh_c[c] = b.theta_c[d.oWh + cj * 5 + c];
-    float a_wh[5] = {0.f, 0.f, 0.f, 0.f, 0.f}, a_b2 = 0.f, a_bh = 0.f;  // running sums over this thread's rows
+    for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+        for (int c = 0; c < 5; ++c) wh_c[cc][c] = b.theta_c[d.oWh + (2 * cp + cc) * 5 + c];
+    float a_wh[2][5], a_b2[2] = {0.f, 0.f};
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc)
+#pragma unroll
+        for (int c = 0; c < 5; ++c) a_wh[cc][c] = 0.f;
+    float a_bh[5] = {0.f, 0.f, 0.f, 0.f, 0.f};  // row threads: sums of dOut over their rows
     float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
 
     auto load_tile = [&](int tile, int buf) {  // 16-byte chunks, zero-filled past the last row
-        float* dst = s_h2 + buf * TR * HP;
+        float* dst = s_h2 + buf * TR * H;
         for (int c = tid; c < TR * (H / 4); c += NTHREADS) {
             const int r = c / (H / 4), k = 4 * (c - r * (H / 4));
             const size_t row = (size_t)tile * TR + r;
             const bool ok = row < R;
-            cp_async16(dst + r * HP + k, b.h2 + (ok ? row : 0) * H + k, ok ? 16 : 0);
+            cp_async16(dst + r * H + k, b.h2 + (ok ? row : 0) * H + k, ok ? 16 : 0);
         }
         cp_async_commit();
     };
+    // Row phase, split in two so that the loads are in flight during the column phase.
+    struct RowIn { float4 o4; float v, adv, ret; int act; bool ok; };
+    auto row_load = [&](int tile) {
+        RowIn in;
+        const size_t i = (size_t)tile * TR + rr;
+        in.ok = tile < ntiles && i < R;
+        if (in.ok) {
+            in.o4 = *reinterpret_cast<const float4*>(b.out5 + i * 8);
+            in.v = b.out5[i * 8 + 4];
+            in.adv = b.adv[i];
+            in.ret = b.ret[i];
+            in.act = b.tact[i];
+        } else {
+            in.o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            in.v = in.adv = in.ret = 0.f;
+            in.act = 0;
+        }
+        return in;
+    };
+    auto row_finish = [&](const RowIn& in, int buf) {
+        float dO[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+        if (in.ok) {
+            const float o[4] = {in.o4.x, in.o4.y, in.o4.z, in.o4.w};
+            const float mx = fmaxf(fmaxf(o[0], o[1]), fmaxf(o[2], o[3]));
+            float ex[4], Z = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { ex[c] = expf(o[c] - mx); Z += ex[c]; }
+            const float logZ = logf(Z);
+            float p[4], lp[4], ent = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
+            const float A = in.adv;
+            const float err = in.v - in.ret;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                dO[c] = rnd<PREC>((-A * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
+            dO[4] = rnd<PREC>(2.f * a.c_v * err * invR);
+            l_pg += -A * (in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3]);
+            l_v += err * err;
+            l_ent += ent;
+#pragma unroll
+            for (int c = 0; c < 5; ++c) a_bh[c] += dO[c];
+        }
+        float4* o4 = reinterpret_cast<float4*>(s_dout + (buf * TR + rr) * 8);
+        o4[0] = make_float4(dO[0], dO[1], dO[2], dO[3]);
+        o4[1] = make_float4(dO[4], 0.f, 0.f, 0.f);
+    };
+
     int it = 0;
-    if ((int)blockIdx.x < ntiles) load_tile(blockIdx.x, 0);
+    if ((int)blockIdx.x < ntiles) {
+        load_tile(blockIdx.x, 0);
+        if (row_thread) row_finish(row_load(blockIdx.x), 0);
+    }
     for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
         const int buf = it & 1;
+        const int next = tile + (int)gridDim.x;
         cp_async_wait<0>();
-        __syncthreads();  // tile `tile` has landed; everyone is done with the other buffer
-        if (tile + (int)gridDim.x < ntiles) load_tile(tile + gridDim.x, buf ^ 1);
-        const float* h2t = s_h2 + buf * TR * HP;
-        // ---- heads, softmax, loss terms, output gradients
-        {
-            float o[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int q = 0; q < QN; ++q) {
-                const int j = hp + PARTS * q;
-                const float x = h2t[hr * HP + j];
-#pragma unroll
-                for (int c = 0; c < 5; ++c) o[c] = fmaf(x, s_wh[j * 5 + c], o[c]);
-            }
-#pragma unroll
-            for (int c = 0; c < 5; ++c) {
-#pragma unroll
-                for (int off = PARTS / 2; off > 0; off >>= 1) o[c] += __shfl_xor_sync(0xFFFFFFFFu, o[c], off);
-                o[c] += s_bh[c];
-            }
-            if (hp == 0) {
-                float dO[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-                const size_t i = (size_t)tile * TR + hr;
-                if (i < R) {
-                    const float mx = fmaxf(fmaxf(o[0], o[1]), fmaxf(o[2], o[3]));
-                    float ex[4], Z = 0.f;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) { ex[c] = expf(o[c] - mx); Z += ex[c]; }
-                    const float logZ = logf(Z);
-                    float p[4], lp[4], ent = 0.f;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
-                    const int act = b.tact[i];
-                    const float A = b.adv[i];
-                    const float err = o[4] - b.ret[i];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        dO[c] = rnd<PREC>((-A * ((c == act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
-                    dO[4] = rnd<PREC>(2.f * a.c_v * err * invR);
-                    l_pg += -A * (act == 0 ? lp[0] : act == 1 ? lp[1] : act == 2 ? lp[2] : lp[3]);
-                    l_v += err * err;
-                    l_ent += ent;
-                }
-                float4* o4 = reinterpret_cast<float4*>(s_dout + hr * 8);
-                o4[0] = make_float4(dO[0], dO[1], dO[2], dO[3]);
-                o4[1] = make_float4(dO[4], 0.f, 0.f, 0.f);
-            }
-        }
-        __syncthreads();
-        // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0, written as 16-bit planes; sums of dWh, db2, dbh
+        __syncthreads();  // this tile's h2 and dOut are in place; everyone is done with the other buffers
+        if (next < ntiles) load_tile(next, buf ^ 1);
+        RowIn nin;
+        if (row_thread) nin = row_load(next);
+        // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0, as 16-bit planes; running sums of dWh and db2
+        const float* h2t = s_h2 + buf * TR * H;
+        const float* dt = s_dout + buf * TR * 8;
 #pragma unroll 4
-        for (int r = 0; r < 16; ++r) {
-            const int e = cg * 16 + r;
+        for (int r = 0; r < 8; ++r) {
+            const int e = rg * 8 + r;
             const size_t i = (size_t)tile * TR + e;
-            const float4 d0 = *reinterpret_cast<const float4*>(s_dout + e * 8);
-            const float d4 = s_dout[e * 8 + 4];
-            const float h2 = h2t[e * HP + cj];
-            float back = d0.x * wh_c[0];
-            back = fmaf(d0.y, wh_c[1], back);
-            back = fmaf(d0.z, wh_c[2], back);
-            back = fmaf(d0.w, wh_c[3], back);
-            back = fmaf(d4, wh_c[4], back);
-            const float dh2 = rnd<PREC>(h2 > 0.f ? back : 0.f);
-            a_wh[0] = fmaf(h2, d0.x, a_wh[0]);
-            a_wh[1] = fmaf(h2, d0.y, a_wh[1]);
-            a_wh[2] = fmaf(h2, d0.z, a_wh[2]);
-            a_wh[3] = fmaf(h2, d0.w, a_wh[3]);
-            a_wh[4] = fmaf(h2, d4, a_wh[4]);
-            a_b2 += dh2;
-            if (cj < 5) a_bh += cj == 0 ? d0.x : cj == 1 ? d0.y : cj == 2 ? d0.z : cj == 3 ? d0.w : d4;
+            const float4 d0 = *reinterpret_cast<const float4*>(dt + e * 8);
+            const float d4 = dt[e * 8 + 4];
+            const float2 h2 = *reinterpret_cast<const float2*>(h2t + e * H + 2 * cp);
+            const float hv[2] = {h2.x, h2.y};
+            float dh[2];
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+                float back = d0.x * wh_c[cc][0];
+                back = fmaf(d0.y, wh_c[cc][1], back);
+                back = fmaf(d0.z, wh_c[cc][2], back);
+                back = fmaf(d0.w, wh_c[cc][3], back);
+                back = fmaf(d4, wh_c[cc][4], back);
+                dh[cc] = rnd<PREC>(hv[cc] > 0.f ? back : 0.f);
+                a_wh[cc][0] = fmaf(hv[cc], d0.x, a_wh[cc][0]);
+                a_wh[cc][1] = fmaf(hv[cc], d0.y, a_wh[cc][1]);
+                a_wh[cc][2] = fmaf(hv[cc], d0.z, a_wh[cc][2]);
+                a_wh[cc][3] = fmaf(hv[cc], d0.w, a_wh[cc][3]);
+                a_wh[cc][4] = fmaf(hv[cc], d4, a_wh[cc][4]);
+                a_b2[cc] += dh[cc];
+            }
             if (i < R) {
-                uint16_t hi16, lo16;
-                split1<PREC>(dh2, hi16, lo16);
-                g_dh2hi[i * H + cj] = hi16;
-                if (PREC == 0) g_dh2lo[i * H + cj] = lo16;
+                uint32_t phi, plo;
+                split2<PREC>(dh[0], dh[1], phi, plo);
+                g_dh2hi[(i * H) / 2 + cp] = phi;
+                if (PREC == 0) g_dh2lo[(i * H) / 2 + cp] = plo;
             }
         }
-        // the loop-top barrier orders these reads of the tile before the buffer is refilled
+        // ---- row phase of the next tile (its inputs were requested before the column phase)
+        if (row_thread && next < ntiles) row_finish(nin, buf ^ 1);
     }
     cp_async_wait<0>();
-    // ---- per-CTA results: dWh, db2, dbh partials (split index = 2*CTA + row group) and loss partials
+    // ---- per-CTA results: dWh, db2 partials (split index = 4*CTA + row group); dbh and loss partials
     {
-        float* part = a.part_small + (size_t)(2 * blockIdx.x + cg) * a.small_stride;
+        float* part = a.part_small + (size_t)(4 * blockIdx.x + rg) * a.small_stride;
 #pragma unroll
-        for (int c = 0; c < 5; ++c) part[(size_t)cj * 5 + c] = a_wh[c];
-        part[(size_t)H * 5 + cj] = a_b2;
-        if (cj < 5) part[(size_t)H * 6 + cj] = a_bh;
+        for (int cc = 0; cc < 2; ++cc) {
+#pragma unroll
+            for (int c = 0; c < 5; ++c) part[(size_t)(2 * cp + cc) * 5 + c] = a_wh[cc][c];
+            part[(size_t)H * 5 + 2 * cp + cc] = a_b2[cc];
+        }
     }
     __syncthreads();
-    if (hp == 0) { s_loss[hr * 4 + 0] = l_pg; s_loss[hr * 4 + 1] = l_v; s_loss[hr * 4 + 2] = l_ent; }
+    if (row_thread) {
+#pragma unroll
+        for (int c = 0; c < 5; ++c) s_fin[rr * 8 + c] = a_bh[c];
+        s_fin[rr * 8 + 5] = l_pg;
+        s_fin[rr * 8 + 6] = l_v;
+        s_fin[rr * 8 + 7] = l_ent;
+    }
     __syncthreads();
-    if (tid < 3) {
+    if (tid < 8) {  // rows in index order
         float s = 0.f;
-        for (int e = 0; e < TR; ++e) s += s_loss[e * 4 + tid];
-        b.loss_part[(size_t)blockIdx.x * 4 + tid] = s;
+        for (int e = 0; e < TR; ++e) s += s_fin[e * 8 + tid];
+        if (tid < 5) {
+            for (int q = 0; q < 4; ++q) a.part_small[(size_t)(4 * blockIdx.x + q) * a.small_stride + (size_t)H * 6 + tid] = q == 0 ? s : 0.f;
+        } else {
+            b.loss_part[(size_t)blockIdx.x * 4 + (tid - 5)] = s;
+        }
     }
 }
 
@@ -665,7 +698,7 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     p->ns_env = splits_for(d.B, tiles_ch, 128);
     const size_t tiles32 = (R + 31) / 32;
     p->heads_grid = (int)(tiles32 < (size_t)HEADS_GRID ? tiles32 : (size_t)HEADS_GRID);
-    p->ns_small = 2 * p->heads_grid;
+    p->ns_small = 4 * p->heads_grid;
     p->small_stride = (size_t)6 * H + 8;
     size_t off = 0;
     p->off_w2 = off; off += (size_t)p->ns_w2 * H * H;

@@ -226,21 +226,19 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
                             *reinterpret_cast<float2*>(b.h2 + ((size_t)t * B + e0 + row) * H + col0) =
                                 make_float2(acc[mt][j][2 * hh], acc[mt][j][2 * hh + 1]);
                     }
-                if (!a.replay) {
 #pragma unroll
-                    for (int cc = 0; cc < 2; ++cc) {
-                        float wh[5];
+                for (int cc = 0; cc < 2; ++cc) {
+                    float wh[5];
 #pragma unroll
-                        for (int c = 0; c < 5; ++c) wh[c] = s_wh[(col0 + cc) * 5 + c];
+                    for (int c = 0; c < 5; ++c) wh[c] = s_wh[(col0 + cc) * 5 + c];
 #pragma unroll
-                        for (int mt = 0; mt < 2; ++mt)
+                    for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-                            for (int hh = 0; hh < 2; ++hh) {
-                                const float h2 = acc[mt][j][2 * hh + cc];
+                        for (int hh = 0; hh < 2; ++hh) {
+                            const float h2 = acc[mt][j][2 * hh + cc];
 #pragma unroll
-                                for (int c = 0; c < 5; ++c) ps[2 * mt + hh][c] = fmaf(h2, wh[c], ps[2 * mt + hh][c]);
-                            }
-                    }
+                            for (int c = 0; c < 5; ++c) ps[2 * mt + hh][c] = fmaf(h2, wh[c], ps[2 * mt + hh][c]);
+                        }
                 }
             }
 #pragma unroll
@@ -261,7 +259,7 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
         }
         __syncthreads();
         // ---- one thread per env: fixed-order sum of the warps' partials, then act and step
-        if (owner && !a.replay) {
+        if (owner) {
             float o[5];
 #pragma unroll
             for (int c = 0; c < 5; ++c) o[c] = 0.f;
@@ -271,10 +269,17 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
 #pragma unroll
             for (int c = 0; c < 5; ++c) o[c] += s_bh[c];
             const int env = e0 + tid;
-            b.tval[(size_t)t * B + env] = o[4];
-            if (t < a.T) {
-                act_and_step(s, a, env, t, o[0], o[1], o[2], o[3], s_walls + tid * 8);
-                s_pos[tid] = s.pos;
+            if (b.out5 && t < a.T) {  // the update reuses the head outputs of every recorded row
+                float4* o5 = reinterpret_cast<float4*>(b.out5 + ((size_t)t * B + env) * 8);
+                o5[0] = make_float4(o[0], o[1], o[2], o[3]);
+                o5[1] = make_float4(o[4], 0.f, 0.f, 0.f);
+            }
+            if (!a.replay) {
+                b.tval[(size_t)t * B + env] = o[4];
+                if (t < a.T) {
+                    act_and_step(s, a, env, t, o[0], o[1], o[2], o[3], s_walls + tid * 8);
+                    s_pos[tid] = s.pos;
+                }
             }
         }
         __syncthreads();
