@@ -144,28 +144,38 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
             if (tid < ME) s_pos[tid] = owner ? b.tpos[(size_t)t * B + e0 + tid] : 0;
             __syncthreads();
         }
-        // ---- layer 1: pairs of consecutive hidden units per thread
-        for (int p = tid; p < ME * H / 2; p += NTHREADS) {
-            const int e = p / (H / 2), k = 2 * (p - e * (H / 2));
-            const float2 bs = *reinterpret_cast<const float2*>(s_base + e * H + k);
-            const float2 w = __ldg(reinterpret_cast<const float2*>(W1 + (size_t)(C + s_pos[e]) * H + k));
-            const float z0 = fmaxf(bs.x + w.x, 0.f), z1 = fmaxf(bs.y + w.y, 0.f);
-            uint32_t phi, plo;
-            split2<PREC>(z0, z1, phi, plo);
-            if (PREC == 0) *reinterpret_cast<uint32_t*>(s_h1lo + e * LD + k) = plo;
-            *reinterpret_cast<uint32_t*>(s_h1hi + e * LD + k) = phi;
-        }
-        __syncthreads();
-        if (b.h1 && t < a.T) {  // save the h1 planes, 16 bytes per thread per trip, coalesced
-            for (int c = tid; c < ME * (H / 8); c += NTHREADS) {
-                const int e = c / (H / 8), k = 8 * (c - e * (H / 8));
-                if (e0 + e < B) {
+        // ---- layer 1: pairs of consecutive hidden units per thread.  All gathers of the agent's W1 row are issued
+        // before any is used (one L2 round trip per step, not one per trip); the fp16 planes go to shared memory for
+        // the MMAs and, for the update's reuse, straight to global memory (4 bytes per lane, 128 bytes per warp).
+        {
+            constexpr int TRIPS = ME * H / 2 / NTHREADS;
+            static_assert(TRIPS * NTHREADS == ME * H / 2, "layer-1 trips must tile the h1 block");
+            const bool save_h1 = b.h1 != nullptr && t < a.T;
+            float2 w[TRIPS];
+#pragma unroll
+            for (int i = 0; i < TRIPS; ++i) {
+                const int p = tid + i * NTHREADS;
+                const int e = p / (H / 2), k = 2 * (p - e * (H / 2));
+                w[i] = __ldg(reinterpret_cast<const float2*>(W1 + (size_t)(C + s_pos[e]) * H + k));
+            }
+#pragma unroll
+            for (int i = 0; i < TRIPS; ++i) {
+                const int p = tid + i * NTHREADS;
+                const int e = p / (H / 2), k = 2 * (p - e * (H / 2));
+                const float2 bs = *reinterpret_cast<const float2*>(s_base + e * H + k);
+                const float z0 = fmaxf(bs.x + w[i].x, 0.f), z1 = fmaxf(bs.y + w[i].y, 0.f);
+                uint32_t phi, plo;
+                split2<PREC>(z0, z1, phi, plo);
+                if (PREC == 0) *reinterpret_cast<uint32_t*>(s_h1lo + e * LD + k) = plo;
+                *reinterpret_cast<uint32_t*>(s_h1hi + e * LD + k) = phi;
+                if (save_h1 && e0 + e < B) {
                     const size_t gi = ((size_t)t * B + e0 + e) * H + k;
-                    *reinterpret_cast<uint4*>(g_h1hi + gi) = *reinterpret_cast<const uint4*>(s_h1hi + e * LD + k);
-                    if (PREC == 0) *reinterpret_cast<uint4*>(g_h1lo + gi) = *reinterpret_cast<const uint4*>(s_h1lo + e * LD + k);
+                    *reinterpret_cast<uint32_t*>(g_h1hi + gi) = phi;
+                    if (PREC == 0) *reinterpret_cast<uint32_t*>(g_h1lo + gi) = plo;
                 }
             }
         }
+        __syncthreads();
         // ---- layer 2 on the tensor pipe: acc[mt][j] = rows 16mt.. x columns 8(wid*NT+j)..
         float acc[2][NT][4];
 #pragma unroll
