@@ -87,23 +87,45 @@ __device__ __forceinline__ void flush_env_stats(EnvLane& s, const RolloutArgs& a
     }
 }
 
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(gsrc), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
 // GAE reverse scan of one env (explicit rounding intrinsics: the standalone kernel and the fused learner agree bitwise):
 //   d_t = 1 - done_t; delta_t = r_t + gamma d_t V_{t+1} - V_t; A_t = delta_t + gamma lambda d_t A_{t+1}; ret_t = A_t + V_t
 __device__ __forceinline__ void gae_scan_env(const Buffers& b, int B, int T, int env, float gamma, float lambda) {
     float A = 0.f;
     float vnext = b.tval[(size_t)T * B + env];
     const float gl = __fmul_rn(gamma, lambda);
-#pragma unroll 4
-    for (int t = T - 1; t >= 0; --t) {
-        const size_t i = (size_t)t * B + env;
-        const float v = b.tval[i];
-        const float r = b.trew[i];
-        const float nd = b.tdone[i] ? 0.f : 1.f;
-        const float delta = __fsub_rn(__fmaf_rn(__fmul_rn(gamma, nd), vnext, r), v);
-        A = __fmaf_rn(__fmul_rn(gl, nd), A, delta);
-        b.adv[i] = A;
-        b.ret[i] = __fadd_rn(A, v);
-        vnext = v;
+    // eight steps at a time: all loads of a chunk are issued before its stores, so the scan pays one memory round trip
+    // per chunk instead of one per step
+    for (int tb = T; tb > 0; tb -= 8) {
+        float v[8], r[8], nd[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int t = tb - 1 - q;
+            if (t >= 0) {
+                const size_t i = (size_t)t * B + env;
+                v[q] = b.tval[i];
+                r[q] = b.trew[i];
+                nd[q] = b.tdone[i] ? 0.f : 1.f;
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int t = tb - 1 - q;
+            if (t >= 0) {
+                const size_t i = (size_t)t * B + env;
+                const float delta = __fsub_rn(__fmaf_rn(__fmul_rn(gamma, nd[q]), vnext, r[q]), v[q]);
+                A = __fmaf_rn(__fmul_rn(gl, nd[q]), A, delta);
+                b.adv[i] = A;
+                b.ret[i] = __fadd_rn(A, v[q]);
+                vnext = v[q];
+            }
+        }
     }
 }
 

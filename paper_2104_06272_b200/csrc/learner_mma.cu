@@ -17,13 +17,6 @@
 
 namespace anakin {
 
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(d), "l"(gsrc), "r"(src_bytes));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
-
 // ----------------------------------------------------------------------------------------------------
 // k_heads_bwd: softmax, loss terms, output gradients and dh2 for flat 32-row tiles (row i = t*B + env).
 // The head outputs (4 logits, value) of every row were saved by the rollout, so no h2 x Wh pass is needed here.

@@ -99,15 +99,14 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
     const float* W1 = b.theta_c + d.oW1;
 
     // ---- prologue: weights and per-env constants on chip
-    {
-        const uint4* src = reinterpret_cast<const uint4*>(b.w2f_hi);
-        uint4* dst = reinterpret_cast<uint4*>(s_w2hi);
-        for (int i = tid; i < H * H * 2 / 16; i += NTHREADS) dst[i] = src[i];
+    // asynchronous copies: every 16-byte chunk is in flight at once, nothing is staged in registers
+    for (int i = tid; i < H * H * 2 / 16; i += NTHREADS) cp_async16(reinterpret_cast<uint4*>(s_w2hi) + i, reinterpret_cast<const uint4*>(b.w2f_hi) + i, 16);
+    for (int i = tid; i < ME * H / 4; i += NTHREADS) {
+        const int e = i / (H / 4), j = 4 * (i - e * (H / 4));
+        const bool ok = e0 + e < B;
+        cp_async16(s_base + e * H + j, b.base + (size_t)(ok ? e0 + e : 0) * H + j, ok ? 16 : 0);
     }
-    for (int i = tid; i < ME * H; i += NTHREADS) {
-        const int e = i / H, j = i - e * H;
-        s_base[i] = (e0 + e < B) ? b.base[(size_t)(e0 + e) * H + j] : 0.f;
-    }
+    cp_async_commit();
     for (int i = tid; i < H * 5; i += NTHREADS) s_wh[i] = b.theta_c[d.oWh + i];
     for (int i = tid; i < H; i += NTHREADS) s_b2[i] = b.theta_c[d.ob2 + i];
     if (tid < 5) s_bh[tid] = b.theta_c[d.obh + tid];
@@ -133,6 +132,7 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
         }
         s_pos[tid] = s.pos;
     }
+    cp_async_wait<0>();
     __syncthreads();
 
     // Saved activations (the update reuses the policy's forward pass: Section 3.1): row i = t*B + env.
