@@ -87,7 +87,7 @@ class ClockSampler:
 
 
 def workload_label(w):
-    return (f"throughput: B={w.B} envs, {w.N}x{w.N} gridworld (obs {w.D}), MLP {w.D}-{w.H}-{w.H}+5, "
+    return (f"{w.name}: B={w.B} envs, {w.N}x{w.N} gridworld (obs {w.D}), MLP {w.D}-{w.H}-{w.H}+5, "
             f"{'fp32' if w.precision == 0 else 'bf16'}, T={w.T}")
 
 
@@ -120,6 +120,25 @@ def kernel_work(w):
     }
 
 
+def max_over_ranks(value: float, world: int, device="cpu") -> float:
+    """The slowest rank's value (the time every multi-GPU number is reported on).  Works on any backend: the tensor
+    lives on `device` ("cuda" under NCCL, "cpu" under gloo)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_frames_per_sec(frames_per_rank: float, world: int, max_seconds: float) -> float:
+    """Replicas only: every rank processes frames_per_rank frames of its own; the job's rate is the sum over ranks
+    divided by the slowest rank's time."""
+    return frames_per_rank * world / max_seconds
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -136,7 +155,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    w = WORKLOADS["throughput"]
+    w = WORKLOADS[args.workload]
     peaks = load_peaks()
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
@@ -174,13 +193,8 @@ def run_ours(args):
     launches = an.launch_count() - n0
     clocks = sampler.stop() if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = float(sum(step_ms))
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    frames = float(w.B) * w.T * K * world
-    value = frames / (total_ms * 1e-3)
+    total_ms = max_over_ranks(float(sum(step_ms)), world, "cuda")
+    value = whole_job_frames_per_sec(float(w.B) * w.T * K, world, total_ms * 1e-3)
 
     # ---- per-kernel pass (events around every launch), same K steps, for the roofline entry
     an.profile_enable(True)
@@ -213,11 +227,8 @@ def run_ours(args):
         h_theta.copy_(h_out)
     barrier()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = float(w.B) * w.T * Ke * world / e2e_s
+    e2e_s = max_over_ranks(e2e_s, world, "cuda")
+    e2e_value = whole_job_frames_per_sec(float(w.B) * w.T * Ke, world, e2e_s)
     assert np.isfinite(st.loss_total) and an.status() == 0
 
     if rank != 0:
@@ -259,13 +270,18 @@ def run_ours(args):
                 "share_of_step": top_ms / tot,
                 "kernels": {k: kernel_line(k, ms, n) for k, (ms, n) in sorted(prof.items(), key=lambda kv: -kv[1][0])}}
 
-    # ---- the oracle on the host cores, bounded sample of the same workload
-    cpu = cpu_baseline(w, iters=2)
+    # ---- the oracle on the host cores, bounded sample of the same workload (about 10-30 s of CPU work)
+    if args.workload == "throughput":
+        cpu = cpu_baseline(w, iters=2)
+    else:
+        mac_per_frame = 3.0 * (w.D * w.H + w.H * w.H + 5 * w.H) + w.H * w.H
+        frames = 5.0e11 / mac_per_frame
+        cpu = cpu_baseline(w, iters=1, B=int(max(16, min(w.B, frames / w.T))))
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": "bf16" if w.precision == 1 else "f32", "data": "synthetic",
         "config": {"workload": workload_label(w), "frames_per_step": w.B * w.T, "seed": seed,
                    "l2": "flushed between timed steps (256 MiB write outside the event brackets)",
                    "multi_gpu": "replicas only" if world > 1 else "single GPU"},
@@ -331,6 +347,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="throughput", choices=list(WORKLOADS),
+                    help="the metric is quoted on 'throughput'; the others are for the per-workload table")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

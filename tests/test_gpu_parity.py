@@ -36,6 +36,13 @@ SMALL = {
     "one_env": Workload("one_env", B=1, N=2, H=32, T=1, iters=1, episode_cap=1, wall_density=0.0),
     "dense_walls": Workload("dense_walls", B=130, N=16, H=32, T=9, iters=1, episode_cap=255, wall_density=0.9),
     "ragged_bf16": Workload("ragged_bf16", B=45, N=6, H=192, T=7, iters=1, precision=1, episode_cap=4),
+    # ragged shapes on the tensor-pipe path (H in {64, 128, 256}): batch tails, T not a multiple of the t-slices,
+    # grids whose cell count is not a multiple of 32, the bf16 operand format
+    "tp_ragged_128": Workload("tp_ragged_128", B=333, N=9, H=128, T=11, iters=1, episode_cap=7),
+    "tp_ragged_256": Workload("tp_ragged_256", B=150, N=12, H=256, T=7, iters=1, episode_cap=9, wall_density=0.35),
+    "tp_ragged_64": Workload("tp_ragged_64", B=97, N=3, H=64, T=3, iters=1, episode_cap=2),
+    "tp_bf16_128": Workload("tp_bf16_128", B=210, N=7, H=128, T=6, iters=1, precision=1, episode_cap=5),
+    "tp_bf16_256": Workload("tp_bf16_256", B=131, N=16, H=256, T=5, iters=1, precision=1),
 }
 
 
