@@ -97,21 +97,22 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.dbg_logits = c.debug_logits ? (float*)take(R * 16) : nullptr;
     b.dbg_gates = c.debug_logits ? (uint32_t*)take(2 * R * (H / 32) * 4) : nullptr;
     b.base = (float*)take(B * H * 4);
-    b.w2f_hi = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
-    b.w2f_lo = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
-    b.w2tf_hi = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
-    b.w2tf_lo = rollout_mma_supported(d.H) ? (uint2*)take(H * H * 2) : nullptr;
-    b.w2p_hi = rollout_mma_supported(d.H) ? (uint16_t*)take(H * H * 2) : nullptr;
-    b.w2p_lo = rollout_mma_supported(d.H) ? (uint16_t*)take(H * H * 2) : nullptr;
+    const bool mma = rollout_mma_supported(d.H), tensor = tensor_path_supported(d.H, c.precision);
+    b.w2f_hi = mma ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2f_lo = mma ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2tf_hi = mma ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2tf_lo = mma ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2p_hi = tensor ? (uint16_t*)take(H * H * 2) : nullptr;
+    b.w2p_lo = mma ? (uint16_t*)take(H * H * 2) : nullptr;
     b.h1 = (float*)take(R * H * 4);
     b.h2 = (float*)take(R * H * 4);
-    b.out5 = rollout_mma_supported(d.H) ? (float*)take(R * 8 * 4) : nullptr;
+    b.out5 = tensor ? (float*)take(R * 8 * 4) : nullptr;
     b.dh2 = (float*)take(R * H * 4);
     b.dh1 = (float*)take(R * H * 4);
     b.dout = (float*)take(R * 8 * 4);
     b.S = (float*)take(4 * B * H * 4);  // up to four t-slices of two 16-bit planes
     size_t part_floats = (size_t)NS * P, loss_blocks = LOSS_BLOCKS;
-    if (rollout_mma_supported(d.H)) {
+    if (tensor) {
         LearnPlan pl;
         learn_mma_plan(d, &pl);
         if (pl.part_floats > part_floats) part_floats = pl.part_floats;
@@ -169,6 +170,12 @@ Blob blob_of(anakin_t* h, int which) {
     }
 }
 
+// 16-bit copies of W2 in the layouts the tensor-core kernels read.
+cudaError_t pack_w2(anakin_t* h) {
+    if (wide_supported(h->d.H, h->cfg.precision)) return launch_pack_w2_wide(h->d, h->b, h->ctx());
+    return launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+}
+
 int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     if (!h) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset) return ANAKIN_E_BAD_STATE;
@@ -180,7 +187,7 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
         h->base_valid = true;
     }
     if (!h->frags_valid) {
-        e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+        e = pack_w2(h);
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->frags_valid = true;
     }
@@ -202,7 +209,7 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     h->gstep += T;
     h->last_T = T;
     h->rollout_pending = true;
-    h->acts_valid = rollout_mma_supported(h->d.H);  // the tensor-pipe rollout saved h1 and h2 of every row
+    h->acts_valid = tensor_path_supported(h->d.H, h->cfg.precision);  // the tensor-core rollouts save h1 and h2 of every row
     h->adv_valid = a.fuse_gae != 0;
     return ANAKIN_OK;
 }
@@ -216,7 +223,7 @@ int replay_activations(anakin_t* h) {
         h->base_valid = true;
     }
     if (!h->frags_valid) {
-        e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+        e = pack_w2(h);
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->frags_valid = true;
     }
@@ -231,7 +238,9 @@ int replay_activations(anakin_t* h) {
     a.replay = 1;
     a.fuse_gae = 0;
     a.gamma = a.lambda = 0.f;
-    {
+    if (wide_supported(h->d.H, h->cfg.precision)) {
+        e = launch_rollout_wide(a, h->ctx());
+    } else {
         Scope sc(h->ctx(), K_REPLAY);
         e = launch_rollout_mma(a, h->cfg.precision, h->stream);
     }
@@ -339,7 +348,7 @@ static int learn_after_gae(anakin_t* h) {
         h->base_valid = true;
     }
     if (!h->frags_valid) {
-        e = launch_pack_w2(h->d, h->b, h->cfg.precision, h->ctx());
+        e = pack_w2(h);
         if (e != cudaSuccess) return fail_cuda(h, e);
         h->frags_valid = true;
     }
@@ -362,7 +371,7 @@ static int learn_after_gae(anakin_t* h) {
         a.gscale = (float)ldexp(1.0, ex);
         a.inv_gscale = (float)ldexp(1.0, -ex);
     }
-    if (rollout_mma_supported(h->d.H)) {
+    if (tensor_path_supported(h->d.H, h->cfg.precision)) {
         if (!h->acts_valid) {
             const int rc = replay_activations(h);
             if (rc != ANAKIN_OK) return rc;
@@ -375,7 +384,7 @@ static int learn_after_gae(anakin_t* h) {
     h->adam_k += 1;
     h->adv_valid = false;
     h->base_valid = false;  // parameters changed
-    h->frags_valid = rollout_mma_supported(h->d.H);  // the tensor-pipe update refreshes the fragment copies itself
+    h->frags_valid = tensor_path_supported(h->d.H, h->cfg.precision);  // the tensor-core update refreshes the 16-bit copies itself
     h->acts_valid = false;
     h->rollout_pending = false;
     return ANAKIN_OK;

@@ -224,6 +224,11 @@ cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c);
 cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c);
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s);  // cudaErrorNotSupported if not covered
 bool rollout_mma_supported(int H);
+bool wide_supported(int H, int prec);         // bf16 workload with a hidden layer too wide for the persistent rollout
+bool tensor_path_supported(int H, int prec);  // either tensor-core path: the update reuses activations the rollout saved
+cudaError_t launch_rollout_wide(const RolloutArgs& a, const Ctx& c);  // T+1 forward passes, or the replay of recorded rows
+cudaError_t launch_pack_w2_wide(const Dims& d, const Buffers& b, const Ctx& c);
+cudaError_t launch_dh1_wide(const LearnArgs& a, const Ctx& c);
 cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);

@@ -4,7 +4,8 @@
 // Podracer paper, Section 3.1): dW2 = h1^T dh2 and the agent plane of dW1 = onehot(pos)^T dh1.  Both operands have the
 // contraction index as their slow (row) index, i.e. they are "MN-major" for the MMA.
 //
-// One CTA owns a 128 x BN output tile (BN = the hidden width, up to 256 accumulator columns in tensor memory) and a
+// One CTA owns a 128 x BN output tile (BN = the hidden width up to 256, else column tiles of 256; the accumulator
+// columns live in tensor memory) and a
 // K range (split-K; partials are summed later in a fixed order).  Per 64-row K chunk:
 //   warp 0 (one lane)  issues TMA loads of the operand planes (64 x 64 boxes, 128-byte swizzle) into a 2-stage ring,
 //   warps 2-5          for the one-hot A operand: write the 0/1 tile straight into the swizzled layout instead of loading it,
@@ -75,7 +76,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
     uint64_t* bars = (uint64_t*)(base + STAGES * Cfg::STAGE);  // full[STAGES], empty[STAGES], done
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 1);
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.x * BM, split = blockIdx.z;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, split = blockIdx.z;
     const int kbeg = split * g.klen, kend = min(g.K, kbeg + g.klen);
     const int nchunks = kend > kbeg ? (kend - kbeg + KC - 1) / KC : 0;
     constexpr uint32_t NBUILD = AMODE == A_PLANES ? 0u : 128u;
@@ -111,8 +112,8 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
                 unsigned char* sb = st + APL * Cfg::A_PLANE;
 #pragma unroll
                 for (int bx = 0; bx < BN / 64; ++bx) {
-                    tc::tma_load_2d(sb + bx * Cfg::BOX, &maps.b_hi, &bars[s], 64 * bx, k0);
-                    if (BPL == 2) tc::tma_load_2d(sb + Cfg::B_PLANE + bx * Cfg::BOX, &maps.b_lo, &bars[s], 64 * bx, k0);
+                    tc::tma_load_2d(sb + bx * Cfg::BOX, &maps.b_hi, &bars[s], n0 + 64 * bx, k0);
+                    if (BPL == 2) tc::tma_load_2d(sb + Cfg::B_PLANE + bx * Cfg::BOX, &maps.b_lo, &bars[s], n0 + 64 * bx, k0);
                 }
             }
             if (!ok) atomicOr(status, DEV_E_WAIT_TIMEOUT);
@@ -206,9 +207,9 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
 #pragma unroll
                 for (int j = 0; j < 32; ++j) r[j] = 0u;  // an empty K range contributes zeros
             }
-            if (m < g.M && c0 < g.N) {
-                float4* dst = reinterpret_cast<float4*>(part + (size_t)m * g.ldc + c0);
-                if (AMODE == A_WALLS && m == g.ones_row) dst = reinterpret_cast<float4*>(part - g.off + g.off_ones + c0);
+            if (m < g.M && n0 + c0 < g.N) {
+                float4* dst = reinterpret_cast<float4*>(part + (size_t)m * g.ldc + n0 + c0);
+                if (AMODE == A_WALLS && m == g.ones_row) dst = reinterpret_cast<float4*>(part - g.off + g.off_ones + n0 + c0);
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
@@ -235,7 +236,7 @@ static cudaError_t launch_t(const GemmTnArgs& g, int splits, int* status, cudaSt
     if (BPL == 2 && !make_tensor_map_2d(&maps.b_lo, g.Blo, (uint64_t)g.K, (uint64_t)g.ldb, 64, bf)) return cudaErrorNotSupported;
     cudaError_t e = cudaFuncSetAttribute(k_gemm_tn_tc<BN, AMODE, APL, BPL, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
     if (e != cudaSuccess) return e;
-    dim3 grid((g.M + Cfg::BM - 1) / Cfg::BM, 1, splits);
+    dim3 grid((g.M + Cfg::BM - 1) / Cfg::BM, (g.N + BN - 1) / BN, splits);
     k_gemm_tn_tc<BN, AMODE, APL, BPL, PREC><<<grid, Cfg::THREADS, Cfg::smem_bytes, s>>>(maps, g, status);
     return cudaGetLastError();
 }
@@ -249,20 +250,21 @@ static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int splits, int* st
     return cudaErrorNotSupported;
 }
 
-// Covered: N = ldb = 64, 128 or 256 (one CTA spans all output columns), klen a multiple of 64, A planes or one-hot A,
+// Covered: N = ldb = 64, 128, 256 or a multiple of 256 (column tiles of 256 on grid.y), klen a multiple of 64, A planes or one-hot A,
 // operand planes as the fp32 workloads (hi+lo fp16) or the bf16 workload (one plane) use them.
 cudaError_t launch_gemm_tn_tc(const GemmTnArgs& g, int amode, int apl, int bpl, int prec, int splits, int* status, cudaStream_t s) {
     const int pl = prec == 1 ? 1 : 2;
     if (g.N != g.ldb || g.klen % 64 != 0 || bpl != pl || (amode == A_PLANES && (apl != pl || g.lda % 64 != 0))) return cudaErrorNotSupported;
     if (amode != A_PLANES && apl != 1) return cudaErrorNotSupported;
+    const int bn = g.N > 256 && g.N % 256 == 0 ? 256 : g.N;
     if (prec == 1) {
-        switch (g.N) {
+        switch (bn) {
             case 64: return launch_bn<64, 1>(g, amode, splits, status, s);
             case 128: return launch_bn<128, 1>(g, amode, splits, status, s);
             case 256: return launch_bn<256, 1>(g, amode, splits, status, s);
         }
     } else {
-        switch (g.N) {
+        switch (bn) {
             case 64: return launch_bn<64, 0>(g, amode, splits, status, s);
             case 128: return launch_bn<128, 0>(g, amode, splits, status, s);
             case 256: return launch_bn<256, 0>(g, amode, splits, status, s);

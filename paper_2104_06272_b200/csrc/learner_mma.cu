@@ -25,21 +25,25 @@ namespace anakin {
 // turns the saved head outputs into output gradients, so that the two phases of different warps overlap and one CTA
 // barrier per tile suffices.  HBM-bound in principle: reads h2 (4 B/elt), writes the dh2 planes (2 x 2 B/elt).
 // ----------------------------------------------------------------------------------------------------
-template <int H, int NW, int PREC>
+// HS = width of the column slab one CTA covers (blockIdx.y picks the slab; HS = H for H <= 256); H2BF: h2 is stored as
+// bf16 (the wide bf16 path) instead of fp32.
+template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
 struct HeadsCfg {
     static constexpr int TR = 32;  // rows per tile
-    static constexpr size_t smem_bytes = (size_t)2 * TR * H * 4 + (size_t)2 * TR * 8 * 4 + (size_t)TR * 8 * 4;
+    static constexpr int ESZ = H2BF ? 2 : 4;
+    static constexpr size_t smem_bytes = (size_t)2 * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + (size_t)TR * 8 * 4;
 };
 
-template <int H, int NW, int PREC>
+template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
 __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
-    using Cfg = HeadsCfg<H, NW, PREC>;
-    constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = H / 2;
+    using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
+    constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = HS / 2, ESZ = Cfg::ESZ;
     static_assert(NTHREADS / HP2 == 4, "four row groups of eight rows");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* s_h2 = reinterpret_cast<float*>(smem_raw);  // [2][TR][H]
-    float* s_dout = s_h2 + 2 * TR * H;                 // [2][TR][8]
-    float* s_fin = s_dout + 2 * TR * 8;                // [TR][8] end-of-kernel reductions
+    unsigned char* s_h2 = smem_raw;                                               // [2][TR][HS] fp32 or bf16
+    float* s_dout = reinterpret_cast<float*>(smem_raw + (size_t)2 * TR * HS * ESZ);  // [2][TR][8]
+    float* s_fin = s_dout + 2 * TR * 8;                                           // [TR][8] end-of-kernel reductions
+    const int c_base = blockIdx.y * HS;  // first hidden unit of this CTA's slab
     const Dims& d = a.d;
     const Buffers& b = a.b;
     const int tid = threadIdx.x;
@@ -58,7 +62,7 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
 #pragma unroll
     for (int cc = 0; cc < 2; ++cc)
 #pragma unroll
-        for (int c = 0; c < 5; ++c) wh_c[cc][c] = b.theta_c[d.oWh + (2 * cp + cc) * 5 + c];
+        for (int c = 0; c < 5; ++c) wh_c[cc][c] = b.theta_c[d.oWh + (c_base + 2 * cp + cc) * 5 + c];
     float a_wh[2][5], a_b2[2] = {0.f, 0.f};
 #pragma unroll
     for (int cc = 0; cc < 2; ++cc)
@@ -68,12 +72,14 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
     float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
 
     auto load_tile = [&](int tile, int buf) {  // 16-byte chunks, zero-filled past the last row
-        float* dst = s_h2 + buf * TR * H;
-        for (int c = tid; c < TR * (H / 4); c += NTHREADS) {
-            const int r = c / (H / 4), k = 4 * (c - r * (H / 4));
+        constexpr int EPC = 16 / ESZ;  // elements per 16-byte chunk
+        unsigned char* dst = s_h2 + (size_t)buf * TR * HS * ESZ;
+        const unsigned char* src0 = reinterpret_cast<const unsigned char*>(b.h2);
+        for (int c = tid; c < TR * (HS / EPC); c += NTHREADS) {
+            const int r = c / (HS / EPC), k = EPC * (c - r * (HS / EPC));
             const size_t row = (size_t)tile * TR + r;
             const bool ok = row < R;
-            cp_async16(dst + r * H + k, b.h2 + (ok ? row : 0) * H + k, ok ? 16 : 0);
+            cp_async16(dst + ((size_t)r * HS + k) * ESZ, src0 + (((ok ? row : 0) * H) + c_base + k) * ESZ, ok ? 16 : 0);
         }
         cp_async_commit();
     };
@@ -139,7 +145,7 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
         RowIn nin;
         if (row_thread) nin = row_load(next);
         // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0, as 16-bit planes; running sums of dWh and db2
-        const float* h2t = s_h2 + buf * TR * H;
+        const unsigned char* h2t = s_h2 + (size_t)buf * TR * HS * ESZ;
         const float* dt = s_dout + buf * TR * 8;
 #pragma unroll 4
         for (int r = 0; r < 8; ++r) {
@@ -147,8 +153,16 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
             const size_t i = (size_t)tile * TR + e;
             const float4 d0 = *reinterpret_cast<const float4*>(dt + e * 8);
             const float d4 = dt[e * 8 + 4];
-            const float2 h2 = *reinterpret_cast<const float2*>(h2t + e * H + 2 * cp);
-            const float hv[2] = {h2.x, h2.y};
+            float hv[2];
+            if (H2BF) {
+                const uint32_t pk = *reinterpret_cast<const uint32_t*>(h2t + ((size_t)e * HS + 2 * cp) * 2);
+                hv[0] = __uint_as_float(pk << 16);          // bf16 -> fp32 is a 16-bit shift
+                hv[1] = __uint_as_float(pk & 0xFFFF0000u);
+            } else {
+                const float2 h2 = *reinterpret_cast<const float2*>(h2t + ((size_t)e * HS + 2 * cp) * 4);
+                hv[0] = h2.x;
+                hv[1] = h2.y;
+            }
             float dh[2];
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
@@ -168,8 +182,8 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
             if (i < R) {
                 uint32_t phi, plo;
                 split2<PREC>(dh[0], dh[1], phi, plo);
-                g_dh2hi[(i * H) / 2 + cp] = phi;
-                if (PREC == 0) g_dh2lo[(i * H) / 2 + cp] = plo;
+                g_dh2hi[(i * H + c_base) / 2 + cp] = phi;
+                if (PREC == 0) g_dh2lo[(i * H + c_base) / 2 + cp] = plo;
             }
         }
         // ---- row phase of the next tile (its inputs were requested before the column phase)
@@ -182,8 +196,8 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
 #pragma unroll
-            for (int c = 0; c < 5; ++c) part[(size_t)(2 * cp + cc) * 5 + c] = a_wh[cc][c];
-            part[(size_t)H * 5 + 2 * cp + cc] = a_b2[cc];
+            for (int c = 0; c < 5; ++c) part[(size_t)(c_base + 2 * cp + cc) * 5 + c] = a_wh[cc][c];
+            part[(size_t)H * 5 + c_base + 2 * cp + cc] = a_b2[cc];
         }
     }
     __syncthreads();
@@ -195,7 +209,7 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
         s_fin[rr * 8 + 7] = l_ent;
     }
     __syncthreads();
-    if (tid < 8) {  // rows in index order
+    if (tid < 8 && blockIdx.y == 0) {  // rows in index order; dbh and the loss terms come from the first slab only
         float s = 0.f;
         for (int e = 0; e < TR; ++e) s += s_fin[e * 8 + tid];
         if (tid < 5) {
@@ -590,12 +604,14 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             split1<PREC>(thc, hi, lo);
             const size_t ef = ((size_t)((k >> 4) * (H / 8) + (n >> 3)) * 32 + (n & 7) * 4 + ((k & 7) >> 1)) * 4 + ((k & 15) >> 3) * 2 + (k & 1);
             const size_t et = ((size_t)((n >> 4) * (H / 8) + (k >> 3)) * 32 + (k & 7) * 4 + ((n & 7) >> 1)) * 4 + ((n & 15) >> 3) * 2 + (n & 1);
-            reinterpret_cast<uint16_t*>(b.w2f_hi)[ef] = hi;
-            reinterpret_cast<uint16_t*>(b.w2f_lo)[ef] = lo;
-            reinterpret_cast<uint16_t*>(b.w2tf_hi)[et] = hi;
-            reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
+            if (b.w2f_hi) {
+                reinterpret_cast<uint16_t*>(b.w2f_hi)[ef] = hi;
+                reinterpret_cast<uint16_t*>(b.w2f_lo)[ef] = lo;
+                reinterpret_cast<uint16_t*>(b.w2tf_hi)[et] = hi;
+                reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
+            }
             b.w2p_hi[i - d.oW2] = hi;
-            b.w2p_lo[i - d.oW2] = lo;
+            if (b.w2p_lo) b.w2p_lo[i - d.oW2] = lo;
         }
     };
     auto region_of = [&](size_t i) {
@@ -654,13 +670,14 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
 }
 
 // Debug record of the ReLU gates from the saved activations (h1 hi plane, h2).
-__global__ void __launch_bounds__(256) k_pack_gates2(Dims d, Buffers b, size_t R) {
+__global__ void __launch_bounds__(256) k_pack_gates2(Dims d, Buffers b, size_t R, int h2_bf16) {
     const int lane = threadIdx.x & 31;
     const size_t words = R * (size_t)(d.H / 32);
     const __nv_bfloat16* h1hi = reinterpret_cast<const __nv_bfloat16*>(b.h1);
     for (size_t w = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5); w < 2 * words; w += (size_t)gridDim.x * 8) {
         bool on;
         if (w < words) on = (__bfloat16_as_ushort(h1hi[w * 32 + lane]) & 0x7FFFu) != 0;  // h1 >= 0: any magnitude bit
+        else if (h2_bf16) on = (reinterpret_cast<const uint16_t*>(b.h2)[(w - words) * 32 + lane] & 0x7FFFu) != 0;
         else on = b.h2[(w - words) * 32 + lane] > 0.f;
         const uint32_t bits = __ballot_sync(0xFFFFFFFFu, on);
         if (lane == 0) b.dbg_gates[w] = bits;
@@ -684,10 +701,15 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     const int H = d.H, C = d.C;
     const size_t R = (size_t)d.B * d.Tmax;
     const int bt = H >= 128 ? 128 : 64;  // gemm tile side
-    const int tiles_hh = ((H + bt - 1) / bt) * ((H + bt - 1) / bt);
+    int tiles_hh = ((H + bt - 1) / bt) * ((H + bt - 1) / bt);
     const int tiles_ch = ((C + 1 + bt - 1) / bt) * ((H + bt - 1) / bt);
+    int tiles_agent = tiles_ch;
+    if (H > 256) {  // wide path: 128 x 256 output tiles in the tcgen05 GEMMs
+        tiles_hh = (H / 128) * (H / 256);
+        tiles_agent = ((C + 127) / 128) * (H / 256);
+    }
     p->ns_w2 = splits_for((int)R, tiles_hh, 256);
-    p->ns_agent = splits_for((int)R, tiles_ch, 256);
+    p->ns_agent = splits_for((int)R, tiles_agent, 256);
     p->ns_env = splits_for(d.B, tiles_ch, 128);
     const size_t tiles32 = (R + 31) / 32;
     p->heads_grid = (int)(tiles32 < (size_t)HEADS_GRID ? tiles32 : (size_t)HEADS_GRID);
@@ -705,11 +727,11 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
 
 #define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
 
-template <int H, int NW, int PREC>
+template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
 static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s) {
-    using Cfg = HeadsCfg<H, NW, PREC>;
-    CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
-    k_heads_bwd<H, NW, PREC><<<grid, NW * 32, Cfg::smem_bytes, s>>>(a);
+    using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
+    CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
+    k_heads_bwd<H, NW, PREC, HS, H2BF><<<dim3(grid, H / HS), NW * 32, Cfg::smem_bytes, s>>>(a);
     return cudaGetLastError();
 }
 
@@ -729,6 +751,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     const int H = d.H, C = d.C, B = d.B, T = a.T;
     const size_t R = (size_t)B * T, RH = (size_t)B * d.Tmax * H;
     cudaStream_t s = c.s;
+    const bool wide = wide_supported(H, PREC);  // bf16 activations in HBM, layer-2 products as large tcgen05 GEMMs
     LearnPlan pl;
     learn_mma_plan(d, &pl);
     a.part_small = b.part + pl.off_small;
@@ -750,7 +773,13 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
             case 64: CK((launch_heads_t<64, 4, PREC>(a, pl.heads_grid, s))); break;
             case 128: CK((launch_heads_t<128, 8, PREC>(a, pl.heads_grid, s))); break;
             case 256: CK((launch_heads_t<256, 16, PREC>(a, pl.heads_grid, s))); break;
-            default: return cudaErrorNotSupported;
+            default:
+                if constexpr (PREC == 1) {
+                    if (wide && H == 512) { CK((launch_heads_t<512, 16, 1, 256, true>(a, pl.heads_grid, s))); break; }
+                    if (wide && H == 1024) { CK((launch_heads_t<1024, 16, 1, 256, true>(a, pl.heads_grid, s))); break; }
+                    if (wide && H == 2048) { CK((launch_heads_t<2048, 16, 1, 256, true>(a, pl.heads_grid, s))); break; }
+                }
+                return cudaErrorNotSupported;
         }
     }
     // t-slices: the tcgen05 dh1 kernel has ceil(B/128)*(H/128) CTAs per slice; slice the T steps so that one wave of
@@ -763,7 +792,9 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         if (ts > T) ts = T;
         if (ts >= 2) a.ts = ts;
     }
-    {
+    if (wide) {
+        CK(launch_dh1_wide(a, c));
+    } else {
         Scope sc(c, K_DH1);
         const cudaError_t etc = launch_dh1_tc(a, PREC, s);  // tcgen05 where covered, else the mma.sync kernel
         if (etc != cudaErrorNotSupported) CK(etc);
@@ -843,7 +874,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     }
     if (b.dbg_gates) {
         Scope sc(c, K_PACK_GATES);
-        k_pack_gates2<<<148 * 8, 256, 0, s>>>(d, b, R);
+        k_pack_gates2<<<148 * 8, 256, 0, s>>>(d, b, R, wide ? 1 : 0);
         CK(cudaGetLastError());
     }
     return cudaSuccess;

@@ -246,6 +246,7 @@ static cudaError_t launch_rollout_p(const RolloutArgs& a, cudaStream_t s) {
 }
 
 cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c) {
+    if (wide_supported(a.d.H, prec) && a.b.w2p_hi) return launch_rollout_wide(a, c);  // three launches per step
     Scope sc(c, K_ROLLOUT);
     const cudaError_t e = launch_rollout_mma(a, prec, c.s);  // tensor-pipe kernel where the shape is covered
     if (e != cudaErrorNotSupported) return e;

@@ -156,7 +156,9 @@ def test_full_size_workloads_on_sampled_envs(bnd, name):
     assert np.isfinite(grads).all() and np.abs(grads).max() > 0
     sl = orc.Dims(w.N, w.H).slices()
     bh = grads[sl["bh"]]
-    assert abs(bh[:4].sum()) <= 1e-3 * np.abs(bh[:4]).max() + 1e-9  # softmax gradients sum to zero in every row
+    # softmax gradients sum to zero in every row; in the bf16 workload each of the four is rounded to bf16 (2^-9) before
+    # the batch sum, so the cancellation is only as good as that rounding
+    assert abs(bh[:4].sum()) <= (1e-3 if w.precision == 0 else 1e-2) * np.abs(bh[:4]).max() + 1e-9
     # loss terms from the recorded data alone: policy term = -mean(A * logp), entropy <= ln 4
     s = an.stats()
     rt = par.rtol_of(w.precision)
