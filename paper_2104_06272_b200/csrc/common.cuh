@@ -229,6 +229,7 @@ bool tensor_path_supported(int H, int prec);  // either tensor-core path: the up
 cudaError_t launch_rollout_wide(const RolloutArgs& a, const Ctx& c);  // T+1 forward passes, or the replay of recorded rows
 cudaError_t launch_pack_w2_wide(const Dims& d, const Buffers& b, const Ctx& c);
 cudaError_t launch_dh1_wide(const LearnArgs& a, const Ctx& c);
+cudaError_t launch_env_base_wide(const Dims& d, const Buffers& b, const Ctx& c);  // cudaErrorNotSupported if not covered
 cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);

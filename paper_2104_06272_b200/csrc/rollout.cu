@@ -8,29 +8,51 @@ namespace anakin {
 // base[b][j] = b1[j] + sum over wall cells c (ascending) of W1[c][j] + W1[2C+goal_b][j].
 // The wall and goal planes of the observation do not change during an env's life, so their contribution
 // to the first layer is computed once per parameter version instead of once per step.
+// One thread owns four hidden units of one env; the W1 rows are fetched eight at a time (independent loads) and added in
+// ascending cell order, the goal row last.
 __global__ void __launch_bounds__(256) k_env_base(Dims d, Buffers b) {
-    const int e = blockIdx.x;
+    const int H4 = d.H / 4;
+    const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= (size_t)d.B * H4) return;
+    const int e = (int)(idx / H4), j4 = (int)(idx - (size_t)e * H4);
     const uint32_t* w = b.walls + (size_t)e * d.W;
-    const float* W1 = b.theta_c + d.oW1;
-    const int goal = b.goal[e];
-    for (int j = threadIdx.x; j < d.H; j += blockDim.x) {
-        float acc = b.theta_c[d.ob1 + j];
-        for (int wi = 0; wi < d.W; ++wi) {
-            uint32_t bits = w[wi];
-            while (bits) {
-                const int c = wi * 32 + (__ffs(bits) - 1);
-                bits &= bits - 1;
-                acc += W1[(size_t)c * d.H + j];
-            }
+    const float4* W1 = reinterpret_cast<const float4*>(b.theta_c + d.oW1) + j4;
+    const int goal_row = 2 * d.C + b.goal[e];
+    float4 acc = reinterpret_cast<const float4*>(b.theta_c + d.ob1)[j4];
+    int wi = 0;
+    uint32_t bits = w[0];
+    bool goal_done = false;
+    auto next_row = [&]() -> int {  // next wall cell in ascending order, then the goal row, then -1
+        while (!bits && wi + 1 < d.W) bits = w[++wi];
+        if (bits) {
+            const int c = wi * 32 + (__ffs(bits) - 1);
+            bits &= bits - 1;
+            return c;
         }
-        acc += W1[(size_t)(2 * d.C + goal) * d.H + j];
-        b.base[(size_t)e * d.H + j] = acc;
+        if (!goal_done) { goal_done = true; return goal_row; }
+        return -1;
+    };
+    for (;;) {
+        int rows[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) rows[q] = next_row();
+        float4 v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = rows[q] >= 0 ? __ldg(W1 + (size_t)rows[q] * H4) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            if (rows[q] >= 0) { acc.x += v[q].x; acc.y += v[q].y; acc.z += v[q].z; acc.w += v[q].w; }
+        }
+        if (rows[7] < 0) break;
     }
+    reinterpret_cast<float4*>(b.base)[idx] = acc;
 }
 
 cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c) {
+    const cudaError_t ew = launch_env_base_wide(d, b, c);  // tensor-core form where it applies
+    if (ew != cudaErrorNotSupported) return ew;
     Scope sc(c, K_ENV_BASE);
-    k_env_base<<<d.B, d.H < 256 ? d.H : 256, 0, c.s>>>(d, b);
+    k_env_base<<<(unsigned)(((size_t)d.B * (d.H / 4) + 255) / 256), 256, 0, c.s>>>(d, b);
     return cudaGetLastError();
 }
 

@@ -27,7 +27,7 @@ bool tensor_path_supported(int H, int prec) { return rollout_mma_supported(H) ||
 
 namespace {
 
-enum : int { EPI_FWD = 0, EPI_GATE = 1 };
+enum : int { EPI_FWD = 0, EPI_GATE = 1, EPI_BASE = 2 };
 
 struct NtArgs {
     int M, N, K;           // C is M x N; M rows starting at row0 of A, out and gate
@@ -35,6 +35,10 @@ struct NtArgs {
     uint16_t* out;         // bf16 [rows][N]
     const float* bias;     // EPI_FWD: [N]
     const uint16_t* gate;  // EPI_GATE: bf16 [rows][N], non-negative; out = gate > 0 ? acc : 0
+    float* outf;           // EPI_BASE: fp32 [rows][N] = acc + bias[n] + addrows[(addrow0 + addidx[m])*N + n]
+    const float* addrows;
+    const uint8_t* addidx;
+    int addrow0;
     int* status;
 };
 
@@ -69,7 +73,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ N
         for (int i = 0; i < 2; ++i) { tc::mbar_init(&tfull[i], 1); tc::mbar_init(&tempty[i], 4); }
         tc::mbar_fence_init();
     }
-    if (EPI == EPI_FWD)
+    if (EPI != EPI_GATE)
         for (int i = tid; i < g.N; i += Cfg::THREADS) s_bias[i] = g.bias[i];
     if (wid == 2) tc::tmem_alloc(tmem_slot, 512);
     tc::tc_fence_before();
@@ -158,6 +162,20 @@ __global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ N
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 tc::tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * BN + c0), r);
+                if (EPI == EPI_BASE) {  // fp32 out: accumulator + bias + this row's extra weight row
+                    if (valid) {
+                        const float4* add = reinterpret_cast<const float4*>(g.addrows + ((size_t)g.addrow0 + g.addidx[m]) * g.N + n0 + c0);
+                        float4* dst = reinterpret_cast<float4*>(g.outf + gi + c0);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 w = __ldg(add + j);
+                            const float* bs = s_bias + n0 + c0 + 4 * j;
+                            dst[j] = make_float4(__uint_as_float(r[4 * j]) + bs[0] + w.x, __uint_as_float(r[4 * j + 1]) + bs[1] + w.y,
+                                                 __uint_as_float(r[4 * j + 2]) + bs[2] + w.z, __uint_as_float(r[4 * j + 3]) + bs[3] + w.w);
+                        }
+                    }
+                    continue;
+                }
                 uint4 gn[4];
                 if (EPI == EPI_GATE && c0 + 32 < BN) {  // next chunk's gates, in flight during this chunk's math
 #pragma unroll
@@ -372,6 +390,26 @@ __global__ void __launch_bounds__(256) k_pack_w2_wide(Dims d, Buffers b) {
     if (i < (size_t)d.H * d.H) b.w2p_hi[i] = __bfloat16_as_ushort(__float2bfloat16_rn(b.theta_c[d.oW2 + i]));
 }
 
+// Operands of the base GEMM: X[env][c] = 1 where cell c of the env is a wall (bf16), and the wall plane of W1 as bf16
+// (exact: the weights are bf16 values in this workload).
+__global__ void __launch_bounds__(256) k_expand_walls(Dims d, Buffers b, uint16_t* X, uint16_t* W1w) {
+    const size_t nx = (size_t)d.B * (d.C / 8), nw = (size_t)d.C * d.H;
+    for (size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x; idx < nx + nw; idx += (size_t)gridDim.x * 256) {
+        if (idx < nx) {
+            const size_t e = idx / (d.C / 8);
+            const int c8 = (int)(idx - e * (d.C / 8));
+            const uint32_t bits = (b.walls[e * d.W + (c8 >> 2)] >> ((c8 & 3) * 8)) & 0xFFu;
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) o[q] = ((bits >> (2 * q)) & 1u ? 0x3F80u : 0u) | ((bits >> (2 * q + 1)) & 1u ? 0x3F800000u : 0u);
+            reinterpret_cast<uint4*>(X)[idx] = make_uint4(o[0], o[1], o[2], o[3]);
+        } else {
+            const size_t i = idx - nx;
+            W1w[i] = __bfloat16_as_ushort(__float2bfloat16_rn(b.theta_c[d.oW1 + i]));
+        }
+    }
+}
+
 #define CKW(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
 
 cudaError_t heads_wide(const RolloutArgs& a, int t, int mode, size_t rows, size_t row0, cudaStream_t s) {
@@ -386,6 +424,36 @@ cudaError_t launch_pack_w2_wide(const Dims& d, const Buffers& b, const Ctx& c) {
     Scope sc(c, K_PACK_W2);
     k_pack_w2_wide<<<(unsigned)(((size_t)d.H * d.H + 255) / 256), 256, 0, c.s>>>(d, b);
     return cudaGetLastError();
+}
+
+// base = b1 + walls x W1[wall plane] + W1[goal row] as one GEMM (K = C cells).  Applies to the buffers of the wide path
+// (bf16 workload: the products 1 x w are exact and the accumulation is fp32); cudaErrorNotSupported otherwise.
+// Uses the dh1 buffer, which is dead outside the update, as scratch for the two bf16 operands.
+cudaError_t launch_env_base_wide(const Dims& d, const Buffers& b, const Ctx& c) {
+    const bool wide_buffers = b.w2p_hi && !b.w2f_hi;
+    if (!wide_buffers || d.C % 64 != 0 || d.H % NtCfg::BN != 0 || d.H > NtCfg::MAXN) return cudaErrorNotSupported;
+    uint16_t* X = reinterpret_cast<uint16_t*>(b.dh1);
+    uint16_t* W1w = X + (size_t)d.B * d.C;
+    NtMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (!make_tensor_map_2d(&maps.a, X, d.B, d.C, 128, true)) return cudaErrorNotSupported;
+    if (!make_tensor_map_2d(&maps.b, W1w, d.C, d.H, 64, true)) return cudaErrorNotSupported;
+    {
+        Scope sc(c, K_ENV_BASE);
+        k_expand_walls<<<148 * 8, 256, 0, c.s>>>(d, b, X, W1w);
+        CKW(cudaGetLastError());
+    }
+    Scope sc(c, K_ENV_BASE);
+    NtArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = d.B; g.N = d.H; g.K = d.C; g.row0 = 0;
+    g.bias = b.theta_c + d.ob1;
+    g.outf = b.base;
+    g.addrows = b.theta_c + d.oW1;
+    g.addidx = b.goal;
+    g.addrow0 = 2 * d.C;
+    g.status = b.status;
+    return launch_nt<EPI_BASE, true>(maps, g, c.s);
 }
 
 // T+1 forward passes (or, in replay mode, one pass over the recorded rows).
