@@ -156,6 +156,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     w = WORKLOADS[args.workload]
+    if args.envs:  # reduced batch for profiler captures; such a run is not a bench line of the named workload
+        w = w.scaled(name=f"{w.name}[B={args.envs}]", B=args.envs)
     peaks = load_peaks()
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
@@ -271,7 +273,9 @@ def run_ours(args):
                 "kernels": {k: kernel_line(k, ms, n) for k, (ms, n) in sorted(prof.items(), key=lambda kv: -kv[1][0])}}
 
     # ---- the oracle on the host cores, bounded sample of the same workload (about 10-30 s of CPU work)
-    if args.workload == "throughput":
+    if args.no_cpu_baseline or rank != 0:
+        cpu = None
+    elif args.workload == "throughput" and not args.envs:
         cpu = cpu_baseline(w, iters=2)
     else:
         mac_per_frame = 3.0 * (w.D * w.H + w.H * w.H + 5 * w.H) + w.H * w.H
@@ -347,6 +351,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiler captures only)")
+    ap.add_argument("--envs", type=int, default=0, help="override the workload's number of envs (small profiler captures only)")
     ap.add_argument("--workload", default="throughput", choices=list(WORKLOADS),
                     help="the metric is quoted on 'throughput'; the others are for the per-workload table")
     args = ap.parse_args()

@@ -31,17 +31,18 @@ template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
 struct HeadsCfg {
     static constexpr int TR = 32;  // rows per tile
     static constexpr int ESZ = H2BF ? 2 : 4;
-    static constexpr size_t smem_bytes = (size_t)2 * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + (size_t)TR * 8 * 4;
+    static constexpr int NST = TR * HS * ESZ >= 32768 ? 3 : 4;  // depth of the h2 ring (tiles in flight = NST - 1)
+    static constexpr size_t smem_bytes = (size_t)NST * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + (size_t)TR * 8 * 4;
 };
 
 template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
 __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
     using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
-    constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = HS / 2, ESZ = Cfg::ESZ;
+    constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = HS / 2, ESZ = Cfg::ESZ, NST = Cfg::NST;
     static_assert(NTHREADS / HP2 == 4, "four row groups of eight rows");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned char* s_h2 = smem_raw;                                               // [2][TR][HS] fp32 or bf16
-    float* s_dout = reinterpret_cast<float*>(smem_raw + (size_t)2 * TR * HS * ESZ);  // [2][TR][8]
+    unsigned char* s_h2 = smem_raw;                                                 // [NST][TR][HS] fp32 or bf16
+    float* s_dout = reinterpret_cast<float*>(smem_raw + (size_t)NST * TR * HS * ESZ);  // [2][TR][8]
     float* s_fin = s_dout + 2 * TR * 8;                                           // [TR][8] end-of-kernel reductions
     const int c_base = blockIdx.y * HS;  // first hidden unit of this CTA's slab
     const Dims& d = a.d;
@@ -54,10 +55,11 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
     const float invR = a.gscale / (float)R;  // output gradients are carried times gscale
     const int ntiles = (int)((R + TR - 1) / TR);
 
-    // column phase: thread = (unit pair cp, row group rg of 8 rows); row phase: one thread per row
+    // column phase: thread = (unit pair cp, row group rg of 8 rows); row phase: the lanes of ONE warp take the 32 rows of
+    // a tile, and the warps take turns (tile after tile), so that no warp issues the row code for a few active lanes
     const int cp = tid % HP2, rg = tid / HP2;
-    const bool row_thread = (tid % NW) == 0;
-    const int rr = tid / NW;
+    const int wid = tid >> 5;
+    const int rr = tid & 31;
     float wh_c[2][5];
 #pragma unroll
     for (int cc = 0; cc < 2; ++cc)
@@ -71,11 +73,11 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
     float a_bh[5] = {0.f, 0.f, 0.f, 0.f, 0.f};  // row threads: sums of dOut over their rows
     float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
 
-    auto load_tile = [&](int tile, int buf) {  // 16-byte chunks, zero-filled past the last row
+    auto load_tile = [&](int tile, int buf) {  // 16-byte chunks, zero-filled past the last row; always commits a group
         constexpr int EPC = 16 / ESZ;  // elements per 16-byte chunk
         unsigned char* dst = s_h2 + (size_t)buf * TR * HS * ESZ;
         const unsigned char* src0 = reinterpret_cast<const unsigned char*>(b.h2);
-        for (int c = tid; c < TR * (HS / EPC); c += NTHREADS) {
+        for (int c = tid; tile < ntiles && c < TR * (HS / EPC); c += NTHREADS) {
             const int r = c / (HS / EPC), k = EPC * (c - r * (HS / EPC));
             const size_t row = (size_t)tile * TR + r;
             const bool ok = row < R;
@@ -132,34 +134,36 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
     };
 
     int it = 0;
-    if ((int)blockIdx.x < ntiles) {
-        load_tile(blockIdx.x, 0);
-        if (row_thread) row_finish(row_load(blockIdx.x), 0);
-    }
+#pragma unroll
+    for (int q = 0; q < NST - 1; ++q) load_tile(blockIdx.x + q * (int)gridDim.x, q);
+    if ((int)blockIdx.x < ntiles && wid == 0) row_finish(row_load(blockIdx.x), 0);
     for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
-        const int buf = it & 1;
+        const int buf = it & 1;  // dOut buffer of this tile
         const int next = tile + (int)gridDim.x;
-        cp_async_wait<0>();
-        __syncthreads();  // this tile's h2 and dOut are in place; everyone is done with the other buffers
-        if (next < ntiles) load_tile(next, buf ^ 1);
+        cp_async_wait<NST - 2>();
+        __syncthreads();  // this tile's h2 and dOut are in place; everyone is done with the buffers of the tile before
+        load_tile(tile + (NST - 1) * (int)gridDim.x, (it + NST - 1) % NST);
+        const bool row_thread = wid == (it + 1) % NW;  // this warp prepares the next tile's output gradients
         RowIn nin;
         if (row_thread) nin = row_load(next);
         // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0, as 16-bit planes; running sums of dWh and db2
-        const unsigned char* h2t = s_h2 + (size_t)buf * TR * HS * ESZ;
-        const float* dt = s_dout + buf * TR * 8;
+        const unsigned char* h2t = s_h2 + ((size_t)(it % NST) * TR + rg * 8) * HS * ESZ + (size_t)2 * cp * ESZ;
+        const float* dt = s_dout + (buf * TR + rg * 8) * 8;
+        const size_t i0 = (size_t)tile * TR + rg * 8;
+        const int rows_left = i0 < R ? (int)((R - i0) < 8 ? (R - i0) : 8) : 0;
+        uint32_t* o_hi = g_dh2hi + (i0 * H + c_base) / 2 + cp;
+        uint32_t* o_lo = g_dh2lo + (i0 * H + c_base) / 2 + cp;
 #pragma unroll 4
         for (int r = 0; r < 8; ++r) {
-            const int e = rg * 8 + r;
-            const size_t i = (size_t)tile * TR + e;
-            const float4 d0 = *reinterpret_cast<const float4*>(dt + e * 8);
-            const float d4 = dt[e * 8 + 4];
+            const float4 d0 = *reinterpret_cast<const float4*>(dt + r * 8);
+            const float d4 = dt[r * 8 + 4];
             float hv[2];
             if (H2BF) {
-                const uint32_t pk = *reinterpret_cast<const uint32_t*>(h2t + ((size_t)e * HS + 2 * cp) * 2);
+                const uint32_t pk = *reinterpret_cast<const uint32_t*>(h2t + (size_t)r * HS * 2);
                 hv[0] = __uint_as_float(pk << 16);          // bf16 -> fp32 is a 16-bit shift
                 hv[1] = __uint_as_float(pk & 0xFFFF0000u);
             } else {
-                const float2 h2 = *reinterpret_cast<const float2*>(h2t + ((size_t)e * HS + 2 * cp) * 4);
+                const float2 h2 = *reinterpret_cast<const float2*>(h2t + (size_t)r * HS * 4);
                 hv[0] = h2.x;
                 hv[1] = h2.y;
             }
@@ -171,19 +175,24 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
                 back = fmaf(d0.z, wh_c[cc][2], back);
                 back = fmaf(d0.w, wh_c[cc][3], back);
                 back = fmaf(d4, wh_c[cc][4], back);
-                dh[cc] = rnd<PREC>(hv[cc] > 0.f ? back : 0.f);
+                dh[cc] = hv[cc] > 0.f ? back : 0.f;
                 a_wh[cc][0] = fmaf(hv[cc], d0.x, a_wh[cc][0]);
                 a_wh[cc][1] = fmaf(hv[cc], d0.y, a_wh[cc][1]);
                 a_wh[cc][2] = fmaf(hv[cc], d0.z, a_wh[cc][2]);
                 a_wh[cc][3] = fmaf(hv[cc], d0.w, a_wh[cc][3]);
                 a_wh[cc][4] = fmaf(hv[cc], d4, a_wh[cc][4]);
-                a_b2[cc] += dh[cc];
             }
-            if (i < R) {
-                uint32_t phi, plo;
-                split2<PREC>(dh[0], dh[1], phi, plo);
-                g_dh2hi[(i * H + c_base) / 2 + cp] = phi;
-                if (PREC == 0) g_dh2lo[(i * H + c_base) / 2 + cp] = plo;
+            uint32_t phi, plo;
+            split2<PREC>(dh[0], dh[1], phi, plo);
+            if (PREC == 1) {  // the bf16 workload rounds dh2: the sums take the rounded values
+                dh[0] = __uint_as_float(phi << 16);
+                dh[1] = __uint_as_float(phi & 0xFFFF0000u);
+            }
+            a_b2[0] += dh[0];
+            a_b2[1] += dh[1];
+            if (r < rows_left) {
+                o_hi[(size_t)r * (H / 2)] = phi;
+                if (PREC == 0) o_lo[(size_t)r * (H / 2)] = plo;
             }
         }
         // ---- row phase of the next tile (its inputs were requested before the column phase)
@@ -201,17 +210,21 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
         }
     }
     __syncthreads();
-    if (row_thread) {
+    {   // every warp has taken turns at the row phase: fold its lanes (fixed tree), then the warps in index order
+        float vals[8] = {a_bh[0], a_bh[1], a_bh[2], a_bh[3], a_bh[4], l_pg, l_v, l_ent};
 #pragma unroll
-        for (int c = 0; c < 5; ++c) s_fin[rr * 8 + c] = a_bh[c];
-        s_fin[rr * 8 + 5] = l_pg;
-        s_fin[rr * 8 + 6] = l_v;
-        s_fin[rr * 8 + 7] = l_ent;
+        for (int c = 0; c < 8; ++c)
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) vals[c] += __shfl_xor_sync(0xFFFFFFFFu, vals[c], off);
+        if (rr == 0) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) s_fin[wid * 8 + c] = vals[c];
+        }
     }
     __syncthreads();
     if (tid < 8 && blockIdx.y == 0) {  // rows in index order; dbh and the loss terms come from the first slab only
         float s = 0.f;
-        for (int e = 0; e < TR; ++e) s += s_fin[e * 8 + tid];
+        for (int e = 0; e < NW; ++e) s += s_fin[e * 8 + tid];
         if (tid < 5) {
             for (int q = 0; q < 4; ++q) a.part_small[(size_t)(4 * blockIdx.x + q) * a.small_stride + (size_t)H * 6 + tid] = q == 0 ? s : 0.f;
         } else {

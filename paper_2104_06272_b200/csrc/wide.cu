@@ -251,42 +251,75 @@ __global__ void __launch_bounds__(256) k_h1_wide(Dims d, Buffers b, const uint8_
     }
 }
 
-// Heads, sampling and env step for 64 rows per CTA.
+// Heads, sampling and env step for 32 rows per CTA: eight warps take four rows each for the head products, then warp 0
+// takes one row per lane for the per-env part (its env state and wall words were requested at kernel start).
 //   mode 0: step t of the rollout (row = env): saves the head outputs and the value, samples, steps the env, records.
 //   mode 1: bootstrap forward after the last step: saves the value only.
 //   mode 2: replay of recorded rows (row = t*B + env): saves the head outputs only.
-constexpr int HW_ROWS = 64;
+constexpr int HW_ROWS = 32;
 
+template <int H>
 __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mode, size_t rows, size_t row0) {
-    extern __shared__ float s_wh[];  // [5][H]
+    constexpr int TRIPS = H / 128;   // a lane covers four consecutive hidden units per trip
+    extern __shared__ __align__(16) float s_wh[];  // [H][5] as stored
     __shared__ float s_out[HW_ROWS][8];
+    __shared__ uint32_t s_walls[HW_ROWS][8];
     const Dims& d = a.d;
     const Buffers& b = a.b;
-    const int H = d.H, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    for (int idx = tid; idx < 5 * H; idx += 256) {
-        const int k = idx / 5, c = idx - 5 * k;
-        s_wh[c * H + k] = b.theta_c[d.oWh + idx];
-    }
-    __syncthreads();
-    const uint16_t* h2b = reinterpret_cast<const uint16_t*>(b.h2);
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const size_t i0 = (size_t)blockIdx.x * HW_ROWS;
-    for (int r = wid; r < HW_ROWS; r += 8) {
-        const size_t i = i0 + r;
-        if (i >= rows) break;
-        const uint2* hp = reinterpret_cast<const uint2*>(h2b + (row0 + i) * H);
-        float acc[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int k4 = lane; k4 < H / 4; k4 += 32) {  // four consecutive hidden units per lane and trip
-            const uint2 v = hp[k4];
-            const float x[4] = {__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
-                                __uint_as_float(v.y & 0xFFFF0000u)};
+    {   // Wh: straight 16-byte copies (the parameter block starts on a 16-byte boundary for these H)
+        const float4* src = reinterpret_cast<const float4*>(b.theta_c + d.oWh);
+        float4* dst = reinterpret_cast<float4*>(s_wh);
 #pragma unroll
-            for (int c = 0; c < 5; ++c) {
-                const float4 w = *reinterpret_cast<const float4*>(s_wh + c * H + 4 * k4);
-                acc[c] = fmaf(x[0], w.x, acc[c]);
-                acc[c] = fmaf(x[1], w.y, acc[c]);
-                acc[c] = fmaf(x[2], w.z, acc[c]);
-                acc[c] = fmaf(x[3], w.w, acc[c]);
+        for (int q = 0; q < (5 * H / 4 + 255) / 256; ++q)
+            if (tid + 256 * q < 5 * H / 4) dst[tid + 256 * q] = __ldg(src + tid + 256 * q);
+    }
+    EnvLane es;
+    es.pos = es.tep = es.start = es.goal = 0;
+    if (mode == 0) {
+        if (tid < HW_ROWS && i0 + tid < rows) {
+            es.pos = b.pos[i0 + tid];
+            es.tep = b.tep[i0 + tid];
+            es.start = b.start[i0 + tid];
+            es.goal = b.goal[i0 + tid];
+        }
+        for (int idx = tid; idx < HW_ROWS * d.W; idx += 256) {
+            const int e = idx / d.W, wi = idx - e * d.W;
+            if (i0 + e < rows) s_walls[e][wi] = b.walls[(i0 + e) * d.W + wi];
+        }
+    }
+    const uint16_t* h2b = reinterpret_cast<const uint16_t*>(b.h2);
+    // a warp walks rows wid, wid+8, ...; the loads of the next row are in flight while this row is reduced
+    uint2 v[TRIPS], vn[TRIPS];
+    auto load_row = [&](int r, uint2 (&dst)[TRIPS]) {
+        const size_t i = i0 + r;
+        const uint2* hp = reinterpret_cast<const uint2*>(h2b + (row0 + (i < rows ? i : 0)) * H);
+#pragma unroll
+        for (int q = 0; q < TRIPS; ++q) dst[q] = (r < HW_ROWS && i < rows) ? __ldg(hp + lane + 32 * q) : make_uint2(0u, 0u);
+    };
+    load_row(wid, v);
+    __syncthreads();
+#pragma unroll 1
+    for (int r = wid; r < HW_ROWS; r += 8) {
+        load_row(r + 8, vn);
+        float acc[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int q = 0; q < TRIPS; ++q) {
+            const float x[4] = {__uint_as_float(v[q].x << 16), __uint_as_float(v[q].x & 0xFFFF0000u), __uint_as_float(v[q].y << 16),
+                                __uint_as_float(v[q].y & 0xFFFF0000u)};
+            // this lane's four units are 20 consecutive floats of Wh (80-byte lane stride: conflict-free 16-byte reads)
+            const float4* wp = reinterpret_cast<const float4*>(s_wh + 20 * (lane + 32 * q));
+            float w[20];
+#pragma unroll
+            for (int j = 0; j < 5; ++j) {
+                const float4 f = wp[j];
+                w[4 * j] = f.x; w[4 * j + 1] = f.y; w[4 * j + 2] = f.z; w[4 * j + 3] = f.w;
             }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int c = 0; c < 5; ++c) acc[c] = fmaf(x[u], w[5 * u + c], acc[c]);
         }
 #pragma unroll
         for (int c = 0; c < 5; ++c)
@@ -296,6 +329,8 @@ __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mo
 #pragma unroll
             for (int c = 0; c < 5; ++c) s_out[r][c] = acc[c] + b.theta_c[d.obh + c];
         }
+#pragma unroll
+        for (int q = 0; q < TRIPS; ++q) v[q] = vn[q];
     }
     __syncthreads();
     if (tid >= HW_ROWS) return;
@@ -304,33 +339,28 @@ __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mo
     unsigned long long n_ep = 0, n_goal = 0, n_steps = 0;
     int bad = 0;
     if (valid) {
-        const float o0 = s_out[tid][0], o1 = s_out[tid][1], o2 = s_out[tid][2], o3 = s_out[tid][3], v = s_out[tid][4];
+        const float o0 = s_out[tid][0], o1 = s_out[tid][1], o2 = s_out[tid][2], o3 = s_out[tid][3], v4 = s_out[tid][4];
         if (mode == 1) {
-            b.tval[(size_t)a.T * d.B + i] = v;
+            b.tval[(size_t)a.T * d.B + i] = v4;
         } else {
             const size_t row = mode == 0 ? (size_t)t * d.B + i : i;
             float4* o = reinterpret_cast<float4*>(b.out5 + row * 8);
             o[0] = make_float4(o0, o1, o2, o3);
-            o[1] = make_float4(v, 0.f, 0.f, 0.f);
+            o[1] = make_float4(v4, 0.f, 0.f, 0.f);
             if (mode == 0) {
-                b.tval[row] = v;
+                b.tval[row] = v4;
                 const int env = (int)i;
-                EnvLane s;
-                s.pos = b.pos[env];
-                s.tep = b.tep[env];
-                s.start = b.start[env];
-                s.goal = b.goal[env];
-                s.n_episodes = s.n_goals = s.n_epsteps = 0;
-                s.bad = 0;
-                act_and_step(s, a, env, t, o0, o1, o2, o3, b.walls + (size_t)env * d.W);
-                b.pos[env] = (uint8_t)s.pos;
-                b.tep[env] = (uint8_t)s.tep;
-                n_ep = s.n_episodes; n_goal = s.n_goals; n_steps = s.n_epsteps; bad = s.bad;
+                es.n_episodes = es.n_goals = es.n_epsteps = 0;
+                es.bad = 0;
+                act_and_step(es, a, env, t, o0, o1, o2, o3, s_walls[tid]);
+                b.pos[env] = (uint8_t)es.pos;
+                b.tep[env] = (uint8_t)es.tep;
+                n_ep = es.n_episodes; n_goal = es.n_goals; n_steps = es.n_epsteps; bad = es.bad;
             }
         }
     }
     if (mode != 0) return;
-    // fold the two warps' counters and add them with integer atomics (order-free totals)
+    // fold the warp's counters and add them with integer atomics (order-free totals)
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         n_ep += __shfl_xor_sync(0xFFFFFFFFu, n_ep, off);
@@ -414,7 +444,13 @@ __global__ void __launch_bounds__(256) k_expand_walls(Dims d, Buffers b, uint16_
 
 cudaError_t heads_wide(const RolloutArgs& a, int t, int mode, size_t rows, size_t row0, cudaStream_t s) {
     const size_t smem = (size_t)5 * a.d.H * sizeof(float);
-    k_heads_wide<<<(unsigned)((rows + HW_ROWS - 1) / HW_ROWS), 256, smem, s>>>(a, t, mode, rows, row0);
+    const unsigned grid = (unsigned)((rows + HW_ROWS - 1) / HW_ROWS);
+    switch (a.d.H) {
+        case 512: k_heads_wide<512><<<grid, 256, smem, s>>>(a, t, mode, rows, row0); break;
+        case 1024: k_heads_wide<1024><<<grid, 256, smem, s>>>(a, t, mode, rows, row0); break;
+        case 2048: k_heads_wide<2048><<<grid, 256, smem, s>>>(a, t, mode, rows, row0); break;
+        default: return cudaErrorNotSupported;
+    }
     return cudaGetLastError();
 }
 
@@ -472,7 +508,7 @@ cudaError_t launch_rollout_wide(const RolloutArgs& a, const Ctx& c) {
     g.out = reinterpret_cast<uint16_t*>(b.h2);
     g.bias = b.theta_c + d.ob2;
     g.status = b.status;
-    auto h1_grid = [](size_t rows, int H) { const size_t n = (rows * (H / 8) + 255) / 256; return (unsigned)(n < 148 * 16 ? n : 148 * 16); };
+    auto h1_grid = [](size_t rows, int H) { return (unsigned)((rows * (H / 8) + 255) / 256); };
     if (a.replay) {
         const size_t R = (size_t)B * a.T;
         {
