@@ -5,8 +5,9 @@
     python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands
 
 One step = one pass of the whole hot path: a T-step rollout of all B envs followed by one A2C/Adam update
-(B*T frames).  Prints ONE JSON line.  With N > 1 (torchrun) every rank runs an independent replica of the
-workload with its own seed ("replicas only": the library has no cross-device exchange step yet).
+(B*T frames).  Prints ONE JSON line.  With N > 1 (torchrun) every rank runs the workload's B envs as one shard of an
+N*B-env job: same seed, env offsets rank*B, and one exchange per step, the mean of the gradients (NCCL all-reduce of P
+floats) between the backward pass and Adam.
 """
 from __future__ import annotations
 
@@ -134,8 +135,8 @@ def max_over_ranks(value: float, world: int, device="cpu") -> float:
 
 
 def whole_job_frames_per_sec(frames_per_rank: float, world: int, max_seconds: float) -> float:
-    """Replicas only: every rank processes frames_per_rank frames of its own; the job's rate is the sum over ranks
-    divided by the slowest rank's time."""
+    """Every rank processes frames_per_rank frames of its own shard; the job's rate is the sum over ranks divided by
+    the slowest rank's time."""
     return frames_per_rank * world / max_seconds
 
 
@@ -160,10 +161,24 @@ def run_ours(args):
         w = w.scaled(name=f"{w.name}[B={args.envs}]", B=args.envs)
     peaks = load_peaks()
     stream = torch.cuda.Stream()
-    with torch.cuda.stream(stream):
-        an = bnd.Anakin(bnd.cfg_from_workload(w, device=local_rank), stream=stream)
-    seed = 1 + rank
-    an.reset(seed)
+    seed = 1
+    if world > 1:
+        from paper_2104_06272_b200 import replicas
+
+        with torch.cuda.stream(stream):
+            rep = replicas.ReplicatedAnakin(w.scaled(B=w.B * world), rank, world, device=local_rank, stream=stream)
+        an = rep.an
+        rep.reset(seed)
+
+        def run_steps(n):
+            rep.run(n)
+    else:
+        with torch.cuda.stream(stream):
+            an = bnd.Anakin(bnd.cfg_from_workload(w, device=local_rank), stream=stream)
+        an.reset(seed)
+
+        def run_steps(n):
+            an.run(n)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
 
     def barrier():
@@ -173,7 +188,7 @@ def run_ours(args):
 
     K, W = args.steps, args.warmup
     # ---- warm-up
-    an.run(W)
+    run_steps(W)
     torch.cuda.synchronize()
 
     # ---- timed region: K steps, each bracketed by events on the library's stream; L2 flushed between steps
@@ -188,7 +203,7 @@ def run_ours(args):
         for a, b in ev:
             flush.fill_(0)
             a.record(stream)
-            an.run(1)
+            run_steps(1)
             b.record(stream)
     barrier()
     t_wall = time.perf_counter() - t_wall0
@@ -203,7 +218,7 @@ def run_ours(args):
     with torch.cuda.stream(stream):
         for _ in range(K):
             flush.fill_(0)
-            an.run(1)
+            run_steps(1)
     prof = an.profile_read()
     an.profile_enable(False)
 
@@ -221,7 +236,7 @@ def run_ours(args):
         an.set(bnd.PARAMS, h_theta)
         an.set(bnd.ENV_POS, h_pos)
         an.set(bnd.ENV_TEP, h_tep)
-        an.run(1)
+        run_steps(1)
         st = an.stats()
         an.get_into(bnd.PARAMS, h_out)
         an.get_into(bnd.ENV_POS, h_pos)
@@ -288,7 +303,8 @@ def run_ours(args):
         "dtype": "bf16" if w.precision == 1 else "f32", "data": "synthetic",
         "config": {"workload": workload_label(w), "frames_per_step": w.B * w.T, "seed": seed,
                    "l2": "flushed between timed steps (256 MiB write outside the event brackets)",
-                   "multi_gpu": "replicas only" if world > 1 else "single GPU"},
+                   "multi_gpu": (f"{world} replicas of B envs each (one job of {world * w.B} envs), gradients averaged with one NCCL "
+                                 "all-reduce per step" if world > 1 else "single GPU")},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": P * 4 + 2 * w.B, "d2h_bytes_per_step": P * 4 + 2 * w.B + 48,
                 "steps": Ke, "what": "set(PARAMS, ENV_POS, ENV_TEP) from pinned host, run(1), get(STATS, PARAMS, ENV_POS, ENV_TEP)"},

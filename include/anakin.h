@@ -76,13 +76,16 @@ typedef struct anakin_cfg {
     int32_t device;       /* CUDA device ordinal the workspace lives on */
     int32_t debug_logits; /* non-zero: debug records -- rollouts also store the 4 logits of every (t, b), updates
                              also store the ReLU gates of every row (DEBUG_LOGITS / DEBUG_GATES blobs) */
-    int32_t reserved;     /* must be 0 */
+    int32_t env_offset;   /* global index of this handle's first env, >= 0 (0 on a single device).  Env b draws its
+                             initial state and its action noise from the Philox counters of env env_offset + b, so
+                             that G handles with B/G envs each and offsets 0, B/G, ... hold exactly the envs of one
+                             handle with B envs (the replicas of Section 3.1, Figure 2 bottom) */
 } anakin_cfg;
 
 /* Blob selectors for anakin_get / anakin_set.  Sizes in bytes for the LAST rollout length T (or T_max where noted). */
 enum {
     ANAKIN_PARAMS = 0,       /* f32[P]                       get/set */
-    ANAKIN_GRADS = 1,        /* f32[P]   last batch-mean gradient      get */
+    ANAKIN_GRADS = 1,        /* f32[P]   last batch-mean gradient      get/set (set: before anakin_apply_grads) */
     ANAKIN_ADAM_M = 2,       /* f32[P]                       get/set */
     ANAKIN_ADAM_V = 3,       /* f32[P]                       get/set */
     ANAKIN_ADAM_STEP = 4,    /* i64[1]  host-side counter; pointer must be HOST   get/set */
@@ -163,6 +166,19 @@ int anakin_gae(anakin_t* h);
 /* Only the update's second half: loss, backward, batch mean and Adam from the ADV and RET blobs as they stand
  * (anakin_learn == anakin_gae followed by anakin_update).  Consumes the pending rollout. */
 int anakin_update(anakin_t* h);
+
+/*
+ * The update split at the point where the paper averages gradients across devices (Section 3.1: the update computed on
+ * each core's batch is averaged with a collective before it is applied).
+ *   anakin_grads        everything anakin_learn does up to and including the batch mean over this handle's B*T rows:
+ *                       fills GRADS and the loss statistics, consumes the pending rollout, leaves parameters and Adam
+ *                       state untouched.  Errors: BAD_STATE if no rollout is pending.
+ *   anakin_apply_grads  one Adam step with the GRADS blob as it stands (after the caller has averaged it over the
+ *                       replicas, on this stream).  Errors: BAD_STATE before the first anakin_reset.
+ * anakin_grads followed by anakin_apply_grads gives bitwise the result of anakin_learn.
+ */
+int anakin_grads(anakin_t* h);
+int anakin_apply_grads(anakin_t* h);
 
 /* iters x ( anakin_rollout(T_max); anakin_learn() ), enqueue-only: no copy and no synchronisation. */
 int anakin_run(anakin_t* h, int iters);

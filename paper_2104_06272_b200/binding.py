@@ -29,7 +29,7 @@ class AnakinCfg(C.Structure):
         ("episode_cap", C.c_int32), ("wall_density", C.c_double),
         ("gamma", C.c_float), ("gae_lambda", C.c_float), ("entropy_coef", C.c_float), ("value_coef", C.c_float),
         ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float),
-        ("precision", C.c_int32), ("device", C.c_int32), ("debug_logits", C.c_int32), ("reserved", C.c_int32),
+        ("precision", C.c_int32), ("device", C.c_int32), ("debug_logits", C.c_int32), ("env_offset", C.c_int32),
     ]
 
 
@@ -45,7 +45,8 @@ OK, E_INVALID_ARG, E_BAD_STATE, E_WORKSPACE_TOO_SMALL, E_UNSUPPORTED_CFG, E_CUDA
 
 EXPORTS = [
     "anakin_workspace_bytes", "anakin_create", "anakin_destroy", "anakin_reset", "anakin_rollout",
-    "anakin_rollout_forced", "anakin_learn", "anakin_gae", "anakin_update", "anakin_run", "anakin_get", "anakin_set",
+    "anakin_rollout_forced", "anakin_learn", "anakin_gae", "anakin_update", "anakin_grads", "anakin_apply_grads",
+    "anakin_run", "anakin_get", "anakin_set",
     "anakin_blob_bytes", "anakin_status", "anakin_launch_count", "anakin_strerror", "anakin_last_cuda_error",
     "anakin_profile_enable", "anakin_profile_read", "anakin_kernel_count", "anakin_kernel_name",
     "anakin_rollout_noalloc",
@@ -61,6 +62,8 @@ _lib.anakin_rollout_forced.argtypes = [_vp, C.c_int, _vp]
 _lib.anakin_learn.argtypes = [_vp]
 _lib.anakin_gae.argtypes = [_vp]
 _lib.anakin_update.argtypes = [_vp]
+_lib.anakin_grads.argtypes = [_vp]
+_lib.anakin_apply_grads.argtypes = [_vp]
 _lib.anakin_run.argtypes = [_vp, C.c_int]
 _lib.anakin_get.argtypes = [_vp, C.c_int, _vp, C.c_size_t, C.c_int]
 _lib.anakin_set.argtypes = [_vp, C.c_int, _vp, C.c_size_t, C.c_int]
@@ -102,20 +105,20 @@ def lib() -> C.CDLL:
 
 def make_cfg(B, N, H, T_max, precision=0, episode_cap=50, wall_density=0.2, gamma=0.99, gae_lambda=0.95,
              entropy_coef=0.01, value_coef=0.5, lr=3e-4, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8, device=0,
-             debug_logits=0) -> AnakinCfg:
+             debug_logits=0, env_offset=0) -> AnakinCfg:
     c = AnakinCfg()
     c.struct_size = C.sizeof(AnakinCfg)
     c.B, c.N, c.H, c.T_max, c.episode_cap, c.wall_density = B, N, H, T_max, episode_cap, wall_density
     c.gamma, c.gae_lambda, c.entropy_coef, c.value_coef = gamma, gae_lambda, entropy_coef, value_coef
     c.lr, c.adam_b1, c.adam_b2, c.adam_eps = lr, adam_b1, adam_b2, adam_eps
-    c.precision, c.device, c.debug_logits, c.reserved = precision, device, debug_logits, 0
+    c.precision, c.device, c.debug_logits, c.env_offset = precision, device, debug_logits, env_offset
     return c
 
 
-def cfg_from_workload(w, device=0, debug_logits=0, T_max=None) -> AnakinCfg:
+def cfg_from_workload(w, device=0, debug_logits=0, T_max=None, env_offset=0) -> AnakinCfg:
     return make_cfg(w.B, w.N, w.H, w.T if T_max is None else T_max, w.precision, w.episode_cap, w.wall_density, w.gamma,
                     w.gae_lambda, w.entropy_coef, w.value_coef, w.lr, w.adam_b1, w.adam_b2, w.adam_eps, device,
-                    debug_logits)
+                    debug_logits, env_offset)
 
 
 def workspace_bytes(cfg: AnakinCfg) -> int:
@@ -193,6 +196,12 @@ class Anakin:
     def update(self):
         self._ck(_lib.anakin_update(self._h))
 
+    def grads(self):
+        self._ck(_lib.anakin_grads(self._h))
+
+    def apply_grads(self):
+        self._ck(_lib.anakin_apply_grads(self._h))
+
     def run(self, iters: int):
         self._ck(_lib.anakin_run(self._h, iters))
 
@@ -214,9 +223,11 @@ class Anakin:
         self._ck(_lib.anakin_get(self._h, which, out.ctypes.data_as(_vp), n, 0))
         return out
 
-    def get_into(self, which: int, host: torch.Tensor):
-        """Copies a blob into a (pinned) host tensor of exactly the blob's size; synchronises."""
-        self._ck(_lib.anakin_get(self._h, which, _vp(host.data_ptr()), host.numel() * host.element_size(), 0))
+    def get_into(self, which: int, out: torch.Tensor):
+        """Copies a blob into a tensor of exactly the blob's size: a (pinned) host tensor (synchronises) or a CUDA
+        tensor on the handle's device (asynchronous, on the handle's stream)."""
+        assert out.is_contiguous()
+        self._ck(_lib.anakin_get(self._h, which, _vp(out.data_ptr()), out.numel() * out.element_size(), 1 if out.is_cuda else 0))
 
     def set(self, which: int, value):
         if which in (ADAM_STEP, GLOBAL_STEP):

@@ -42,7 +42,7 @@ int validate(const anakin_cfg* c) {
     if (c->B < 1 || c->T_max < 1 || c->episode_cap < 1 || c->episode_cap > 255) return ANAKIN_E_INVALID_ARG;
     if (!(c->wall_density >= 0.0 && c->wall_density < 1.0)) return ANAKIN_E_INVALID_ARG;
     if (c->precision != ANAKIN_PRECISION_FP32 && c->precision != ANAKIN_PRECISION_BF16) return ANAKIN_E_INVALID_ARG;
-    if (c->reserved != 0) return ANAKIN_E_INVALID_ARG;
+    if (c->env_offset < 0 || (double)c->env_offset + (double)c->B > 2147483647.0) return ANAKIN_E_INVALID_ARG;
     if (c->N < 2 || c->N > 16) return ANAKIN_E_UNSUPPORTED_CFG;
     const int hj = c->H / 32;
     if (c->H % 32 != 0) return ANAKIN_E_UNSUPPORTED_CFG;
@@ -145,7 +145,7 @@ Blob blob_of(anakin_t* h, int which) {
     const size_t B = d.B, T = h->last_T > 0 ? h->last_T : d.Tmax, R = B * T, P = d.P;
     switch (which) {
         case ANAKIN_PARAMS: return {b.theta, P * 4, true, false, false};
-        case ANAKIN_GRADS: return {b.grads, P * 4, false, false, false};
+        case ANAKIN_GRADS: return {b.grads, P * 4, true, false, false};
         case ANAKIN_ADAM_M: return {b.adam_m, P * 4, true, false, false};
         case ANAKIN_ADAM_V: return {b.adam_v, P * 4, true, false, false};
         case ANAKIN_ADAM_STEP: return {&h->adam_k, 8, true, true, false};
@@ -268,7 +268,8 @@ int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void
     const int rc = validate(cfg);
     if (rc != ANAKIN_OK) return rc;
     if (!dev_workspace || ((uintptr_t)dev_workspace & 255u)) return ANAKIN_E_INVALID_ARG;
-    const Dims d = make_dims(cfg->B, cfg->N, cfg->H, cfg->T_max);
+    Dims d = make_dims(cfg->B, cfg->N, cfg->H, cfg->T_max);
+    d.env0 = cfg->env_offset;
     const int NS = choose_splits(d);
     const size_t need = carve(*cfg, d, NS, nullptr, nullptr);
     if (bytes < need) return ANAKIN_E_WORKSPACE_TOO_SMALL;
@@ -339,8 +340,8 @@ int anakin_gae(anakin_t* h) {
     return ANAKIN_OK;
 }
 
-// The update proper, from ADV/RET as they stand.
-static int learn_after_gae(anakin_t* h) {
+// The update proper, from ADV/RET as they stand.  phase 0: through Adam; phase 1: stop at the batch-mean gradient.
+static int learn_after_gae(anakin_t* h, int phase) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
@@ -364,6 +365,7 @@ static int learn_after_gae(anakin_t* h) {
     a.beta2 = h->cfg.adam_b2;
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
+    a.phase = phase;
     {   // smallest power of two >= R: keeps the scaled output gradients O(1) for the fp16 operand format
         const double Rrows = (double)h->d.B * (double)h->last_T;
         int ex = 0;
@@ -381,12 +383,14 @@ static int learn_after_gae(anakin_t* h) {
         e = launch_learn(a, h->cfg.precision, h->ctx());
     }
     if (e != cudaSuccess) return fail_cuda(h, e);
-    h->adam_k += 1;
     h->adv_valid = false;
-    h->base_valid = false;  // parameters changed
-    h->frags_valid = tensor_path_supported(h->d.H, h->cfg.precision);  // the tensor-core update refreshes the 16-bit copies itself
     h->acts_valid = false;
     h->rollout_pending = false;
+    if (phase == 0) {
+        h->adam_k += 1;
+        h->base_valid = false;  // parameters changed
+        h->frags_valid = tensor_path_supported(h->d.H, h->cfg.precision);  // the tensor-core update refreshes the 16-bit copies itself
+    }
     return ANAKIN_OK;
 }
 
@@ -397,13 +401,43 @@ int anakin_learn(anakin_t* h) {
         const int rc = anakin_gae(h);
         if (rc != ANAKIN_OK) return rc;
     }
-    return learn_after_gae(h);
+    return learn_after_gae(h, 0);
 }
 
 int anakin_update(anakin_t* h) {
     if (!h) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
-    return learn_after_gae(h);
+    return learn_after_gae(h, 0);
+}
+
+int anakin_grads(anakin_t* h) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
+    if (!h->adv_valid) {
+        const int rc = anakin_gae(h);
+        if (rc != ANAKIN_OK) return rc;
+    }
+    return learn_after_gae(h, 1);
+}
+
+int anakin_apply_grads(anakin_t* h) {
+    if (!h) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset) return ANAKIN_E_BAD_STATE;
+    LearnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.d = h->d;
+    a.b = h->b;
+    a.lr = h->cfg.lr;
+    a.beta1 = h->cfg.adam_b1;
+    a.beta2 = h->cfg.adam_b2;
+    a.eps = h->cfg.adam_eps;
+    a.adam_k = (int)(h->adam_k + 1);
+    const cudaError_t e = launch_adam_only(a, h->cfg.precision, h->ctx());
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->adam_k += 1;
+    h->base_valid = false;  // parameters changed
+    h->frags_valid = tensor_path_supported(h->d.H, h->cfg.precision);  // every element of the 16-bit copies of W2 was rewritten
+    return ANAKIN_OK;
 }
 
 int anakin_run(anakin_t* h, int iters) {

@@ -21,11 +21,13 @@ enum : int {
 
 struct Dims {
     int B, N, C, D, H, W, Tmax;  // envs, grid side, cells, obs features, hidden, wall words per env, max T
+    int env0;                    // global index of env 0 (Philox counters use env0 + b)
     size_t oW1, ob1, oW2, ob2, oWh, obh, P;
 };
 
 inline Dims make_dims(int B, int N, int H, int Tmax) {
     Dims d;
+    d.env0 = 0;
     d.B = B; d.N = N; d.C = N * N; d.D = 3 * d.C; d.H = H; d.W = (d.C + 31) / 32; d.Tmax = Tmax;
     d.oW1 = 0;
     d.ob1 = d.oW1 + (size_t)d.D * H;
@@ -139,6 +141,7 @@ struct LearnArgs {
     float c_v, c_e;
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
+    int phase;   // 0: reduce the partials and apply Adam; 1: reduce only (GRADS and loss statistics)
     // tensor-pipe path
     int ts;               // t-slices of the dh1 kernel: S holds ts*B rows (slice z, env b at row z*B + b)
     float gscale, inv_gscale;  // power of two carried by every gradient-side tensor, divided out in the reduction
@@ -234,6 +237,7 @@ cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx&
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c);
+cudaError_t launch_adam_only(const LearnArgs& a, int prec, const Ctx& c);  // Adam from GRADS as they stand
 cudaError_t launch_dh1_tc(const LearnArgs& a, int prec, cudaStream_t s);  // tcgen05 dh1 kernel; cudaErrorNotSupported if not covered  // needs the activations the rollout saved
 cudaError_t launch_refresh_compute_params(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 

@@ -25,7 +25,7 @@ __device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, i
     const float x0 = expf(l0 - mx), x1 = expf(l1 - mx), x2 = expf(l2 - mx), x3 = expf(l3 - mx);
     const float Z = ((x0 + x1) + x2) + x3;
     const float c0 = x0 / Z, c1 = c0 + x1 / Z, c2 = c1 + x2 / Z;
-    const U4 r = philox4x32_10((uint32_t)env, a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
+    const U4 r = philox4x32_10((uint32_t)(a.d.env0 + env), a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
     const float u = uniform24(r.x);
     int act = (u >= c0) + (u >= c1) + (u >= c2);
     if (a.forced) {

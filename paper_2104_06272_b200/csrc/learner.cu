@@ -285,16 +285,18 @@ __global__ void __launch_bounds__(256) k_reduce_adam(LearnArgs a, size_t R, int 
         float g = 0.f;
         for (int s = 0; s < a.NS; ++s) g += b.part[(size_t)s * d.P + i];
         b.grads[i] = g;
-        const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * g;
-        const float v = a.beta2 * b.adam_v[i] + (1.f - a.beta2) * g * g;
-        b.adam_m[i] = m;
-        b.adam_v[i] = v;
-        const float mhat = m / s_c[0], vhat = v / s_c[1];
-        const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
-        b.theta[i] = th;
-        if (PREC == 1) {
-            const bool is_bias = (i >= d.ob1 && i < d.oW2) || (i >= d.ob2 && i < d.oWh) || i >= d.obh;
-            b.theta_c[i] = is_bias ? th : round_bf16(th);
+        if (a.phase == 0) {  // phase 1 stops at the gradient
+            const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * g;
+            const float v = a.beta2 * b.adam_v[i] + (1.f - a.beta2) * g * g;
+            b.adam_m[i] = m;
+            b.adam_v[i] = v;
+            const float mhat = m / s_c[0], vhat = v / s_c[1];
+            const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
+            b.theta[i] = th;
+            if (PREC == 1) {
+                const bool is_bias = (i >= d.ob1 && i < d.oW2) || (i >= d.ob2 && i < d.oWh) || i >= d.obh;
+                b.theta_c[i] = is_bias ? th : round_bf16(th);
+            }
         }
     }
     if (blockIdx.x == 0 && threadIdx.x < 3) {

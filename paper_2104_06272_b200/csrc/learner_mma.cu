@@ -579,6 +579,57 @@ static cudaError_t launch_gemm_tn(const GemmTnArgs& g, int rows_m, int splits, c
     return cudaGetLastError();
 }
 
+// One Adam step of parameter i with gradient g (Kingma & Ba, Algorithm 1), plus the refreshed 16-bit copies.
+// c[0] = 1 - beta1^k, c[1] = 1 - beta2^k.
+template <int PREC>
+__device__ __forceinline__ void adam_step(const LearnArgs& a, const float* c, size_t i, float g) {
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * g;
+    const float v = a.beta2 * b.adam_v[i] + (1.f - a.beta2) * g * g;
+    b.adam_m[i] = m;
+    b.adam_v[i] = v;
+    const float mhat = m / c[0], vhat = v / c[1];
+    const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
+    b.theta[i] = th;
+    float thc = th;
+    if (PREC == 1) {
+        const bool is_bias = (i >= d.ob1 && i < d.oW2) || (i >= d.ob2 && i < d.oWh) || i >= d.obh;
+        thc = is_bias ? th : round_bf16(th);
+        b.theta_c[i] = thc;
+    }
+    // refresh the tensor-pipe copies of W2 in place (fragment layouts as in k_pack_w2, and the row-major planes)
+    if (b.w2p_hi && i >= d.oW2 && i < d.ob2) {
+        const int H = d.H;
+        const int k = (int)((i - d.oW2) / H), n = (int)((i - d.oW2) % H);
+        uint16_t hi, lo;
+        split1<PREC>(thc, hi, lo);
+        if (b.w2f_hi) {
+            const size_t ef = ((size_t)((k >> 4) * (H / 8) + (n >> 3)) * 32 + (n & 7) * 4 + ((k & 7) >> 1)) * 4 + ((k & 15) >> 3) * 2 + (k & 1);
+            const size_t et = ((size_t)((n >> 4) * (H / 8) + (k >> 3)) * 32 + (k & 7) * 4 + ((n & 7) >> 1)) * 4 + ((n & 15) >> 3) * 2 + (n & 1);
+            reinterpret_cast<uint16_t*>(b.w2f_hi)[ef] = hi;
+            reinterpret_cast<uint16_t*>(b.w2f_lo)[ef] = lo;
+            reinterpret_cast<uint16_t*>(b.w2tf_hi)[et] = hi;
+            reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
+        }
+        b.w2p_hi[i - d.oW2] = hi;
+        if (b.w2p_lo) b.w2p_lo[i - d.oW2] = lo;
+    }
+}
+
+// Adam from the GRADS blob as it stands (the second half of an update whose gradient was averaged over replicas).
+template <int PREC>
+__global__ void __launch_bounds__(256) k_adam_only(LearnArgs a) {
+    __shared__ float s_c[2];
+    if (threadIdx.x == 0) {
+        s_c[0] = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
+        s_c[1] = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
+    }
+    __syncthreads();
+    const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    if (i < a.d.P) adam_step<PREC>(a, s_c, i, a.b.grads[i]);
+}
+
 // ----------------------------------------------------------------------------------------------------
 // k_reduce_adam2: fixed-order sums of each parameter region's partials, then Adam (Kingma & Ba, Algorithm 1).
 // ----------------------------------------------------------------------------------------------------
@@ -592,40 +643,11 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
         s_c[1] = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
     }
     __syncthreads();
-    // Applies the batch-mean gradient of parameter i: statistics, Adam, refreshed 16-bit copies.
+    // Batch-mean gradient of parameter i, then (phase 0) its Adam step.
     auto apply = [&](size_t i, float gsum) {
         gsum *= a.inv_gscale;  // exact: a power of two
         b.grads[i] = gsum;
-        const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * gsum;
-        const float v = a.beta2 * b.adam_v[i] + (1.f - a.beta2) * gsum * gsum;
-        b.adam_m[i] = m;
-        b.adam_v[i] = v;
-        const float mhat = m / s_c[0], vhat = v / s_c[1];
-        const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
-        b.theta[i] = th;
-        float thc = th;
-        if (PREC == 1) {
-            const bool is_bias = (i >= d.ob1 && i < d.oW2) || (i >= d.ob2 && i < d.oWh) || i >= d.obh;
-            thc = is_bias ? th : round_bf16(th);
-            b.theta_c[i] = thc;
-        }
-        // refresh the tensor-pipe copies of W2 in place (fragment layouts as in k_pack_w2, and the row-major planes)
-        if (i >= d.oW2 && i < d.ob2) {
-            const int H = d.H;
-            const int k = (int)((i - d.oW2) / H), n = (int)((i - d.oW2) % H);
-            uint16_t hi, lo;
-            split1<PREC>(thc, hi, lo);
-            const size_t ef = ((size_t)((k >> 4) * (H / 8) + (n >> 3)) * 32 + (n & 7) * 4 + ((k & 7) >> 1)) * 4 + ((k & 15) >> 3) * 2 + (k & 1);
-            const size_t et = ((size_t)((n >> 4) * (H / 8) + (k >> 3)) * 32 + (k & 7) * 4 + ((n & 7) >> 1)) * 4 + ((n & 15) >> 3) * 2 + (n & 1);
-            if (b.w2f_hi) {
-                reinterpret_cast<uint16_t*>(b.w2f_hi)[ef] = hi;
-                reinterpret_cast<uint16_t*>(b.w2f_lo)[ef] = lo;
-                reinterpret_cast<uint16_t*>(b.w2tf_hi)[et] = hi;
-                reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
-            }
-            b.w2p_hi[i - d.oW2] = hi;
-            if (b.w2p_lo) b.w2p_lo[i - d.oW2] = lo;
-        }
+        if (a.phase == 0) adam_step<PREC>(a, s_c, i, gsum);
     };
     auto region_of = [&](size_t i) {
         int r = 0;
@@ -891,6 +913,14 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         CK(cudaGetLastError());
     }
     return cudaSuccess;
+}
+
+cudaError_t launch_adam_only(const LearnArgs& a, int prec, const Ctx& c) {
+    Scope sc(c, K_REDUCE_ADAM);
+    const unsigned nb = (unsigned)((a.d.P + 255) / 256);
+    if (prec == 1) k_adam_only<1><<<nb, 256, 0, c.s>>>(a);
+    else k_adam_only<0><<<nb, 256, 0, c.s>>>(a);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c) {

@@ -73,6 +73,7 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     RolloutArgs a;
     memset(&a, 0, sizeof(a));
     a.d = make_dims(cfg->B, cfg->N, cfg->H, cfg->T_max);
+    a.d.env0 = cfg->env_offset;
     Buffers& b = a.b;
     b.theta = b.theta_c = const_cast<float*>(dev_params);
     b.walls = const_cast<uint32_t*>(dev_walls);

@@ -10,13 +10,14 @@ namespace anakin {
 __global__ void __launch_bounds__(128) k_reset_env(Dims d, Buffers b, uint32_t k0, uint32_t k1, uint32_t thr) {
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= d.B) return;
-    const U4 x = philox4x32_10((uint32_t)e, 0, 0, STREAM_ENV, k0, k1);
+    const uint32_t ge = (uint32_t)(d.env0 + e);  // global env index
+    const U4 x = philox4x32_10(ge, 0, 0, STREAM_ENV, k0, k1);
     const uint32_t s = (uint32_t)(((uint64_t)x.x * (uint32_t)d.C) >> 32);
     uint32_t g = (uint32_t)(((uint64_t)x.y * (uint32_t)(d.C - 1)) >> 32);
     if (g >= s) g += 1;
     uint32_t word = 0;
     for (int c4 = 0; c4 * 4 < d.C; ++c4) {
-        const U4 y = philox4x32_10((uint32_t)e, (uint32_t)(1 + c4), 0, STREAM_ENV, k0, k1);
+        const U4 y = philox4x32_10(ge, (uint32_t)(1 + c4), 0, STREAM_ENV, k0, k1);
         const uint32_t ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {

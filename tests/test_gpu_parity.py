@@ -251,7 +251,7 @@ def test_state_errors(bnd):
     with pytest.raises(bnd.AnakinError):
         an.learn()  # the rollout was consumed
     with pytest.raises(bnd.AnakinError):
-        an.set(bnd.GRADS, np.zeros(an.P, np.float32))  # read-only blob
+        an.set(bnd.STATS, torch.zeros(an.blob_bytes(bnd.STATS), dtype=torch.uint8))  # read-only blob
     with pytest.raises(bnd.AnakinError):
         an.set(bnd.PARAMS, np.zeros(an.P - 1, np.float32))  # wrong size
     # a forced action outside 0..3 sets the sticky device status instead of faulting
