@@ -104,7 +104,7 @@ def kernel_work(w):
     p3 = 1 if w.precision == 1 else 3
     p2 = 1 if w.precision == 1 else 2
     pl = 2 if w.precision == 1 else 4  # bytes per element of a 16-bit operand stored as (hi[, lo]) planes
-    return {
+    work = {
         # name: (bound, executed flops, bytes)
         "rollout": ("tensor", p3 * 2.0 * B * (T + 1) * H * H, R * (15.0 + pl * H + 4.0 * H) + B * 4),
         "dh1": ("tensor", p3 * 2.0 * R * H * H, R * H * (2.0 * pl + 2.0)),
@@ -119,6 +119,20 @@ def kernel_work(w):
         "reduce_adam": ("hbm", P * 12.0, P * 28.0),
         "replay": ("tensor", p3 * 2.0 * R * H * H, R * H * (pl + 4.0)),
     }
+    if w.precision == 1 and H in (512, 1024):
+        # wide bf16 path: three launches per env step (h1 gather, layer-2 GEMM, heads + env step), bf16 activations in HBM
+        work.update({
+            "h1": ("hbm", B * H * 2.0, B * H * (4.0 + 2.0) + B),                  # per step: base fp32 in, h1 bf16 out
+            "fwd2": ("tensor", 2.0 * B * H * H, B * H * 4.0 + H * H * 2.0),       # per step: h1 in, h2 out, W2
+            "rollout": ("hbm", B * H * 10.0, B * H * 2.0 + B * 47.0),             # per step: h2 in, records out
+            "heads_bwd": ("hbm", R * H * 22.0, R * H * 4.0 + R * 42.0),           # h2 in, dh2 out (bf16 each)
+            "dh1": ("tensor", 2.0 * R * H * H, R * H * 6.0),                      # dh2 in, h1 gates in, dh1 out
+            "sum_over_t": ("hbm", R * H * 1.0, R * H * 2.0 + B * H * 4.0),
+            "dw2": ("tensor", 2.0 * R * H * H, R * H * 4.0),
+            "dw1_agent": ("tensor", 2.0 * R * C * H, R * H * 2.0 + R),
+            "env_base": ("tensor", 2.0 * B * C * H, B * H * 4.0 + B * C * 2.0),   # two launches: operand expansion + GEMM
+        })
+    return work
 
 
 def max_over_ranks(value: float, world: int, device="cpu") -> float:
