@@ -87,6 +87,11 @@ class ClockSampler:
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu capture
+# summarised under profiles/ for the same kernel source; None for workloads without a capture at full size.
+NCU_TRAFFIC_BYTES = {("throughput", "rollout"): 5.5e6 + 221.0e6}
+
+
 def workload_label(w):
     return (f"{w.name}: B={w.B} envs, {w.N}x{w.N} gridworld (obs {w.D}), MLP {w.D}-{w.H}-{w.H}+5, "
             f"{'fp32' if w.precision == 0 else 'bf16'}, T={w.T}")
@@ -297,7 +302,7 @@ def run_ours(args):
         achieved, peak, unit = nbytes / per_launch_s / 1e9, peaks["hbm_gbs"], "GB/s"
         peak_note = f"HBM copy bandwidth, {peaks['source']}"
     roofline = {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": None, "peak_source": peak_note, "us_per_launch": per_launch_s * 1e6,
+                "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)), "peak_source": peak_note, "us_per_launch": per_launch_s * 1e6,
                 "share_of_step": top_ms / tot,
                 "kernels": {k: kernel_line(k, ms, n) for k, (ms, n) in sorted(prof.items(), key=lambda kv: -kv[1][0])}}
 

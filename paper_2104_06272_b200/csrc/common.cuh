@@ -238,6 +238,9 @@ cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, floa
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_adam_only(const LearnArgs& a, int prec, const Ctx& c);  // Adam from GRADS as they stand
+bool dh1_agent_tc_supported(const Dims& d);
+// dh1, S and the agent plane of dW1 in one tcgen05 kernel; cudaErrorNotSupported if not covered
+cudaError_t launch_dh1_agent_tc(const LearnArgs& a, int prec, int grid_x, float* part_agent, size_t part_stride, cudaStream_t s);
 cudaError_t launch_dh1_tc(const LearnArgs& a, int prec, cudaStream_t s);  // tcgen05 dh1 kernel; cudaErrorNotSupported if not covered  // needs the activations the rollout saved
 cudaError_t launch_refresh_compute_params(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 

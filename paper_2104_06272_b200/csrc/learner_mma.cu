@@ -732,6 +732,22 @@ static int splits_for(int K, int tiles, int min_k) {
     return ns < 1 ? 1 : ns;
 }
 
+// Launch shape of the fused dh1 + agent-plane kernel: one CTA per SM.  Few env tiles: slice the steps; many: let a CTA
+// walk several tiles, so that the number of agent-plane partials stays at most one per CTA row.
+static void dh1a_shape(const Dims& d, int T, int* grid_x, int* ts) {
+    const int m_tiles = (d.B + 127) / 128, n_tiles = d.H / 64;
+    *grid_x = m_tiles;
+    *ts = 1;
+    if (m_tiles * n_tiles >= 148) {
+        *grid_x = 148 / n_tiles > 0 ? 148 / n_tiles : 1;
+    } else {
+        int t = 148 / (m_tiles * n_tiles);
+        if (t > 4) t = 4;
+        if (t > T) t = T;
+        if (t >= 2) *ts = t;
+    }
+}
+
 void learn_mma_plan(const Dims& d, LearnPlan* p) {
     const int H = d.H, C = d.C;
     const size_t R = (size_t)d.B * d.Tmax;
@@ -745,6 +761,11 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     }
     p->ns_w2 = splits_for((int)R, tiles_hh, 256);
     p->ns_agent = splits_for((int)R, tiles_agent, 256);
+    if (dh1_agent_tc_supported(d)) {  // the fused kernel writes one agent-plane partial per (CTA row, t slice)
+        int gx, ts;
+        dh1a_shape(d, d.Tmax, &gx, &ts);
+        if (gx * ts > p->ns_agent) p->ns_agent = gx * ts;
+    }
     p->ns_env = splits_for(d.B, tiles_ch, 128);
     const size_t tiles32 = (R + 31) / 32;
     p->heads_grid = (int)(tiles32 < (size_t)HEADS_GRID ? tiles32 : (size_t)HEADS_GRID);
@@ -820,14 +841,31 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     // t-slices: the tcgen05 dh1 kernel has ceil(B/128)*(H/128) CTAs per slice; slice the T steps so that one wave of
     // CTAs covers the SMs.  The mma.sync fall-back keeps one slice.
     a.ts = 1;
-    if (H == 128 || H == 256) {
+    bool fused_agent = false;  // dh1, S and the agent plane of dW1 in one kernel (dh1 stays on chip)
+    if (!wide && dh1_agent_tc_supported(d)) {
+        int gx, ts;
+        dh1a_shape(d, T, &gx, &ts);
+        a.ts = ts;
+        Scope sc(c, K_DH1);
+        const cudaError_t ef = launch_dh1_agent_tc(a, PREC, gx, b.part + pl.off_agent, CH, s);
+        if (ef == cudaSuccess) {
+            fused_agent = true;
+            a.reg[1].ns = gx * ts;
+        } else if (ef != cudaErrorNotSupported) {
+            return ef;
+        } else {
+            a.ts = 1;
+        }
+    }
+    if (!fused_agent && (H == 128 || H == 256)) {
         const int per_slice = ((B + 127) / 128) * (H / 128);
         int ts = 148 / per_slice;
         if (ts > 4) ts = 4;
         if (ts > T) ts = T;
         if (ts >= 2) a.ts = ts;
     }
-    if (wide) {
+    if (fused_agent) {
+    } else if (wide) {
         CK(launch_dh1_wide(a, c));
     } else {
         Scope sc(c, K_DH1);
@@ -867,7 +905,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     g.idx = b.tpos;
     g.Bhi = dh1hi; g.Blo = dh1hi + RH;
     g.part = b.part + pl.off_agent; g.stride = CH; g.off = 0;
-    {
+    if (!fused_agent) {
         Scope sc(c, K_DW1_AGENT);
         cudaError_t e = launch_gemm_tn_tc(g, A_ONEHOT, 1, PL, PREC, pl.ns_agent, b.status, s);
         if (e == cudaErrorNotSupported) {
