@@ -14,19 +14,49 @@ struct EnvLane {
     int bad;
 };
 
+// The part of an interaction that does not depend on the policy's output: the Philox uniform of (env, step) and, for
+// each of the four actions, the cell the agent would end up in.  A kernel can compute it while it waits for memory or
+// for the tensor pipe, so that only the softmax and the selection remain once the logits are known.
+struct StepPre {
+    float u;
+    int np[4];  // 0 up, 1 right, 2 down, 3 left; blocked moves stay in place
+};
+
 // walls: this env's wall words (shared memory), 8 words.
-__device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
-                                             float l3, const uint32_t* walls) {
-    const Buffers& b = a.b;
+__device__ __forceinline__ StepPre step_prepare(const EnvLane& s, const RolloutArgs& a, int env, int t, const uint32_t* walls) {
+    StepPre p;
+    const U4 r = philox4x32_10((uint32_t)(a.d.env0 + env), a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
+    p.u = uniform24(r.x);
     const int N = a.d.N;
+    const int row = s.pos / N, col = s.pos - row * N;
+#pragma unroll
+    for (int act = 0; act < 4; ++act) {
+        int nr = row, nc = col;
+        if (act == 0) nr = row - 1;
+        else if (act == 1) nc = col + 1;
+        else if (act == 2) nr = row + 1;
+        else nc = col - 1;
+        int np = s.pos;
+        if (nr >= 0 && nr < N && nc >= 0 && nc < N) {
+            const int cand = nr * N + nc;
+            if (!((walls[cand >> 5] >> (cand & 31)) & 1u)) np = cand;
+        }
+        p.np[act] = np;
+    }
+    return p;
+}
+
+// Categorical sampling from the 4 logits (inverse CDF against the prepared uniform), the env transition and the records.
+__device__ __forceinline__ void act_and_step_pre(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
+                                                 float l3, const StepPre& pre) {
+    const Buffers& b = a.b;
     const size_t i = (size_t)t * a.d.B + env;
     // softmax and inverse CDF: c0 = p0, c1 = c0 + p1, c2 = c1 + p2; a = [u>=c0] + [u>=c1] + [u>=c2]
     const float mx = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
     const float x0 = expf(l0 - mx), x1 = expf(l1 - mx), x2 = expf(l2 - mx), x3 = expf(l3 - mx);
     const float Z = ((x0 + x1) + x2) + x3;
     const float c0 = x0 / Z, c1 = c0 + x1 / Z, c2 = c1 + x2 / Z;
-    const U4 r = philox4x32_10((uint32_t)(a.d.env0 + env), a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
-    const float u = uniform24(r.x);
+    const float u = pre.u;
     int act = (u >= c0) + (u >= c1) + (u >= c2);
     if (a.forced) {
         act = a.forced[i];
@@ -37,18 +67,7 @@ __device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, i
     b.tpos[i] = (uint8_t)s.pos;
     b.tact[i] = (int8_t)act;
     if (b.dbg_logits) reinterpret_cast<float4*>(b.dbg_logits)[i] = make_float4(l0, l1, l2, l3);
-    // gridworld: 0 up, 1 right, 2 down, 3 left; blocked moves stay in place
-    const int row = s.pos / N, col = s.pos - row * N;
-    int nr = row, nc = col;
-    if (act == 0) nr = row - 1;
-    else if (act == 1) nc = col + 1;
-    else if (act == 2) nr = row + 1;
-    else nc = col - 1;
-    int np = s.pos;
-    if (nr >= 0 && nr < N && nc >= 0 && nc < N) {
-        const int cand = nr * N + nc;
-        if (!((walls[cand >> 5] >> (cand & 31)) & 1u)) np = cand;
-    }
+    const int np = act == 0 ? pre.np[0] : act == 1 ? pre.np[1] : act == 2 ? pre.np[2] : pre.np[3];
     const int te = s.tep + 1;
     float rew = 0.f;
     int done = 0;
@@ -66,6 +85,12 @@ __device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, i
     }
     b.trew[i] = rew;
     b.tdone[i] = (uint8_t)done;
+}
+
+__device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
+                                             float l3, const uint32_t* walls) {
+    const StepPre pre = step_prepare(s, a, env, t, walls);
+    act_and_step_pre(s, a, env, t, l0, l1, l2, l3, pre);
 }
 
 // Warp 0 holds every owner thread: fold the per-env counters and add them with integer atomics (order-free totals).

@@ -144,34 +144,39 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
             if (tid < ME) s_pos[tid] = owner ? b.tpos[(size_t)t * B + e0 + tid] : 0;
             __syncthreads();
         }
-        // ---- layer 1: pairs of consecutive hidden units per thread.  All gathers of the agent's W1 row are issued
+        // ---- layer 1: eight consecutive hidden units per thread and trip.  All gathers of the agent's W1 row are issued
         // before any is used (one L2 round trip per step, not one per trip); the fp16 planes go to shared memory for
-        // the MMAs and, for the update's reuse, straight to global memory (4 bytes per lane, 128 bytes per warp).
+        // the MMAs and, for the update's reuse, straight to global memory (16 bytes per lane).
         {
-            constexpr int TRIPS = ME * H / 2 / NTHREADS;
-            static_assert(TRIPS * NTHREADS == ME * H / 2, "layer-1 trips must tile the h1 block");
+            constexpr int TRIPS = ME * H / 8 / NTHREADS;
+            static_assert(TRIPS * NTHREADS == ME * H / 8, "layer-1 trips must tile the h1 block");
             const bool save_h1 = b.h1 != nullptr && t < a.T;
-            float2 w[TRIPS];
+            float4 w[TRIPS][2];
 #pragma unroll
             for (int i = 0; i < TRIPS; ++i) {
                 const int p = tid + i * NTHREADS;
-                const int e = p / (H / 2), k = 2 * (p - e * (H / 2));
-                w[i] = __ldg(reinterpret_cast<const float2*>(W1 + (size_t)(C + s_pos[e]) * H + k));
+                const int e = p / (H / 8), k = 8 * (p - e * (H / 8));
+                const float4* wp = reinterpret_cast<const float4*>(W1 + (size_t)(C + s_pos[e]) * H + k);
+                w[i][0] = __ldg(wp);
+                w[i][1] = __ldg(wp + 1);
             }
 #pragma unroll
             for (int i = 0; i < TRIPS; ++i) {
                 const int p = tid + i * NTHREADS;
-                const int e = p / (H / 2), k = 2 * (p - e * (H / 2));
-                const float2 bs = *reinterpret_cast<const float2*>(s_base + e * H + k);
-                const float z0 = fmaxf(bs.x + w[i].x, 0.f), z1 = fmaxf(bs.y + w[i].y, 0.f);
-                uint32_t phi, plo;
-                split2<PREC>(z0, z1, phi, plo);
-                if (PREC == 0) *reinterpret_cast<uint32_t*>(s_h1lo + e * LD + k) = plo;
-                *reinterpret_cast<uint32_t*>(s_h1hi + e * LD + k) = phi;
+                const int e = p / (H / 8), k = 8 * (p - e * (H / 8));
+                const float4 b0 = *reinterpret_cast<const float4*>(s_base + e * H + k);
+                const float4 b1 = *reinterpret_cast<const float4*>(s_base + e * H + k + 4);
+                uint4 hi, lo;
+                split2<PREC>(fmaxf(b0.x + w[i][0].x, 0.f), fmaxf(b0.y + w[i][0].y, 0.f), hi.x, lo.x);
+                split2<PREC>(fmaxf(b0.z + w[i][0].z, 0.f), fmaxf(b0.w + w[i][0].w, 0.f), hi.y, lo.y);
+                split2<PREC>(fmaxf(b1.x + w[i][1].x, 0.f), fmaxf(b1.y + w[i][1].y, 0.f), hi.z, lo.z);
+                split2<PREC>(fmaxf(b1.z + w[i][1].z, 0.f), fmaxf(b1.w + w[i][1].w, 0.f), hi.w, lo.w);
+                if (PREC == 0) *reinterpret_cast<uint4*>(s_h1lo + e * LD + k) = lo;
+                *reinterpret_cast<uint4*>(s_h1hi + e * LD + k) = hi;
                 if (save_h1 && e0 + e < B) {
                     const size_t gi = ((size_t)t * B + e0 + e) * H + k;
-                    *reinterpret_cast<uint32_t*>(g_h1hi + gi) = phi;
-                    if (PREC == 0) *reinterpret_cast<uint32_t*>(g_h1lo + gi) = plo;
+                    *reinterpret_cast<uint4*>(g_h1hi + gi) = hi;
+                    if (PREC == 0) *reinterpret_cast<uint4*>(g_h1lo + gi) = lo;
                 }
             }
         }
@@ -251,20 +256,26 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
                         }
                 }
             }
+            // sum over the four lanes of a quad with a transposing exchange: after two rounds lane t4 holds the total
+            // of ONE of the four rows (15 shuffles instead of 40), and every lane stores its row
+            float q2[2][5];
+            const bool b0 = t4 & 1, b1 = t4 & 2;
 #pragma unroll
-            for (int r = 0; r < 4; ++r)
+            for (int c = 0; c < 5; ++c) {
 #pragma unroll
-                for (int c = 0; c < 5; ++c) {
-                    ps[r][c] += __shfl_xor_sync(0xFFFFFFFFu, ps[r][c], 1);
-                    ps[r][c] += __shfl_xor_sync(0xFFFFFFFFu, ps[r][c], 2);
+                for (int i = 0; i < 2; ++i) {
+                    const float send = b0 ? ps[i][c] : ps[2 + i][c];
+                    const float keep = b0 ? ps[2 + i][c] : ps[i][c];
+                    q2[i][c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 1);
                 }
-            if (t4 == 0) {
+            }
+            const int r = (b0 ? 2 : 0) + (b1 ? 1 : 0);
+            const int row = 16 * (r >> 1) + 8 * (r & 1) + g;
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const int row = 16 * (r >> 1) + 8 * (r & 1) + g;
-#pragma unroll
-                    for (int c = 0; c < 5; ++c) s_red[(wid * ME + row) * 5 + c] = ps[r][c];
-                }
+            for (int c = 0; c < 5; ++c) {
+                const float send = b1 ? q2[0][c] : q2[1][c];
+                const float keep = b1 ? q2[1][c] : q2[0][c];
+                s_red[(wid * ME + row) * 5 + c] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 2);
             }
         }
         __syncthreads();
