@@ -35,6 +35,8 @@ struct Dh1aCfg {
     static constexpr int A_STAGE = PL * A_BOX;
     static constexpr int D_TILE = PL * BM * 128;         // dh1 tile: 128 k-rows (envs) x 64 cols, MN-major, hi (and lo)
     static constexpr int O_TILE = 2 * BM * 128;          // one-hot tile: 128 k-rows (envs) x 128 cells (two 64-wide boxes)
+    static constexpr int ACCW = PL * BN;                 // accumulator width: the hi x lo term has its own 64 columns
+    static constexpr int TMEM_COLS = 3 * ACCW <= 256 ? 256 : 512;
     static constexpr int BARS = 256;
     static constexpr int MAX_SMEM = 232448 - 1024;       // 227 KB per CTA minus alignment slack
     static constexpr int RING = MAX_SMEM - BARS - W_BYTES - D_TILE - O_TILE;
@@ -51,9 +53,10 @@ template <int H, int PREC>
 __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1aMaps maps, LearnArgs a, float* part_agent, size_t part_stride) {
     using Cfg = Dh1aCfg<H, PREC>;
     constexpr int BM = Cfg::BM, BN = Cfg::BN, KC = Cfg::KC, PL = Cfg::PL, NCH = Cfg::NCH, STAGES = Cfg::STAGES;
+    constexpr int PREFETCH = 3 * NCH;  // chunks between the L2 prefetch of a box and its load (three steps)
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    unsigned char* sW = base;                                   // [PL][NCH] boxes
+    unsigned char* sW = base;                                   // [NCH][PL] boxes: the lo box follows the hi box of its k chunk
     unsigned char* sA = sW + Cfg::W_BYTES;                      // [STAGES][PL] boxes
     unsigned char* sD = sA + STAGES * Cfg::A_STAGE;             // dh1 tile, hi plane then lo plane
     unsigned char* sO = sD + Cfg::D_TILE;                       // one-hot tile, two boxes of 64 cells
@@ -86,7 +89,7 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
         tc::mbar_init(tiles_free, 1);
         tc::mbar_fence_init();
     }
-    if (wid == 2) tc::tmem_alloc(tmem_slot, 256);
+    if (wid == 2) tc::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
     // the one-hot tile starts all zero; every step clears the element it set the step before
     for (int i = tid; i < Cfg::O_TILE / 16; i += Cfg::THREADS) reinterpret_cast<uint4*>(sO)[i] = make_uint4(0u, 0u, 0u, 0u);
     tc::fence_proxy_async();
@@ -94,7 +97,8 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t acc_agent = tmem + 2 * BN;
+    constexpr int ACCW = Cfg::ACCW;
+    const uint32_t acc_agent = tmem + 2 * ACCW;
     int my_tiles = 0;  // env tiles this CTA walks
     for (int mt = blockIdx.x; mt < m_tiles; mt += gridDim.x) ++my_tiles;
     const int G = my_tiles * nsteps;  // steps of this CTA, all env tiles together (the pipelines run across tiles)
@@ -105,12 +109,21 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
             tc::mbar_expect_tx(wfull, Cfg::W_BYTES);
 #pragma unroll
             for (int kc = 0; kc < NCH; ++kc) {
-                tc::tma_load_2d(sW + kc * Cfg::W_BOX, &maps.w_hi, wfull, kc * KC, n0);
-                if (PL == 2) tc::tma_load_2d(sW + (NCH + kc) * Cfg::W_BOX, &maps.w_lo, wfull, kc * KC, n0);
+                tc::tma_load_2d(sW + PL * kc * Cfg::W_BOX, &maps.w_hi, wfull, kc * KC, n0);
+                if (PL == 2) tc::tma_load_2d(sW + (PL * kc + 1) * Cfg::W_BOX, &maps.w_lo, wfull, kc * KC, n0);
             }
             for (int c = 0; c < G * NCH && ok; ++c) {
                 const int s = c % STAGES, g = c / NCH, kc = c - g * NCH;
                 const int e0 = ((int)blockIdx.x + (g / nsteps) * (int)gridDim.x) * BM, t = t0 + g % nsteps;
+                {   // pull the boxes of a later chunk towards L2 now, so that their TMA load is an L2 hit
+                    const int cp = c + PREFETCH;
+                    if (cp < G * NCH) {
+                        const int gp = cp / NCH, kp = cp - gp * NCH;
+                        const int ep = ((int)blockIdx.x + (gp / nsteps) * (int)gridDim.x) * BM, tp = t0 + gp % nsteps;
+                        tc::tma_prefetch_2d(&maps.a_hi, kp * KC, tp * B + ep);
+                        if (PL == 2) tc::tma_prefetch_2d(&maps.a_lo, kp * KC, tp * B + ep);
+                    }
+                }
                 if (c >= STAGES) ok = tc::mbar_wait(&empty[s], ((c / STAGES) - 1) & 1);
                 if (!ok) break;
                 tc::mbar_expect_tx(&full[s], Cfg::A_STAGE);
@@ -123,9 +136,13 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
         }
     } else if (wid == 1) {
         if (lane == 0) {  // ---- MMA issuer
+            // Operand fetch from shared memory bounds these MMAs, so terms that share an A operand are issued as ONE
+            // instruction over a wider B: [W_hi | W_lo] (N = 128) for a_hi, and [dh1_hi | dh1_lo] for the one-hot.
             const uint32_t idesc = tc::umma_idesc<PREC>(BM, BN, false, false);
-            const uint32_t idesc_agent = tc::umma_idesc<PREC>(128, BN, true, true);
-            // agent-plane product of step v: 8 k16 steps over the 128 envs, one term per dh1 plane (the one-hot is exact)
+            const uint32_t idesc_w = tc::umma_idesc<PREC>(BM, ACCW, false, false);
+            const uint32_t idesc_agent = tc::umma_idesc<PREC>(128, ACCW, true, true);
+            // agent-plane product of step v: 8 k16 steps over the 128 envs (the one-hot is exact; columns 64.. of the
+            // accumulator collect the dh1 lo plane's share)
             auto agent_mma = [&](int v) {
                 ok = tc::mbar_wait(tiles_full, (uint32_t)v & 1u);
                 if (!ok) return;
@@ -133,9 +150,8 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
 #pragma unroll
                 for (int k16 = 0; k16 < BM / 16; ++k16) {
                     const uint64_t od = tc::umma_desc(sO + k16 * 2048, BM * 128, 1024);  // cells 64.. are one box further
-                    const uint64_t dh = tc::umma_desc(sD + k16 * 2048, BM * 128, 1024);
+                    const uint64_t dh = tc::umma_desc(sD + k16 * 2048, BM * 128, 1024);  // the lo plane is the next box
                     tc::umma(acc_agent, od, dh, idesc_agent, (v > 0 || k16 > 0) ? 1u : 0u);
-                    if (PL == 2) tc::umma(acc_agent, od, tc::umma_desc(sD + BM * 128 + k16 * 2048, BM * 128, 1024), idesc_agent, 1u);
                 }
                 tc::umma_commit(tiles_free);
             };
@@ -145,7 +161,7 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
                 if (u >= 2) ok = tc::mbar_wait(&tempty[buf], ((u >> 1) - 1) & 1);  // epilogue of step u-2 has drained it
                 if (!ok) break;
                 tc::tc_fence_after();
-                const uint32_t acc = tmem + (uint32_t)(buf * BN);
+                const uint32_t acc = tmem + (uint32_t)(buf * ACCW);
                 for (int kc = 0; kc < NCH && ok; ++kc) {
                     const int c = u * NCH + kc, s = c % STAGES;
                     ok = tc::mbar_wait(&full[s], (c / STAGES) & 1);
@@ -156,14 +172,10 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
                     for (int k16 = 0; k16 < KC / 16; ++k16) {
                         // K-major operands: 16 k = 32 bytes further along the swizzled 128-byte rows
                         const uint64_t a_hi = tc::umma_desc(sa + k16 * 32, 16, 1024);
-                        const uint64_t w_hi = tc::umma_desc(sW + kc * Cfg::W_BOX + k16 * 32, 16, 1024);
-                        uint32_t accum = (kc > 0 || k16 > 0) ? 1u : 0u;
-                        if (PL == 2) {
-                            tc::umma(acc, tc::umma_desc(sa + Cfg::A_BOX + k16 * 32, 16, 1024), w_hi, idesc, accum);
-                            tc::umma(acc, a_hi, tc::umma_desc(sW + (NCH + kc) * Cfg::W_BOX + k16 * 32, 16, 1024), idesc, 1u);
-                            accum = 1u;
-                        }
-                        tc::umma(acc, a_hi, w_hi, idesc, accum);
+                        const uint64_t w_hi = tc::umma_desc(sW + PL * kc * Cfg::W_BOX + k16 * 32, 16, 1024);  // lo rows follow
+                        const uint32_t accum = (kc > 0 || k16 > 0) ? 1u : 0u;
+                        tc::umma(acc, a_hi, w_hi, idesc_w, accum);  // columns 0-63: hi x hi; 64-127: hi x lo
+                        if (PL == 2) tc::umma(acc, tc::umma_desc(sa + Cfg::A_BOX + k16 * 32, 16, 1024), w_hi, idesc, 1u);  // lo x hi
                     }
                     tc::umma_commit(&empty[s]);
                 }
@@ -201,9 +213,18 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
                 if (!ok) break;
                 tc::tc_fence_after();
                 uint32_t r0[32], r1[32];
-                const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * BN);
+                const uint32_t taddr = tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * ACCW);
                 tc::tmem_ld32(taddr, r0);
                 tc::tmem_ld32(taddr + 32, r1);
+                if (PL == 2) {  // add the hi x lo term
+                    uint32_t r2[32];
+                    tc::tmem_ld32(taddr + 64, r2);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r0[j] = __float_as_uint(__uint_as_float(r0[j]) + __uint_as_float(r2[j]));
+                    tc::tmem_ld32(taddr + 96, r2);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r1[j] = __float_as_uint(__uint_as_float(r1[j]) + __uint_as_float(r2[j]));
+                }
                 tc::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&tempty[buf]);  // the issuer may overwrite this accumulator now
@@ -279,6 +300,12 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
             uint32_t r[32];
             if (got && G > 0) {
                 tc::tmem_ld32(acc_agent + ((uint32_t)(32 * q) << 16) + (uint32_t)(32 * half), r);
+                if (PL == 2) {  // the dh1 lo plane's share
+                    uint32_t r2[32];
+                    tc::tmem_ld32(acc_agent + ((uint32_t)(32 * q) << 16) + (uint32_t)(64 + 32 * half), r2);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                }
             } else {
 #pragma unroll
                 for (int j = 0; j < 32; ++j) r[j] = 0u;  // an empty slice contributes zeros
@@ -294,7 +321,7 @@ __global__ void __launch_bounds__(192, 1) k_dh1a_tc(const __grid_constant__ Dh1a
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (wid == 2) tc::tmem_dealloc(tmem, 256);
+    if (wid == 2) tc::tmem_dealloc(tmem, Cfg::TMEM_COLS);
 }
 
 template <int H, int PREC>

@@ -45,6 +45,10 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, u
                  "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
                  : "memory");
 }
+// Asks L2 to fetch the box a later tma_load_2d of the same coordinates will read (no shared memory, no completion).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
 // Makes generic-proxy writes to shared memory (ordinary stores) visible to the async proxy (TMA, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
