@@ -201,7 +201,7 @@ struct Scope {
 };
 
 // Operands of the split-K "TN" GEMMs  C[m][n] = sum_k A[k][m] B[k][n]  (weight gradients).
-enum : int { A_PLANES = 0, A_ONEHOT = 1, A_WALLS = 2 };
+enum : int { A_PLANES = 0, A_ONEHOT = 1, A_WALLS = 2, A_ENV = 3 };  // A_ENV: row tile 0 = A_WALLS, row tile 1 = A_ONEHOT of idx2
 
 struct GemmTnArgs {
     int M, N, K, klen;
@@ -216,6 +216,11 @@ struct GemmTnArgs {
     float* part;                     // out: part[split*stride + off + m*ldc + n]; row ones_row goes to off_ones + n
     size_t stride, off, off_ones;
     int ldc;
+    // A_ENV only: the second row tile is the one-hot of idx2 (M2 rows), written to part2[split*stride2 + m*ldc + n]
+    const uint8_t* idx2;
+    int M2;
+    float* part2;
+    size_t stride2;
 };
 
 // tcgen05 version (tensor memory accumulators, TMA-fed); cudaErrorNotSupported when the shape is not covered.

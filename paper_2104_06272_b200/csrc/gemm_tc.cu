@@ -76,7 +76,10 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
     uint64_t* bars = (uint64_t*)(base + STAGES * Cfg::STAGE);  // full[STAGES], empty[STAGES], done
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 1);
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, split = blockIdx.z;
+    // A_ENV: two row tiles with different synthesized A operands (wall bits + ones row; one-hot of idx2), each with its own M space
+    const int amode = AMODE == A_ENV ? (blockIdx.x == 0 ? A_WALLS : A_ONEHOT) : AMODE;
+    const int m0 = AMODE == A_ENV ? 0 : blockIdx.x * BM, n0 = blockIdx.y * BN, split = blockIdx.z;
+    const uint8_t* oh_idx = (AMODE == A_ENV) ? g.idx2 : g.idx;
     const int kbeg = split * g.klen, kend = min(g.K, kbeg + g.klen);
     const int nchunks = kend > kbeg ? (kend - kbeg + KC - 1) / KC : 0;
     constexpr uint32_t NBUILD = AMODE == A_PLANES ? 0u : 128u;
@@ -153,12 +156,12 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
                 if (ok && c >= STAGES) ok = tc::mbar_wait(&bars[STAGES + s], ((c / STAGES) - 1) & 1);
                 unsigned char* sa = base + s * Cfg::STAGE;
                 // element (k, m) of the tile lives in box m/64 at byte  k*128 + (((m%64)/8) ^ (k%8))*16 + (m%8)*2
-                if (AMODE == A_ONEHOT) {
+                if (amode == A_ONEHOT) {
                     uint4* z = reinterpret_cast<uint4*>(sa);
                     for (int i = bt; i < Cfg::A_PLANE / 16; i += 128) z[i] = make_uint4(0u, 0u, 0u, 0u);
                     asm volatile("bar.sync 1, 128;" ::: "memory");  // zeros before ones
                     if (bt < KC && k0 + bt < kend) {
-                        const int m = (int)g.idx[g.kmod ? (k0 + bt) % g.kmod : (k0 + bt)] - m0;
+                        const int m = (int)oh_idx[g.kmod ? (k0 + bt) % g.kmod : (k0 + bt)] - m0;
                         if (m >= 0 && m < BM) {
                             const int k = bt;
                             const uint32_t off = (m >> 6) * Cfg::BOX + k * 128 + ((((m & 63) >> 3) ^ (k & 7)) << 4) + (m & 7) * 2;
@@ -198,7 +201,9 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
         __syncwarp();
         const int q = wid & 3;
         const int m = m0 + 32 * q + lane;
-        float* part = g.part + (size_t)split * g.stride + g.off;
+        const bool second = AMODE == A_ENV && blockIdx.x == 1;
+        const int Mrows = second ? g.M2 : g.M;
+        float* part = second ? g.part2 + (size_t)split * g.stride2 : g.part + (size_t)split * g.stride + g.off;
         for (int c0 = 0; c0 < BN; c0 += 32) {
             uint32_t r[32];
             if (nchunks > 0 && got) {
@@ -207,9 +212,9 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
 #pragma unroll
                 for (int j = 0; j < 32; ++j) r[j] = 0u;  // an empty K range contributes zeros
             }
-            if (m < g.M && n0 + c0 < g.N) {
+            if (m < Mrows && n0 + c0 < g.N) {
                 float4* dst = reinterpret_cast<float4*>(part + (size_t)m * g.ldc + n0 + c0);
-                if (AMODE == A_WALLS && m == g.ones_row) dst = reinterpret_cast<float4*>(part - g.off + g.off_ones + n0 + c0);
+                if (amode == A_WALLS && m == g.ones_row) dst = reinterpret_cast<float4*>(part - g.off + g.off_ones + n0 + c0);
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
@@ -236,7 +241,7 @@ static cudaError_t launch_t(const GemmTnArgs& g, int splits, int* status, cudaSt
     if (BPL == 2 && !make_tensor_map_2d(&maps.b_lo, g.Blo, (uint64_t)g.K, (uint64_t)g.ldb, 64, bf)) return cudaErrorNotSupported;
     cudaError_t e = cudaFuncSetAttribute(k_gemm_tn_tc<BN, AMODE, APL, BPL, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
     if (e != cudaSuccess) return e;
-    dim3 grid((g.M + Cfg::BM - 1) / Cfg::BM, (g.N + BN - 1) / BN, splits);
+    dim3 grid(AMODE == A_ENV ? 2 : (g.M + Cfg::BM - 1) / Cfg::BM, (g.N + BN - 1) / BN, splits);
     k_gemm_tn_tc<BN, AMODE, APL, BPL, PREC><<<grid, Cfg::THREADS, Cfg::smem_bytes, s>>>(maps, g, status);
     return cudaGetLastError();
 }
@@ -247,6 +252,7 @@ static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int splits, int* st
     if (amode == A_PLANES) return launch_t<BN, A_PLANES, PL, PL, PREC>(g, splits, status, s);
     if (amode == A_ONEHOT) return launch_t<BN, A_ONEHOT, 1, PL, PREC>(g, splits, status, s);
     if (amode == A_WALLS && g.M <= 128) return launch_t<BN, A_WALLS, 1, PL, PREC>(g, splits, status, s);
+    if (amode == A_ENV && g.M <= 128 && g.M2 <= 128) return launch_t<BN, A_ENV, 1, PL, PREC>(g, splits, status, s);
     return cudaErrorNotSupported;
 }
 

@@ -657,7 +657,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
         return r;
     };
     // Parameters before b2 (W1, b1, W2) have at most ~128 partials: one thread each, partials added in index order,
-    // eight loads in flight.  The tail (b2 | Wh | bh) has two partials per CTA of the heads kernel: one warp per
+    // sixteen loads in flight.  The tail (b2 | Wh | bh) has two partials per CTA of the heads kernel: one warp per
     // parameter, lane l adds partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
     const int nb_main = (int)((d.ob2 + 255) / 256);
     if ((int)blockIdx.x < nb_main) {
@@ -667,12 +667,19 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             const float* p = rg.part + (i - rg.start);
             float gsum = 0.f;
             int s = 0;
-            for (; s + 8 <= rg.ns; s += 8) {
-                float v[8];
+            for (; s + 16 <= rg.ns; s += 16) {
+                float v[16];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
+                for (int q = 0; q < 16; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) gsum += v[q];
+                for (int q = 0; q < 16; ++q) gsum += v[q];
+            }
+            for (; s + 4 <= rg.ns; s += 4) {
+                float v[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) gsum += v[q];
             }
             for (; s < rg.ns; ++s) gsum += p[(size_t)s * rg.stride];
             apply(i, gsum);
@@ -684,7 +691,15 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             const PartRegion& rg = a.reg[region_of(i)];
             const float* p = rg.part + (i - rg.start);
             float gsum = 0.f;
-            for (int s = lane; s < rg.ns; s += 32) gsum += p[(size_t)s * rg.stride];
+            int s = lane;
+            for (; s + 32 * 7 < rg.ns; s += 32 * 8) {  // eight loads in flight per lane
+                float v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + 32 * q) * rg.stride];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) gsum += v[q];
+            }
+            for (; s < rg.ns; s += 32) gsum += p[(size_t)s * rg.stride];
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, off);
             if (lane == 0) apply(i, gsum);
@@ -919,25 +934,35 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     g.Bhi = Shi; g.Blo = Shi + (size_t)a.ts * B * H;
     g.walls = b.walls; g.W = d.W; g.ones_row = C; g.M = C + 1;
     g.part = b.part + pl.off_walls; g.stride = (size_t)(C + 1) * H; g.off = 0; g.off_ones = CH;
-    {
+    bool env_planes_done = false;
+    if (PREC == 0) {  // both planes in one launch: row tile 0 = wall bits + ones row, row tile 1 = one-hot of the goal cell
+        g.idx2 = b.goal; g.M2 = C; g.part2 = b.part + pl.off_goal; g.stride2 = CH;
         Scope sc(c, K_DW1_WALLS);
-        cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_WALLS, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
-        if (e == cudaErrorNotSupported) {
-            if (H >= 128) e = launch_gemm_tn<128, 128, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
-            else e = launch_gemm_tn<64, 64, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
-        }
-        CK(e);
+        const cudaError_t e = launch_gemm_tn_tc(g, A_ENV, 1, 2, PREC, pl.ns_env, b.status, s);
+        if (e == cudaSuccess) env_planes_done = true;
+        else if (e != cudaErrorNotSupported) return e;
     }
-    g.M = C; g.ones_row = -1; g.idx = b.goal;
-    g.part = b.part + pl.off_goal; g.stride = CH;
-    {
-        Scope sc(c, K_DW1_GOAL);
-        cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_ONEHOT, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
-        if (e == cudaErrorNotSupported) {
-            if (H >= 128) e = launch_gemm_tn<128, 128, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
-            else e = launch_gemm_tn<64, 64, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
+    if (!env_planes_done) {
+        {
+            Scope sc(c, K_DW1_WALLS);
+            cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_WALLS, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
+            if (e == cudaErrorNotSupported) {
+                if (H >= 128) e = launch_gemm_tn<128, 128, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
+                else e = launch_gemm_tn<64, 64, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
+            }
+            CK(e);
         }
-        CK(e);
+        g.M = C; g.ones_row = -1; g.idx = b.goal;
+        g.part = b.part + pl.off_goal; g.stride = CH;
+        {
+            Scope sc(c, K_DW1_GOAL);
+            cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_ONEHOT, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
+            if (e == cudaErrorNotSupported) {
+                if (H >= 128) e = launch_gemm_tn<128, 128, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
+                else e = launch_gemm_tn<64, 64, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
+            }
+            CK(e);
+        }
     }
     {
         Scope sc(c, K_REDUCE_ADAM);
