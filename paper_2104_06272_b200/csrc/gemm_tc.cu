@@ -247,11 +247,16 @@ static cudaError_t launch_t(const GemmTnArgs& g, int splits, int* status, cudaSt
 }
 
 template <int BN, int PREC>
-static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int splits, int* status, cudaStream_t s) {
+static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int bpl, int splits, int* status, cudaStream_t s) {
     constexpr int PL = PREC == 1 ? 1 : 2;
+    if (PREC == 1 && bpl == 2) {  // bf16 workload with a two-term B (the sum over t of dh1): synthesized A only
+        if (amode == A_ONEHOT) return launch_t<BN, A_ONEHOT, 1, 2, PREC>(g, splits, status, s);
+        if (amode == A_WALLS) return launch_t<BN, A_WALLS, 1, 2, PREC>(g, splits, status, s);
+        return cudaErrorNotSupported;
+    }
     if (amode == A_PLANES) return launch_t<BN, A_PLANES, PL, PL, PREC>(g, splits, status, s);
     if (amode == A_ONEHOT) return launch_t<BN, A_ONEHOT, 1, PL, PREC>(g, splits, status, s);
-    if (amode == A_WALLS && g.M <= 128) return launch_t<BN, A_WALLS, 1, PL, PREC>(g, splits, status, s);
+    if (amode == A_WALLS) return launch_t<BN, A_WALLS, 1, PL, PREC>(g, splits, status, s);
     if (amode == A_ENV && g.M <= 128 && g.M2 <= 128) return launch_t<BN, A_ENV, 1, PL, PREC>(g, splits, status, s);
     return cudaErrorNotSupported;
 }
@@ -260,20 +265,22 @@ static cudaError_t launch_bn(const GemmTnArgs& g, int amode, int splits, int* st
 // operand planes as the fp32 workloads (hi+lo fp16) or the bf16 workload (one plane) use them.
 cudaError_t launch_gemm_tn_tc(const GemmTnArgs& g, int amode, int apl, int bpl, int prec, int splits, int* status, cudaStream_t s) {
     const int pl = prec == 1 ? 1 : 2;
-    if (g.N != g.ldb || g.klen % 64 != 0 || bpl != pl || (amode == A_PLANES && (apl != pl || g.lda % 64 != 0))) return cudaErrorNotSupported;
+    if (g.N != g.ldb || g.klen % 64 != 0 || (bpl != pl && !(prec == 1 && bpl == 2 && amode != A_PLANES)) ||
+        (amode == A_PLANES && (apl != pl || g.lda % 64 != 0)))
+        return cudaErrorNotSupported;
     if (amode != A_PLANES && apl != 1) return cudaErrorNotSupported;
     const int bn = g.N > 256 && g.N % 256 == 0 ? 256 : g.N;
     if (prec == 1) {
         switch (bn) {
-            case 64: return launch_bn<64, 1>(g, amode, splits, status, s);
-            case 128: return launch_bn<128, 1>(g, amode, splits, status, s);
-            case 256: return launch_bn<256, 1>(g, amode, splits, status, s);
+            case 64: return launch_bn<64, 1>(g, amode, bpl, splits, status, s);
+            case 128: return launch_bn<128, 1>(g, amode, bpl, splits, status, s);
+            case 256: return launch_bn<256, 1>(g, amode, bpl, splits, status, s);
         }
     } else {
         switch (bn) {
-            case 64: return launch_bn<64, 0>(g, amode, splits, status, s);
-            case 128: return launch_bn<128, 0>(g, amode, splits, status, s);
-            case 256: return launch_bn<256, 0>(g, amode, splits, status, s);
+            case 64: return launch_bn<64, 0>(g, amode, bpl, splits, status, s);
+            case 128: return launch_bn<128, 0>(g, amode, bpl, splits, status, s);
+            case 256: return launch_bn<256, 0>(g, amode, bpl, splits, status, s);
         }
     }
     return cudaErrorNotSupported;

@@ -945,7 +945,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     if (!env_planes_done) {
         {
             Scope sc(c, K_DW1_WALLS);
-            cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_WALLS, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
+            cudaError_t e = launch_gemm_tn_tc(g, A_WALLS, 1, 2, PREC, pl.ns_env, b.status, s);
             if (e == cudaErrorNotSupported) {
                 if (H >= 128) e = launch_gemm_tn<128, 128, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
                 else e = launch_gemm_tn<64, 64, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
@@ -956,7 +956,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         g.part = b.part + pl.off_goal; g.stride = CH;
         {
             Scope sc(c, K_DW1_GOAL);
-            cudaError_t e = PREC == 0 ? launch_gemm_tn_tc(g, A_ONEHOT, 1, 2, PREC, pl.ns_env, b.status, s) : cudaErrorNotSupported;
+            cudaError_t e = launch_gemm_tn_tc(g, A_ONEHOT, 1, 2, PREC, pl.ns_env, b.status, s);
             if (e == cudaErrorNotSupported) {
                 if (H >= 128) e = launch_gemm_tn<128, 128, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
                 else e = launch_gemm_tn<64, 64, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);

@@ -333,7 +333,8 @@ __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mo
         for (int q = 0; q < TRIPS; ++q) v[q] = vn[q];
     }
     __syncthreads();
-    if (tid >= HW_ROWS) return;
+    __shared__ int s_pos[HW_ROWS];
+    if (tid < HW_ROWS) {
     const size_t i = i0 + tid;
     const bool valid = i < rows;
     unsigned long long n_ep = 0, n_goal = 0, n_steps = 0;
@@ -355,11 +356,12 @@ __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mo
                 act_and_step(es, a, env, t, o0, o1, o2, o3, s_walls[tid]);
                 b.pos[env] = (uint8_t)es.pos;
                 b.tep[env] = (uint8_t)es.tep;
+                s_pos[tid] = es.pos;
                 n_ep = es.n_episodes; n_goal = es.n_goals; n_steps = es.n_epsteps; bad = es.bad;
             }
         }
     }
-    if (mode != 0) return;
+    if (mode == 0) {
     // fold the warp's counters and add them with integer atomics (order-free totals)
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -374,6 +376,31 @@ __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mo
         if (n_steps) atomicAdd((unsigned long long*)&b.stats->episode_steps, n_steps);
         if (blockIdx.x == 0 && tid == 0) atomicAdd((unsigned long long*)&b.stats->frames, (unsigned long long)d.B);
         if (bad) atomicOr(b.status, bad);
+    }
+    }
+    }
+    if (mode != 0) return;
+    // ---- layer 1 of the NEXT step for this CTA's envs, from the positions just produced (rows (t+1)*B + env):
+    // 8 threads per env, 16-byte chunks interleaved so that a row's lanes read and write contiguous memory
+    __syncthreads();
+    {
+        const int rl = tid >> 3, q = tid & 7;
+        const size_t env = i0 + rl;
+        if (env < rows) {
+            const float4* bp = reinterpret_cast<const float4*>(b.base + env * H);
+            const float4* wp = reinterpret_cast<const float4*>(b.theta_c + d.oW1 + ((size_t)d.C + s_pos[rl]) * H);
+            uint4* out = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(b.h1) + ((size_t)(t + 1) * d.B + env) * H);
+#pragma unroll 4
+            for (int ch = q; ch < H / 8; ch += 8) {
+                const float4 b0 = bp[2 * ch], b1 = bp[2 * ch + 1], w0 = __ldg(wp + 2 * ch), w1 = __ldg(wp + 2 * ch + 1);
+                uint4 o;
+                o.x = pack_bf16(__float2bfloat16_rn(fmaxf(b0.x + w0.x, 0.f)), __float2bfloat16_rn(fmaxf(b0.y + w0.y, 0.f)));
+                o.y = pack_bf16(__float2bfloat16_rn(fmaxf(b0.z + w0.z, 0.f)), __float2bfloat16_rn(fmaxf(b0.w + w0.w, 0.f)));
+                o.z = pack_bf16(__float2bfloat16_rn(fmaxf(b1.x + w1.x, 0.f)), __float2bfloat16_rn(fmaxf(b1.y + w1.y, 0.f)));
+                o.w = pack_bf16(__float2bfloat16_rn(fmaxf(b1.z + w1.z, 0.f)), __float2bfloat16_rn(fmaxf(b1.w + w1.w, 0.f)));
+                out[ch] = o;
+            }
+        }
     }
 }
 
@@ -526,7 +553,7 @@ cudaError_t launch_rollout_wide(const RolloutArgs& a, const Ctx& c) {
     }
     for (int t = 0; t <= a.T; ++t) {
         const size_t row0 = (size_t)t * B;
-        {
+        if (t == 0) {  // later steps: the heads kernel of step t-1 writes the h1 rows of step t
             Scope sc(c, K_H1);
             k_h1_wide<<<h1_grid(B, H), 256, 0, c.s>>>(d, b, b.pos, B, row0);
             CKW(cudaGetLastError());
