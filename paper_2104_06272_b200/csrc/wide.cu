@@ -11,14 +11,14 @@
 //
 // k_gemm_nt_tc: C[m][n] = sum_k A[m][k] Bop[k][n] with A row-major (K-major for the MMA).  One persistent CTA per SM walks
 // 128 x 256 output tiles (n fastest, so that the CTAs running together share A tiles through L2):
-//   warp 0 (one lane)  TMA producer: 64-wide k chunks of A (128 rows) and B (256 columns) into a 4-stage ring
+//   warp 0 (one lane)  TMA producer: 64-wide k chunks of A (128 rows) and B (256 columns) into a 3-stage ring
 //   warp 1 (one lane)  tcgen05.mma issuer, four k16 MMAs per chunk into one of two 256-column fp32 accumulators in TMEM
-//   warps 2-5          epilogue of tile i while the MMAs of tile i+1 run: tcgen05.ld, bias + ReLU (or gate), bf16, store
+//   warps 2-9          epilogue of tile i while the MMAs of tile i+1 run: tcgen05.ld, bias + ReLU (or gate), bf16, store
 // B is either K-major (rows = n: W2 as stored, for dh2 W2^T) or MN-major (rows = k: W2 as stored, for h1 W2).
 // Every wait is bounded; a timeout raises DEV_E_WAIT_TIMEOUT and the CTA unwinds (tensor memory freed).
 #include <cstring>
 
-#include "tc_common.cuh"
+#include "wide_gemm.cuh"
 
 namespace anakin {
 
@@ -27,33 +27,16 @@ bool tensor_path_supported(int H, int prec) { return rollout_mma_supported(H) ||
 
 namespace {
 
-enum : int { EPI_FWD = 0, EPI_GATE = 1, EPI_BASE = 2 };
-
-struct NtArgs {
-    int M, N, K;           // C is M x N; M rows starting at row0 of A, out and gate
-    int row0;
-    uint16_t* out;         // bf16 [rows][N]
-    const float* bias;     // EPI_FWD: [N]
-    const uint16_t* gate;  // EPI_GATE: bf16 [rows][N], non-negative; out = gate > 0 ? acc : 0
-    float* outf;           // EPI_BASE: fp32 [rows][N] = acc + bias[n] + addrows[(addrow0 + addidx[m])*N + n]
-    const float* addrows;
-    const uint8_t* addidx;
-    int addrow0;
-    int* status;
-};
-
-struct NtMaps {
-    CUtensorMap a, b;
-};
+using namespace widegemm;
 
 struct NtCfg {
-    static constexpr int BM = 128, BN = 256, KC = 64, STAGES = 4, THREADS = 192, MAXN = 2048;
+    static constexpr int BM = 128, BN = NT_BN, KC = 64, STAGES = 3, THREADS = 320, MAXN = NT_MAXN;
     static constexpr int A_BYTES = BM * KC * 2, B_BYTES = BN * KC * 2, STAGE = A_BYTES + B_BYTES;
-    static constexpr size_t smem_bytes = (size_t)STAGES * STAGE + 1024 /*alignment slack*/ + 256 /*barriers, tmem slot*/ + MAXN * 4;
+    static constexpr size_t smem_bytes = (size_t)STAGES * STAGE + 1024 /*alignment slack*/ + 256 /*barriers, tmem slot*/ + MAXN * 4 + NT_EPI_WARPS * NT_STAGE_BYTES;
 };
 
 template <int EPI, bool B_MN>
-__global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ NtMaps maps, NtArgs g) {
+__global__ void __launch_bounds__(320, 1) k_gemm_nt_tc(const __grid_constant__ NtMaps maps, NtArgs g) {
     using Cfg = NtCfg;
     constexpr int BM = Cfg::BM, BN = Cfg::BN, KC = Cfg::KC, STAGES = Cfg::STAGES;
     extern __shared__ unsigned char smem_raw[];
@@ -65,12 +48,13 @@ __global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ N
     uint64_t* tempty = tfull + 2;         // [2] accumulator drained (4 epilogue warps arrive)
     uint32_t* tmem_slot = (uint32_t*)(tempty + 2);
     float* s_bias = (float*)(base + STAGES * Cfg::STAGE + 256);
+    unsigned char* s_stage = (unsigned char*)(s_bias + NT_MAXN);  // [NT_EPI_WARPS][NT_STAGE_BYTES]
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
     const int nt = g.N / BN, mt = (g.M + BM - 1) / BM, ntiles = mt * nt, nch = g.K / KC;
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
-        for (int i = 0; i < 2; ++i) { tc::mbar_init(&tfull[i], 1); tc::mbar_init(&tempty[i], 4); }
+        for (int i = 0; i < 2; ++i) { tc::mbar_init(&tfull[i], 1); tc::mbar_init(&tempty[i], NT_EPI_WARPS); }
         tc::mbar_fence_init();
     }
     if (EPI != EPI_GATE)
@@ -100,7 +84,8 @@ __global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ N
 #pragma unroll
                         for (int bx = 0; bx < BN / 64; ++bx) tc::tma_load_2d(sb + bx * 8192, &maps.b, &full[s], n0 + 64 * bx, kc * KC);
                     } else {
-                        tc::tma_load_2d(sb, &maps.b, &full[s], kc * KC, n0);
+                        tc::tma_load_2d(sb, &maps.b, &full[s], kc * KC, n0);  // two boxes of 128 rows (n)
+                        tc::tma_load_2d(sb + Cfg::B_BYTES / 2, &maps.b, &full[s], kc * KC, n0 + BN / 2);
                     }
                 }
             }
@@ -138,7 +123,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ N
         }
     } else {
         // ---- epilogue warps: accumulator lanes 32*(wid%4)..+31 = output rows
-        const int q = wid & 3;
+        const int q = wid & 3, half = (wid - 2) >> 2;
         int u = 0;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++u) {
             const int buf = u & 1;
@@ -146,66 +131,12 @@ __global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ N
             const int m = m0 + 32 * q + lane;
             const bool valid = m < g.M;
             const size_t gi = ((size_t)g.row0 + (valid ? m : 0)) * g.N + n0;
-            if (EPI == EPI_GATE && valid) {  // pull this row's gate bytes (512 B) towards L2 while the MMAs run
-#pragma unroll
-                for (int l = 0; l < 4; ++l) asm volatile("prefetch.global.L2 [%0];" ::"l"(g.gate + gi + 64 * l));
-            }
+            if (EPI == EPI_GATE && valid) nt_prefetch_gate(g, gi);  // towards L2 while the MMAs run
             ok = tc::mbar_wait(&tfull[buf], (u >> 1) & 1);
             if (!ok) break;
             tc::tc_fence_after();
-            uint4 gt[4];
-            if (EPI == EPI_GATE) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) gt[j] = valid ? __ldg(reinterpret_cast<const uint4*>(g.gate + gi) + j) : make_uint4(0u, 0u, 0u, 0u);
-            }
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                tc::tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * BN + c0), r);
-                if (EPI == EPI_BASE) {  // fp32 out: accumulator + bias + this row's extra weight row
-                    if (valid) {
-                        const float4* add = reinterpret_cast<const float4*>(g.addrows + ((size_t)g.addrow0 + g.addidx[m]) * g.N + n0 + c0);
-                        float4* dst = reinterpret_cast<float4*>(g.outf + gi + c0);
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 w = __ldg(add + j);
-                            const float* bs = s_bias + n0 + c0 + 4 * j;
-                            dst[j] = make_float4(__uint_as_float(r[4 * j]) + bs[0] + w.x, __uint_as_float(r[4 * j + 1]) + bs[1] + w.y,
-                                                 __uint_as_float(r[4 * j + 2]) + bs[2] + w.z, __uint_as_float(r[4 * j + 3]) + bs[3] + w.w);
-                        }
-                    }
-                    continue;
-                }
-                uint4 gn[4];
-                if (EPI == EPI_GATE && c0 + 32 < BN) {  // next chunk's gates, in flight during this chunk's math
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        gn[j] = valid ? __ldg(reinterpret_cast<const uint4*>(g.gate + gi + c0 + 32) + j) : make_uint4(0u, 0u, 0u, 0u);
-                }
-                uint32_t pk[16];
-                const uint32_t* gw = reinterpret_cast<const uint32_t*>(gt);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float x0 = __uint_as_float(r[2 * j]), x1 = __uint_as_float(r[2 * j + 1]);
-                    if (EPI == EPI_FWD) {
-                        x0 = fmaxf(x0 + s_bias[n0 + c0 + 2 * j], 0.f);
-                        x1 = fmaxf(x1 + s_bias[n0 + c0 + 2 * j + 1], 0.f);
-                    } else {
-                        x0 = (gw[j] & 0x00007FFFu) ? x0 : 0.f;  // gate >= 0: "> 0" is "any magnitude bit set"
-                        x1 = (gw[j] & 0x7FFF0000u) ? x1 : 0.f;
-                    }
-                    pk[j] = pack_bf16(__float2bfloat16_rn(x0), __float2bfloat16_rn(x1));
-                }
-                if (valid) {
-                    uint4* dst = reinterpret_cast<uint4*>(g.out + gi + c0);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                }
-                if (EPI == EPI_GATE && c0 + 32 < BN) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) gt[j] = gn[j];
-                }
-            }
+            nt_epilogue_warp<EPI>(g, s_bias, s_stage + (wid - 2) * NT_STAGE_BYTES, tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * BN), m - lane, n0, lane,
+                                  half * (BN / 2), (half + 1) * (BN / 2));
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&tempty[buf]);  // the issuer may overwrite this accumulator now
@@ -220,6 +151,10 @@ __global__ void __launch_bounds__(192, 1) k_gemm_nt_tc(const __grid_constant__ N
 template <int EPI, bool B_MN>
 cudaError_t launch_nt(const NtMaps& maps, const NtArgs& g, cudaStream_t s) {
     if (g.N % NtCfg::BN != 0 || g.K % NtCfg::KC != 0 || g.N > NtCfg::MAXN || g.M < 1) return cudaErrorNotSupported;
+    if (g.M >= 2 * NtCfg::BM) {  // the CTA-pair kernel (256 x 256 tiles) where there are rows for it
+        const cudaError_t ep = launch_nt_pair(EPI, B_MN, maps, g, s);
+        if (ep != cudaErrorNotSupported) return ep;
+    }
     const cudaError_t e = cudaFuncSetAttribute(k_gemm_nt_tc<EPI, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)NtCfg::smem_bytes);
     if (e != cudaSuccess) return e;
     const int ntiles = ((g.M + NtCfg::BM - 1) / NtCfg::BM) * (g.N / NtCfg::BN);
@@ -580,7 +515,7 @@ cudaError_t launch_dh1_wide(const LearnArgs& a, const Ctx& c) {
     NtMaps maps;
     memset(&maps, 0, sizeof(maps));
     if (!make_tensor_map_2d(&maps.a, b.dh2, R, H, 128, true)) return cudaErrorNotSupported;
-    if (!make_tensor_map_2d(&maps.b, b.w2p_hi, H, H, 256, true)) return cudaErrorNotSupported;
+    if (!make_tensor_map_2d(&maps.b, b.w2p_hi, H, H, 128, true)) return cudaErrorNotSupported;
     NtArgs g;
     memset(&g, 0, sizeof(g));
     g.M = (int)R; g.N = H; g.K = H; g.row0 = 0;
