@@ -53,13 +53,18 @@ bool make_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint6
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int APL, int BPL>
+// DEEP: as many stages as fit (plane operands, TMA-latency-bound); otherwise two, so that two CTAs share an SM (the
+// synthesized-A modes are bound by their builder threads, and a second CTA hides them).
+template <int BN, int APL, int BPL, bool DEEP>
 struct GemmTcCfg {
-    static constexpr int BM = 128, KC = 64, STAGES = 2, THREADS = 192;
+    static constexpr int BM = 128, KC = 64, THREADS = 192;
     static constexpr int BOX = 64 * 64 * 2;                  // one 64 x 64 box of 16-bit elements
     static constexpr int A_PLANE = (BM / 64) * BOX;          // 16 KB
     static constexpr int B_PLANE = (BN / 64) * BOX;
     static constexpr int STAGE = APL * A_PLANE + BPL * B_PLANE;
+    // as many stages as fit beside the slack (the loads are latency-bound: bytes in flight set the rate), at most 4
+    static constexpr int FIT = (232448 - 1024 - 128) / STAGE;
+    static constexpr int STAGES = !DEEP ? 2 : (FIT >= 4 ? 4 : (FIT >= 2 ? FIT : 2));
     static constexpr size_t smem_bytes = (size_t)STAGES * STAGE + 1024 /*alignment slack*/ + 128 /*barriers, tmem slot*/;
 };
 
@@ -69,7 +74,7 @@ struct GemmTcMaps {
 
 template <int BN, int AMODE, int APL, int BPL, int PREC>
 __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ GemmTcMaps maps, GemmTnArgs g, int* status) {
-    using Cfg = GemmTcCfg<BN, APL, BPL>;
+    using Cfg = GemmTcCfg<BN, APL, BPL, AMODE == A_PLANES>;
     constexpr int BM = Cfg::BM, KC = Cfg::KC, STAGES = Cfg::STAGES;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // the swizzle needs 1024-byte alignment
@@ -229,7 +234,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
 
 template <int BN, int AMODE, int APL, int BPL, int PREC>
 static cudaError_t launch_t(const GemmTnArgs& g, int splits, int* status, cudaStream_t s) {
-    using Cfg = GemmTcCfg<BN, APL, BPL>;
+    using Cfg = GemmTcCfg<BN, APL, BPL, AMODE == A_PLANES>;
     GemmTcMaps maps;
     memset(&maps, 0, sizeof(maps));
     const bool bf = PREC == 1;

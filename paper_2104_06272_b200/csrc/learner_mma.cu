@@ -776,6 +776,9 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     }
     p->ns_w2 = splits_for((int)R, tiles_hh, 256);
     p->ns_agent = splits_for((int)R, tiles_agent, 256);
+    if (H > 256) {  // the bf16 GEMM CTAs of the wide path take a whole SM each (four 48 KB stages): one wave
+        p->ns_w2 = 148 / tiles_hh > 0 ? 148 / tiles_hh : 1;
+    }
     if (dh1_agent_tc_supported(d)) {  // the fused kernel writes one agent-plane partial per (CTA row, t slice)
         int gx, ts;
         dh1a_shape(d, d.Tmax, &gx, &ts);
