@@ -89,7 +89,7 @@ class ClockSampler:
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu capture
 # summarised under profiles/ for the same kernel source; None for workloads without a capture at full size.
-NCU_TRAFFIC_BYTES = {("throughput", "rollout"): 5.5e6 + 221.0e6}
+NCU_TRAFFIC_BYTES = {("throughput", "rollout"): 5.6e6 + 223.5e6}
 
 
 def workload_label(w):
@@ -125,11 +125,11 @@ def kernel_work(w):
         "replay": ("tensor", p3 * 2.0 * R * H * H, R * H * (pl + 4.0)),
     }
     if w.precision == 1 and H in (512, 1024):
-        # wide bf16 path: three launches per env step (h1 gather, layer-2 GEMM, heads + env step), bf16 activations in HBM
+        # wide bf16 path: two launches per env step (layer-2 GEMM; heads + env step + next step's h1), bf16 activations in HBM
         work.update({
-            "h1": ("hbm", B * H * 2.0, B * H * (4.0 + 2.0) + B),                  # per step: base fp32 in, h1 bf16 out
+            "h1": ("hbm", B * H * 2.0, B * H * (4.0 + 2.0) + B),                  # first step only: base fp32 in, h1 bf16 out
             "fwd2": ("tensor", 2.0 * B * H * H, B * H * 4.0 + H * H * 2.0),       # per step: h1 in, h2 out, W2
-            "rollout": ("hbm", B * H * 10.0, B * H * 2.0 + B * 47.0),             # per step: h2 in, records out
+            "rollout": ("hbm", B * H * 12.0, B * H * 8.0 + B * 47.0),             # per step: h2 in, records out; base in, next h1 out
             "heads_bwd": ("hbm", R * H * 22.0, R * H * 4.0 + R * 42.0),           # h2 in, dh2 out (bf16 each)
             "dh1": ("tensor", 2.0 * R * H * H, R * H * 6.0),                      # dh2 in, h1 gates in, dh1 out
             "sum_over_t": ("hbm", R * H * 1.0, R * H * 2.0 + B * H * 4.0),
