@@ -234,6 +234,223 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
 }
 
 // ----------------------------------------------------------------------------------------------------
+// k_heads_bwd_tc: the same step for the bf16 workload with bf16 h2 in HBM (wide layers), with both small products on
+// the tensor pipe (mma.sync m16n8k16, bf16 inputs are exact here, fp32 accumulate):
+//   dh2 tile [32 rows x 16 cols per warp] = dOut [rows x 16 (5 used)] x Wh^T [16 x cols], then the gate and bf16;
+//   dWh [16 cols per warp x 8 (5 used)] += h2^T [cols x 32 rows] x dOut [32 rows x 8]   (accumulators live all kernel).
+// A CTA owns a 256-column slab (blockIdx.y) and walks 32-row tiles; the row phase (softmax, loss, dOut) is as in
+// k_heads_bwd.  dh2 goes through a shared staging tile and leaves as whole 512-byte row segments.
+// ----------------------------------------------------------------------------------------------------
+template <int H>
+struct HeadsTcCfg {
+    static constexpr int TR = 32, HS = 256, NW = 16, NST = 4;
+    static constexpr int LD = HS + 8;  // bf16 pitch of the shared tiles (16-byte skew: conflict-free fragment access)
+    static constexpr size_t smem_bytes = (size_t)(NST + 2) * TR * LD * 2 + (size_t)2 * TR * 8 * 2 + (size_t)2 * 8 * (TR + 8) * 2 + NW * 8 * 4;
+};
+
+template <int H>
+__global__ void __launch_bounds__(512, 2) k_heads_bwd_tc(LearnArgs a) {
+    using Cfg = HeadsTcCfg<H>;
+    constexpr int TR = Cfg::TR, HS = Cfg::HS, NW = Cfg::NW, NST = Cfg::NST, LD = Cfg::LD, LDT = TR + 8;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __nv_bfloat16* s_h2 = reinterpret_cast<__nv_bfloat16*>(smem_raw);  // [NST][TR][LD]
+    __nv_bfloat16* s_o = s_h2 + NST * TR * LD;                         // [2][TR][LD] dh2 staging
+    __nv_bfloat16* s_dA = s_o + 2 * TR * LD;                           // [2][TR][8]   dOut rows (c fastest)
+    __nv_bfloat16* s_dT = s_dA + 2 * TR * 8;                           // [2][8][LDT]  dOut transposed (row fastest)
+    float* s_fin = reinterpret_cast<float*>(s_dT + 2 * 8 * LDT);       // [NW][8]
+    const int c_base = blockIdx.y * HS;
+    const Dims& d = a.d;
+    const Buffers& b = a.b;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, g = lane >> 2, t4 = lane & 3;
+    const size_t R = (size_t)d.B * a.T;
+    const float invR = a.gscale / (float)R;
+    const int ntiles = (int)((R + TR - 1) / TR);
+    const uint16_t* g_h2 = reinterpret_cast<const uint16_t*>(b.h2);
+    uint16_t* g_dh2 = reinterpret_cast<uint16_t*>(b.dh2);
+    const int col0 = 16 * wid;  // this warp's 16 columns inside the slab
+
+    // B fragments of Wh^T for the warp's two n8 tiles: k = head index (5 used of 16), n = column
+    uint32_t whf[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const float* w = b.theta_c + d.oWh + (size_t)(c_base + col0 + 8 * j + g) * 5;
+        const float w0 = 2 * t4 < 5 ? w[2 * t4] : 0.f, w1 = 2 * t4 + 1 < 5 ? w[2 * t4 + 1] : 0.f;
+        whf[j] = pack_bf16(__float2bfloat16_rn(w0), __float2bfloat16_rn(w1));
+    }
+    for (int i = tid; i < 2 * 8 * LDT; i += 512) s_dT[i] = __float2bfloat16_rn(0.f);  // rows 5..7 stay zero
+    float acc_wh[4] = {0.f, 0.f, 0.f, 0.f};
+    float a_b2[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    float a_bh[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+    float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
+
+    auto load_tile = [&](int tile, int buf) {  // 16-byte chunks, zero-filled past the last row; always commits a group
+        __nv_bfloat16* dst = s_h2 + buf * TR * LD;
+        for (int c = tid; tile < ntiles && c < TR * (HS / 8); c += 512) {
+            const int r = c / (HS / 8), k = 8 * (c - r * (HS / 8));
+            const size_t row = (size_t)tile * TR + r;
+            const bool ok = row < R;
+            cp_async16(dst + r * LD + k, g_h2 + (ok ? row : 0) * H + c_base + k, ok ? 16 : 0);
+        }
+        cp_async_commit();
+    };
+    struct RowIn { float4 o4; float v, adv, ret; int act; bool ok; };
+    auto row_load = [&](int tile) {
+        RowIn in;
+        const size_t i = (size_t)tile * TR + lane;
+        in.ok = tile < ntiles && i < R;
+        in.o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        in.v = in.adv = in.ret = 0.f;
+        in.act = 0;
+        if (in.ok) {
+            in.o4 = *reinterpret_cast<const float4*>(b.out5 + i * 8);
+            in.v = b.out5[i * 8 + 4];
+            in.adv = b.adv[i];
+            in.ret = b.ret[i];
+            in.act = b.tact[i];
+        }
+        return in;
+    };
+    auto row_finish = [&](const RowIn& in, int buf) {  // lane = row of the tile
+        float dO[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+        if (in.ok) {
+            const float o[4] = {in.o4.x, in.o4.y, in.o4.z, in.o4.w};
+            const float mx = fmaxf(fmaxf(o[0], o[1]), fmaxf(o[2], o[3]));
+            float ex[4], Z = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { ex[c] = expf(o[c] - mx); Z += ex[c]; }
+            const float logZ = logf(Z);
+            float p[4], lp[4], ent = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
+            const float A = in.adv, err = in.v - in.ret;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) dO[c] = round_bf16((-A * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
+            dO[4] = round_bf16(2.f * a.c_v * err * invR);
+            l_pg += -A * (in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3]);
+            l_v += err * err;
+            l_ent += ent;
+#pragma unroll
+            for (int c = 0; c < 5; ++c) a_bh[c] += dO[c];
+        }
+        uint4 pk;
+        pk.x = pack_bf16(__float2bfloat16_rn(dO[0]), __float2bfloat16_rn(dO[1]));
+        pk.y = pack_bf16(__float2bfloat16_rn(dO[2]), __float2bfloat16_rn(dO[3]));
+        pk.z = pack_bf16(__float2bfloat16_rn(dO[4]), __float2bfloat16_rn(0.f));
+        pk.w = 0u;
+        *reinterpret_cast<uint4*>(s_dA + (buf * TR + lane) * 8) = pk;
+#pragma unroll
+        for (int c = 0; c < 5; ++c) s_dT[(buf * 8 + c) * LDT + lane] = __float2bfloat16_rn(dO[c]);
+    };
+    // staged dh2 tile -> global: thread = (row, 16-column piece), 32 bytes each, rows in whole 512-byte segments
+    auto copy_out = [&](int tile, int buf) {
+        const int r = tid >> 4, c16 = (tid & 15) * 16;
+        const size_t row = (size_t)tile * TR + r;
+        if (row < R) {
+            const uint4* src = reinterpret_cast<const uint4*>(s_o + (buf * TR + r) * LD + c16);
+            uint4* dst = reinterpret_cast<uint4*>(g_dh2 + row * H + c_base + c16);
+            dst[0] = src[0];
+            dst[1] = src[1];
+        }
+    };
+
+    int it = 0, prev_tile = -1;
+#pragma unroll
+    for (int q = 0; q < NST - 1; ++q) load_tile(blockIdx.x + q * (int)gridDim.x, q);
+    __syncthreads();  // the zeroed rows of s_dT are in place before the first row phase writes beside them
+    if ((int)blockIdx.x < ntiles && wid == 0) row_finish(row_load(blockIdx.x), 0);
+    const int jm = lane >> 3, r8 = lane & 7;  // ldmatrix addressing: matrix index, row inside the matrix
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
+        const int buf = it & 1;
+        const int next = tile + (int)gridDim.x;
+        cp_async_wait<NST - 2>();
+        __syncthreads();  // this tile's h2 and dOut are in place; the staging tile of the tile before is complete
+        load_tile(tile + (NST - 1) * (int)gridDim.x, (it + NST - 1) % NST);
+        const bool row_warp = wid == (it + 1) % NW;  // this warp prepares the next tile's output gradients
+        RowIn nin;
+        if (row_warp) nin = row_load(next);
+        if (prev_tile >= 0) copy_out(prev_tile, buf ^ 1);
+        const __nv_bfloat16* h2t = s_h2 + (it % NST) * TR * LD;
+        __nv_bfloat16* ot = s_o + buf * TR * LD;
+        // ---- dh2 = (dOut Wh^T) gated by h2 > 0: A = dOut rows (k = head index; only k < 8 can be non-zero)
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            uint32_t af[4];
+            af[0] = *reinterpret_cast<const uint32_t*>(s_dA + (buf * TR + 16 * mt + g) * 8 + 2 * t4);
+            af[1] = *reinterpret_cast<const uint32_t*>(s_dA + (buf * TR + 16 * mt + g + 8) * 8 + 2 * t4);
+            af[2] = af[3] = 0u;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float c[4] = {0.f, 0.f, 0.f, 0.f};
+                mma_bf16(c, af, whf[j], 0u);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int row = 16 * mt + 8 * hh + g, col = col0 + 8 * j + 2 * t4;
+                    const uint32_t hv = *reinterpret_cast<const uint32_t*>(h2t + row * LD + col);  // h2 >= 0: any magnitude bit = "> 0"
+                    const float v0 = (hv & 0x00007FFFu) ? c[2 * hh] : 0.f, v1 = (hv & 0x7FFF0000u) ? c[2 * hh + 1] : 0.f;
+                    const __nv_bfloat162 pk = __floats2bfloat162_rn(v0, v1);
+                    const uint32_t pku = *reinterpret_cast<const uint32_t*>(&pk);
+                    *reinterpret_cast<uint32_t*>(ot + row * LD + col) = pku;
+                    a_b2[j][0] += __uint_as_float(pku << 16);  // the sums take the rounded values
+                    a_b2[j][1] += __uint_as_float(pku & 0xFFFF0000u);
+                }
+            }
+        }
+        // ---- dWh += h2^T dOut: A[m = column][k = row] comes transposed out of the [row][column] tile
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+            uint32_t af[4];
+            ldmatrix_x4_trans(af, h2t + (16 * ks + 8 * (jm >> 1) + r8) * LD + col0 + 8 * (jm & 1));
+            const uint32_t b0 = *reinterpret_cast<const uint32_t*>(s_dT + (buf * 8 + g) * LDT + 16 * ks + 2 * t4);
+            const uint32_t b1 = *reinterpret_cast<const uint32_t*>(s_dT + (buf * 8 + g) * LDT + 16 * ks + 2 * t4 + 8);
+            mma_bf16(acc_wh, af, b0, b1);
+        }
+        // ---- row phase of the next tile (its inputs were requested before the tensor work)
+        if (row_warp && next < ntiles) row_finish(nin, buf ^ 1);
+        prev_tile = tile;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    if (prev_tile >= 0) copy_out(prev_tile, (it - 1) & 1);
+    // ---- per-CTA results (split index = CTA): dWh from the accumulator fragments, db2 folded over the 8 row lanes
+    float* part = a.part_small + (size_t)(4 * blockIdx.x) * a.small_stride;
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int col = c_base + col0 + g + 8 * hh;
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc)
+            if (2 * t4 + cc < 5) part[(size_t)col * 5 + 2 * t4 + cc] = acc_wh[2 * hh + cc];
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+            float v = a_b2[j][cc];
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 8);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 16);
+            if (g == 0) part[(size_t)H * 5 + c_base + col0 + 8 * j + 2 * t4 + cc] = v;
+        }
+    {   // every warp has taken turns at the row phase: fold its lanes (fixed tree), then the warps in index order
+        float vals[8] = {a_bh[0], a_bh[1], a_bh[2], a_bh[3], a_bh[4], l_pg, l_v, l_ent};
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) vals[c] += __shfl_xor_sync(0xFFFFFFFFu, vals[c], off);
+        if (lane == 0) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) s_fin[wid * 8 + c] = vals[c];
+        }
+    }
+    __syncthreads();
+    if (tid < 8 && blockIdx.y == 0) {  // dbh and the loss terms come from the first slab only
+        float sum = 0.f;
+        for (int e = 0; e < NW; ++e) sum += s_fin[e * 8 + tid];
+        if (tid < 5) part[(size_t)H * 6 + tid] = sum;
+        else b.loss_part[(size_t)blockIdx.x * 4 + (tid - 5)] = sum;
+    }
+}
+
+// ----------------------------------------------------------------------------------------------------
 // k_dh1: dh1 = (dh2 W2^T) gated by h1 > 0 on the tensor pipe, and S = sum over t of dh1.
 // A CTA owns 64 envs x BN output columns and walks t = 0..T-1.  Its slice of W2 (BN rows, all K, hi and lo planes)
 // stays in shared memory for the whole kernel; the dh2 planes stream through a cp.async ring in 64-wide k chunks
@@ -809,6 +1026,14 @@ static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s) 
     return cudaGetLastError();
 }
 
+template <int H>
+static cudaError_t launch_heads_tc_t(const LearnArgs& a, int grid, cudaStream_t s) {
+    using Cfg = HeadsTcCfg<H>;
+    CK(cudaFuncSetAttribute(k_heads_bwd_tc<H>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
+    k_heads_bwd_tc<H><<<dim3(grid, H / Cfg::HS), 512, Cfg::smem_bytes, s>>>(a);
+    return cudaGetLastError();
+}
+
 template <int H, int BN, int PREC>
 static cudaError_t launch_dh1_t(const LearnArgs& a, cudaStream_t s) {
     using Cfg = Dh1Cfg<H, BN, PREC>;
@@ -849,9 +1074,12 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
             case 256: CK((launch_heads_t<256, 16, PREC>(a, pl.heads_grid, s))); break;
             default:
                 if constexpr (PREC == 1) {
-                    if (wide && H == 512) { CK((launch_heads_t<512, 16, 1, 256, true>(a, pl.heads_grid, s))); break; }
-                    if (wide && H == 1024) { CK((launch_heads_t<1024, 16, 1, 256, true>(a, pl.heads_grid, s))); break; }
-                    if (wide && H == 2048) { CK((launch_heads_t<2048, 16, 1, 256, true>(a, pl.heads_grid, s))); break; }
+                    if (wide) {  // tensor-pipe version: one partial slot per CTA (slot 4 * CTA of the small region)
+                        for (int q = 5; q <= 7; ++q) { a.reg[q].ns = pl.heads_grid; a.reg[q].stride = 4 * pl.small_stride; }
+                        if (H == 512) { CK((launch_heads_tc_t<512>(a, pl.heads_grid, s))); break; }
+                        if (H == 1024) { CK((launch_heads_tc_t<1024>(a, pl.heads_grid, s))); break; }
+                        if (H == 2048) { CK((launch_heads_tc_t<2048>(a, pl.heads_grid, s))); break; }
+                    }
                 }
                 return cudaErrorNotSupported;
         }
