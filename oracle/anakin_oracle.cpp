@@ -147,8 +147,11 @@ void env_init(uint64_t seed, int B, int N, double density, uint32_t* walls, uint
 // 1 right (col+1), 2 down (row+1), 3 left (col-1).  A move into a wall or off the grid leaves the agent
 // in place.  Reaching the goal pays 1 and ends the episode; the step cap ends it with reward 0.  On
 // episode end the env resets itself to its seeded start inside the same step.
+// The paper's env interface is generic (any `initial_state` / `step` written as array code); `kind` selects a
+// second env with the same state and observation: kind 1 = torus, where a move off an edge re-enters at the
+// opposite edge (walls still block).
 void env_step(const Dims& d, const uint32_t* walls, uint8_t start, uint8_t goal, int cap,
-              uint8_t* pos, uint8_t* tep, int action, float* reward, uint8_t* done) {
+              uint8_t* pos, uint8_t* tep, int action, float* reward, uint8_t* done, int kind = 0) {
     const int N = d.N;
     const int row = *pos / N, col = *pos % N;
     int nr = row, nc = col;
@@ -156,6 +159,10 @@ void env_step(const Dims& d, const uint32_t* walls, uint8_t start, uint8_t goal,
     else if (action == 1) nc = col + 1;
     else if (action == 2) nr = row + 1;
     else nc = col - 1;
+    if (kind == 1) {
+        nr = (nr + N) % N;
+        nc = (nc + N) % N;
+    }
     int np = *pos;
     if (nr >= 0 && nr < N && nc >= 0 && nc < N) {
         const int cand = nr * N + nc;
@@ -481,6 +488,11 @@ void orc_env_step(int N, const uint32_t* walls, uint8_t start, uint8_t goal, int
     env_step(make_dims(N, 16), walls, start, goal, cap, pos, tep, action, reward, done);
 }
 
+void orc_env_step_kind(int kind, int N, const uint32_t* walls, uint8_t start, uint8_t goal, int cap, uint8_t* pos,
+                       uint8_t* tep, int action, float* reward, uint8_t* done) {
+    env_step(make_dims(N, 16), walls, start, goal, cap, pos, tep, action, reward, done, kind);
+}
+
 void orc_observe(int N, const uint32_t* walls, uint8_t pos, uint8_t goal, float* x) {
     observe(make_dims(N, 16), walls, pos, goal, x);
 }
@@ -536,11 +548,11 @@ void orc_sample_from_logits(uint64_t seed, uint32_t gstep0, int T, int B, const 
 // state the action was taken in, the action, reward, done, value and log-probability.  After the last
 // step the value of the current state is stored in value[T][b] (the bootstrap).
 // Env dynamic state (pos, tep) is updated in place; the global step counter advances by T (caller).
-void orc_rollout(int N, int H, int prec, int B, int T, int cap, const float* theta, const uint32_t* walls,
-                 const uint8_t* start, const uint8_t* goal, uint8_t* pos, uint8_t* tep, uint64_t seed,
-                 uint32_t gstep0, const int8_t* forced /*nullable [T][B]*/, uint8_t* tpos, int8_t* tact,
-                 uint8_t* tdone, float* trew, float* tval /*[T+1][B]*/, float* tlogp,
-                 float* tlogits /*nullable [T][B][4]*/, uint8_t* tnear /*nullable*/) {
+void orc_rollout_kind(int kind, int N, int H, int prec, int B, int T, int cap, const float* theta, const uint32_t* walls,
+                      const uint8_t* start, const uint8_t* goal, uint8_t* pos, uint8_t* tep, uint64_t seed,
+                      uint32_t gstep0, const int8_t* forced /*nullable [T][B]*/, uint8_t* tpos, int8_t* tact,
+                      uint8_t* tdone, float* trew, float* tval /*[T+1][B]*/, float* tlogp,
+                      float* tlogits /*nullable [T][B][4]*/, uint8_t* tnear /*nullable*/) {
     const Dims d = make_dims(N, H);
     const std::vector<float> cp = compute_params(d, theta, prec);
 #pragma omp parallel
@@ -570,10 +582,18 @@ void orc_rollout(int N, int H, int prec, int B, int T, int cap, const float* the
                 tact[i] = (int8_t)a;
                 tlogp[i] = lp;
                 if (tnear) tnear[i] = nr;
-                env_step(d, w, start[b], goal[b], cap, &pos[b], &tep[b], a, &trew[i], &tdone[i]);
+                env_step(d, w, start[b], goal[b], cap, &pos[b], &tep[b], a, &trew[i], &tdone[i], kind);
             }
         }
     }
+}
+
+void orc_rollout(int N, int H, int prec, int B, int T, int cap, const float* theta, const uint32_t* walls,
+                 const uint8_t* start, const uint8_t* goal, uint8_t* pos, uint8_t* tep, uint64_t seed,
+                 uint32_t gstep0, const int8_t* forced, uint8_t* tpos, int8_t* tact, uint8_t* tdone, float* trew,
+                 float* tval, float* tlogp, float* tlogits, uint8_t* tnear) {
+    orc_rollout_kind(0, N, H, prec, B, T, cap, theta, walls, start, goal, pos, tep, seed, gstep0, forced, tpos, tact, tdone,
+                     trew, tval, tlogp, tlogits, tnear);
 }
 
 // Generalised advantage estimation, reverse scan over t for each env:

@@ -125,15 +125,18 @@ def param_init(seed: int, N: int, H: int) -> np.ndarray:
     return theta
 
 
-def env_step(N: int, walls_b: np.ndarray, start: int, goal: int, cap: int, pos: int, tep: int, action: int):
+GRID, TORUS = 0, 1  # env kinds: walls and borders block / walls block and borders wrap around
+
+
+def env_step(N: int, walls_b: np.ndarray, start: int, goal: int, cap: int, pos: int, tep: int, action: int, kind: int = GRID):
     """One env, one step.  Returns (pos', tep', reward, done)."""
     w = np.ascontiguousarray(walls_b, dtype=np.uint32)
     p = C.c_uint8(pos)
     t = C.c_uint8(tep)
     r = C.c_float(0)
     dn = C.c_uint8(0)
-    lib().orc_env_step(C.c_int(N), _p(w), C.c_uint8(start), C.c_uint8(goal), C.c_int(cap), C.byref(p), C.byref(t),
-                       C.c_int(action), C.byref(r), C.byref(dn))
+    lib().orc_env_step_kind(C.c_int(kind), C.c_int(N), _p(w), C.c_uint8(start), C.c_uint8(goal), C.c_int(cap), C.byref(p),
+                            C.byref(t), C.c_int(action), C.byref(r), C.byref(dn))
     return int(p.value), int(t.value), float(r.value), int(dn.value)
 
 
@@ -203,7 +206,7 @@ class Trajectory:
     near: np.ndarray  # u8 [T][B]  uniform within 1e-5 of a CDF boundary
 
 
-def rollout(N, H, prec, T, cap, theta, walls, start, goal, pos, tep, seed, gstep0, forced=None) -> Trajectory:
+def rollout(N, H, prec, T, cap, theta, walls, start, goal, pos, tep, seed, gstep0, forced=None, kind: int = GRID) -> Trajectory:
     """Runs T steps for all envs; pos/tep (uint8 arrays) are updated in place."""
     B = walls.shape[0]
     tr = Trajectory(
@@ -213,10 +216,10 @@ def rollout(N, H, prec, T, cap, theta, walls, start, goal, pos, tep, seed, gstep
     if forced is not None:
         forced = np.ascontiguousarray(forced, dtype=np.int8)
         assert forced.shape == (T, B)
-    lib().orc_rollout(C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), C.c_int(cap), _p(theta), _p(walls),
-                      _p(start), _p(goal), _p(pos), _p(tep), C.c_uint64(seed), C.c_uint32(gstep0), _p(forced),
-                      _p(tr.pos), _p(tr.action), _p(tr.done), _p(tr.reward), _p(tr.value), _p(tr.logp), _p(tr.logits),
-                      _p(tr.near))
+    lib().orc_rollout_kind(C.c_int(kind), C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), C.c_int(cap), _p(theta),
+                           _p(walls), _p(start), _p(goal), _p(pos), _p(tep), C.c_uint64(seed), C.c_uint32(gstep0), _p(forced),
+                           _p(tr.pos), _p(tr.action), _p(tr.done), _p(tr.reward), _p(tr.value), _p(tr.logp), _p(tr.logits),
+                           _p(tr.near))
     return tr
 
 
@@ -282,7 +285,8 @@ class Agent:
     library keeps (params, Adam moments and step, env static/dynamic state, global step counter)."""
 
     def __init__(self, B, N, H, T, prec=0, cap=50, density=0.2, gamma=0.99, lam=0.95, c_e=0.01, c_v=0.5, lr=3e-4,
-                 b1=0.9, b2=0.999, eps=1e-8):
+                 b1=0.9, b2=0.999, eps=1e-8, kind=GRID):
+        self.kind = kind
         self.B, self.N, self.H, self.T, self.prec, self.cap, self.density = B, N, H, T, prec, cap, density
         self.gamma, self.lam, self.c_e, self.c_v = gamma, lam, c_e, c_v
         self.lr, self.b1, self.b2, self.eps = lr, b1, b2, eps
@@ -304,7 +308,7 @@ class Agent:
     def rollout(self, T=None, forced=None) -> Trajectory:
         T = self.T if T is None else T
         self.traj = rollout(self.N, self.H, self.prec, T, self.cap, self.theta, self.walls, self.start, self.goal,
-                            self.pos, self.tep, self.seed, self.gstep, forced)
+                            self.pos, self.tep, self.seed, self.gstep, forced, self.kind)
         self.gstep += T
         return self.traj
 

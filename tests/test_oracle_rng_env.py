@@ -278,3 +278,93 @@ def test_observation_planes(N):
         assert (x[:C] == bits[b]).all()
         assert x[C:2 * C].argmax() == start[b] and x[C:2 * C].sum() == 1
         assert x[2 * C:].argmax() == goal[b] and x[2 * C:].sum() == 1
+
+
+# ---- second env ("torus": a move off an edge re-enters at the opposite edge; walls still block) ----
+def test_torus_step_hand_traced_episode():
+    cells, steps, meta = load_trace(os.path.join(GOLDEN, "torus_trace_5x5.txt"))
+    w = np.zeros(1, np.uint32)
+    for c in cells:
+        w[0] |= np.uint32(1 << c)
+    pos, tep = meta["start"], 0
+    for a, p0, t0, p1, t1, r, dn in steps:
+        assert (pos, tep) == (p0, t0)
+        pos, tep, rew, done = orc.env_step(5, w, meta["start"], meta["goal"], meta["cap"], pos, tep, a, orc.TORUS)
+        assert (pos, tep, rew, done) == (p1, t1, float(r), dn)
+
+
+def test_torus_without_walls_is_addition_modulo_n():
+    """Closed form: on an empty board the position after any action sequence is start + sum of displacements, each
+    coordinate modulo N (until the goal is entered)."""
+    N, cap = 7, 255
+    w = np.zeros(2, np.uint32)
+    rng = np.random.default_rng(3)
+    disp = [(-1, 0), (0, 1), (1, 0), (0, -1)]
+    for trial in range(20):
+        start, goal = (int(x) for x in rng.choice(N * N, 2, replace=False))
+        pos, tep = start, 0
+        r, c = divmod(start, N)
+        for k in range(200):
+            a = int(rng.integers(0, 4))
+            r, c = (r + disp[a][0]) % N, (c + disp[a][1]) % N
+            pos, tep, rew, done = orc.env_step(N, w, start, goal, cap, pos, tep, a, orc.TORUS)
+            if r * N + c == goal:
+                assert (rew, done, pos, tep) == (1.0, 1, start, 0)
+                break
+            assert (rew, done, pos, tep) == (0.0, 0, r * N + c, k + 1)
+
+
+def test_torus_and_grid_agree_away_from_the_edges_and_differ_on_them():
+    N, cap = 6, 50
+    w = np.zeros(2, np.uint32)
+    w[0] = np.uint32(1 << 14)  # one wall at (2, 2)
+    for pos in range(N * N):
+        if pos == 14:
+            continue
+        r, c = divmod(pos, N)
+        for a, (dr, dc) in enumerate([(-1, 0), (0, 1), (1, 0), (0, -1)]):
+            g = orc.env_step(N, w, 0, 35, cap, pos, 0, a, orc.GRID)
+            t = orc.env_step(N, w, 0, 35, cap, pos, 0, a, orc.TORUS)
+            inside = 0 <= r + dr < N and 0 <= c + dc < N
+            if inside:
+                assert g == t
+            else:
+                assert g[0] == pos or g[3] == 1  # the grid blocks at the edge
+                want = ((r + dr) % N) * N + (c + dc) % N
+                assert t[0] == (0 if want == 35 else want)  # entering the goal (cell 35) restarts at the start cell 0
+
+
+@pytest.mark.parametrize("N", [5, 8])
+def test_torus_invariants_under_random_actions(N):
+    B, steps, cap = 32, 300, 50
+    C = N * N
+    walls, start, goal = orc.env_init(23, B, N, 0.2)
+    bits = unpack_walls(walls, C)
+    rng = np.random.default_rng(6)
+    for b in range(B):
+        # brute-force component of the start cell under wrap-around adjacency
+        seen, todo = {int(start[b])}, [int(start[b])]
+        while todo:
+            p = todo.pop()
+            r, c = divmod(p, N)
+            for nr, nc in (((r - 1) % N, c), (r, (c + 1) % N), ((r + 1) % N, c), (r, (c - 1) % N)):
+                q = nr * N + nc
+                if not bits[b, q] and q not in seen:
+                    seen.add(q)
+                    todo.append(q)
+        pos, tep, since = int(start[b]), 0, 0
+        for _ in range(steps):
+            a = int(rng.integers(0, 4))
+            r0, c0 = divmod(pos, N)
+            tr, tc = [((r0 - 1) % N, c0), (r0, (c0 + 1) % N), ((r0 + 1) % N, c0), (r0, (c0 - 1) % N)][a]
+            land = pos if bits[b, tr * N + tc] else tr * N + tc
+            npos, ntep, rew, done = orc.env_step(N, walls[b], int(start[b]), int(goal[b]), cap, pos, tep, a, orc.TORUS)
+            since += 1
+            assert (rew == 1.0) == (land == goal[b])
+            if land == goal[b] or since >= cap:
+                assert done == 1 and npos == start[b] and ntep == 0
+                since = 0
+            else:
+                assert done == 0 and npos == land and ntep == since
+            assert not bits[b, npos] and npos in seen and ntep < cap
+            pos, tep = npos, ntep
