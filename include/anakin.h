@@ -61,6 +61,11 @@ enum {
 enum { ANAKIN_PRECISION_FP32 = 0, ANAKIN_PRECISION_BF16 = 1 };
 
 /* Plain-old-data configuration.  struct_size must be sizeof(anakin_cfg) (ABI versioning). */
+/* Environments (Section 3.1: any `initial_state` / `step` written as array code).  GRID: a move off the board or into a
+ * wall leaves the agent in place.  TORUS: a move off an edge re-enters at the opposite edge; walls still block. */
+#define ANAKIN_ENV_GRID 0
+#define ANAKIN_ENV_TORUS 1
+
 typedef struct anakin_cfg {
     uint32_t struct_size;
     int32_t B;            /* environments, >= 1 */
@@ -80,6 +85,8 @@ typedef struct anakin_cfg {
                              initial state and its action noise from the Philox counters of env env_offset + b, so
                              that G handles with B/G envs each and offsets 0, B/G, ... hold exactly the envs of one
                              handle with B envs (the replicas of Section 3.1, Figure 2 bottom) */
+    int32_t env_kind;     /* ANAKIN_ENV_*: which `step` the envs run (same state, same observation planes) */
+    int32_t reserved;     /* must be 0 */
 } anakin_cfg;
 
 /* Blob selectors for anakin_get / anakin_set.  Sizes in bytes for the LAST rollout length T (or T_max where noted). */

@@ -29,7 +29,7 @@ class AnakinCfg(C.Structure):
         ("episode_cap", C.c_int32), ("wall_density", C.c_double),
         ("gamma", C.c_float), ("gae_lambda", C.c_float), ("entropy_coef", C.c_float), ("value_coef", C.c_float),
         ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float),
-        ("precision", C.c_int32), ("device", C.c_int32), ("debug_logits", C.c_int32), ("env_offset", C.c_int32),
+        ("precision", C.c_int32), ("device", C.c_int32), ("debug_logits", C.c_int32), ("env_offset", C.c_int32), ("env_kind", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -83,6 +83,7 @@ _lib.anakin_kernel_name.argtypes = [C.c_int]
 _lib.anakin_kernel_name.restype = C.c_char_p
 _lib.anakin_rollout_noalloc.argtypes = [C.POINTER(AnakinCfg), C.c_uint64, C.c_int64, C.c_int] + [_vp] * 13
 NOALLOC_MAX_BH = 1048576
+ENV_GRID, ENV_TORUS = 0, 1  # anakin_cfg.env_kind
 
 _BLOB_DTYPE = {
     PARAMS: np.float32, GRADS: np.float32, ADAM_M: np.float32, ADAM_V: np.float32, ENV_WALLS: np.uint32,
@@ -105,20 +106,21 @@ def lib() -> C.CDLL:
 
 def make_cfg(B, N, H, T_max, precision=0, episode_cap=50, wall_density=0.2, gamma=0.99, gae_lambda=0.95,
              entropy_coef=0.01, value_coef=0.5, lr=3e-4, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8, device=0,
-             debug_logits=0, env_offset=0) -> AnakinCfg:
+             debug_logits=0, env_offset=0, env_kind=0) -> AnakinCfg:
     c = AnakinCfg()
     c.struct_size = C.sizeof(AnakinCfg)
     c.B, c.N, c.H, c.T_max, c.episode_cap, c.wall_density = B, N, H, T_max, episode_cap, wall_density
     c.gamma, c.gae_lambda, c.entropy_coef, c.value_coef = gamma, gae_lambda, entropy_coef, value_coef
     c.lr, c.adam_b1, c.adam_b2, c.adam_eps = lr, adam_b1, adam_b2, adam_eps
     c.precision, c.device, c.debug_logits, c.env_offset = precision, device, debug_logits, env_offset
+    c.env_kind, c.reserved = env_kind, 0
     return c
 
 
 def cfg_from_workload(w, device=0, debug_logits=0, T_max=None, env_offset=0) -> AnakinCfg:
     return make_cfg(w.B, w.N, w.H, w.T if T_max is None else T_max, w.precision, w.episode_cap, w.wall_density, w.gamma,
                     w.gae_lambda, w.entropy_coef, w.value_coef, w.lr, w.adam_b1, w.adam_b2, w.adam_eps, device,
-                    debug_logits, env_offset)
+                    debug_logits, env_offset, getattr(w, "env_kind", 0))
 
 
 def workspace_bytes(cfg: AnakinCfg) -> int:

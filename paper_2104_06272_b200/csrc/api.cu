@@ -42,6 +42,8 @@ int validate(const anakin_cfg* c) {
     if (c->B < 1 || c->T_max < 1 || c->episode_cap < 1 || c->episode_cap > 255) return ANAKIN_E_INVALID_ARG;
     if (!(c->wall_density >= 0.0 && c->wall_density < 1.0)) return ANAKIN_E_INVALID_ARG;
     if (c->precision != ANAKIN_PRECISION_FP32 && c->precision != ANAKIN_PRECISION_BF16) return ANAKIN_E_INVALID_ARG;
+    if (c->reserved != 0) return ANAKIN_E_INVALID_ARG;
+    if (c->env_kind != ANAKIN_ENV_GRID && c->env_kind != ANAKIN_ENV_TORUS) return ANAKIN_E_UNSUPPORTED_CFG;
     if (c->env_offset < 0 || (double)c->env_offset + (double)c->B > 2147483647.0) return ANAKIN_E_INVALID_ARG;
     if (c->N < 2 || c->N > 16) return ANAKIN_E_UNSUPPORTED_CFG;
     const int hj = c->H / 32;
@@ -199,6 +201,7 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     a.gstep0 = (uint32_t)h->gstep;
     a.key0 = (uint32_t)(h->seed & 0xFFFFFFFFu);
     a.key1 = (uint32_t)(h->seed >> 32);
+    a.env_kind = h->cfg.env_kind;
     a.forced = forced;
     a.replay = 0;
     a.fuse_gae = rollout_mma_supported(h->d.H) ? 1 : 0;
@@ -234,6 +237,7 @@ int replay_activations(anakin_t* h) {
     a.cap = h->cfg.episode_cap;
     a.gstep0 = 0;
     a.key0 = a.key1 = 0;
+    a.env_kind = h->cfg.env_kind;
     a.forced = nullptr;
     a.replay = 1;
     a.fuse_gae = 0;

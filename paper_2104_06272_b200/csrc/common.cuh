@@ -118,6 +118,7 @@ struct RolloutArgs {
     int cap;
     uint32_t gstep0;
     uint32_t key0, key1;
+    int env_kind;          // ANAKIN_ENV_*: the transition rule (env_step.cuh)
     const int8_t* forced;  // nullable
     int replay;            // 1: recompute and save the activations of the recorded rows only (no sampling, no env step)
     int fuse_gae;          // 1: after the last step each env's owner thread also runs the GAE scan (fills ADV, RET)

@@ -22,8 +22,26 @@ struct StepPre {
     int np[4];  // 0 up, 1 right, 2 down, 3 left; blocked moves stay in place
 };
 
+// The env's movement rule as a compile-time plug-in: target(row, col, action, N) = the cell the move aims at, or -1
+// when it leaves the board.  Everything else of `step` (walls, clock, goal, restart, records) is shared.
+struct GridMoves {  // borders block
+    static __device__ __forceinline__ int target(int row, int col, int act, int N) {
+        const int nr = act == 0 ? row - 1 : act == 2 ? row + 1 : row, nc = act == 1 ? col + 1 : act == 3 ? col - 1 : col;
+        return (nr >= 0 && nr < N && nc >= 0 && nc < N) ? nr * N + nc : -1;
+    }
+};
+struct TorusMoves {  // borders wrap around
+    static __device__ __forceinline__ int target(int row, int col, int act, int N) {
+        int nr = act == 0 ? row - 1 : act == 2 ? row + 1 : row, nc = act == 1 ? col + 1 : act == 3 ? col - 1 : col;
+        nr = nr < 0 ? N - 1 : nr >= N ? 0 : nr;
+        nc = nc < 0 ? N - 1 : nc >= N ? 0 : nc;
+        return nr * N + nc;
+    }
+};
+
 // walls: this env's wall words (shared memory), 8 words.
-__device__ __forceinline__ StepPre step_prepare(const EnvLane& s, const RolloutArgs& a, int env, int t, const uint32_t* walls) {
+template <class Moves>
+__device__ __forceinline__ StepPre step_prepare_t(const EnvLane& s, const RolloutArgs& a, int env, int t, const uint32_t* walls) {
     StepPre p;
     const U4 r = philox4x32_10((uint32_t)(a.d.env0 + env), a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
     p.u = uniform24(r.x);
@@ -31,19 +49,15 @@ __device__ __forceinline__ StepPre step_prepare(const EnvLane& s, const RolloutA
     const int row = s.pos / N, col = s.pos - row * N;
 #pragma unroll
     for (int act = 0; act < 4; ++act) {
-        int nr = row, nc = col;
-        if (act == 0) nr = row - 1;
-        else if (act == 1) nc = col + 1;
-        else if (act == 2) nr = row + 1;
-        else nc = col - 1;
+        const int cand = Moves::target(row, col, act, N);
         int np = s.pos;
-        if (nr >= 0 && nr < N && nc >= 0 && nc < N) {
-            const int cand = nr * N + nc;
-            if (!((walls[cand >> 5] >> (cand & 31)) & 1u)) np = cand;
-        }
+        if (cand >= 0 && !((walls[cand >> 5] >> (cand & 31)) & 1u)) np = cand;
         p.np[act] = np;
     }
     return p;
+}
+__device__ __forceinline__ StepPre step_prepare(const EnvLane& s, const RolloutArgs& a, int env, int t, const uint32_t* walls) {
+    return a.env_kind == ANAKIN_ENV_TORUS ? step_prepare_t<TorusMoves>(s, a, env, t, walls) : step_prepare_t<GridMoves>(s, a, env, t, walls);
 }
 
 // Categorical sampling from the 4 logits (inverse CDF against the prepared uniform), the env transition and the records.

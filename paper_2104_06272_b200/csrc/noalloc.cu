@@ -103,6 +103,7 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     a.gstep0 = (uint32_t)global_step;
     a.key0 = (uint32_t)(seed & 0xFFFFFFFFu);
     a.key1 = (uint32_t)(seed >> 32);
+    a.env_kind = cfg->env_kind;
     a.forced = nullptr;
     a.replay = 0;
     a.fuse_gae = 0;  // the caller gets the trajectory only

@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(256) k_rollout(RolloutArgs a) {
     const Buffers& b = a.b;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int e0 = blockIdx.x * ME;
-    const int B = d.B, C = d.C, N = d.N;
+    const int B = d.B, C = d.C;
     const float* W1 = b.theta_c + d.oW1;
     const float* W2 = b.theta_c + d.oW2;
     const float* b2 = b.theta_c + d.ob2;
@@ -164,53 +164,18 @@ __global__ void __launch_bounds__(256) k_rollout(RolloutArgs a) {
             const int env = e0 + tid;
             const float l0 = s_out[tid * 8 + 0], l1 = s_out[tid * 8 + 1], l2 = s_out[tid * 8 + 2], l3 = s_out[tid * 8 + 3];
             b.tval[(size_t)t * B + env] = s_out[tid * 8 + 4];
-            if (t < a.T) {
-                const size_t i = (size_t)t * B + env;
-                const float mx = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
-                const float x0 = expf(l0 - mx), x1 = expf(l1 - mx), x2 = expf(l2 - mx), x3 = expf(l3 - mx);
-                const float Z = ((x0 + x1) + x2) + x3;
-                const float c0 = x0 / Z, c1 = c0 + x1 / Z, c2 = c1 + x2 / Z;
-                const U4 r = philox4x32_10((uint32_t)(a.d.env0 + env), a.gstep0 + (uint32_t)t, 0, STREAM_ACT, a.key0, a.key1);
-                const float u = uniform24(r.x);
-                int act = (u >= c0) + (u >= c1) + (u >= c2);
-                if (a.forced) {
-                    act = a.forced[i];
-                    if (act < 0 || act > 3) { bad |= DEV_E_BAD_ACTION; act &= 3; }
-                }
-                const float la = act == 0 ? l0 : act == 1 ? l1 : act == 2 ? l2 : l3;
-                b.tlogp[i] = (la - mx) - logf(Z);
-                b.tpos[i] = (uint8_t)my_pos;
-                b.tact[i] = (int8_t)act;
-                if (b.dbg_logits) reinterpret_cast<float4*>(b.dbg_logits)[i] = make_float4(l0, l1, l2, l3);
-                // env step
-                const int row = my_pos / N, col = my_pos - row * N;
-                int nr = row, nc = col;
-                if (act == 0) nr = row - 1;
-                else if (act == 1) nc = col + 1;
-                else if (act == 2) nr = row + 1;
-                else nc = col - 1;
-                int np = my_pos;
-                if (nr >= 0 && nr < N && nc >= 0 && nc < N) {
-                    const int cand = nr * N + nc;
-                    if (!((s_walls[tid * 8 + (cand >> 5)] >> (cand & 31)) & 1u)) np = cand;
-                }
-                const int te = my_tep + 1;
-                float rew = 0.f;
-                int done = 0;
-                if (np == my_goal) { rew = 1.f; done = 1; }
-                else if (te >= a.cap) { done = 1; }
-                if (done) {
-                    n_episodes += 1;
-                    n_goals += (np == my_goal);
-                    n_epsteps += te;
-                    my_pos = my_start;
-                    my_tep = 0;
-                } else {
-                    my_pos = np;
-                    my_tep = te;
-                }
-                b.trew[i] = rew;
-                b.tdone[i] = (uint8_t)done;
+            if (t < a.T) {  // the shared per-env step (env_step.cuh): sample, transition rule of the configured env, records
+                EnvLane es;
+                es.pos = my_pos; es.tep = my_tep; es.start = my_start; es.goal = my_goal;
+                es.n_episodes = es.n_goals = es.n_epsteps = 0;
+                es.bad = 0;
+                act_and_step(es, a, env, t, l0, l1, l2, l3, s_walls + tid * 8);
+                my_pos = es.pos;
+                my_tep = es.tep;
+                n_episodes += es.n_episodes;
+                n_goals += es.n_goals;
+                n_epsteps += es.n_epsteps;
+                bad |= es.bad;
                 s_pos[tid] = my_pos;
             }
         }

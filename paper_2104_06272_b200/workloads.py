@@ -32,6 +32,7 @@ class Workload:
     adam_b1: float = 0.9
     adam_b2: float = 0.999
     adam_eps: float = 1e-8
+    env_kind: int = 0  # 0 = gridworld (borders block), 1 = torus (borders wrap around)
 
     @property
     def C(self):

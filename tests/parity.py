@@ -64,7 +64,7 @@ def check_rollout(an, bnd, w, seed, st, T, forced=None, envs=None):
     pos, tep = st["pos"][sel].copy(), st["tep"][sel].copy()
     tr = orc.rollout(w.N, w.H, w.precision, T, w.episode_cap, st["theta"], np.ascontiguousarray(st["walls"][sel]),
                      st["start"][sel].copy(), st["goal"][sel].copy(), pos, tep, seed, st["gstep"],
-                     forced=np.ascontiguousarray(g["action"][:, sel]))
+                     forced=np.ascontiguousarray(g["action"][:, sel]), kind=w.env_kind)
     if forced is not None:
         assert (g["action"] == forced).all()
     assert (g["pos"][:, sel] == tr.pos).all(), "recorded positions differ"

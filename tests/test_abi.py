@@ -41,7 +41,7 @@ def test_cfg_struct_matches_header_size(bnd):
     with pytest.raises(bnd.AnakinError) as e:
         bnd.workspace_bytes(cfg)
     assert e.value.code == bnd.E_INVALID_ARG
-    assert C.sizeof(bnd.AnakinCfg) == 80 and C.sizeof(bnd.AnakinStats) == 48
+    assert C.sizeof(bnd.AnakinCfg) == 88 and C.sizeof(bnd.AnakinStats) == 48
 
 
 @pytest.mark.parametrize("kw,code", [

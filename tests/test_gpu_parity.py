@@ -43,6 +43,11 @@ SMALL = {
     "tp_ragged_64": Workload("tp_ragged_64", B=97, N=3, H=64, T=3, iters=1, episode_cap=2),
     "tp_bf16_128": Workload("tp_bf16_128", B=210, N=7, H=128, T=6, iters=1, precision=1, episode_cap=5),
     "tp_bf16_256": Workload("tp_bf16_256", B=131, N=16, H=256, T=5, iters=1, precision=1),
+    # the second env (torus: moves wrap around the edges) on every rollout path: persistent tensor-pipe kernel,
+    # FFMA kernel, wide bf16 path
+    "torus_tp_256": Workload("torus_tp_256", B=140, N=6, H=256, T=12, iters=1, episode_cap=9, env_kind=1),
+    "torus_ffma_96": Workload("torus_ffma_96", B=77, N=5, H=96, T=12, iters=1, episode_cap=9, env_kind=1),
+    "torus_wide_512": Workload("torus_wide_512", B=70, N=8, H=512, T=6, iters=1, precision=1, episode_cap=9, env_kind=1),
 }
 
 
@@ -307,3 +312,36 @@ def test_update_from_set_trajectory_recomputes_the_forward_pass(bnd):
     c.learn()
     d.learn()
     assert (c.get(bnd.GRADS).view(np.uint32) == d.get(bnd.GRADS).view(np.uint32)).all()
+
+
+def test_torus_env_free_running_and_different_from_the_grid(bnd):
+    """The second env kind: the library and the oracle agent, both running freely from one seed, record the same
+    trajectory; and the same seed under the grid rule gives a different one (some move crosses an edge)."""
+    w = WORKLOADS["tiny"].scaled(name="tiny_torus", B=96, T=24, env_kind=1)
+    an = make(bnd, w)
+    ag = orc.Agent(w.B, w.N, w.H, w.T, w.precision, w.episode_cap, w.wall_density, np.float32(w.gamma),
+                   np.float32(w.gae_lambda), np.float32(w.entropy_coef), np.float32(w.value_coef), np.float32(w.lr),
+                   np.float32(w.adam_b1), np.float32(w.adam_b2), np.float32(w.adam_eps), kind=orc.TORUS)
+    an.reset(4)
+    ag.reset(4)
+    an.rollout()
+    tr = ag.rollout()
+    g = par.gpu_traj(an, bnd, w.T)
+    mism = g["action"] != tr.action
+    assert not (mism & (tr.near == 0)).any()
+    if mism.any():
+        pytest.skip("a near-boundary sample diverged the free-running comparison")
+    assert (g["pos"] == tr.pos).all() and (g["reward"] == tr.reward).all() and (g["done"] == tr.done).all()
+    # a wrap really happened: some recorded step changes the column by N-1 or the row by N-1
+    pos = np.concatenate([tr.pos, an.get(bnd.ENV_POS)[None, :]], axis=0).astype(np.int64)
+    dr, dc = np.abs(np.diff(pos // w.N, axis=0)), np.abs(np.diff(pos % w.N, axis=0))
+    moved_by_wrap = ((dr == w.N - 1) | (dc == w.N - 1)) & (tr.done == 0)
+    assert moved_by_wrap.any()
+    grid = make(bnd, w.scaled(env_kind=0))
+    grid.reset(4)
+    grid.rollout()
+    assert not (par.gpu_traj(grid, bnd, w.T)["pos"] == g["pos"]).all()
+    an.learn()
+    ag.learn()
+    par.assert_close(an.get(bnd.GRADS), ag.grads, 1e-4, "grads")
+    assert an.status() == 0
