@@ -320,7 +320,11 @@ template <typename S>
 void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const uint32_t* walls,
                    const uint8_t* goal, const uint8_t* tpos, const int8_t* tact, const S* adv,
                    const S* ret, double c_v, double c_e, S* grads /*nullable*/, double loss4[4],
-                   const uint32_t* gate1 = nullptr, const uint32_t* gate2 = nullptr, double* gate_info /*[6]*/ = nullptr) {
+                   const uint32_t* gate1 = nullptr, const uint32_t* gate2 = nullptr, double* gate_info /*[6]*/ = nullptr,
+                   const S* logp_old = nullptr, double clip = 0.0) {
+    // logp_old != nullptr selects the clipped-surrogate policy term (PPO, Schulman et al. 2017, Eq. 7) in place of the
+    // plain policy-gradient term:  -min(r A, clip(r, 1-eps, 1+eps) A),  r = pi(a|s) / pi_old(a|s) = exp(logp - logp_old).
+    // Its gradient is that of -r A where the unclipped product is the smaller one (ties included) and zero elsewhere.
     const size_t R = (size_t)B * T;
     const int GW = (d.H + 31) / 32;
     const std::vector<S> cp = compute_params(d, theta, prec);
@@ -365,14 +369,23 @@ void loss_and_grad(const Dims& d, int prec, int B, int T, const S* theta, const 
             const double A = (double)adv[i];
             const double V = (double)out[4];
             const double err = V - (double)ret[i];
-            l_pg += -A * s.logp[a];
+            double pg_coef = 1.0;  // d(policy term)/d(logp[a]) = -A * pg_coef
+            if (logp_old) {
+                const double r = std::exp(s.logp[a] - (double)logp_old[i]);
+                const double rc = std::min(std::max(r, 1.0 - clip), 1.0 + clip);
+                const bool unclipped = r * A <= rc * A;
+                l_pg += -std::min(r * A, rc * A);
+                pg_coef = unclipped ? r : 0.0;
+            } else {
+                l_pg += -A * s.logp[a];
+            }
             l_v += err * err;
             l_ent += s.entropy;
             if (!grads) continue;
             // output gradients (already divided by R)
             S dOut[5];
             for (int k = 0; k < 4; ++k) {
-                const double dz = (-A * ((k == a ? 1.0 : 0.0) - s.p[k]) + c_e * s.p[k] * (s.logp[k] + s.entropy)) / (double)R;
+                const double dz = (-A * pg_coef * ((k == a ? 1.0 : 0.0) - s.p[k]) + c_e * s.p[k] * (s.logp[k] + s.entropy)) / (double)R;
                 dOut[k] = maybe_bf16((S)dz, prec);
             }
             dOut[4] = maybe_bf16((S)(2.0 * c_v * err / (double)R), prec);
@@ -627,6 +640,22 @@ void orc_learn_f64(int N, int H, int B, int T, const double* theta, const uint32
                    const uint8_t* tpos, const int8_t* tact, const double* adv, const double* ret, double c_v,
                    double c_e, double* grads /*nullable*/, double* loss4) {
     loss_and_grad<double>(make_dims(N, H), 0, B, T, theta, walls, goal, tpos, tact, adv, ret, c_v, c_e, grads, loss4);
+}
+
+// The same with the clipped-surrogate policy term (logp_old = log-probabilities recorded when the actions were taken).
+void orc_learn_ppo_f32(int N, int H, int prec, int B, int T, const float* theta, const uint32_t* walls,
+                       const uint8_t* goal, const uint8_t* tpos, const int8_t* tact, const float* adv,
+                       const float* ret, const float* logp_old, double clip, double c_v, double c_e, float* grads,
+                       double* loss4, const uint32_t* gate1, const uint32_t* gate2, double* gate_info) {
+    loss_and_grad<float>(make_dims(N, H), prec, B, T, theta, walls, goal, tpos, tact, adv, ret, c_v, c_e, grads, loss4,
+                         gate1, gate2, gate_info, logp_old, clip);
+}
+
+void orc_learn_ppo_f64(int N, int H, int B, int T, const double* theta, const uint32_t* walls, const uint8_t* goal,
+                       const uint8_t* tpos, const int8_t* tact, const double* adv, const double* ret,
+                       const double* logp_old, double clip, double c_v, double c_e, double* grads, double* loss4) {
+    loss_and_grad<double>(make_dims(N, H), 0, B, T, theta, walls, goal, tpos, tact, adv, ret, c_v, c_e, grads, loss4,
+                          nullptr, nullptr, nullptr, logp_old, clip);
 }
 
 // Adam (Kingma & Ba, Algorithm 1), k = step index AFTER the increment (first call: k = 1):

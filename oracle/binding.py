@@ -236,8 +236,9 @@ def gae(gamma: float, lam: float, reward: np.ndarray, value: np.ndarray, done: n
     return adv, ret
 
 
-def learn(N, H, prec, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, want_grads=True, gates=None):
-    """fp32-storage loss and batch-mean gradient.  Returns (grads f32 [P] or None, loss[4] f64), plus a
+def learn(N, H, prec, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, want_grads=True, gates=None,
+          logp_old=None, clip=0.0):
+    """fp32-storage loss and batch-mean gradient; with `logp_old` the policy term is the clipped surrogate (PPO).  Returns (grads f32 [P] or None, loss[4] f64), plus a
     gate report when `gates` = (gate1, gate2) uint32 bitmaps [R][ceil(H/32)] recorded by the implementation
     under test are given: the backward pass then takes the ReLU gate decisions from them."""
     T, B = tpos.shape
@@ -249,10 +250,17 @@ def learn(N, H, prec, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.0
         g2 = np.ascontiguousarray(gates[1], np.uint32)
         assert g1.size == g2.size == T * B * ((H + 31) // 32)
         info = np.zeros(6, np.float64)
-    lib().orc_learn_f32(C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), _p(theta), _p(walls), _p(goal),
-                        _p(np.ascontiguousarray(tpos, np.uint8)), _p(np.ascontiguousarray(tact, np.int8)),
-                        _p(np.ascontiguousarray(adv, np.float32)), _p(np.ascontiguousarray(ret, np.float32)),
-                        C.c_double(c_v), C.c_double(c_e), _p(grads), _p(loss), _p(g1), _p(g2), _p(info))
+    if logp_old is None:
+        lib().orc_learn_f32(C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), _p(theta), _p(walls), _p(goal),
+                            _p(np.ascontiguousarray(tpos, np.uint8)), _p(np.ascontiguousarray(tact, np.int8)),
+                            _p(np.ascontiguousarray(adv, np.float32)), _p(np.ascontiguousarray(ret, np.float32)),
+                            C.c_double(c_v), C.c_double(c_e), _p(grads), _p(loss), _p(g1), _p(g2), _p(info))
+    else:
+        lib().orc_learn_ppo_f32(C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), _p(theta), _p(walls), _p(goal),
+                                _p(np.ascontiguousarray(tpos, np.uint8)), _p(np.ascontiguousarray(tact, np.int8)),
+                                _p(np.ascontiguousarray(adv, np.float32)), _p(np.ascontiguousarray(ret, np.float32)),
+                                _p(np.ascontiguousarray(logp_old, np.float32)), C.c_double(clip), C.c_double(c_v),
+                                C.c_double(c_e), _p(grads), _p(loss), _p(g1), _p(g2), _p(info))
     if gates is not None:
         report = {"layer1": dict(mismatched=int(info[0]), max_abs_z=float(info[1]), rms_z=float(info[2])),
                   "layer2": dict(mismatched=int(info[3]), max_abs_z=float(info[4]), rms_z=float(info[5]))}
@@ -260,11 +268,18 @@ def learn(N, H, prec, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.0
     return grads, loss
 
 
-def learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, want_grads=True):
+def learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, want_grads=True, logp_old=None, clip=0.0):
     T, B = tpos.shape
     theta = np.ascontiguousarray(theta, np.float64)
     grads = np.zeros(Dims(N, H).P, np.float64) if want_grads else None
     loss = np.zeros(4, np.float64)
+    if logp_old is not None:
+        lib().orc_learn_ppo_f64(C.c_int(N), C.c_int(H), C.c_int(B), C.c_int(T), _p(theta), _p(walls), _p(goal),
+                                _p(np.ascontiguousarray(tpos, np.uint8)), _p(np.ascontiguousarray(tact, np.int8)),
+                                _p(np.ascontiguousarray(adv, np.float64)), _p(np.ascontiguousarray(ret, np.float64)),
+                                _p(np.ascontiguousarray(logp_old, np.float64)), C.c_double(clip), C.c_double(c_v),
+                                C.c_double(c_e), _p(grads), _p(loss))
+        return grads, loss
     lib().orc_learn_f64(C.c_int(N), C.c_int(H), C.c_int(B), C.c_int(T), _p(theta), _p(walls), _p(goal),
                         _p(np.ascontiguousarray(tpos, np.uint8)), _p(np.ascontiguousarray(tact, np.int8)),
                         _p(np.ascontiguousarray(adv, np.float64)), _p(np.ascontiguousarray(ret, np.float64)),
@@ -319,6 +334,18 @@ class Agent:
                                       self.adv, self.ret, self.c_v, self.c_e)
         self.k += 1
         adam(self.theta, self.grads, self.m, self.v, self.k, self.lr, self.b1, self.b2, self.eps)
+        self.traj = None
+
+    def learn_ppo(self, epochs: int, clip: float):
+        """`epochs` full-batch Adam steps on the clipped surrogate of the pending trajectory (advantages and recorded
+        log-probabilities stay fixed; the forward pass is recomputed with the current parameters every epoch)."""
+        tr = self.traj
+        self.adv, self.ret = gae(self.gamma, self.lam, tr.reward, tr.value, tr.done)
+        for _ in range(epochs):
+            self.grads, self.loss = learn(self.N, self.H, self.prec, self.theta, self.walls, self.goal, tr.pos, tr.action,
+                                          self.adv, self.ret, self.c_v, self.c_e, logp_old=tr.logp, clip=clip)
+            self.k += 1
+            adam(self.theta, self.grads, self.m, self.v, self.k, self.lr, self.b1, self.b2, self.eps)
         self.traj = None
 
     def run(self, iters: int):

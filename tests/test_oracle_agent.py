@@ -474,3 +474,96 @@ def test_recorded_relu_gates_override_only_the_backward_decision():
     W2c = changed[s["W2"]].reshape(H, H)
     assert W2c[:, 5].any() and not np.delete(W2c, 5, axis=1).any()  # only column 5 of dW2
     assert not changed[s["Wh"]].any() and not changed[s["bh"]].any()  # heads see h2, not its gate
+
+
+# ------------------------------------------------------------------------------------------------
+# clipped-surrogate objective (PPO, Schulman et al. 2017, Eq. 7) on the same trajectory buffers
+# ------------------------------------------------------------------------------------------------
+def ppo_batch(seed, spread):
+    """tiny_batch plus recorded log-probabilities: the current policy's, shifted by N(0, spread) so that ratios spread
+    around 1."""
+    N, H = 5, 16
+    d = orc.Dims(N, H)
+    walls, goal, tpos, tact, adv, ret = tiny_batch(seed, B=6, T=5)
+    theta = random_params(200 + seed, d.P, 0.3).astype(np.float64)
+    T, B = tpos.shape
+    x = np.stack([orc.observe(N, walls[b], int(tpos[t, b]), int(goal[b])) for t in range(T) for b in range(B)])
+    out, z1, z2 = numpy_forward64(theta, N, H, x)
+    lg = torch.log_softmax(torch.from_numpy(out[:, :4]), dim=1).numpy()
+    logp_now = lg[np.arange(T * B), tact.ravel().astype(int)].reshape(T, B)
+    rng = np.random.default_rng(seed + 1)
+    return N, H, d, walls, goal, tpos, tact, adv, ret, theta, out, lg, logp_now, logp_now - spread * rng.standard_normal((T, B)), (z1, z2)
+
+
+def test_ppo_loss_matches_numpy_restatement_and_reduces_to_a2c_at_ratio_one():
+    N, H, d, walls, goal, tpos, tact, adv, ret, theta, out, lg, logp_now, logp_old, _ = ppo_batch(3, 0.3)
+    eps = 0.2
+    _, loss = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, 0.5, 0.01, want_grads=False, logp_old=logp_old, clip=eps)
+    r = np.exp(logp_now - logp_old)
+    pg = -np.minimum(r * adv, np.clip(r, 1 - eps, 1 + eps) * adv).mean()
+    assert (np.abs(r - 1) > eps).any() and (np.abs(r - 1) < eps).any()  # both branches are exercised
+    assert abs(loss[1] - pg) < 1e-12
+    # recorded log-probabilities equal to the current ones: ratio 1 everywhere, the gradient is the A2C gradient
+    g_ppo, l_ppo = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, 0.5, 0.01, logp_old=logp_now, clip=eps)
+    g_a2c, l_a2c = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, 0.5, 0.01)
+    assert np.allclose(g_ppo, g_a2c, rtol=1e-12, atol=1e-15)
+    assert abs(l_ppo[1] - (-(adv).mean())) < 1e-12  # -mean(1 * A)
+    assert np.allclose(l_ppo[2:], l_a2c[2:])
+
+
+def test_ppo_rows_on_the_clipped_side_carry_no_policy_gradient():
+    N, H, d, walls, goal, tpos, tact, adv, ret, theta, out, lg, logp_now, _, _ = ppo_batch(4, 0.0)
+    eps = 0.2
+    # every row far on the clipped side: ratio 2 with positive advantage, ratio 0.5 with negative advantage
+    logp_old = np.where(adv > 0, logp_now - np.log(2.0), logp_now + np.log(2.0))
+    g_ppo, _ = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, 0.5, 0.01, logp_old=logp_old, clip=eps)
+    g_zero, _ = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, np.zeros_like(adv), ret, 0.5, 0.01)
+    assert np.allclose(g_ppo, g_zero, rtol=1e-12, atol=1e-15)  # only the value and entropy terms are left
+    # the other side (ratio 2 with negative advantage) is NOT clipped: gradient = A2C gradient scaled by the ratio
+    logp_old2 = np.where(adv > 0, logp_now + np.log(2.0), logp_now - np.log(2.0))
+    g2, _ = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, 0.5, 0.01, logp_old=logp_old2, clip=eps)
+    r = np.exp(logp_now - logp_old2)
+    g_scaled, _ = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, adv * r, ret, 0.5, 0.01)
+    assert np.allclose(g2, g_scaled, rtol=1e-10, atol=1e-14)
+
+
+def test_ppo_gradient_matches_central_finite_differences_fp64():
+    eps, c_v, c_e = 0.2, 0.5, 0.01
+    for seed in range(60):  # a draw with no ReLU kink and no ratio near a clip boundary
+        N, H, d, walls, goal, tpos, tact, adv, ret, theta, out, lg, logp_now, logp_old, (z1, z2) = ppo_batch(seed, 0.3)
+        r = np.exp(logp_now - logp_old)
+        if min(np.abs(z1).min(), np.abs(z2).min()) > 1e-3 and np.abs(np.abs(r - 1) - eps).min() > 1e-3:
+            break
+    else:
+        pytest.fail("no kink-free draw found")
+    grads, _ = orc.learn_f64(N, H, theta, walls, goal, tpos, tact, adv, ret, c_v, c_e, logp_old=logp_old, clip=eps)
+    s = d.slices()
+    rng = np.random.default_rng(1)
+    idx = list(range(s["b2"].start, s["b2"].stop)) + list(range(s["Wh"].start, s["bh"].stop))
+    idx += list(rng.choice(np.arange(s["W1"].start, s["W1"].stop), 100, replace=False))
+    idx += list(rng.choice(np.arange(s["W2"].start, s["W2"].stop), 100, replace=False))
+    h, scale = 1e-5, np.sqrt((grads**2).mean())
+    for i in idx:
+        tp, tm = theta.copy(), theta.copy()
+        tp[i] += h
+        tm[i] -= h
+        lp = orc.learn_f64(N, H, tp, walls, goal, tpos, tact, adv, ret, c_v, c_e, want_grads=False, logp_old=logp_old, clip=eps)[1][0]
+        lm = orc.learn_f64(N, H, tm, walls, goal, tpos, tact, adv, ret, c_v, c_e, want_grads=False, logp_old=logp_old, clip=eps)[1][0]
+        fd = (lp - lm) / (2 * h)
+        assert abs(fd - grads[i]) <= 1e-6 * (abs(fd) + scale), (i, fd, grads[i])
+
+
+def test_agent_ppo_first_epoch_is_the_a2c_step():
+    """The recorded log-probabilities are the policy's own at rollout time, so epoch 1 has ratio 1 everywhere."""
+    a, b = orc.Agent(32, 5, 32, 8), orc.Agent(32, 5, 32, 8)
+    for ag in (a, b):
+        ag.reset(9)
+        ag.rollout()
+    a.learn()
+    b.learn_ppo(1, 0.2)
+    assert np.allclose(a.grads, b.grads, rtol=2e-5, atol=1e-9)  # exp(logp - logp) = 1 up to the fp32 record of logp
+    c = orc.Agent(32, 5, 32, 8)
+    c.reset(9)
+    c.rollout()
+    c.learn_ppo(3, 0.2)
+    assert c.k == 3 and not np.allclose(c.theta, b.theta)
