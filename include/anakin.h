@@ -187,6 +187,16 @@ int anakin_update(anakin_t* h);
 int anakin_grads(anakin_t* h);
 int anakin_apply_grads(anakin_t* h);
 
+/*
+ * Another objective over the same trajectory buffers (Section 3.2 names "a suitable RL objective"; this one is the
+ * clipped surrogate of PPO, Schulman et al. 2017, Eq. 7): GAE once, then `epochs` full-batch Adam steps in which the
+ * policy term of a row is -min(r A, clip(r, 1-clip_eps, 1+clip_eps) A), r = pi(a|s) / pi_old(a|s) from the recorded
+ * TRAJ_LOGP; value and entropy terms as in anakin_learn.  Every epoch after the first recomputes the forward pass of
+ * the recorded rows with the current parameters.  The first epoch equals anakin_learn's step (r = 1 everywhere).
+ * Consumes the pending rollout.  Errors: BAD_STATE if none is pending; INVALID_ARG for epochs < 1 or clip_eps <= 0.
+ */
+int anakin_learn_ppo(anakin_t* h, int epochs, float clip_eps);
+
 /* iters x ( anakin_rollout(T_max); anakin_learn() ), enqueue-only: no copy and no synchronisation. */
 int anakin_run(anakin_t* h, int iters);
 

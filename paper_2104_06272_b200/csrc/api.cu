@@ -345,7 +345,7 @@ int anakin_gae(anakin_t* h) {
 }
 
 // The update proper, from ADV/RET as they stand.  phase 0: through Adam; phase 1: stop at the batch-mean gradient.
-static int learn_after_gae(anakin_t* h, int phase) {
+static int learn_after_gae(anakin_t* h, int phase, float ppo_clip = 0.f, bool consume = true) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
@@ -370,6 +370,7 @@ static int learn_after_gae(anakin_t* h, int phase) {
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
     a.phase = phase;
+    a.ppo_clip = ppo_clip;
     {   // smallest power of two >= R: keeps the scaled output gradients O(1) for the fp16 operand format
         const double Rrows = (double)h->d.B * (double)h->last_T;
         int ex = 0;
@@ -387,9 +388,11 @@ static int learn_after_gae(anakin_t* h, int phase) {
         e = launch_learn(a, h->cfg.precision, h->ctx());
     }
     if (e != cudaSuccess) return fail_cuda(h, e);
-    h->adv_valid = false;
-    h->acts_valid = false;
-    h->rollout_pending = false;
+    h->acts_valid = false;  // saved activations belong to the parameters they were computed with
+    if (consume) {
+        h->adv_valid = false;
+        h->rollout_pending = false;
+    }
     if (phase == 0) {
         h->adam_k += 1;
         h->base_valid = false;  // parameters changed
@@ -412,6 +415,20 @@ int anakin_update(anakin_t* h) {
     if (!h) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
     return learn_after_gae(h, 0);
+}
+
+int anakin_learn_ppo(anakin_t* h, int epochs, float clip_eps) {
+    if (!h || epochs < 1 || !(clip_eps > 0.f)) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
+    if (!h->adv_valid) {
+        const int rc = anakin_gae(h);
+        if (rc != ANAKIN_OK) return rc;
+    }
+    for (int e = 0; e < epochs; ++e) {
+        const int rc = learn_after_gae(h, 0, clip_eps, e == epochs - 1);
+        if (rc != ANAKIN_OK) return rc;
+    }
+    return ANAKIN_OK;
 }
 
 int anakin_grads(anakin_t* h) {

@@ -110,6 +110,21 @@ __device__ inline float uniform24(uint32_t x) { return (float)(x >> 8) * (1.0f /
 __device__ inline float round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 template <int PREC> __device__ inline float rnd(float x) { return PREC == 1 ? round_bf16(x) : x; }
 
+// Policy term of one row.  Adds the term to l_pg and returns the factor f with d(term)/d(logit k) = -A f (1{k=a} - p_k).
+//   clip <= 0: plain policy gradient  -A log pi(a|s)                                   f = 1
+//   clip  > 0: clipped surrogate (PPO, Schulman et al. 2017, Eq. 7)  -min(r A, clip(r, 1-clip, 1+clip) A),
+//              r = exp(log pi(a|s) - logp_old);  f = r where the unclipped product is the smaller one (ties included), else 0
+__device__ __forceinline__ float policy_term(float A, float lpa, float logp_old, float clip, float& l_pg) {
+    if (clip <= 0.f) {
+        l_pg += -A * lpa;
+        return 1.f;
+    }
+    const float r = expf(lpa - logp_old), rc = fminf(fmaxf(r, 1.f - clip), 1.f + clip);
+    const float u = r * A, c = rc * A;
+    l_pg += -fminf(u, c);
+    return u <= c ? r : 0.f;
+}
+
 // launch parameter blocks --------------------------------------------------------------------------
 struct RolloutArgs {
     Dims d;
@@ -143,6 +158,7 @@ struct LearnArgs {
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
     int phase;   // 0: reduce the partials and apply Adam; 1: reduce only (GRADS and loss statistics)
+    float ppo_clip;  // > 0: the policy term is the clipped surrogate over the recorded log-probabilities (TRAJ_LOGP)
     // tensor-pipe path
     int ts;               // t-slices of the dh1 kernel: S holds ts*B rows (slice z, env b at row z*B + b)
     float gscale, inv_gscale;  // power of two carried by every gradient-side tensor, divided out in the reduction

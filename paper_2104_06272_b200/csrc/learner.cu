@@ -140,7 +140,7 @@ struct EpPartial {  // split-K partial of a weight gradient, in flat parameter l
 //   dh2 = (dOut Wh^T) masked by h2 > 0
 // ----------------------------------------------------------------------------------------------------
 template <int PREC>
-__global__ void __launch_bounds__(256) k_heads_loss(Dims d, Buffers b, size_t R, float c_v, float c_e) {
+__global__ void __launch_bounds__(256) k_heads_loss(Dims d, Buffers b, size_t R, float c_v, float c_e, float ppo_clip) {
     __shared__ float s_loss[8][3];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int H = d.H;
@@ -174,14 +174,16 @@ __global__ void __launch_bounds__(256) k_heads_loss(Dims d, Buffers b, size_t R,
         const float A = b.adv[i];
         const float err = o[4] - b.ret[i];
         float dO[5];
+        float lpg_row = 0.f;
+        const float pf = policy_term(A, act == 0 ? lp[0] : act == 1 ? lp[1] : act == 2 ? lp[2] : lp[3], ppo_clip > 0.f ? b.tlogp[i] : 0.f, ppo_clip, lpg_row);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) dO[c] = rnd<PREC>((-A * ((c == act ? 1.f : 0.f) - p[c]) + c_e * p[c] * (lp[c] + ent)) * invR);
+        for (int c = 0; c < 4; ++c) dO[c] = rnd<PREC>((-A * pf * ((c == act ? 1.f : 0.f) - p[c]) + c_e * p[c] * (lp[c] + ent)) * invR);
         dO[4] = rnd<PREC>(2.f * c_v * err * invR);
         if (lane == 0) {
             float4* o4 = reinterpret_cast<float4*>(b.dout + i * 8);
             o4[0] = make_float4(dO[0], dO[1], dO[2], dO[3]);
             o4[1] = make_float4(dO[4], 0.f, 0.f, 0.f);
-            l_pg += -A * (act == 0 ? lp[0] : act == 1 ? lp[1] : act == 2 ? lp[2] : lp[3]);
+            l_pg += lpg_row;
             l_v += err * err;
             l_ent += ent;
         }
@@ -357,7 +359,7 @@ static cudaError_t launch_learn_p(const LearnArgs& a, const Ctx& c) {
     const int lb = (int)((R + 7) / 8 < (size_t)LOSS_BLOCKS ? (R + 7) / 8 : LOSS_BLOCKS);
     {
         Scope sc(c, K_HEADS_LOSS);
-        k_heads_loss<PREC><<<lb, 256, 0, s>>>(d, b, R, a.c_v, a.c_e);
+        k_heads_loss<PREC><<<lb, 256, 0, s>>>(d, b, R, a.c_v, a.c_e, a.ppo_clip);
         CK(cudaGetLastError());
     }
     // dh1 = (dh2 W2^T) masked

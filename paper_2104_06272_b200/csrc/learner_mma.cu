@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
         cp_async_commit();
     };
     // Row phase, split in two so that the loads are in flight during the column phase.
-    struct RowIn { float4 o4; float v, adv, ret; int act; bool ok; };
+    struct RowIn { float4 o4; float v, adv, ret, lpo; int act; bool ok; };
     auto row_load = [&](int tile) {
         RowIn in;
         const size_t i = (size_t)tile * TR + rr;
@@ -95,11 +95,12 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
             in.o4 = *reinterpret_cast<const float4*>(b.out5 + i * 8);
             in.v = b.out5[i * 8 + 4];
             in.adv = b.adv[i];
+            in.lpo = a.ppo_clip > 0.f ? b.tlogp[i] : 0.f;
             in.ret = b.ret[i];
             in.act = b.tact[i];
         } else {
             in.o4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            in.v = in.adv = in.ret = 0.f;
+            in.v = in.adv = in.ret = in.lpo = 0.f;
             in.act = 0;
         }
         return in;
@@ -118,11 +119,11 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
             for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
             const float A = in.adv;
             const float err = in.v - in.ret;
+            const float pf = policy_term(A, in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3], in.lpo, a.ppo_clip, l_pg);
 #pragma unroll
             for (int c = 0; c < 4; ++c)
-                dO[c] = rnd<PREC>((-A * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
+                dO[c] = rnd<PREC>((-A * pf * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
             dO[4] = rnd<PREC>(2.f * a.c_v * err * invR);
-            l_pg += -A * (in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3]);
             l_v += err * err;
             l_ent += ent;
 #pragma unroll
@@ -293,18 +294,19 @@ __global__ void __launch_bounds__(512, 2) k_heads_bwd_tc(LearnArgs a) {
         }
         cp_async_commit();
     };
-    struct RowIn { float4 o4; float v, adv, ret; int act; bool ok; };
+    struct RowIn { float4 o4; float v, adv, ret, lpo; int act; bool ok; };
     auto row_load = [&](int tile) {
         RowIn in;
         const size_t i = (size_t)tile * TR + lane;
         in.ok = tile < ntiles && i < R;
         in.o4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        in.v = in.adv = in.ret = 0.f;
+        in.v = in.adv = in.ret = in.lpo = 0.f;
         in.act = 0;
         if (in.ok) {
             in.o4 = *reinterpret_cast<const float4*>(b.out5 + i * 8);
             in.v = b.out5[i * 8 + 4];
             in.adv = b.adv[i];
+            in.lpo = a.ppo_clip > 0.f ? b.tlogp[i] : 0.f;
             in.ret = b.ret[i];
             in.act = b.tact[i];
         }
@@ -323,10 +325,10 @@ __global__ void __launch_bounds__(512, 2) k_heads_bwd_tc(LearnArgs a) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
             const float A = in.adv, err = in.v - in.ret;
+            const float pf = policy_term(A, in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3], in.lpo, a.ppo_clip, l_pg);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) dO[c] = round_bf16((-A * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
+            for (int c = 0; c < 4; ++c) dO[c] = round_bf16((-A * pf * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
             dO[4] = round_bf16(2.f * a.c_v * err * invR);
-            l_pg += -A * (in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3]);
             l_v += err * err;
             l_ent += ent;
 #pragma unroll
