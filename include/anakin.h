@@ -8,7 +8,7 @@
  * (Section 3.1: the host only schedules); the workload is self-contained and deterministic given a seed
  * (Section 3.1).
  *
- * Workload (the paper says only "small neural networks and grid-world environments", Section 4.1; the
+ * Workload (Section 4.1 of the paper describes it only as small networks on grid-world environments; the
  * concrete rules are this library's):
  *   env      N x N integer gridworld per env, C = N*N cells; per-env wall mask, start and goal cell drawn from the
  *            seed; actions 0 up (row-1), 1 right (col+1), 2 down (row+1), 3 left (col-1); a move into a wall or
@@ -188,7 +188,7 @@ int anakin_grads(anakin_t* h);
 int anakin_apply_grads(anakin_t* h);
 
 /*
- * Another objective over the same trajectory buffers (Section 3.2 names "a suitable RL objective"; this one is the
+ * Another objective over the same trajectory buffers (Section 3.2 leaves the choice of objective open; this one is the
  * clipped surrogate of PPO, Schulman et al. 2017, Eq. 7): GAE once, then `epochs` full-batch Adam steps in which the
  * policy term of a row is -min(r A, clip(r, 1-clip_eps, 1+clip_eps) A), r = pi(a|s) / pi_old(a|s) from the recorded
  * TRAJ_LOGP; value and entropy terms as in anakin_learn.  Every epoch after the first recomputes the forward pass of
