@@ -73,15 +73,24 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
     float a_bh[5] = {0.f, 0.f, 0.f, 0.f, 0.f};  // row threads: sums of dOut over their rows
     float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
 
-    auto load_tile = [&](int tile, int buf) {  // 16-byte chunks, zero-filled past the last row; always commits a group
-        constexpr int EPC = 16 / ESZ;  // elements per 16-byte chunk
-        unsigned char* dst = s_h2 + (size_t)buf * TR * HS * ESZ;
-        const unsigned char* src0 = reinterpret_cast<const unsigned char*>(b.h2);
-        for (int c = tid; tile < ntiles && c < TR * (HS / EPC); c += NTHREADS) {
-            const int r = c / (HS / EPC), k = EPC * (c - r * (HS / EPC));
-            const size_t row = (size_t)tile * TR + r;
-            const bool ok = row < R;
-            cp_async16(dst + ((size_t)r * HS + k) * ESZ, src0 + (((ok ? row : 0) * H) + c_base + k) * ESZ, ok ? 16 : 0);
+    // h2 tile loads: 16-byte chunks, zero-filled past the last row; a thread's chunks of one tile differ by a fixed number
+    // of rows, so one address is formed per tile and the rest are constant offsets.  Always commits a group.
+    constexpr int EPC = 16 / ESZ;             // elements per 16-byte chunk
+    constexpr int CPR = HS / EPC;             // chunks per row
+    constexpr int RPP = NTHREADS / CPR;       // rows per pass of the whole CTA
+    static_assert(NTHREADS % CPR == 0 && TR % RPP == 0, "the tile must split into whole passes");
+    const int l_r = tid / CPR, l_k = EPC * (tid % CPR);
+    const unsigned char* src_base = reinterpret_cast<const unsigned char*>(b.h2) + (size_t)(c_base + l_k) * ESZ;
+    auto load_tile = [&](int tile, int buf) {
+        if (tile < ntiles) {
+            const size_t row0 = (size_t)tile * TR + l_r;
+            unsigned char* dst = s_h2 + ((size_t)(buf * TR + l_r) * HS + l_k) * ESZ;
+            const unsigned char* src = src_base + row0 * H * ESZ;
+#pragma unroll
+            for (int j = 0; j < TR / RPP; ++j) {
+                const bool ok = row0 + j * RPP < R;
+                cp_async16(dst + (size_t)j * RPP * HS * ESZ, ok ? src + (size_t)j * RPP * H * ESZ : src_base, ok ? 16 : 0);
+            }
         }
         cp_async_commit();
     };
@@ -154,7 +163,8 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
         const int rows_left = i0 < R ? (int)((R - i0) < 8 ? (R - i0) : 8) : 0;
         uint32_t* o_hi = g_dh2hi + (i0 * H + c_base) / 2 + cp;
         uint32_t* o_lo = g_dh2lo + (i0 * H + c_base) / 2 + cp;
-#pragma unroll 4
+        const bool full = rows_left == 8;  // all but the last tile: stores without per-row predicates
+#pragma unroll
         for (int r = 0; r < 8; ++r) {
             const float4 d0 = *reinterpret_cast<const float4*>(dt + r * 8);
             const float d4 = dt[r * 8 + 4];
@@ -191,9 +201,9 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
             }
             a_b2[0] += dh[0];
             a_b2[1] += dh[1];
-            if (r < rows_left) {
-                o_hi[(size_t)r * (H / 2)] = phi;
-                if (PREC == 0) o_lo[(size_t)r * (H / 2)] = plo;
+            if (full || r < rows_left) {
+                o_hi[r * (H / 2)] = phi;
+                if (PREC == 0) o_lo[r * (H / 2)] = plo;
             }
         }
         // ---- row phase of the next tile (its inputs were requested before the column phase)
