@@ -310,7 +310,7 @@ def run_ours(args):
     if args.no_cpu_baseline or rank != 0:
         cpu = None
     elif args.workload == "throughput" and not args.envs:
-        cpu = cpu_baseline(w, iters=2)
+        cpu = cpu_baseline(w, iters=6)
     else:
         mac_per_frame = 3.0 * (w.D * w.H + w.H * w.H + 5 * w.H) + w.H * w.H
         frames = 5.0e11 / mac_per_frame
@@ -383,7 +383,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiler captures only)")

@@ -71,7 +71,8 @@ struct RolloutMmaCfg {
         + (size_t)PLANES * ME * LD * 2       // h1 hi (and lo)
         + (size_t)NW * ME * 5 * 4            // per-warp head partials
         + (size_t)(H * 5 + H + 8) * 4        // Wh, b2, bh
-        + (size_t)ME * 8 * 4 + ME * 4;       // walls, pos
+        + (size_t)ME * 8 * 4 + ME * 4        // walls, pos
+        + (size_t)ME * 8;                    // prepared half of the next interaction
 };
 
 template <int H, int NW, int PREC>
@@ -89,6 +90,7 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
     float* s_bh = s_b2 + H;                                                    // [8]
     uint32_t* s_walls = reinterpret_cast<uint32_t*>(s_bh + 8);                 // [ME][8]
     int* s_pos = reinterpret_cast<int*>(s_walls + ME * 8);                     // [ME]
+    uint2* s_pre = reinterpret_cast<uint2*>(s_pos + ME);                       // [ME]
 
     const Dims& d = a.d;
     const Buffers& b = a.b;
@@ -181,6 +183,14 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
             }
         }
         __syncthreads();
+        // The logits-independent half of the interaction (the Philox uniform, the four candidate cells) is taken by the
+        // owner threads now, under the other warps' tensor work, so that only softmax and selection follow the heads.
+        // It waits in shared memory (two words per env) rather than in registers, which the MMA loop needs.
+        const bool acting = owner && !a.replay && t < a.T;
+        if (acting) {
+            const StepPre pre = step_prepare(s, a, e0 + tid, t, s_walls + tid * 8);
+            s_pre[tid] = make_uint2(__float_as_uint(pre.u), (uint32_t)pre.np[0] | ((uint32_t)pre.np[1] << 8) | ((uint32_t)pre.np[2] << 16) | ((uint32_t)pre.np[3] << 24));
+        }
         // ---- layer 2 on the tensor pipe: acc[mt][j] = rows 16mt.. x columns 8(wid*NT+j)..
         float acc[2][NT][4];
 #pragma unroll
@@ -297,8 +307,13 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
             }
             if (!a.replay) {
                 b.tval[(size_t)t * B + env] = o[4];
-                if (t < a.T) {
-                    act_and_step(s, a, env, t, o[0], o[1], o[2], o[3], s_walls + tid * 8);
+                if (acting) {
+                    const uint2 pk = s_pre[tid];
+                    StepPre pre;
+                    pre.u = __uint_as_float(pk.x);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) pre.np[q] = (pk.y >> (8 * q)) & 0xFF;
+                    act_and_step_pre(s, a, env, t, o[0], o[1], o[2], o[3], pre);
                     s_pos[tid] = s.pos;
                 }
             }
