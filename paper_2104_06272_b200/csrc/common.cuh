@@ -138,6 +138,7 @@ struct RolloutArgs {
     int replay;            // 1: recompute and save the activations of the recorded rows only (no sampling, no env step)
     int fuse_gae;          // 1: after the last step each env's owner thread also runs the GAE scan (fills ADV, RET)
     float gamma, lambda;
+    int gae_smem;          // set by the tensor-pipe rollout's launcher: the fused scan reads its inputs from shared memory
 };
 
 // One parameter range and where its split-K partial sums live: partial s of parameter i is part[s*stride + (i - start)].

@@ -61,17 +61,20 @@ __device__ __forceinline__ StepPre step_prepare(const EnvLane& s, const RolloutA
 }
 
 // Categorical sampling from the 4 logits (inverse CDF against the prepared uniform), the env transition and the records.
-__device__ __forceinline__ void act_and_step_pre(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
-                                                 float l3, const StepPre& pre) {
+// Returns bit 0 = the episode ended at this step, bit 1 = it ended at the goal (reward 1).
+__device__ __forceinline__ int act_and_step_pre(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
+                                                float l3, const StepPre& pre) {
     const Buffers& b = a.b;
     const size_t i = (size_t)t * a.d.B + env;
     // softmax and inverse CDF: c0 = p0, c1 = c0 + p1, c2 = c1 + p2; a = [u>=c0] + [u>=c1] + [u>=c2]
     const float mx = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
     const float x0 = expf(l0 - mx), x1 = expf(l1 - mx), x2 = expf(l2 - mx), x3 = expf(l3 - mx);
     const float Z = ((x0 + x1) + x2) + x3;
-    const float c0 = x0 / Z, c1 = c0 + x1 / Z, c2 = c1 + x2 / Z;
-    const float u = pre.u;
-    int act = (u >= c0) + (u >= c1) + (u >= c2);
+    // the comparisons u >= c_k are taken as u Z >= x0 + .. + x_k: no division, and the same decision except within
+    // rounding (1e-7) of a boundary
+    const float s01 = x0 + x1, s012 = s01 + x2;
+    const float uz = pre.u * Z;
+    int act = (uz >= x0) + (uz >= s01) + (uz >= s012);
     if (a.forced) {
         act = a.forced[i];
         if (act < 0 || act > 3) { s.bad |= DEV_E_BAD_ACTION; act &= 3; }
@@ -99,6 +102,7 @@ __device__ __forceinline__ void act_and_step_pre(EnvLane& s, const RolloutArgs& 
     }
     b.trew[i] = rew;
     b.tdone[i] = (uint8_t)done;
+    return done | (rew != 0.f ? 2 : 0);
 }
 
 __device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
@@ -165,6 +169,27 @@ __device__ __forceinline__ void gae_scan_env(const Buffers& b, int B, int T, int
                 vnext = v[q];
             }
         }
+    }
+}
+
+// The same scan over a copy of one CTA's values and outcomes kept in shared memory by the rollout (value row t of the
+// CTA's env e at sv[t*ME + e], outcome code of act_and_step_pre at sc[t*ME + e]): no global load on the serial chain.
+// Same operations in the same order as gae_scan_env, so the results are bitwise equal.
+__device__ __forceinline__ void gae_scan_env_smem(const Buffers& b, int B, int T, int env, float gamma, float lambda, const float* sv,
+                                                  const uint8_t* sc, int ME, int e) {
+    float A = 0.f;
+    float vnext = sv[T * ME + e];
+    const float gl = __fmul_rn(gamma, lambda);
+    for (int t = T - 1; t >= 0; --t) {
+        const size_t i = (size_t)t * B + env;
+        const float v = sv[t * ME + e];
+        const int code = sc[t * ME + e];
+        const float nd = (code & 1) ? 0.f : 1.f, r = (code & 2) ? 1.f : 0.f;
+        const float delta = __fsub_rn(__fmaf_rn(__fmul_rn(gamma, nd), vnext, r), v);
+        A = __fmaf_rn(__fmul_rn(gl, nd), A, delta);
+        b.adv[i] = A;
+        b.ret[i] = __fadd_rn(A, v);
+        vnext = v;
     }
 }
 

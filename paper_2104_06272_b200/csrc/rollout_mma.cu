@@ -73,10 +73,12 @@ struct RolloutMmaCfg {
         + (size_t)(H * 5 + H + 8) * 4        // Wh, b2, bh
         + (size_t)ME * 8 * 4 + ME * 4        // walls, pos
         + (size_t)ME * 8;                    // prepared half of the next interaction
+    // values and outcomes of the CTA's envs for the GAE scan at the end (only when the scan is fused and they fit)
+    static constexpr size_t gae_bytes(int T) { return (size_t)(T + 1) * ME * 4 + (size_t)T * ME; }
 };
 
 template <int H, int NW, int PREC>
-__global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(RolloutArgs a) {
+__global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(RolloutArgs a) {
     using Cfg = RolloutMmaCfg<H, NW, PREC>;
     constexpr int ME = Cfg::ME, NT = Cfg::NT, KS = Cfg::KS, LD = Cfg::LD, NTHREADS = NW * 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -91,6 +93,8 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
     uint32_t* s_walls = reinterpret_cast<uint32_t*>(s_bh + 8);                 // [ME][8]
     int* s_pos = reinterpret_cast<int*>(s_walls + ME * 8);                     // [ME]
     uint2* s_pre = reinterpret_cast<uint2*>(s_pos + ME);                       // [ME]
+    float* s_gv = reinterpret_cast<float*>(s_pre + ME);                        // [T+1][ME] (a.gae_smem only)
+    uint8_t* s_gc = reinterpret_cast<uint8_t*>(s_gv + (a.T + 1) * ME);         // [T][ME]
 
     const Dims& d = a.d;
     const Buffers& b = a.b;
@@ -307,13 +311,15 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
             }
             if (!a.replay) {
                 b.tval[(size_t)t * B + env] = o[4];
+                if (a.gae_smem) s_gv[t * ME + tid] = o[4];
                 if (acting) {
                     const uint2 pk = s_pre[tid];
                     StepPre pre;
                     pre.u = __uint_as_float(pk.x);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) pre.np[q] = (pk.y >> (8 * q)) & 0xFF;
-                    act_and_step_pre(s, a, env, t, o[0], o[1], o[2], o[3], pre);
+                    const int code = act_and_step_pre(s, a, env, t, o[0], o[1], o[2], o[3], pre);
+                    if (a.gae_smem) s_gc[t * ME + tid] = (uint8_t)code;
                     s_pos[tid] = s.pos;
                 }
             }
@@ -325,17 +331,27 @@ __global__ void __launch_bounds__(NW * 32, (NW <= 8 ? 2 : 1)) k_rollout_mma(Roll
         b.pos[e0 + tid] = (uint8_t)s.pos;
         b.tep[e0 + tid] = (uint8_t)s.tep;
         // the owner thread wrote this env's rewards, values and done flags itself: it can scan them right away
-        if (a.fuse_gae) gae_scan_env(b, B, a.T, e0 + tid, a.gamma, a.lambda);
+        if (a.gae_smem) gae_scan_env_smem(b, B, a.T, e0 + tid, a.gamma, a.lambda, s_gv, s_gc, ME, tid);
+        else if (a.fuse_gae) gae_scan_env(b, B, a.T, e0 + tid, a.gamma, a.lambda);
     }
     if (tid < 32) flush_env_stats(s, a);
 }
 
+constexpr size_t MAX_DYN_SMEM = 232448;  // 227 KB of dynamic shared memory per CTA
+
 template <int H, int NW, int PREC>
-static cudaError_t launch_t(const RolloutArgs& a, cudaStream_t s) {
+static cudaError_t launch_t(const RolloutArgs& a0, cudaStream_t s) {
     using Cfg = RolloutMmaCfg<H, NW, PREC>;
-    cudaError_t e = cudaFuncSetAttribute(k_rollout_mma<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
+    RolloutArgs a = a0;
+    size_t smem = Cfg::smem_bytes;
+    a.gae_smem = 0;
+    if (a.fuse_gae && !a.replay && smem + Cfg::gae_bytes(a.T) <= MAX_DYN_SMEM) {
+        a.gae_smem = 1;
+        smem += Cfg::gae_bytes(a.T);
+    }
+    cudaError_t e = cudaFuncSetAttribute(k_rollout_mma<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MAX_DYN_SMEM);
     if (e != cudaSuccess) return e;
-    k_rollout_mma<H, NW, PREC><<<(a.d.B + Cfg::ME - 1) / Cfg::ME, NW * 32, Cfg::smem_bytes, s>>>(a);
+    k_rollout_mma<H, NW, PREC><<<(a.d.B + Cfg::ME - 1) / Cfg::ME, NW * 32, smem, s>>>(a);
     return cudaGetLastError();
 }
 
@@ -354,7 +370,7 @@ cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
         switch (a.d.H) {
             case 64: return launch_t<64, 4, 0>(a, s);
             case 128: return launch_t<128, 8, 0>(a, s);
-            case 256: return launch_t<256, 16, 0>(a, s);
+            case 256: return launch_t<256, 8, 0>(a, s);
         }
     }
     return cudaErrorNotSupported;
