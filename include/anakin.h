@@ -237,10 +237,10 @@ const char* anakin_kernel_name(int id);
  * a control loop whose memory budget is fixed at start-up, a plug-in inside an application that owns the
  * allocator, a process that must never synchronise the device (cudaMalloc and cudaFree may).  This call needs no
  * handle and no workspace.  The caller passes the rollout's inputs and outputs as DEVICE pointers; the only
- * scratch the rollout uses (B*H floats, plus a 256 KiB repacked copy of the second-layer weights) is a fixed
+ * scratch the rollout uses (B*H floats, plus two 256 KiB repacked copies of the second-layer weights) is a fixed
  * array compiled into the library, so
  *     B * H  <=  ANAKIN_NOALLOC_MAX_BH  (1,048,576 floats = 4 MiB),
- * and every GPU that loads the library holds those 4.25 MiB until the process exits.  Larger sizes return
+ * and every GPU that loads the library holds those 4.5 MiB until the process exits.  Larger sizes return
  * ANAKIN_E_WORKSPACE_TOO_SMALL (with a message on stderr); precision must be ANAKIN_PRECISION_FP32
  * (ANAKIN_E_UNSUPPORTED_CFG otherwise).  The call itself calls no cudaMalloc / cudaFree and no allocating library
  * routine; it enqueues one small memset and up to three kernels on `cuda_stream` and returns without synchronising.

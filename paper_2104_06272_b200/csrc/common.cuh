@@ -250,6 +250,7 @@ cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c);
 cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c);
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s);  // cudaErrorNotSupported if not covered
 bool rollout_mma_supported(int H);
+cudaError_t launch_rollout_pair(const RolloutArgs& a, cudaStream_t s);  // CTA-pair tcgen05 rollout (H = 256, fp32); cudaErrorNotSupported otherwise
 bool wide_supported(int H, int prec);         // bf16 workload with a hidden layer too wide for the persistent rollout
 bool tensor_path_supported(int H, int prec);  // either tensor-core path: the update reuses activations the rollout saved
 cudaError_t launch_rollout_wide(const RolloutArgs& a, const Ctx& c);  // T+1 forward passes, or the replay of recorded rows

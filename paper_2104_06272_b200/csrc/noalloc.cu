@@ -4,7 +4,7 @@
 // fixed memory budget handed out at start-up, a plug-in inside a host application that owns the allocator, a
 // process that must not synchronise the device (cudaMalloc and cudaFree may) -- and that therefore cannot size
 // and provide the library's workspace either.  Such a caller passes only the rollout's inputs and outputs; the
-// scratch the rollout needs (the per-env first-layer constant `base`, B*H floats, and a repacked copy of the
+// scratch the rollout needs (the per-env first-layer constant `base`, B*H floats, and two repacked copies of the
 // second-layer weights) lives in a file-scope device array of fixed size inside this library.
 //
 // The array below is device memory reserved in every CUDA context that loads the library, from load to exit,
@@ -21,11 +21,12 @@ namespace {
 
 constexpr size_t kMaxBaseFloats = ANAKIN_NOALLOC_MAX_BH;  // B*H limit (floats)
 constexpr size_t kW2FragBytes = 2 * 256 * 256 * 2;          // W2 as tensor-pipe fragments, hi and lo planes (H <= 256)
+constexpr size_t kW2PlaneBytes = 2 * 256 * 256 * 2;         // W2 row-major as 16-bit hi and lo planes (H <= 256)
 constexpr size_t kTailBytes = 256;                          // statistics block + status word
 constexpr int kMaxDevices = 64;
 
-// [ base: kMaxBaseFloats floats | W2 fragments hi, lo | anakin_stats | status word ]
-static __device__ __align__(256) unsigned char g_noalloc_scratch[kMaxBaseFloats * sizeof(float) + kW2FragBytes + kTailBytes];
+// [ base: kMaxBaseFloats floats | W2 fragments hi, lo | W2 planes hi, lo | anakin_stats | status word ]
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kMaxBaseFloats * sizeof(float) + kW2FragBytes + kW2PlaneBytes + kTailBytes];
 
 unsigned char* g_scratch_ptr[kMaxDevices] = {nullptr};  // device address of the array, per device ordinal
 
@@ -92,8 +93,10 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     if (rollout_mma_supported(cfg->H)) {  // same kernel choice as the handle-based rollout
         b.w2f_hi = reinterpret_cast<uint2*>(frag);
         b.w2f_lo = reinterpret_cast<uint2*>(frag + kW2FragBytes / 2);
+        b.w2p_hi = reinterpret_cast<uint16_t*>(frag + kW2FragBytes);
+        b.w2p_lo = reinterpret_cast<uint16_t*>(frag + kW2FragBytes + kW2PlaneBytes / 2);
     }
-    unsigned char* tail = frag + kW2FragBytes;
+    unsigned char* tail = frag + kW2FragBytes + kW2PlaneBytes;
     b.stats = reinterpret_cast<anakin_stats*>(tail);
     b.status = reinterpret_cast<int*>(tail + 128);
     // the tail holds accumulators and a sticky status word left by the previous call: start them at zero

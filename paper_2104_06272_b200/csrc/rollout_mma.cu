@@ -33,13 +33,14 @@ __global__ void __launch_bounds__(256) k_pack_w2(Dims d, Buffers b) {
     b.w2f_hi[idx] = hi;
     b.w2f_lo[idx] = lo;
     // the same for W2^T (the backward pass contracts over W2's second index): B[k][n] = W2[n][k]
-    if (!b.w2tf_hi) return;
-    split2<PREC>(W2[(size_t)n * H + ks4[0]], W2[(size_t)n * H + ks4[1]], hi.x, lo.x);
-    split2<PREC>(W2[(size_t)n * H + ks4[2]], W2[(size_t)n * H + ks4[3]], hi.y, lo.y);
-    b.w2tf_hi[idx] = hi;
-    b.w2tf_lo[idx] = lo;
+    if (b.w2tf_hi) {
+        split2<PREC>(W2[(size_t)n * H + ks4[0]], W2[(size_t)n * H + ks4[1]], hi.x, lo.x);
+        split2<PREC>(W2[(size_t)n * H + ks4[2]], W2[(size_t)n * H + ks4[3]], hi.y, lo.y);
+        b.w2tf_hi[idx] = hi;
+        b.w2tf_lo[idx] = lo;
+    }
     // and W2 itself as row-major hi / lo planes: this thread covers elements 4*idx .. 4*idx+3
-    if (!b.w2p_hi) return;
+    if (!b.w2p_hi || !b.w2p_lo) return;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         uint16_t h16, l16;
@@ -360,6 +361,10 @@ bool rollout_mma_supported(int H) { return H == 64 || H == 128 || H == 256; }
 // Returns cudaErrorNotSupported when the shape is not covered by the tensor-pipe kernel.
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
     if (!a.b.w2f_hi || !rollout_mma_supported(a.d.H)) return cudaErrorNotSupported;
+    if (prec == 0) {  // the CTA-pair kernel on the 5th-generation tensor cores where it covers the shape
+        const cudaError_t e = launch_rollout_pair(a, s);
+        if (e != cudaErrorNotSupported) return e;
+    }
     if (prec == 1) {
         switch (a.d.H) {
             case 64: return launch_t<64, 4, 1>(a, s);
