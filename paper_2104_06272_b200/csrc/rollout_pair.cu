@@ -13,11 +13,13 @@
 //   heads     a thread = one hidden unit j: bias, ReLU, h2 stores (one 128-byte line per env and warp); the warp's
 //             32 units x 32 envs go to shared memory as fp16 (hi, lo) terms and come back transposed (ldmatrix.trans)
 //             as A fragments of warp-level MMAs against Wh: out[env][c] = sum_j h2[j][env] Wh[j][c]; the eight 32-unit
-//             partials of an env meet in the shared memory of the CTA that owns it (remote stores for the peer's envs)
-//   env       one thread per env: softmax, Philox inverse-CDF sample, gridworld step, time-major records
-// Two cluster barriers per step (operands ready; head partials delivered) and one CTA barrier (new positions).  The
-// only bounded waits are on mbarriers (weights landed, MMAs finished); a timeout raises DEV_E_WAIT_TIMEOUT and the
-// CTA keeps walking through the barriers to the exit, where tensor memory is freed.
+//             partials of an env meet in the shared memory of the CTA that owns it, sent as asynchronous remote stores
+//             that count their bytes on the owner's mbarrier
+//   env       (ninth warp) one thread per env: softmax, Philox inverse-CDF sample, gridworld step, time-major records
+// Inside a step the CTAs of a pair meet only through mbarriers (operand blocks written -> issuer; MMAs finished ->
+// workers; partials landed -> owners) and each CTA has one barrier of its own (new positions); the cluster barrier is
+// used at start and exit only.  Every mbarrier wait is bounded; a timeout raises DEV_E_WAIT_TIMEOUT and the threads keep
+// walking through the barriers to the exit, where tensor memory is freed.
 #include <cstring>
 
 #include "tc_common.cuh"
