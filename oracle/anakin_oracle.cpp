@@ -627,6 +627,34 @@ void orc_gae(int T, int B, double gamma, double lambda, const float* rew, const 
     }
 }
 
+// V-trace targets (Espeholt et al. 2018, "IMPALA", Eq. 1 and Remark 1 in its recursive form), reverse scan over t for
+// each env.  The trajectory was generated by a behaviour policy mu (its log-probabilities logp_mu were recorded when the
+// actions were taken); pi is the policy being updated (logp_pi, and the values V, come from the current parameters):
+//   w_t = exp(logp_pi_t - logp_mu_t);  rho_t = min(rho_bar, w_t);  c_t = min(c_bar, w_t);  d_t = 1 - done_t
+//   delta_t = rho_t (r_t + gamma d_t V_{t+1} - V_t)
+//   e_t = delta_t + gamma d_t c_t e_{t+1},  e_T = 0          (e_t = v_t - V_t)
+//   ret_t = v_t = V_t + e_t                                   value target
+//   adv_t = rho_t (r_t + gamma d_t v_{t+1} - V_t),  v_T = V_T  policy-gradient advantage
+// An episode end (goal or time-out) cuts both the bootstrap and the trace, as in the GAE scan.
+void orc_vtrace(int T, int B, double gamma, double rho_bar, double c_bar, const float* rew, const float* val /*[T+1][B]*/,
+                const uint8_t* done, const float* logp_pi, const float* logp_mu, float* adv, float* ret) {
+    for (int b = 0; b < B; ++b) {
+        double e_next = 0.0;
+        for (int t = T - 1; t >= 0; --t) {
+            const size_t i = (size_t)t * B + b;
+            const double w = std::exp((double)logp_pi[i] - (double)logp_mu[i]);
+            const double rho = std::min(rho_bar, w), c = std::min(c_bar, w);
+            const double dt = 1.0 - (double)done[i];
+            const double v_next = (double)val[i + B] + e_next;
+            const double delta = rho * ((double)rew[i] + gamma * dt * (double)val[i + B] - (double)val[i]);
+            const double e = delta + gamma * dt * c * e_next;
+            adv[i] = (float)(rho * ((double)rew[i] + gamma * dt * v_next - (double)val[i]));
+            ret[i] = (float)((double)val[i] + e);
+            e_next = e;
+        }
+    }
+}
+
 void orc_learn_f32(int N, int H, int prec, int B, int T, const float* theta, const uint32_t* walls,
                    const uint8_t* goal, const uint8_t* tpos, const int8_t* tact, const float* adv,
                    const float* ret, double c_v, double c_e, float* grads, double* loss4,

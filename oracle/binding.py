@@ -236,6 +236,22 @@ def gae(gamma: float, lam: float, reward: np.ndarray, value: np.ndarray, done: n
     return adv, ret
 
 
+def vtrace(gamma: float, rho_bar: float, c_bar: float, reward, value, done, logp_pi, logp_mu):
+    """V-trace value targets and policy-gradient advantages (IMPALA, Eq. 1): returns (adv, ret) f32 [T][B]."""
+    reward = np.ascontiguousarray(reward, np.float32)
+    value = np.ascontiguousarray(value, np.float32)
+    done = np.ascontiguousarray(done, np.uint8)
+    logp_pi = np.ascontiguousarray(logp_pi, np.float32)
+    logp_mu = np.ascontiguousarray(logp_mu, np.float32)
+    T, B = reward.shape
+    assert value.shape == (T + 1, B) and done.shape == (T, B) and logp_pi.shape == (T, B) and logp_mu.shape == (T, B)
+    adv = np.empty((T, B), np.float32)
+    ret = np.empty((T, B), np.float32)
+    lib().orc_vtrace(C.c_int(T), C.c_int(B), C.c_double(gamma), C.c_double(rho_bar), C.c_double(c_bar), _p(reward), _p(value),
+                     _p(done), _p(logp_pi), _p(logp_mu), _p(adv), _p(ret))
+    return adv, ret
+
+
 def learn(N, H, prec, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, want_grads=True, gates=None,
           logp_old=None, clip=0.0):
     """fp32-storage loss and batch-mean gradient; with `logp_old` the policy term is the clipped surrogate (PPO).  Returns (grads f32 [P] or None, loss[4] f64), plus a
