@@ -197,6 +197,24 @@ int anakin_apply_grads(anakin_t* h);
  */
 int anakin_learn_ppo(anakin_t* h, int epochs, float clip_eps);
 
+/*
+ * A third objective over the same buffers: the off-policy correction of the paper's other agent (Section 3.2 names
+ * V-trace; defined in Espeholt et al. 2018, "IMPALA", Eq. 1).  The pending trajectory was generated by the policy whose
+ * log-probabilities are in TRAJ_LOGP (the behaviour policy mu); the policy being updated (pi) is the handle's current
+ * parameters, which differ from mu's after an earlier epoch, after anakin_set(PARAMS), or when the trajectory was
+ * written with anakin_set.  Each of the `epochs` steps
+ *   1. takes the head outputs of the recorded rows under the current parameters (the rollout's saved ones when the
+ *      parameters have not changed since; otherwise the forward pass is recomputed, including the value of the state
+ *      after the last step = the env state as it stands, ENV_POS),
+ *   2. fills ADV and RET by the reverse scan   w = pi(a|s)/mu(a|s), rho = min(rho_bar, w), c = min(c_bar, w), d = 1 - done,
+ *      delta = rho (r + gamma d V' - V),  v - V = delta + gamma d c (v' - V'),  RET = v,  ADV = rho (r + gamma d v' - V),
+ *   3. runs the update of anakin_update (policy gradient with ADV, value regression to RET, entropy bonus, Adam).
+ * With pi = mu and both levels >= 1 it is the A2C update with GAE at lambda = 1.  Consumes the pending rollout.
+ * Errors: BAD_STATE if none is pending; INVALID_ARG for epochs < 1 or a negative level; UNSUPPORTED_CFG on hidden widths
+ * whose rollout does not save the head outputs (the generic non-tensor path).
+ */
+int anakin_learn_vtrace(anakin_t* h, int epochs, float rho_bar, float c_bar);
+
 /* iters x ( anakin_rollout(T_max); anakin_learn() ), enqueue-only: no copy and no synchronisation. */
 int anakin_run(anakin_t* h, int iters);
 

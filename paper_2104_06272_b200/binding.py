@@ -45,7 +45,7 @@ OK, E_INVALID_ARG, E_BAD_STATE, E_WORKSPACE_TOO_SMALL, E_UNSUPPORTED_CFG, E_CUDA
 
 EXPORTS = [
     "anakin_workspace_bytes", "anakin_create", "anakin_destroy", "anakin_reset", "anakin_rollout",
-    "anakin_rollout_forced", "anakin_learn", "anakin_gae", "anakin_update", "anakin_grads", "anakin_apply_grads", "anakin_learn_ppo",
+    "anakin_rollout_forced", "anakin_learn", "anakin_gae", "anakin_update", "anakin_grads", "anakin_apply_grads", "anakin_learn_ppo", "anakin_learn_vtrace",
     "anakin_run", "anakin_get", "anakin_set",
     "anakin_blob_bytes", "anakin_status", "anakin_launch_count", "anakin_strerror", "anakin_last_cuda_error",
     "anakin_profile_enable", "anakin_profile_read", "anakin_kernel_count", "anakin_kernel_name",
@@ -65,6 +65,7 @@ _lib.anakin_update.argtypes = [_vp]
 _lib.anakin_grads.argtypes = [_vp]
 _lib.anakin_apply_grads.argtypes = [_vp]
 _lib.anakin_learn_ppo.argtypes = [_vp, C.c_int, C.c_float]
+_lib.anakin_learn_vtrace.argtypes = [_vp, C.c_int, C.c_float, C.c_float]
 _lib.anakin_run.argtypes = [_vp, C.c_int]
 _lib.anakin_get.argtypes = [_vp, C.c_int, _vp, C.c_size_t, C.c_int]
 _lib.anakin_set.argtypes = [_vp, C.c_int, _vp, C.c_size_t, C.c_int]
@@ -207,6 +208,9 @@ class Anakin:
 
     def learn_ppo(self, epochs: int, clip_eps: float):
         self._ck(_lib.anakin_learn_ppo(self._h, epochs, C.c_float(clip_eps)))
+
+    def learn_vtrace(self, epochs: int, rho_bar: float = 1.0, c_bar: float = 1.0):
+        self._ck(_lib.anakin_learn_vtrace(self._h, epochs, C.c_float(rho_bar), C.c_float(c_bar)))
 
     def run(self, iters: int):
         self._ck(_lib.anakin_run(self._h, iters))

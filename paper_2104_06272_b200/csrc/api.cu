@@ -109,6 +109,7 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.h1 = (float*)take(R * H * 4);
     b.h2 = (float*)take(R * H * 4);
     b.out5 = tensor ? (float*)take(R * 8 * 4) : nullptr;
+    b.vboot = tensor ? (float*)take(B * 4) : nullptr;
     b.dh2 = (float*)take(R * H * 4);
     b.dh1 = (float*)take(R * H * 4);
     b.dout = (float*)take(R * 8 * 4);
@@ -217,8 +218,9 @@ int do_rollout(anakin_t* h, int T, const int8_t* forced) {
     return ANAKIN_OK;
 }
 
-// Recomputes and saves the activations of the pending trajectory's rows (positions from TRAJ_POS).
-int replay_activations(anakin_t* h) {
+// Recomputes and saves the activations of the pending trajectory's rows (positions from TRAJ_POS); with_boot: also the
+// value of the current env state (the state after the last recorded step) under the current parameters, into vboot.
+int replay_activations(anakin_t* h, bool with_boot = false) {
     cudaError_t e;
     if (!h->base_valid) {
         e = launch_env_base(h->d, h->b, h->ctx());
@@ -239,7 +241,7 @@ int replay_activations(anakin_t* h) {
     a.key0 = a.key1 = 0;
     a.env_kind = h->cfg.env_kind;
     a.forced = nullptr;
-    a.replay = 1;
+    a.replay = with_boot ? 2 : 1;
     a.fuse_gae = 0;
     a.gamma = a.lambda = 0.f;
     if (wide_supported(h->d.H, h->cfg.precision)) {
@@ -431,6 +433,39 @@ int anakin_learn_ppo(anakin_t* h, int epochs, float clip_eps) {
     return ANAKIN_OK;
 }
 
+int anakin_learn_vtrace(anakin_t* h, int epochs, float rho_bar, float c_bar) {
+    if (!h || epochs < 1 || !(rho_bar >= 0.f) || !(c_bar >= 0.f)) return ANAKIN_E_INVALID_ARG;
+    if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
+    if (!tensor_path_supported(h->d.H, h->cfg.precision)) return ANAKIN_E_UNSUPPORTED_CFG;  // needs the saved head outputs
+    for (int ep = 0; ep < epochs; ++ep) {
+        cudaError_t e;
+        if (!h->base_valid) {
+            e = launch_env_base(h->d, h->b, h->ctx());
+            if (e != cudaSuccess) return fail_cuda(h, e);
+            h->base_valid = true;
+        }
+        if (!h->frags_valid) {
+            e = pack_w2(h);
+            if (e != cudaSuccess) return fail_cuda(h, e);
+            h->frags_valid = true;
+        }
+        // Head outputs of the recorded rows under the current parameters: the rollout's own when nothing has changed since
+        // (then the recorded bootstrap row is the current one too), else a replay that also evaluates the final state.
+        const float* boot = h->b.tval + (size_t)h->last_T * h->d.B;
+        if (!h->acts_valid) {
+            const int rc = replay_activations(h, true);
+            if (rc != ANAKIN_OK) return rc;
+            boot = h->b.vboot;
+        }
+        e = launch_vtrace(h->d, h->b, h->last_T, h->cfg.gamma, rho_bar, c_bar, boot, h->ctx());
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        h->adv_valid = true;
+        const int rc = learn_after_gae(h, 0, 0.f, ep == epochs - 1);
+        if (rc != ANAKIN_OK) return rc;
+    }
+    return ANAKIN_OK;
+}
+
 int anakin_grads(anakin_t* h) {
     if (!h) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
@@ -539,7 +574,7 @@ int anakin_kernel_count(void) { return K_COUNT; }
 const char* anakin_kernel_name(int id) {
     static const char* names[K_COUNT] = {"reset_env", "reset_params", "refresh_params", "env_base", "rollout", "gae", "h1",
                                          "fwd2", "heads_loss", "dh1", "dw2", "colsums", "sum_over_t", "dw1_agent",
-                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates", "pack_w2", "heads_bwd", "replay"};
+                                         "dw1_walls", "dw1_goal", "reduce_adam", "loss_total", "pack_gates", "pack_w2", "heads_bwd", "replay", "vtrace"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "";
 }
 

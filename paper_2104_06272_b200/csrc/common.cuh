@@ -71,6 +71,7 @@ struct Buffers {
     float* h1;       // [R][H]
     float* h2;       // [R][H]
     float* out5;     // [R][8] head outputs (4 logits, value) of every recorded row, saved by the tensor-pipe rollout
+    float* vboot;    // [B] value of the state after the last recorded step under the CURRENT parameters (replay mode 2)
     float* dh2;      // [R][H]
     float* dh1;      // [R][H]
     float* dout;     // [R][8]  (5 used)
@@ -135,7 +136,8 @@ struct RolloutArgs {
     uint32_t key0, key1;
     int env_kind;          // ANAKIN_ENV_*: the transition rule (env_step.cuh)
     const int8_t* forced;  // nullable
-    int replay;            // 1: recompute and save the activations of the recorded rows only (no sampling, no env step)
+    int replay;            // 1: recompute and save the activations of the recorded rows only (no sampling, no env step);
+                           // 2: the same, plus one forward of the current env state whose value goes to Buffers::vboot
     int fuse_gae;          // 1: after the last step each env's owner thread also runs the GAE scan (fills ADV, RET)
     float gamma, lambda;
     int gae_smem;          // set by the tensor-pipe rollout's launcher: the fused scan reads its inputs from shared memory
@@ -178,7 +180,7 @@ void learn_mma_plan(const Dims& d, LearnPlan* p);
 // Kernel identifiers (anakin_kernel_name / anakin_profile_read index by these).
 enum KernelId : int {
     K_RESET_ENV = 0, K_RESET_PARAMS, K_REFRESH_PARAMS, K_ENV_BASE, K_ROLLOUT, K_GAE, K_H1, K_FWD2, K_HEADS_LOSS, K_DH1,
-    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_PACK_W2, K_HEADS_BWD, K_REPLAY, K_COUNT
+    K_DW2, K_COLSUMS, K_SUM_OVER_T, K_DW1_AGENT, K_DW1_WALLS, K_DW1_GOAL, K_REDUCE_ADAM, K_LOSS_TOTAL, K_PACK_GATES, K_PACK_W2, K_HEADS_BWD, K_REPLAY, K_VTRACE, K_COUNT
 };
 
 // Optional per-kernel timing with CUDA events on the launching stream (off by default).
@@ -259,6 +261,8 @@ cudaError_t launch_dh1_wide(const LearnArgs& a, const Ctx& c);
 cudaError_t launch_env_base_wide(const Dims& d, const Buffers& b, const Ctx& c);  // cudaErrorNotSupported if not covered
 cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c);
+// V-trace scan over the recorded rows: current-policy logits and values from out5, bootstrap values from `boot` [B].
+cudaError_t launch_vtrace(const Dims& d, const Buffers& b, int T, float gamma, float rho_bar, float c_bar, const float* boot, const Ctx& c);
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_adam_only(const LearnArgs& a, int prec, const Ctx& c);  // Adam from GRADS as they stand

@@ -256,4 +256,64 @@ cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, floa
     return cudaGetLastError();
 }
 
+// ----------------------------------------------------------------------------------------------------
+// V-trace targets (Espeholt et al. 2018, IMPALA, Eq. 1; recursive form), lane = env, reverse scan over t.  mu = the policy
+// that acted (recorded log-probabilities), pi = the current parameters (head outputs of the recorded rows in out5):
+//   w = exp(logp_pi - logp_mu); rho = min(rho_bar, w); c = min(c_bar, w); d = 1 - done
+//   delta = rho (r + gamma d V' - V);  e = delta + gamma d c e';  ret = V + e;  adv = rho (r + gamma d (V' + e') - V)
+// Four steps per memory round trip.
+// ----------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_vtrace(Dims d, Buffers b, int T, float gamma, float rho_bar, float c_bar, const float* boot) {
+    const int env = blockIdx.x * blockDim.x + threadIdx.x;
+    if (env >= d.B) return;
+    const int B = d.B;
+    float e_next = 0.f, v_next = boot[env];
+    for (int tb = T; tb > 0; tb -= 4) {
+        float4 lg[4];
+        float v[4], r[4], nd[4], lmu[4];
+        int act[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int t = tb - 1 - q;
+            if (t >= 0) {
+                const size_t i = (size_t)t * B + env;
+                const float4* o = reinterpret_cast<const float4*>(b.out5 + i * 8);
+                lg[q] = o[0];
+                v[q] = o[1].x;
+                r[q] = b.trew[i];
+                nd[q] = b.tdone[i] ? 0.f : 1.f;
+                lmu[q] = b.tlogp[i];
+                act[q] = b.tact[i];
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int t = tb - 1 - q;
+            if (t >= 0) {
+                const size_t i = (size_t)t * B + env;
+                const float l0 = lg[q].x, l1 = lg[q].y, l2 = lg[q].z, l3 = lg[q].w;
+                const float mx = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
+                const float Z = ((expf(l0 - mx) + expf(l1 - mx)) + expf(l2 - mx)) + expf(l3 - mx);
+                const float la = act[q] == 0 ? l0 : act[q] == 1 ? l1 : act[q] == 2 ? l2 : l3;
+                const float lpi = (la - mx) - logf(Z);
+                const float w = expf(lpi - lmu[q]);
+                const float rho = fminf(rho_bar, w), c = fminf(c_bar, w);
+                const float gd = gamma * nd[q];
+                const float delta = rho * ((r[q] + gd * v_next) - v[q]);
+                const float e = delta + gd * c * e_next;
+                b.adv[i] = rho * ((r[q] + gd * (v_next + e_next)) - v[q]);
+                b.ret[i] = v[q] + e;
+                e_next = e;
+                v_next = v[q];
+            }
+        }
+    }
+}
+
+cudaError_t launch_vtrace(const Dims& d, const Buffers& b, int T, float gamma, float rho_bar, float c_bar, const float* boot, const Ctx& c) {
+    Scope sc(c, K_VTRACE);
+    k_vtrace<<<(d.B + 127) / 128, 128, 0, c.s>>>(d, b, T, gamma, rho_bar, c_bar, boot);
+    return cudaGetLastError();
+}
+
 }  // namespace anakin

@@ -145,10 +145,10 @@ __global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(Rol
     // Saved activations (the update reuses the policy's forward pass: Section 3.1): row i = t*B + env.
     __nv_bfloat16* g_h1hi = reinterpret_cast<__nv_bfloat16*>(b.h1);
     __nv_bfloat16* g_h1lo = g_h1hi + (size_t)B * d.Tmax * H;
-    const int t_end = a.replay ? a.T - 1 : a.T;  // replay recomputes the T recorded rows only (no bootstrap row)
+    const int t_end = a.replay == 1 ? a.T - 1 : a.T;  // replay recomputes the T recorded rows (mode 2: and the current state)
     for (int t = 0; t <= t_end; ++t) {
-        if (a.replay) {  // positions come from the recorded trajectory
-            if (tid < ME) s_pos[tid] = owner ? b.tpos[(size_t)t * B + e0 + tid] : 0;
+        if (a.replay) {  // positions come from the recorded trajectory (row T: the env state as it stands)
+            if (tid < ME) s_pos[tid] = owner ? (t < a.T ? b.tpos[(size_t)t * B + e0 + tid] : b.pos[e0 + tid]) : 0;
             __syncthreads();
         }
         // ---- layer 1: eight consecutive hidden units per thread and trip.  All gathers of the agent's W1 row are issued
@@ -310,6 +310,7 @@ __global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(Rol
                 o5[0] = make_float4(o[0], o[1], o[2], o[3]);
                 o5[1] = make_float4(o[4], 0.f, 0.f, 0.f);
             }
+            if (a.replay == 2 && t == a.T) b.vboot[env] = o[4];
             if (!a.replay) {
                 b.tval[(size_t)t * B + env] = o[4];
                 if (a.gae_smem) s_gv[t * ME + tid] = o[4];

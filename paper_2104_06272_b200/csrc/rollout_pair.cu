@@ -163,10 +163,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg::THREADS, 1)
     __nv_bfloat16* g_h1lo = g_h1hi + (size_t)B * d.Tmax * H;
     const uint32_t idesc_w = tc::umma_idesc<0>(256, 128, true, false), idesc_n = tc::umma_idesc<0>(256, 64, true, false);
 
-    const int t_end = a.replay ? a.T - 1 : a.T;  // replay recomputes the T recorded rows only (no bootstrap row)
+    const int t_end = a.replay == 1 ? a.T - 1 : a.T;  // replay recomputes the T recorded rows (mode 2: and the current state)
     for (int t = 0; t <= t_end; ++t) {
         if (a.replay) {  // positions come from the recorded trajectory
-            if (ow >= 0) s_pos[ow] = owner ? b.tpos[(size_t)t * B + e0 + ow] : 0;
+            if (ow >= 0) s_pos[ow] = owner ? (t < a.T ? b.tpos[(size_t)t * B + e0 + ow] : b.pos[e0 + ow]) : 0;
             __syncthreads();
         }
         if (tid == NWT) tc::mbar_expect_tx(pfull, 8 * ME * 5 * 4);  // this step's head partials, counted as they land
@@ -334,6 +334,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg::THREADS, 1)
                 o5[0] = make_float4(o[0], o[1], o[2], o[3]);
                 o5[1] = make_float4(o[4], 0.f, 0.f, 0.f);
             }
+            if (a.replay == 2 && t == a.T) b.vboot[env] = o[4];
             if (!a.replay) {
                 b.tval[(size_t)t * B + env] = o[4];
                 if (a.gae_smem) s_gv[t * ME + ow] = o[4];

@@ -191,6 +191,7 @@ __global__ void __launch_bounds__(256) k_h1_wide(Dims d, Buffers b, const uint8_
 //   mode 0: step t of the rollout (row = env): saves the head outputs and the value, samples, steps the env, records.
 //   mode 1: bootstrap forward after the last step: saves the value only.
 //   mode 2: replay of recorded rows (row = t*B + env): saves the head outputs only.
+//   mode 3: forward of the current env state under the current parameters: saves the value to vboot.
 constexpr int HW_ROWS = 32;
 
 template <int H>
@@ -278,6 +279,8 @@ __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mo
         const float o0 = s_out[tid][0], o1 = s_out[tid][1], o2 = s_out[tid][2], o3 = s_out[tid][3], v4 = s_out[tid][4];
         if (mode == 1) {
             b.tval[(size_t)a.T * d.B + i] = v4;
+        } else if (mode == 3) {
+            b.vboot[i] = v4;
         } else {
             const size_t row = mode == 0 ? (size_t)t * d.B + i : i;
             float4* o = reinterpret_cast<float4*>(b.out5 + row * 8);
@@ -483,8 +486,25 @@ cudaError_t launch_rollout_wide(const RolloutArgs& a, const Ctx& c) {
             g.M = (int)R; g.row0 = 0;
             CKW((launch_nt<EPI_FWD, true>(maps, g, c.s)));
         }
-        Scope sc(c, K_REPLAY);
-        return heads_wide(a, 0, 2, R, 0, c.s);
+        {
+            Scope sc(c, K_REPLAY);
+            CKW(heads_wide(a, 0, 2, R, 0, c.s));
+        }
+        if (a.replay == 2) {  // one more forward on the env state as it stands, in the B rows after the recorded ones
+            {
+                Scope sc(c, K_REPLAY);
+                k_h1_wide<<<h1_grid(B, H), 256, 0, c.s>>>(d, b, b.pos, B, R);
+                CKW(cudaGetLastError());
+            }
+            {
+                Scope sc(c, K_REPLAY);
+                g.M = B; g.row0 = (int)R;
+                CKW((launch_nt<EPI_FWD, true>(maps, g, c.s)));
+            }
+            Scope sc(c, K_REPLAY);
+            return heads_wide(a, 0, 3, B, R, c.s);
+        }
+        return cudaSuccess;
     }
     for (int t = 0; t <= a.T; ++t) {
         const size_t row0 = (size_t)t * B;
