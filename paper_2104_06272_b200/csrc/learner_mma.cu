@@ -934,17 +934,33 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             if (lane == 0) apply(i, gsum);
         }
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+    // Loss statistics: the first warp of the last CTA (the one with the least other work) adds the per-CTA partials of
+    // the heads kernel, lane l taking partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x < 32) {
+        const int lane = threadIdx.x;
         float l[3];
+#pragma unroll
         for (int c = 0; c < 3; ++c) {
             float s = 0.f;
-            for (int q = 0; q < loss_blocks; ++q) s += b.loss_part[(size_t)q * 4 + c];
+            int q = lane;
+            for (; q + 32 * 3 < loss_blocks; q += 32 * 4) {  // four loads in flight per lane
+                float v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) v[u] = b.loss_part[(size_t)(q + 32 * u) * 4 + c];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) s += v[u];
+            }
+            for (; q < loss_blocks; q += 32) s += b.loss_part[(size_t)q * 4 + c];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
             l[c] = s / (float)R;
         }
-        b.stats->loss_pg = l[0];
-        b.stats->loss_value = l[1];
-        b.stats->entropy = l[2];
-        b.stats->loss_total = l[0] + a.c_v * l[1] - a.c_e * l[2];
+        if (lane == 0) {
+            b.stats->loss_pg = l[0];
+            b.stats->loss_value = l[1];
+            b.stats->entropy = l[2];
+            b.stats->loss_total = l[0] + a.c_v * l[1] - a.c_e * l[2];
+        }
     }
 }
 
