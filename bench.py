@@ -256,10 +256,10 @@ def run_ours(args):
         an.set(bnd.ENV_POS, h_pos)
         an.set(bnd.ENV_TEP, h_tep)
         run_steps(1)
-        st = an.stats()
-        an.get_into(bnd.PARAMS, h_out)
-        an.get_into(bnd.ENV_POS, h_pos)
-        an.get_into(bnd.ENV_TEP, h_tep)
+        an.get_into(bnd.PARAMS, h_out, wait=False)   # device -> pinned host, enqueued behind the pass
+        an.get_into(bnd.ENV_POS, h_pos, wait=False)
+        an.get_into(bnd.ENV_TEP, h_tep, wait=False)
+        st = an.stats()                              # synchronises: everything above has landed
         h_theta.copy_(h_out)
     barrier()
     e2e_s = time.perf_counter() - t0

@@ -26,8 +26,10 @@
  *     allocated by the caller (e.g. a torch uint8 tensor) and alive until anakin_destroy().  The library
  *     allocates no device memory.  The handle itself is host memory owned by the library.
  *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  All work is
- *     enqueued on it.  reset/rollout/learn/run are asynchronous; get/set with a HOST pointer and
- *     anakin_status synchronise the stream before returning.
+ *     enqueued on it.  reset/rollout/learn/run are asynchronous; anakin_get with a HOST pointer and
+ *     anakin_status synchronise the stream before returning; anakin_set with a HOST pointer is enqueued (pageable
+ *     memory is staged by the runtime before the call returns; a page-locked source buffer must stay unchanged until
+ *     the stream has run the copy).
  *   - A handle is not thread-safe.  Different handles (different workspaces) are independent.
  *   - Unsupported shapes are refused with ANAKIN_E_UNSUPPORTED_CFG; there is no CPU fallback.
  *
@@ -219,8 +221,10 @@ int anakin_learn_vtrace(anakin_t* h, int epochs, float rho_bar, float c_bar);
 int anakin_run(anakin_t* h, int iters);
 
 /*
- * Copy a blob out of / into the workspace.  `ptr` is a host pointer (ptr_is_device = 0; the call synchronises the
- * stream) or a device pointer (ptr_is_device = 1; asynchronous on the stream).  `bytes` must equal the blob's
+ * Copy a blob out of / into the workspace.  `ptr` is a host pointer (ptr_is_device = 0; anakin_get synchronises the
+ * stream, anakin_set only enqueues: see the conventions above) or a device pointer (ptr_is_device = 1; asynchronous
+ * on the stream), or a PAGE-LOCKED host pointer (ptr_is_device = 2; asynchronous on the stream in both directions: the
+ * data of an anakin_get is there once the caller has synchronised the stream, e.g. with anakin_status).  `bytes` must equal the blob's
  * size.  Setting any TRAJ_* / ADV / RET blob marks a rollout of the last used length as pending, so the stages
  * can be driven with the other side's data.  Errors: INVALID_ARG (unknown blob, wrong size, read-only blob).
  */

@@ -233,11 +233,19 @@ class Anakin:
         self._ck(_lib.anakin_get(self._h, which, out.ctypes.data_as(_vp), n, 0))
         return out
 
-    def get_into(self, which: int, out: torch.Tensor):
-        """Copies a blob into a tensor of exactly the blob's size: a (pinned) host tensor (synchronises) or a CUDA
-        tensor on the handle's device (asynchronous, on the handle's stream)."""
+    def get_into(self, which: int, out: torch.Tensor, wait: bool = True):
+        """Copies a blob into a tensor of exactly the blob's size: a host tensor (synchronises; with wait=False and a pinned
+        tensor the copy is only enqueued and the caller synchronises later, e.g. with status()) or a CUDA tensor on the
+        handle's device (asynchronous, on the handle's stream)."""
         assert out.is_contiguous()
-        self._ck(_lib.anakin_get(self._h, which, _vp(out.data_ptr()), out.numel() * out.element_size(), 1 if out.is_cuda else 0))
+        if out.is_cuda:
+            kind = 1
+        elif not wait:
+            assert out.is_pinned(), "an asynchronous read needs page-locked host memory"
+            kind = 2
+        else:
+            kind = 0
+        self._ck(_lib.anakin_get(self._h, which, _vp(out.data_ptr()), out.numel() * out.element_size(), kind))
 
     def set(self, which: int, value):
         if which in (ADAM_STEP, GLOBAL_STEP):

@@ -523,7 +523,11 @@ static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is
         if (to_lib) memcpy(bl.ptr, ptr, bytes); else memcpy(ptr, bl.ptr, bytes);
         return ANAKIN_OK;
     }
-    const cudaMemcpyKind kind = ptr_is_device ? cudaMemcpyDeviceToDevice : (to_lib ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost);
+    if (ptr_is_device < 0 || ptr_is_device > 2) return ANAKIN_E_INVALID_ARG;
+    // 2 = page-locked host memory, asynchronous: the runtime infers the direction from the (unified) addresses
+    const cudaMemcpyKind kind = ptr_is_device == 1 ? cudaMemcpyDeviceToDevice
+                              : ptr_is_device == 2 ? cudaMemcpyDefault
+                              : (to_lib ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost);
     cudaError_t e = to_lib ? cudaMemcpyAsync(bl.ptr, ptr, bytes, kind, h->stream) : cudaMemcpyAsync(ptr, bl.ptr, bytes, kind, h->stream);
     if (e != cudaSuccess) return fail_cuda(h, e);
     if (to_lib) {
@@ -542,7 +546,10 @@ static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is
             h->rollout_pending = true;
         }
     }
-    if (!ptr_is_device) {
+    // A read into host memory must have landed when the call returns.  A write from host memory is stream-ordered like
+    // everything else: the runtime stages pageable memory before cudaMemcpyAsync returns, and a page-locked source is the
+    // caller's to keep unchanged until the stream has run the copy.
+    if (!ptr_is_device && !to_lib) {
         e = cudaStreamSynchronize(h->stream);
         if (e != cudaSuccess) return fail_cuda(h, e);
     }

@@ -345,3 +345,28 @@ def test_torus_env_free_running_and_different_from_the_grid(bnd):
     ag.learn()
     par.assert_close(an.get(bnd.GRADS), ag.grads, 1e-4, "grads")
     assert an.status() == 0
+
+
+def test_asynchronous_copies_through_page_locked_host_memory(bnd):
+    """ptr_is_device = 2: blobs move to and from pinned host buffers in stream order without a synchronisation per call;
+    after one synchronising call the data is what the synchronous copies give."""
+    import torch
+
+    w = WORKLOADS["tiny"]
+    an = make(bnd, w, debug=0)
+    an.reset(4)
+    an.rollout()
+    an.learn()
+    want = {b: an.get(b) for b in (bnd.PARAMS, bnd.ENV_POS, bnd.TRAJ_VALUE)}
+    bufs = {b: torch.empty(v.size, dtype=torch.from_numpy(v).dtype).pin_memory() for b, v in want.items()}
+    for b, t in bufs.items():
+        an.get_into(b, t, wait=False)
+    assert an.status() == 0  # synchronises
+    for b, t in bufs.items():
+        assert np.array_equal(t.numpy(), want[b])
+    # and the other way: a pinned source, enqueued, then read back
+    src = torch.from_numpy(want[bnd.PARAMS] * np.float32(0.5)).pin_memory()
+    an.set(bnd.PARAMS, src)
+    assert np.array_equal(an.get(bnd.PARAMS), src.numpy())
+    with pytest.raises(bnd.AnakinError):
+        an._ck(bnd._lib.anakin_get(an._h, bnd.PARAMS, bufs[bnd.PARAMS].data_ptr(), bufs[bnd.PARAMS].numel() * 4, 3))
