@@ -196,6 +196,23 @@ def test_runs_are_bitwise_deterministic(bnd):
     assert (an2.get(bnd.PARAMS) != outs[0][0]).any()
 
 
+def test_long_runs_of_the_benchmarked_workload_are_bitwise_reproducible(bnd):
+    """The CTA pairs of the tcgen05 rollout hand operand tiles, accumulators and head partials to each other through
+    mbarriers only; a missed ordering would show as a run that differs from its twin.  100 passes of the full-size
+    throughput workload (3,300 rollout steps on 64 pairs), twice."""
+    w = WORKLOADS["throughput"]
+    outs = []
+    for _ in range(2):
+        an = make(bnd, w, debug=0)
+        an.reset(2)
+        an.run(100)
+        outs.append((an.get(bnd.PARAMS), an.get(bnd.TRAJ_ACTION), an.get(bnd.TRAJ_VALUE), an.get(bnd.ADV)))
+        assert an.status() == 0
+    for a, b in zip(*outs):
+        assert (a.view(np.uint8) == b.view(np.uint8)).all()
+    assert np.isfinite(outs[0][0]).all()
+
+
 def test_checkpoint_resume_is_bitwise(bnd):
     w = SMALL["large_batch_s"].scaled(B=300, T=8)
     a = make(bnd, w, debug=0)
