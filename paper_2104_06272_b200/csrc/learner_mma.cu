@@ -886,7 +886,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
         return r;
     };
     // Parameters before b2 (W1, b1, W2) have at most ~128 partials: one thread each, partials added in index order,
-    // sixteen loads in flight.  The tail (b2 | Wh | bh) has two partials per CTA of the heads kernel: one warp per
+    // thirty-two loads in flight.  The tail (b2 | Wh | bh) has two partials per CTA of the heads kernel: one warp per
     // parameter, lane l adds partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
     const int nb_main = (int)((d.ob2 + 255) / 256);
     if ((int)blockIdx.x < nb_main) {
@@ -895,22 +895,16 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
             const PartRegion& rg = a.reg[region_of(i)];
             const float* p = rg.part + (i - rg.start);
             float gsum = 0.f;
-            int s = 0;
-            for (; s + 16 <= rg.ns; s += 16) {
-                float v[16];
+            // thirty-two loads in flight per memory round trip (the ragged last batch is predicated, not split up);
+            // the additions stay in index order
+            for (int s = 0; s < rg.ns; s += 32) {
+                float v[32];
 #pragma unroll
-                for (int q = 0; q < 16; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
+                for (int q = 0; q < 32; ++q) v[q] = s + q < rg.ns ? p[(size_t)(s + q) * rg.stride] : 0.f;
 #pragma unroll
-                for (int q = 0; q < 16; ++q) gsum += v[q];
+                for (int q = 0; q < 32; ++q)
+                    if (s + q < rg.ns) gsum += v[q];
             }
-            for (; s + 4 <= rg.ns; s += 4) {
-                float v[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) v[q] = p[(size_t)(s + q) * rg.stride];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) gsum += v[q];
-            }
-            for (; s < rg.ns; ++s) gsum += p[(size_t)s * rg.stride];
             apply(i, gsum);
         }
     } else {
