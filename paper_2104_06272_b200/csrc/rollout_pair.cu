@@ -39,7 +39,7 @@ struct PairCfg {
         2 * (size_t)A_PLANE + B_BYTES + (size_t)ME * H * 4    // W2 planes, operand tile, base
         + 64                                                  // barriers, tensor-memory slot
         + (size_t)8 * ME * 5 * 4                              // head partials: 8 blocks of 32 hidden units
-        + 8 * 4 + (size_t)ME * 8 * 4 + ME * 4 + ME * 8;       // bh, walls, pos, prepared step
+        + 8 * 4 + (size_t)ME * 8 * 4 + ME * 4;                // bh, walls, pos
     static constexpr size_t gae_bytes(int T) { return (size_t)(T + 1) * ME * 4 + (size_t)T * ME; }
 };
 
@@ -74,8 +74,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg::THREADS, 1)
     float* s_bh = s_red + 8 * ME * 5;                                               // [8]
     uint32_t* s_walls = reinterpret_cast<uint32_t*>(s_bh + 8);                      // [ME][8]
     int* s_pos = reinterpret_cast<int*>(s_walls + ME * 8);                          // [ME]
-    uint2* s_pre = reinterpret_cast<uint2*>(s_pos + ME);                            // [ME]
-    float* s_gv = reinterpret_cast<float*>(s_pre + ME);                             // [T+1][ME] (a.gae_smem only)
+    float* s_gv = reinterpret_cast<float*>(s_pos + ME);                             // [T+1][ME] (a.gae_smem only)
     uint8_t* s_gc = reinterpret_cast<uint8_t*>(s_gv + (a.T + 1) * ME);              // [T][ME]
 
     const Dims& d = a.d;
