@@ -89,7 +89,7 @@ class ClockSampler:
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu capture
 # summarised under profiles/ for the same kernel source; None for workloads without a capture at full size.
-NCU_TRAFFIC_BYTES = {("throughput", "rollout"): 4.7e6 + 215.7e6}
+NCU_TRAFFIC_BYTES = {("throughput", "rollout"): 4.7e6 + 216.7e6}
 
 
 def workload_label(w):
