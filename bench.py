@@ -24,7 +24,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2104_06272_b200.workloads import WORKLOADS  # noqa: E402
+from paper_2104_06272_b200.workloads import ORDER, WORKLOADS  # noqa: E402
 
 METRIC = "env_frames_per_sec_act_plus_learn"
 UNIT = "frames/s"
@@ -87,9 +87,36 @@ class ClockSampler:
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons), "samples": len(sm)}
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the ncu capture
-# summarised under profiles/ for the same kernel source; None for workloads without a capture at full size.
-NCU_TRAFFIC_BYTES = {("throughput", "rollout"): 4.7e6 + 216.7e6}
+# Which ncu summary under profiles/ covers a (workload, profiler kernel name) pair, and the source file of that kernel.
+# The summary carries the counters (a table row "dram__bytes_read / write | X MB / Y MB") and the SHA-256 of the kernel's
+# source file at capture time ("kernel source: <file> sha256 <hex>"); counters of a kernel that has changed since are
+# not reported.
+PROFILE_OF = {
+    ("throughput", "rollout"): ("rollout_pair__throughput.md", "rollout_pair.cu"),
+    ("throughput", "dh1"): ("dh1a_tc__throughput.md", "dh1a_tc.cu"),
+    ("throughput", "dw2"): ("gemm_tn_tc_dw2__throughput.md", "gemm_tc.cu"),
+    ("throughput", "heads_bwd"): ("heads_bwd__throughput.md", "learner_mma.cu"),
+}
+
+
+def ncu_traffic_bytes(workload: str, kernel: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu summary, or None when there is no
+    summary for this kernel and workload or the kernel's source has changed since the capture."""
+    import hashlib
+    import re
+
+    ent = PROFILE_OF.get((workload, kernel))
+    if ent is None:
+        return None
+    prof, src = os.path.join(ROOT, "profiles", ent[0]), os.path.join(ROOT, "paper_2104_06272_b200", "csrc", ent[1])
+    if not (os.path.exists(prof) and os.path.exists(src)):
+        return None
+    text = open(prof).read()
+    m = re.search(r"dram__bytes_read / write \| ([\d.]+) MB / ([\d.]+) MB", text)
+    h = re.search(r"kernel source: \S+ sha256 ([0-9a-f]{64})", text)
+    if not m or not h or h.group(1) != hashlib.sha256(open(src, "rb").read()).hexdigest():
+        return None
+    return (float(m.group(1)) + float(m.group(2))) * 1e6
 
 
 def workload_label(w):
@@ -159,6 +186,111 @@ def whole_job_frames_per_sec(frames_per_rank: float, world: int, max_seconds: fl
     return frames_per_rank * world / max_seconds
 
 
+def time_steps(an, run_steps, w, K, W, stream, flush, barrier, rank, local_rank, world):
+    """W untimed steps, then K steps each bracketed by CUDA events on the library's stream with the L2 flushed between
+    them (outside the brackets), clocks sampled meanwhile; then the same K steps once more with events around every
+    kernel launch.  Returns (frames/s over all ranks, total ms (max over ranks), launches, clocks, per-kernel times,
+    wall seconds of the timed region)."""
+    import torch
+
+    run_steps(W)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    n0 = an.launch_count()
+    barrier()
+    t_wall0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        for a, b in ev:
+            flush.fill_(0)
+            a.record(stream)
+            run_steps(1)
+            b.record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    launches = an.launch_count() - n0
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = max_over_ranks(float(sum(step_ms)), world, "cuda")
+    value = whole_job_frames_per_sec(float(w.B) * w.T * K, world, total_ms * 1e-3)
+    an.profile_enable(True)
+    with torch.cuda.stream(stream):
+        for _ in range(K):
+            flush.fill_(0)
+            run_steps(1)
+    prof = an.profile_read()
+    an.profile_enable(False)
+    return value, total_ms, launches, clocks, prof, t_wall
+
+
+def roofline_of(w, prof, K, peaks, clocks):
+    """Roofline entry of the dominant kernel (largest total time in the per-kernel pass) plus one line per kernel.
+    Tensor kernels: executed FLOPs / duration against the measured cuBLAS bf16 figure -- the burst figure when the SM
+    clock stayed near its maximum during the timed region (short kernels, no power cap), the sustained one otherwise;
+    both fractions are printed."""
+    work = kernel_work(w)
+    tot = sum(ms for ms, _ in prof.values())
+
+    def kernel_line(k, ms, n):
+        line = {"us_per_launch": ms / n * 1e3, "launches_per_step": n / K, "share": ms / tot}
+        if k in work:
+            bnd_, fl, by = work[k]
+            sec = ms / n * 1e-3
+            line["bound"] = bnd_
+            line["tflops"] = fl / sec / 1e12
+            line["gbs"] = by / sec / 1e9
+        return line
+
+    top = max(prof, key=lambda k: prof[k][0])
+    top_ms, top_n = prof[top]
+    bound, flops, nbytes = work.get(top, ("hbm", 0.0, 0.0))
+    per_launch_s = top_ms / top_n * 1e-3
+    sm_max = (clocks or {}).get("sm_max_mhz") or peaks["sm_max_mhz"]
+    sm_now = (clocks or {}).get("sm_mhz") or sm_max
+    extra = {}
+    if bound == "alu":
+        achieved, peak, unit = flops / per_launch_s / 1e12, FP32_ALU_TFLOPS_PER_MHZ * sm_max, "TFLOP/s"
+        peak_note = f"fp32 FMA peak = 148 SMs x 128 lanes x 2 x {sm_max:.0f} MHz (derived)"
+    elif bound == "tensor":
+        achieved, unit = flops / per_launch_s / 1e12, "TFLOP/s"
+        at_full_clock = sm_now >= 0.9 * sm_max
+        peak = peaks["bf16_tflops"] if at_full_clock else peaks["bf16_tflops_sustained"]
+        extra = {"frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"]}
+        peak_note = (f"dense 16-bit tensor throughput (cuBLAS bf16, {'burst: SM clock at ' if at_full_clock else 'sustained: SM clock at '}"
+                     f"{sm_now:.0f} of {sm_max:.0f} MHz during the timed region), {peaks['source']}; achieved counts executed FLOPs "
+                     "(3 fp16 MMAs per fp32 product)")
+    else:
+        achieved, peak, unit = nbytes / per_launch_s / 1e9, peaks["hbm_gbs"], "GB/s"
+        peak_note = f"HBM copy bandwidth, {peaks['source']}"
+    base_name = w.name.split("[")[0]
+    out = {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+           "traffic": ncu_traffic_bytes(base_name, top) if base_name == w.name else None, "peak_source": peak_note,
+           "us_per_launch": per_launch_s * 1e6, "share_of_step": top_ms / tot,
+           "kernels": {k: kernel_line(k, ms, n) for k, (ms, n) in sorted(prof.items(), key=lambda kv: -kv[1][0])}}
+    out.update(extra)
+    return out
+
+
+def time_other_workload(bnd, w, stream, flush, local_rank, peaks, seed, K=4, W=3):
+    """A short device-timed run of another workload (same event / flush method as the headline), for the per-workload
+    table: frames/s, ms per step, clocks of that segment, the dominant kernel and its roofline fraction."""
+    import torch
+
+    with torch.cuda.stream(stream):
+        an = bnd.Anakin(bnd.cfg_from_workload(w, device=local_rank), stream=stream)
+    an.reset(seed)
+    value, total_ms, launches, clocks, prof, _ = time_steps(an, an.run, w, K, W, stream, flush, torch.cuda.synchronize, 0, local_rank, 1)
+    ok = an.status() == 0 and bool(np.isfinite(an.stats().loss_total))
+    rl = roofline_of(w, prof, K, peaks, clocks)
+    del an
+    torch.cuda.empty_cache()
+    return {"workload": workload_label(w), "value": value, "unit": UNIT, "ms_per_step": total_ms / K, "steps": K, "warmup": W,
+            "dtype": "bf16" if w.precision == 1 else "f32", "gpu_launches": int(launches), "clocks": clocks, "status_ok": ok,
+            "roofline": rl}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -206,40 +338,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     K, W = args.steps, args.warmup
-    # ---- warm-up
-    run_steps(W)
-    torch.cuda.synchronize()
-
-    # ---- timed region: K steps, each bracketed by events on the library's stream; L2 flushed between steps
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    n0 = an.launch_count()
-    barrier()
-    t_wall0 = time.perf_counter()
-    with torch.cuda.stream(stream):
-        for a, b in ev:
-            flush.fill_(0)
-            a.record(stream)
-            run_steps(1)
-            b.record(stream)
-    barrier()
-    t_wall = time.perf_counter() - t_wall0
-    launches = an.launch_count() - n0
-    clocks = sampler.stop() if rank == 0 else None
-    step_ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = max_over_ranks(float(sum(step_ms)), world, "cuda")
-    value = whole_job_frames_per_sec(float(w.B) * w.T * K, world, total_ms * 1e-3)
-
-    # ---- per-kernel pass (events around every launch), same K steps, for the roofline entry
-    an.profile_enable(True)
-    with torch.cuda.stream(stream):
-        for _ in range(K):
-            flush.fill_(0)
-            run_steps(1)
-    prof = an.profile_read()
-    an.profile_enable(False)
+    value, total_ms, launches, clocks, prof, t_wall = time_steps(an, run_steps, w, K, W, stream, flush, barrier, rank, local_rank, world)
 
     # ---- end to end through the C ABI with host buffers: per step, parameters and env state go host->device
     # from pinned memory, one act+learn pass runs, statistics and parameters come back
@@ -272,39 +371,16 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel
-    work = kernel_work(w)
+    roofline = roofline_of(w, prof, K, peaks, clocks)
 
-    def kernel_line(k, ms, n):
-        line = {"us_per_launch": ms / n * 1e3, "launches_per_step": n / K, "share": ms / tot}
-        if k in work:
-            bnd_, fl, by = work[k]
-            sec = ms / n * 1e-3
-            line["bound"] = bnd_
-            line["tflops"] = fl / sec / 1e12
-            line["gbs"] = by / sec / 1e9
-        return line
-
-    tot = sum(ms for ms, _ in prof.values())
-    top = max(prof, key=lambda k: prof[k][0])
-    top_ms, top_n = prof[top]
-    bound, flops, nbytes = work.get(top, ("hbm", 0.0, 0.0))
-    per_launch_s = top_ms / top_n * 1e-3
-    sm_mhz = (clocks or {}).get("sm_max_mhz") or peaks["sm_max_mhz"]
-    if bound == "alu":
-        achieved, peak, unit = flops / per_launch_s / 1e12, FP32_ALU_TFLOPS_PER_MHZ * sm_mhz, "TFLOP/s"
-        peak_note = f"fp32 FMA peak = 148 SMs x 128 lanes x 2 x {sm_mhz:.0f} MHz (derived)"
-    elif bound == "tensor":
-        achieved, peak, unit = flops / per_launch_s / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s"
-        peak_note = (f"dense 16-bit tensor throughput (cuBLAS bf16, sustained), {peaks['source']}; achieved counts executed "
-                     "FLOPs (3 fp16 MMAs per fp32 product)")
-    else:
-        achieved, peak, unit = nbytes / per_launch_s / 1e9, peaks["hbm_gbs"], "GB/s"
-        peak_note = f"HBM copy bandwidth, {peaks['source']}"
-    roofline = {"kernel": top, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES.get((w.name, top)), "peak_source": peak_note, "us_per_launch": per_launch_s * 1e6,
-                "share_of_step": top_ms / tot,
-                "kernels": {k: kernel_line(k, ms, n) for k, (ms, n) in sorted(prof.items(), key=lambda kv: -kv[1][0])}}
+    # ---- the other workloads, device-timed the same way (short runs): one entry each
+    others = None
+    if world == 1 and not args.envs and not args.no_workloads and args.workload == "throughput":
+        others = {}
+        for name in ORDER:
+            if name == args.workload:
+                continue
+            others[name] = time_other_workload(bnd, WORKLOADS[name], stream, flush, local_rank, peaks, seed)
 
     # ---- the oracle on the host cores, bounded sample of the same workload (about 10-30 s of CPU work)
     if args.no_cpu_baseline or rank != 0:
@@ -332,6 +408,8 @@ def run_ours(args):
         "roofline": roofline,
         "cpu_baseline": cpu,
     }
+    if others is not None:
+        out["workloads"] = others
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -387,6 +465,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiler captures only)")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--envs", type=int, default=0, help="override the workload's number of envs (small profiler captures only)")
     ap.add_argument("--workload", default="throughput", choices=list(WORKLOADS),
                     help="the metric is quoted on 'throughput'; the others are for the per-workload table")

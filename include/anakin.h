@@ -184,10 +184,15 @@ int anakin_update(anakin_t* h);
  *                       state untouched.  Errors: BAD_STATE if no rollout is pending.
  *   anakin_apply_grads  one Adam step with the GRADS blob as it stands (after the caller has averaged it over the
  *                       replicas, on this stream).  Errors: BAD_STATE before the first anakin_reset.
+ *   anakin_apply_grads_mean   the same step for a GRADS blob that holds the SUM of the replicas' gradients (what a
+ *                       sum all-reduce leaves): the kernel divides by n_replicas first and stores the mean back into
+ *                       GRADS, so the caller's exchange needs no arithmetic of its own.  n_replicas = 1 is
+ *                       anakin_apply_grads.  Errors: INVALID_ARG for n_replicas < 1.
  * anakin_grads followed by anakin_apply_grads gives bitwise the result of anakin_learn.
  */
 int anakin_grads(anakin_t* h);
 int anakin_apply_grads(anakin_t* h);
+int anakin_apply_grads_mean(anakin_t* h, int n_replicas);
 
 /*
  * Another objective over the same trajectory buffers (Section 3.2 leaves the choice of objective open; this one is the
@@ -236,6 +241,15 @@ size_t anakin_blob_bytes(anakin_t* h, int which);
 
 /* Synchronises the stream and returns the sticky device status word (0 = clean) in *device_status. */
 int anakin_status(anakin_t* h, int* device_status);
+
+/*
+ * Self-test of the bounded device-side waits.  Every wait inside the tensor-core kernels (on an mbarrier that a TMA
+ * copy, an MMA or a peer CTA completes) gives up after a clock limit, raises bit 4 (a bounded wait gave up) in the
+ * sticky status word and lets the kernel return.  This call enqueues a one-CTA kernel that waits, with the given limit
+ * in SM clocks (1 .. 2e9), on a barrier nobody arrives on: afterwards anakin_status reports bit 4 and every other call
+ * works as before (anakin_reset clears the word).  It never spins past the limit and never traps.
+ */
+int anakin_selftest_wait_timeout(anakin_t* h, int64_t limit_clocks);
 
 /* Number of kernel launches enqueued by this handle since creation (host-side counter). */
 uint64_t anakin_launch_count(anakin_t* h);
@@ -290,6 +304,17 @@ int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int64_t global_
                            uint8_t* dev_traj_pos, int8_t* dev_traj_action, uint8_t* dev_traj_done,
                            float* dev_traj_reward, float* dev_traj_value, float* dev_traj_logp,
                            void* cuda_stream);
+
+/*
+ * Device status of the last anakin_rollout_noalloc call on the current device.  (No counterpart in the paper either.)
+ * That call has no handle, so anakin_status cannot serve it: its sticky status word (0 = clean; the same bits as
+ * anakin_status reports: a start position outside the grid or on a wall, a bounded device-side wait that gave up)
+ * sits in the library's built-in array.  This call copies the word out on `cuda_stream` -- pass the stream the rollout
+ * was enqueued on -- and SYNCHRONISES that stream; it allocates nothing.  Returns ANAKIN_OK with *device_status = 0,
+ * or ANAKIN_E_DEVICE_STATUS with the word: then the trajectory the rollout wrote is not to be trusted.  The next
+ * anakin_rollout_noalloc call clears the word, so read it before enqueueing another one.
+ */
+int anakin_noalloc_status(void* cuda_stream, int* device_status);
 
 /* Static description of an error code. */
 const char* anakin_strerror(int code);

@@ -45,11 +45,11 @@ OK, E_INVALID_ARG, E_BAD_STATE, E_WORKSPACE_TOO_SMALL, E_UNSUPPORTED_CFG, E_CUDA
 
 EXPORTS = [
     "anakin_workspace_bytes", "anakin_create", "anakin_destroy", "anakin_reset", "anakin_rollout",
-    "anakin_rollout_forced", "anakin_learn", "anakin_gae", "anakin_update", "anakin_grads", "anakin_apply_grads", "anakin_learn_ppo", "anakin_learn_vtrace",
+    "anakin_rollout_forced", "anakin_learn", "anakin_gae", "anakin_update", "anakin_grads", "anakin_apply_grads", "anakin_apply_grads_mean", "anakin_learn_ppo", "anakin_learn_vtrace",
     "anakin_run", "anakin_get", "anakin_set",
     "anakin_blob_bytes", "anakin_status", "anakin_launch_count", "anakin_strerror", "anakin_last_cuda_error",
     "anakin_profile_enable", "anakin_profile_read", "anakin_kernel_count", "anakin_kernel_name",
-    "anakin_rollout_noalloc",
+    "anakin_rollout_noalloc", "anakin_noalloc_status", "anakin_selftest_wait_timeout",
 ]
 
 _vp = C.c_void_p
@@ -64,6 +64,7 @@ _lib.anakin_gae.argtypes = [_vp]
 _lib.anakin_update.argtypes = [_vp]
 _lib.anakin_grads.argtypes = [_vp]
 _lib.anakin_apply_grads.argtypes = [_vp]
+_lib.anakin_apply_grads_mean.argtypes = [_vp, C.c_int]
 _lib.anakin_learn_ppo.argtypes = [_vp, C.c_int, C.c_float]
 _lib.anakin_learn_vtrace.argtypes = [_vp, C.c_int, C.c_float, C.c_float]
 _lib.anakin_run.argtypes = [_vp, C.c_int]
@@ -84,6 +85,8 @@ _lib.anakin_kernel_count.argtypes = []
 _lib.anakin_kernel_name.argtypes = [C.c_int]
 _lib.anakin_kernel_name.restype = C.c_char_p
 _lib.anakin_rollout_noalloc.argtypes = [C.POINTER(AnakinCfg), C.c_uint64, C.c_int64, C.c_int] + [_vp] * 13
+_lib.anakin_selftest_wait_timeout.argtypes = [_vp, C.c_int64]
+_lib.anakin_noalloc_status.argtypes = [_vp, C.POINTER(C.c_int)]
 NOALLOC_MAX_BH = 1048576
 ENV_GRID, ENV_TORUS = 0, 1  # anakin_cfg.env_kind
 
@@ -145,6 +148,15 @@ def rollout_noalloc(cfg: AnakinCfg, seed: int, global_step: int, T: int, params,
                                            *[_vp(t.data_ptr()) for t in ts], _vp(s.cuda_stream)))
 
 
+def noalloc_status(stream=None) -> tuple[int, int]:
+    """anakin_noalloc_status: (return code, device status word) of the last rollout_noalloc call on the current
+    device; synchronises the stream."""
+    s = stream if stream is not None else torch.cuda.current_stream()
+    st = C.c_int(0)
+    rc = int(_lib.anakin_noalloc_status(_vp(s.cuda_stream), C.byref(st)))
+    return rc, int(st.value)
+
+
 class Anakin:
     """anakin_create / reset / rollout / learn / run over a torch-owned workspace and stream."""
 
@@ -203,8 +215,9 @@ class Anakin:
     def grads(self):
         self._ck(_lib.anakin_grads(self._h))
 
-    def apply_grads(self):
-        self._ck(_lib.anakin_apply_grads(self._h))
+    def apply_grads(self, n_replicas: int = 1):
+        """Adam from GRADS; n_replicas > 1: GRADS holds the sum over that many replicas (divided on the device)."""
+        self._ck(_lib.anakin_apply_grads_mean(self._h, C.c_int(n_replicas)))
 
     def learn_ppo(self, epochs: int, clip_eps: float):
         self._ck(_lib.anakin_learn_ppo(self._h, epochs, C.c_float(clip_eps)))
@@ -266,6 +279,10 @@ class Anakin:
         if rc not in (OK, E_DEVICE_STATUS):
             self._ck(rc)
         return int(st.value)
+
+    def selftest_wait_timeout(self, limit_clocks: int = 1_000_000):
+        """Enqueues the one-CTA kernel whose bounded wait must run out (status bit 4 afterwards)."""
+        self._ck(_lib.anakin_selftest_wait_timeout(self._h, C.c_int64(limit_clocks)))
 
     def launch_count(self) -> int:
         return int(_lib.anakin_launch_count(self._h))

@@ -372,6 +372,7 @@ static int learn_after_gae(anakin_t* h, int phase, float ppo_clip = 0.f, bool co
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
     a.phase = phase;
+    a.grad_div = 1.f;
     a.ppo_clip = ppo_clip;
     {   // smallest power of two >= R: keeps the scaled output gradients O(1) for the fp16 operand format
         const double Rrows = (double)h->d.B * (double)h->last_T;
@@ -476,8 +477,10 @@ int anakin_grads(anakin_t* h) {
     return learn_after_gae(h, 1);
 }
 
-int anakin_apply_grads(anakin_t* h) {
-    if (!h) return ANAKIN_E_INVALID_ARG;
+int anakin_apply_grads(anakin_t* h) { return anakin_apply_grads_mean(h, 1); }
+
+int anakin_apply_grads_mean(anakin_t* h, int n_replicas) {
+    if (!h || n_replicas < 1) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset) return ANAKIN_E_BAD_STATE;
     LearnArgs a;
     memset(&a, 0, sizeof(a));
@@ -488,6 +491,7 @@ int anakin_apply_grads(anakin_t* h) {
     a.beta2 = h->cfg.adam_b2;
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
+    a.grad_div = (float)n_replicas;
     const cudaError_t e = launch_adam_only(a, h->cfg.precision, h->ctx());
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->adam_k += 1;
@@ -572,6 +576,14 @@ int anakin_status(anakin_t* h, int* device_status) {
     if (e != cudaSuccess) return fail_cuda(h, e);
     *device_status = st;
     return st == 0 ? ANAKIN_OK : ANAKIN_E_DEVICE_STATUS;
+}
+
+int anakin_selftest_wait_timeout(anakin_t* h, int64_t limit_clocks) {
+    if (!h || limit_clocks < 1 || limit_clocks > 2000000000LL) return ANAKIN_E_INVALID_ARG;
+    const cudaError_t e = launch_selftest_wait(h->b.status, (long long)limit_clocks, nullptr, h->stream);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    ++h->launches;
+    return ANAKIN_OK;
 }
 
 uint64_t anakin_launch_count(anakin_t* h) { return h ? h->launches : 0; }

@@ -161,6 +161,7 @@ struct LearnArgs {
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
     int phase;   // 0: reduce the partials and apply Adam; 1: reduce only (GRADS and loss statistics)
+    float grad_div;  // Adam-only launch: > 1 = GRADS holds a sum over this many replicas, divided here into their mean
     float ppo_clip;  // > 0: the policy term is the clipped surrogate over the recorded log-probabilities (TRAJ_LOGP)
     // tensor-pipe path
     int ts;               // t-slices of the dh1 kernel: S holds ts*B rows (slice z, env b at row z*B + b)
@@ -206,7 +207,7 @@ struct Ctx {
 
 // Counts one kernel launch and, when profiling, brackets it with two events.
 struct Scope {
-    const Ctx& c;
+    const Ctx c;  // by value: launch sites may pass a temporary
     cudaEvent_t b = nullptr;
     Scope(const Ctx& ctx, int id) : c(ctx) {
         ++*c.launches;
@@ -270,6 +271,7 @@ bool dh1_agent_tc_supported(const Dims& d);
 // dh1, S and the agent plane of dW1 in one tcgen05 kernel; cudaErrorNotSupported if not covered
 cudaError_t launch_dh1_agent_tc(const LearnArgs& a, int prec, int grid_x, float* part_agent, size_t part_stride, cudaStream_t s);
 cudaError_t launch_dh1_tc(const LearnArgs& a, int prec, cudaStream_t s);  // tcgen05 dh1 kernel; cudaErrorNotSupported if not covered  // needs the activations the rollout saved
+cudaError_t launch_selftest_wait(int* status, long long limit_clocks, long long* waited_clocks, cudaStream_t s);
 cudaError_t launch_refresh_compute_params(const Dims& d, const Buffers& b, int prec, const Ctx& c);
 
 }  // namespace anakin

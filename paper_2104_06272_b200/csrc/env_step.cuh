@@ -39,6 +39,16 @@ struct TorusMoves {  // borders wrap around
     }
 };
 
+// A state handed in from outside (anakin_set, the handle-less rollout) may not be a legal one.  Start, goal and agent
+// must be cells of the board, and the agent does not stand on a wall: anything else raises DEV_E_BAD_STATE and is
+// replaced (start and goal by cell 0, the agent by the start cell), so that every later index stays inside its array.
+// walls: this env's wall words.
+__device__ __forceinline__ void check_env_state(EnvLane& s, int C, const uint32_t* walls) {
+    if (s.start >= C) { s.bad |= DEV_E_BAD_STATE; s.start = 0; }
+    if (s.goal >= C) { s.bad |= DEV_E_BAD_STATE; s.goal = 0; }
+    if (s.pos >= C || ((walls[s.pos >> 5] >> (s.pos & 31)) & 1u)) { s.bad |= DEV_E_BAD_STATE; s.pos = s.start; }
+}
+
 // walls: this env's wall words (shared memory), 8 words.
 template <class Moves>
 __device__ __forceinline__ StepPre step_prepare_t(const EnvLane& s, const RolloutArgs& a, int env, int t, const uint32_t* walls) {

@@ -12,6 +12,11 @@
 //   warp 1 (one lane)  issues tcgen05.mma: for fp32 workloads three MMAs per k16 (lo*hi, hi*lo, hi*hi fp16 terms) into one
 //                      fp32 accumulator; commits free the stage,
 //   warps 2-5          after the last chunk: tcgen05.ld the accumulator and store the partial tile.
+// Long K ranges (plane operands): the tensor core's fp32 accumulation rounds toward zero, which biases a sum of many
+// thousand MMAs by more than the fp32 workloads' 1e-4 bound (measured: -2e-4 after 65,536 rows).  The K range of a CTA
+// is therefore cut into groups of GROUP chunks; the groups alternate between two accumulators in tensor memory, and
+// while the MMAs of one group run, warps 2-5 add the previous group's accumulator into the partial tile in global
+// memory with ordinary (round-to-nearest) fp32 additions, in group order.
 // Every wait is bounded; a timeout raises DEV_E_WAIT_TIMEOUT in the status word and the CTA unwinds (tensor memory freed).
 #include <cstdio>
 #include <cstring>
@@ -66,6 +71,10 @@ struct GemmTcCfg {
     static constexpr int FIT = (232448 - 1024 - 128) / STAGE;
     static constexpr int STAGES = !DEEP ? 2 : (FIT >= 4 ? 4 : (FIT >= 2 ? FIT : 2));
     static constexpr size_t smem_bytes = (size_t)STAGES * STAGE + 1024 /*alignment slack*/ + 128 /*barriers, tmem slot*/;
+    // plane operands: two accumulators, a group of GROUP 64-row chunks (2048 rows, 384 MMAs of an fp32 product) each
+    static constexpr bool FLUSH = DEEP;
+    static constexpr int GROUP = 32;
+    static constexpr int TMEM_COLS = FLUSH ? 2 * BN : BN;
 };
 
 struct GemmTcMaps {
@@ -78,8 +87,12 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
     constexpr int BM = Cfg::BM, KC = Cfg::KC, STAGES = Cfg::STAGES;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // the swizzle needs 1024-byte alignment
-    uint64_t* bars = (uint64_t*)(base + STAGES * Cfg::STAGE);  // full[STAGES], empty[STAGES], done
-    uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 1);
+    uint64_t* bars = (uint64_t*)(base + STAGES * Cfg::STAGE);  // full[STAGES], empty[STAGES], accfull[2], accempty[2]
+    uint64_t* accfull = bars + 2 * STAGES;
+    uint64_t* accempty = accfull + 2;
+    uint32_t* tmem_slot = (uint32_t*)(accempty + 2);
+    constexpr bool FLUSH = Cfg::FLUSH;
+    constexpr int GROUP = Cfg::GROUP;
     const int tid = threadIdx.x, wid = tid >> 5, lane = tid & 31;
     // A_ENV: two row tiles with different synthesized A operands (wall bits + ones row; one-hot of idx2), each with its own M space
     const int amode = AMODE == A_ENV ? (blockIdx.x == 0 ? A_WALLS : A_ONEHOT) : AMODE;
@@ -87,14 +100,15 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
     const uint8_t* oh_idx = (AMODE == A_ENV) ? g.idx2 : g.idx;
     const int kbeg = split * g.klen, kend = min(g.K, kbeg + g.klen);
     const int nchunks = kend > kbeg ? (kend - kbeg + KC - 1) / KC : 0;
+    const int ngroups = FLUSH ? (nchunks + GROUP - 1) / GROUP : (nchunks > 0 ? 1 : 0);
     constexpr uint32_t NBUILD = AMODE == A_PLANES ? 0u : 128u;
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&bars[s], 1 + NBUILD); tc::mbar_init(&bars[STAGES + s], 1); }
-        tc::mbar_init(&bars[2 * STAGES], 1);
+        for (int q = 0; q < 2; ++q) { tc::mbar_init(&accfull[q], 1); tc::mbar_init(&accempty[q], 128); }
         tc::mbar_fence_init();
     }
-    if (wid == 2) tc::tmem_alloc(tmem_slot, BN);
+    if (wid == 2) tc::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
@@ -131,7 +145,11 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
             const uint32_t idesc = tc::umma_idesc<PREC>(BM, BN, true, true);
             for (int c = 0; c < nchunks && ok; ++c) {
                 const int s = c % STAGES;
-                ok = tc::mbar_wait(&bars[s], (c / STAGES) & 1);
+                const int grp = FLUSH ? c / GROUP : 0, cg = FLUSH ? c - grp * GROUP : c;  // accumulator group, chunk within it
+                const uint32_t acc = tmem + (uint32_t)((grp & 1) * BN);
+                // the third and later groups reuse an accumulator: wait until the epilogue warps have read it out
+                if (FLUSH && cg == 0 && grp >= 2) ok = tc::mbar_wait(&accempty[grp & 1], ((grp >> 1) - 1) & 1);
+                if (ok) ok = tc::mbar_wait(&bars[s], (c / STAGES) & 1);
                 if (!ok) break;
                 tc::tc_fence_after();
                 unsigned char* sa = base + s * Cfg::STAGE;
@@ -141,15 +159,15 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
                     // 16 k rows = two 8-row groups = 2048 bytes further into every box
                     const uint64_t a_hi = tc::umma_desc(sa + k16 * 2048, Cfg::BOX, 1024);
                     const uint64_t b_hi = tc::umma_desc(sb + k16 * 2048, Cfg::BOX, 1024);
-                    uint32_t accum = (c > 0 || k16 > 0) ? 1u : 0u;
-                    if (APL == 2) { tc::umma(tmem, tc::umma_desc(sa + Cfg::A_PLANE + k16 * 2048, Cfg::BOX, 1024), b_hi, idesc, accum); accum = 1u; }
-                    if (BPL == 2) { tc::umma(tmem, a_hi, tc::umma_desc(sb + Cfg::B_PLANE + k16 * 2048, Cfg::BOX, 1024), idesc, accum); accum = 1u; }
-                    tc::umma(tmem, a_hi, b_hi, idesc, accum);
+                    uint32_t accum = (cg > 0 || k16 > 0) ? 1u : 0u;
+                    if (APL == 2) { tc::umma(acc, tc::umma_desc(sa + Cfg::A_PLANE + k16 * 2048, Cfg::BOX, 1024), b_hi, idesc, accum); accum = 1u; }
+                    if (BPL == 2) { tc::umma(acc, a_hi, tc::umma_desc(sb + Cfg::B_PLANE + k16 * 2048, Cfg::BOX, 1024), idesc, accum); accum = 1u; }
+                    tc::umma(acc, a_hi, b_hi, idesc, accum);
                 }
                 tc::umma_commit(&bars[STAGES + s]);  // frees the stage when these MMAs are done
+                if (c == nchunks - 1 || (FLUSH && cg == GROUP - 1)) tc::umma_commit(&accfull[grp & 1]);  // this group's sum is complete
             }
-            if (ok) tc::umma_commit(&bars[2 * STAGES]);
-            else atomicOr(status, DEV_E_WAIT_TIMEOUT);
+            if (!ok) atomicOr(status, DEV_E_WAIT_TIMEOUT);
         }
     } else {
         // ---- warps 2-5: builders of a synthesized A tile, then the epilogue
@@ -198,38 +216,52 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
             }
             if (!ok && lane == 0) atomicOr(status, DEV_E_WAIT_TIMEOUT);
         }
-        // epilogue: warp w reads accumulator lanes 32*(w%4)..+31 = output rows
-        bool got = true;
-        if (nchunks > 0) got = tc::mbar_wait(&bars[2 * STAGES], 0);
-        if (!got && lane == 0) atomicOr(status, DEV_E_WAIT_TIMEOUT);
-        tc::tc_fence_after();
-        __syncwarp();
+        // epilogue: warp w reads accumulator lanes 32*(w%4)..+31 = output rows.  Group 0 writes the partial tile, every
+        // later group adds to what this same thread wrote (program order; round-to-nearest additions in group order).
         const int q = wid & 3;
         const int m = m0 + 32 * q + lane;
         const bool second = AMODE == A_ENV && blockIdx.x == 1;
         const int Mrows = second ? g.M2 : g.M;
         float* part = second ? g.part2 + (size_t)split * g.stride2 : g.part + (size_t)split * g.stride + g.off;
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-            uint32_t r[32];
-            if (nchunks > 0 && got) {
-                tc::tmem_ld32(tmem + ((uint32_t)(32 * q) << 16) + (uint32_t)c0, r);
-            } else {
+        bool got = true;
+        for (int grp = 0; grp < (ngroups > 0 ? ngroups : 1); ++grp) {
+            if (ngroups > 0 && got) got = tc::mbar_wait(&accfull[grp & 1], (grp >> 1) & 1);
+            tc::tc_fence_after();
+            __syncwarp();
+            const uint32_t acc = tmem + (uint32_t)((grp & 1) * BN) + ((uint32_t)(32 * q) << 16);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                if (ngroups > 0 && got) {
+                    tc::tmem_ld32(acc + (uint32_t)c0, r);
+                } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = 0u;  // an empty K range contributes zeros
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;  // an empty K range contributes zeros
+                }
+                if (m < Mrows && n0 + c0 < g.N) {
+                    float4* dst = reinterpret_cast<float4*>(part + (size_t)m * g.ldc + n0 + c0);
+                    if (amode == A_WALLS && m == g.ones_row) dst = reinterpret_cast<float4*>(part - g.off + g.off_ones + n0 + c0);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
+                                               __uint_as_float(r[4 * j + 3]));
+                        if (grp > 0) {
+                            const float4 o = dst[j];
+                            v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                        }
+                        dst[j] = v;
+                    }
+                }
             }
-            if (m < Mrows && n0 + c0 < g.N) {
-                float4* dst = reinterpret_cast<float4*>(part + (size_t)m * g.ldc + n0 + c0);
-                if (amode == A_WALLS && m == g.ones_row) dst = reinterpret_cast<float4*>(part - g.off + g.off_ones + n0 + c0);
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    dst[j] = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]), __uint_as_float(r[4 * j + 2]),
-                                         __uint_as_float(r[4 * j + 3]));
+            if (FLUSH && grp + 2 < ngroups) {  // hand the accumulator back to the issuer
+                tc::tc_fence_before();
+                tc::mbar_arrive(&accempty[grp & 1]);
             }
         }
+        if (!got && lane == 0) atomicOr(status, DEV_E_WAIT_TIMEOUT);
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (wid == 2) tc::tmem_dealloc(tmem, BN);
+    if (wid == 2) tc::tmem_dealloc(tmem, Cfg::TMEM_COLS);
 }
 
 template <int BN, int AMODE, int APL, int BPL, int PREC>

@@ -856,7 +856,14 @@ __global__ void __launch_bounds__(256) k_adam_only(LearnArgs a) {
     }
     __syncthreads();
     const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
-    if (i < a.d.P) adam_step<PREC>(a, s_c, i, a.b.grads[i]);
+    if (i < a.d.P) {
+        float g = a.b.grads[i];
+        if (a.grad_div > 1.f) {  // the mean over the replicas (Section 3.1), taken where the sum is consumed
+            g = g / a.grad_div;
+            a.b.grads[i] = g;
+        }
+        adam_step<PREC>(a, s_c, i, g);
+    }
 }
 
 // ----------------------------------------------------------------------------------------------------

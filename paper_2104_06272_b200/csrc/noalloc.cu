@@ -117,3 +117,19 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     if (launch_rollout(a, cfg->precision, ctx) != cudaSuccess) return ANAKIN_E_CUDA;
     return ANAKIN_OK;
 }
+
+// The sticky status word of the last anakin_rollout_noalloc call on the current device lives in the array's tail, where
+// no caller can see it; this call brings it out (a 4-byte stream-ordered copy, then a stream synchronisation).
+extern "C" int anakin_noalloc_status(void* cuda_stream, int* device_status) {
+    if (!device_status) return ANAKIN_E_INVALID_ARG;
+    unsigned char* scratch = nullptr;
+    if (scratch_for_current_device(&scratch) != cudaSuccess) return ANAKIN_E_CUDA;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const unsigned char* tail = scratch + kMaxBaseFloats * sizeof(float) + kW2FragBytes + kW2PlaneBytes;
+    int st = 0;
+    cudaError_t e = cudaMemcpyAsync(&st, tail + 128, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return ANAKIN_E_CUDA;
+    *device_status = st;
+    return st == 0 ? ANAKIN_OK : ANAKIN_E_DEVICE_STATUS;
+}

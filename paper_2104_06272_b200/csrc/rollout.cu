@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(256) k_env_base(Dims d, Buffers b) {
     const int e = (int)(idx / H4), j4 = (int)(idx - (size_t)e * H4);
     const uint32_t* w = b.walls + (size_t)e * d.W;
     const float4* W1 = reinterpret_cast<const float4*>(b.theta_c + d.oW1) + j4;
-    const int goal_row = 2 * d.C + b.goal[e];
+    const int goal_row = 2 * d.C + min((int)b.goal[e], d.C - 1);  // (the rollout flags a goal outside the board)
     float4 acc = reinterpret_cast<const float4*>(b.theta_c + d.ob1)[j4];
     int wi = 0;
     uint32_t bits = w[0];
@@ -99,10 +99,20 @@ __global__ void __launch_bounds__(256) k_rollout(RolloutArgs a) {
             my_goal = b.goal[e0 + tid];
             for (int wi = 0; wi < 8; ++wi) s_walls[tid * 8 + wi] = wi < d.W ? b.walls[(size_t)(e0 + tid) * d.W + wi] : 0u;
         }
-        s_pos[tid] = my_pos;
     }
     unsigned long long n_episodes = 0, n_goals = 0, n_epsteps = 0;
     int bad = 0;
+    if (tid < ME) {
+        if (owner) {
+            EnvLane es;
+            es.pos = my_pos; es.tep = my_tep; es.start = my_start; es.goal = my_goal;
+            es.bad = 0;
+            check_env_state(es, C, s_walls + tid * 8);
+            my_pos = es.pos; my_start = es.start; my_goal = es.goal;
+            bad |= es.bad;
+        }
+        s_pos[tid] = my_pos;
+    }
     __syncthreads();
 
     for (int t = 0; t <= a.T; ++t) {

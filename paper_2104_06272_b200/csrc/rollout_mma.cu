@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(Rol
             s.tep = b.tep[e0 + tid];
             s.start = b.start[e0 + tid];
             s.goal = b.goal[e0 + tid];
+            check_env_state(s, C, s_walls + tid * 8);
         }
         s_pos[tid] = s.pos;
     }
@@ -148,7 +149,7 @@ __global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(Rol
     const int t_end = a.replay == 1 ? a.T - 1 : a.T;  // replay recomputes the T recorded rows (mode 2: and the current state)
     for (int t = 0; t <= t_end; ++t) {
         if (a.replay) {  // positions come from the recorded trajectory (row T: the env state as it stands)
-            if (tid < ME) s_pos[tid] = owner ? (t < a.T ? b.tpos[(size_t)t * B + e0 + tid] : b.pos[e0 + tid]) : 0;
+            if (tid < ME) s_pos[tid] = owner ? min((int)(t < a.T ? b.tpos[(size_t)t * B + e0 + tid] : b.pos[e0 + tid]), C - 1) : 0;
             __syncthreads();
         }
         // ---- layer 1: eight consecutive hidden units per thread and trip.  All gathers of the agent's W1 row are issued

@@ -150,6 +150,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg::THREADS, 1)
             s.tep = b.tep[e0 + ow];
             s.start = b.start[e0 + ow];
             s.goal = b.goal[e0 + ow];
+            check_env_state(s, C, s_walls + ow * 8);
         }
         s_pos[ow] = s.pos;
     }
@@ -165,7 +166,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg::THREADS, 1)
     const int t_end = a.replay == 1 ? a.T - 1 : a.T;  // replay recomputes the T recorded rows (mode 2: and the current state)
     for (int t = 0; t <= t_end; ++t) {
         if (a.replay) {  // positions come from the recorded trajectory
-            if (ow >= 0) s_pos[ow] = owner ? (t < a.T ? b.tpos[(size_t)t * B + e0 + ow] : b.pos[e0 + ow]) : 0;
+            if (ow >= 0) s_pos[ow] = owner ? min((int)(t < a.T ? b.tpos[(size_t)t * B + e0 + ow] : b.pos[e0 + ow]), C - 1) : 0;
             __syncthreads();
         }
         if (tid == NWT) tc::mbar_expect_tx(pfull, 8 * ME * 5 * 4);  // this step's head partials, counted as they land

@@ -21,9 +21,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait on a phase parity: gives up after about a second of SM clock and returns false (the caller raises the
-// sticky status word and unwinds: no wait in this library can spin forever).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Bounded wait on a phase parity: gives up after `limit_clocks` of SM clock (default: about a second) and returns false
+// (the caller raises the sticky status word and unwinds: no wait in this library can spin forever).
+constexpr long long kWaitLimitClocks = 2000000000LL;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit_clocks = kWaitLimitClocks) {
     const uint32_t addr = smem_u32(bar);
     const long long t0 = clock64();
     do {
@@ -33,7 +34,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
                      : "r"(addr), "r"(parity)
                      : "memory");
         if (ok) return true;
-    } while (clock64() - t0 < 2000000000LL);
+    } while (clock64() - t0 < limit_clocks);
     return false;
 }
 

@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(256) k_h1_wide(Dims d, Buffers b, const uint8_
         const size_t i = idx / H8;
         const int j8 = (int)(idx - i * H8);
         const int env = (int)(i % d.B);
-        const int p = pos[i];
+        const int p = min((int)pos[i], d.C - 1);  // a position handed in from outside stays inside the plane
         const float4* bp = reinterpret_cast<const float4*>(b.base + (size_t)env * H) + 2 * j8;
         const float4* wp = reinterpret_cast<const float4*>(W1a + (size_t)p * H) + 2 * j8;
         const float4 b0 = bp[0], b1 = bp[1], w0 = __ldg(wp), w1 = __ldg(wp + 1);
@@ -291,6 +291,7 @@ __global__ void __launch_bounds__(256) k_heads_wide(RolloutArgs a, int t, int mo
                 const int env = (int)i;
                 es.n_episodes = es.n_goals = es.n_epsteps = 0;
                 es.bad = 0;
+                check_env_state(es, d.C, s_walls[tid]);
                 act_and_step(es, a, env, t, o0, o1, o2, o3, s_walls[tid]);
                 b.pos[env] = (uint8_t)es.pos;
                 b.tep[env] = (uint8_t)es.tep;

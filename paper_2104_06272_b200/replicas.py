@@ -22,14 +22,14 @@ def shard_of(B: int, rank: int, world: int) -> tuple[int, int]:
     return rank * (B // world), B // world
 
 
-def mean_over_replicas_(flat: torch.Tensor, group=None, always: bool = False) -> torch.Tensor:
-    """In-place mean of a tensor over the ranks of `group` (sum all-reduce, then one division by the group size).
-    `always` runs the collective even in a group of one (to exercise the backend)."""
+def sum_over_replicas_(flat: torch.Tensor, group=None, always: bool = False) -> int:
+    """In-place SUM of a tensor over the ranks of `group` (one all-reduce); returns the group size, by which the
+    consumer divides (the library does that inside its Adam kernel: `apply_grads(n_replicas)`).  `always` runs the
+    collective even in a group of one (to exercise the backend)."""
     world = dist.get_world_size(group) if dist.is_initialized() else 1
     if world > 1 or (always and dist.is_initialized()):
         dist.all_reduce(flat, op=dist.ReduceOp.SUM, group=group)
-        flat.div_(world)
-    return flat
+    return world
 
 
 class ReplicatedAnakin:
@@ -50,12 +50,13 @@ class ReplicatedAnakin:
         an = self.an
         an.rollout()
         an.grads()
+        n = 1
         if self.world > 1 or self.always_exchange:
             with torch.cuda.stream(an.stream):  # the copies, the collective and Adam are ordered on the handle's stream
                 an.get_into(bnd.GRADS, self.gbuf)
-                mean_over_replicas_(self.gbuf, self.group, self.always_exchange)
+                n = sum_over_replicas_(self.gbuf, self.group, self.always_exchange)
                 an.set(bnd.GRADS, self.gbuf)
-        an.apply_grads()
+        an.apply_grads(n)  # the division by the number of replicas happens in the Adam kernel
 
     def run(self, iters: int):
         for _ in range(iters):

@@ -8,6 +8,7 @@ from oracle import binding as orc
 
 RTOL_FP32 = 1e-4
 RTOL_BF16 = 2e-2
+MARGINS: dict = {}  # name of the last compared tensors -> worst |error| / bound (printed by the full-size tests)
 
 
 def rtol_of(prec: int) -> float:
@@ -25,6 +26,8 @@ def assert_close(got, want, rtol, name):
     err = np.abs(got - want)
     bound = rtol * (np.abs(want) + rms)
     bad = err > bound
+    if want.size:
+        MARGINS[name] = float((err / np.maximum(bound, 1e-300)).max())  # worst error as a fraction of its bound
     if bad.any():
         i = int(np.argmax(err - bound))
         raise AssertionError(f"{name}: {int(bad.sum())}/{got.size} outside rtol={rtol}; worst at {i}: got {got[i]!r} "
@@ -120,9 +123,13 @@ def check_learn(an, bnd, w, st, g, gadv, gret):
     ograds, oloss, rep = orc.learn(w.N, w.H, w.precision, st["theta"], st["walls"], st["goal"], g["pos"], g["action"], gadv,
                                    gret, np.float32(w.value_coef), np.float32(w.entropy_coef), gates=(gates[0], gates[1]))
     for layer, r in rep.items():
-        # a gate may differ only where the pre-activation is within rounding of zero, and only rarely
+        # a gate may differ only where the pre-activation is within rounding of zero, and only rarely: fp32 and fp64 sums
+        # of O(1) terms differ by ~1e-7, so about 1e-7 of the gates can fall on the other side; 1e-5 of them (plus a floor
+        # for tiny cases) leaves two orders of margin and is far below one CTA tile of mis-gated units on any workload
         assert r["max_abs_z"] <= 10 * rtol * r["rms_z"], (layer, r)
-        assert r["mismatched"] <= 5 + 20 * rtol * R * w.H, (layer, r)
+        assert r["mismatched"] <= 10 + 1e-5 * R * w.H, (layer, r)
+    print(f"{w.name}: gate decisions differing from the oracle's own: layer1 {rep['layer1']['mismatched']}, "
+          f"layer2 {rep['layer2']['mismatched']} of {R * w.H} each")
     ggrads = an.get(bnd.GRADS)
     d = orc.Dims(w.N, w.H)
     for name, sl in d.slices().items():

@@ -96,6 +96,21 @@ def test_one_iteration_stage_by_stage(bnd, name):
     print(name, "near-boundary samples:", counts, counts2)
 
 
+def free_running_seed(ag, iters, learn=True):
+    """First seed for which the ORACLE's own free run draws no uniform within 1e-5 of a CDF boundary (about one sample in
+    17,000 does): on such a run the library has no excuse for a different action, so nothing needs to be skipped."""
+    for seed in range(1, 50):
+        ag.reset(seed)
+        clean = True
+        for _ in range(iters):
+            clean = clean and not ag.rollout().near.any()
+            if learn:
+                ag.learn()
+        if clean:
+            return seed
+    raise AssertionError("no seed without near-boundary samples")
+
+
 def test_tiny_free_running_end_to_end(bnd):
     """The tiny workload, both sides run freely for its 2 iterations from one seed: same actions, same
     trajectories, parameters within tolerance."""
@@ -104,16 +119,15 @@ def test_tiny_free_running_end_to_end(bnd):
     ag = orc.Agent(w.B, w.N, w.H, w.T, w.precision, w.episode_cap, w.wall_density, np.float32(w.gamma),
                    np.float32(w.gae_lambda), np.float32(w.entropy_coef), np.float32(w.value_coef), np.float32(w.lr),
                    np.float32(w.adam_b1), np.float32(w.adam_b2), np.float32(w.adam_eps))
-    an.reset(1)
-    ag.reset(1)
+    seed = free_running_seed(ag, w.iters)
+    an.reset(seed)
+    ag.reset(seed)
     for it in range(w.iters):
         an.rollout()
         tr = ag.rollout()
         g = par.gpu_traj(an, bnd, w.T)
-        mism = g["action"] != tr.action
-        assert not (mism & (tr.near == 0)).any()
-        if mism.any():
-            pytest.skip("a near-boundary sample diverged the free-running comparison")
+        assert not tr.near.any()
+        assert (g["action"] == tr.action).all()  # no sample of this run is near a CDF boundary: every action must agree
         assert (g["pos"] == tr.pos).all() and (g["reward"] == tr.reward).all() and (g["done"] == tr.done).all()
         par.assert_close(g["value"], tr.value, 1e-4, "values")
         an.learn()
@@ -142,7 +156,8 @@ def test_throughput_workload_full_size(bnd):
 def test_full_size_workloads_on_sampled_envs(bnd, name):
     """Full-size launches of the three large workloads.  The oracle replays a sample of envs for the acting
     stage and for GAE; the learner's full-batch gradient is checked through properties that hold at any size
-    (it is compared element by element on the reduced-batch versions above)."""
+    (it is compared element by element on the reduced-batch versions above and, at full size, in
+    test_full_size_learner_element_by_element)."""
     w = WORKLOADS[name]
     an = make(bnd, w)
     an.reset(2)
@@ -177,6 +192,66 @@ def test_full_size_workloads_on_sampled_envs(bnd, name):
     assert np.abs(step).max() <= w.lr * 1.01 and (step[grads == 0] == 0).all()
     assert an.status() == 0
     print(name, counts)
+
+
+@pytest.mark.parametrize("name", ["memory_bound", "large_batch", "tensor_core"])
+def test_full_size_learner_element_by_element(bnd, name):
+    """The three large workloads at their full sizes, in the launch configuration the benchmark times: one whole
+    update (gradient of every parameter block, loss terms, Adam moments, parameters, step) against the oracle run on
+    the library's full trajectory.  The split-K counts, wave counts and partial-buffer sizes the update takes at these
+    sizes occur nowhere else.  The oracle needs about 0.5-2.5 minutes of all host cores per case."""
+    w = WORKLOADS[name]
+    an = make(bnd, w)
+    an.reset(2)
+    an.set(bnd.PARAMS, random_params(5, w.P, 0.15 if w.H <= 256 else 0.05))  # non-zero biases
+    st = par.gpu_state(an, bnd)
+    an.rollout()
+    T = w.T
+    g = dict(pos=an.get(bnd.TRAJ_POS).reshape(T, w.B), action=an.get(bnd.TRAJ_ACTION).reshape(T, w.B),
+             done=an.get(bnd.TRAJ_DONE).reshape(T, w.B), reward=an.get(bnd.TRAJ_REWARD).reshape(T, w.B),
+             value=an.get(bnd.TRAJ_VALUE).reshape(T + 1, w.B))
+    gadv, gret = par.check_gae(an, bnd, w, g, T)  # the whole batch: the scan is cheap on the CPU too
+    par.MARGINS.clear()
+    try:
+        par.check_learn(an, bnd, w, st, g, gadv, gret)
+    finally:
+        print(name, "worst error / bound:", {k: round(v, 3) for k, v in par.MARGINS.items()})
+    assert an.status() == 0
+
+
+def test_bounded_device_wait_runs_out_and_reports(bnd):
+    """A device-side wait that cannot end must give up, raise the 'bounded wait gave up' bit and return; the context
+    stays usable and a reset clears the word.  The wait here is on a barrier nothing arrives on, with a short limit."""
+    w = SMALL["tp_ragged_256"]
+    an = make(bnd, w, debug=0)
+    an.reset(1)
+    an.rollout()
+    assert an.status() == 0
+    an.selftest_wait_timeout(2_000_000)  # about a millisecond of SM clock
+    assert an.status() == 4
+    an.learn()  # the context and the handle still work ...
+    assert np.isfinite(an.get(bnd.PARAMS)).all()
+    assert an.status() == 4  # ... and the word is sticky
+    an.reset(1)
+    assert an.status() == 0
+    with pytest.raises(bnd.AnakinError):
+        an.selftest_wait_timeout(0)
+
+
+def test_profiler_brackets_replay_launches(bnd):
+    """Per-kernel event timing around a PPO update of two epochs: the second epoch replays the forward pass once, and
+    its launch must be bracketed like every other (one 'replay' record, a finite duration)."""
+    w = SMALL["tp_ragged_128"]
+    an = make(bnd, w, debug=0)
+    an.reset(3)
+    an.rollout()
+    an.profile_enable(True)
+    an.learn_ppo(2, 0.2)
+    prof = an.profile_read()
+    an.profile_enable(False)
+    assert prof["replay"][1] == 1 and 0 < prof["replay"][0] < 100.0
+    assert prof["heads_bwd"][1] == 2
+    assert an.status() == 0
 
 
 def test_runs_are_bitwise_deterministic(bnd):
@@ -339,15 +414,13 @@ def test_torus_env_free_running_and_different_from_the_grid(bnd):
     ag = orc.Agent(w.B, w.N, w.H, w.T, w.precision, w.episode_cap, w.wall_density, np.float32(w.gamma),
                    np.float32(w.gae_lambda), np.float32(w.entropy_coef), np.float32(w.value_coef), np.float32(w.lr),
                    np.float32(w.adam_b1), np.float32(w.adam_b2), np.float32(w.adam_eps), kind=orc.TORUS)
-    an.reset(4)
-    ag.reset(4)
+    seed = free_running_seed(ag, 1, learn=False)
+    an.reset(seed)
+    ag.reset(seed)
     an.rollout()
     tr = ag.rollout()
     g = par.gpu_traj(an, bnd, w.T)
-    mism = g["action"] != tr.action
-    assert not (mism & (tr.near == 0)).any()
-    if mism.any():
-        pytest.skip("a near-boundary sample diverged the free-running comparison")
+    assert not tr.near.any() and (g["action"] == tr.action).all()
     assert (g["pos"] == tr.pos).all() and (g["reward"] == tr.reward).all() and (g["done"] == tr.done).all()
     # a wrap really happened: some recorded step changes the column by N-1 or the row by N-1
     pos = np.concatenate([tr.pos, an.get(bnd.ENV_POS)[None, :]], axis=0).astype(np.int64)
@@ -355,7 +428,7 @@ def test_torus_env_free_running_and_different_from_the_grid(bnd):
     moved_by_wrap = ((dr == w.N - 1) | (dc == w.N - 1)) & (tr.done == 0)
     assert moved_by_wrap.any()
     grid = make(bnd, w.scaled(env_kind=0))
-    grid.reset(4)
+    grid.reset(seed)
     grid.rollout()
     assert not (par.gpu_traj(grid, bnd, w.T)["pos"] == g["pos"]).all()
     an.learn()

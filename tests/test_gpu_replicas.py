@@ -13,6 +13,10 @@ CASES = {
     "mma_h64": WORKLOADS["tiny"].scaled(name="mma_h64", B=256, T=16),
     "ffma_h96": WORKLOADS["tiny"].scaled(name="ffma_h96", B=192, H=96, T=8),
     "wide_bf16": WORKLOADS["tensor_core"].scaled(name="wide_bf16", B=256, H=512, T=4),
+    # the kernels the large workloads run: the warp-level tensor rollout at H = 128 and the CTA-pair tcgen05 rollout at
+    # H = 256, each with a shard boundary (env_offset) that is not a multiple of its envs per CTA
+    "mma_h128": WORKLOADS["memory_bound"].scaled(name="mma_h128", B=2 * 176, T=12),
+    "pair_h256": WORKLOADS["throughput"].scaled(name="pair_h256", B=2 * 208, T=10),
 }
 
 
@@ -85,11 +89,13 @@ def test_two_shards_hold_the_envs_of_one_handle_and_their_mean_gradient_is_the_f
     rtol = 1e-5 if w.precision == 0 else 2e-3  # summation order only (bf16 workload: plus the split of the bf16-rounded sums)
     rms = np.sqrt((gfull**2).mean())
     assert (np.abs(gmean - gfull) <= rtol * (np.abs(gfull) + rms)).all()
-    # the exchange: every shard receives the mean, applies it, and the replicas stay identical
-    avg = torch.from_numpy(gmean.astype(np.float32)).cuda()
+    # the exchange: every shard receives the SUM (what the all-reduce leaves), the Adam kernel divides by the number of
+    # replicas, and the replicas stay identical
+    total = torch.from_numpy(shards[0].get(bnd.GRADS)).cuda() + torch.from_numpy(shards[1].get(bnd.GRADS)).cuda()
     for sh in shards:
-        sh.set(bnd.GRADS, avg)
-        sh.apply_grads()
+        sh.set(bnd.GRADS, total)
+        sh.apply_grads(G)
+        assert np.array_equal(sh.get(bnd.GRADS), (total / G).cpu().numpy())  # GRADS now reads as the mean
     assert np.array_equal(shards[0].get(bnd.PARAMS), shards[1].get(bnd.PARAMS))
     full.apply_grads()
     p_full, p_sh = full.get(bnd.PARAMS).astype(np.float64), shards[0].get(bnd.PARAMS).astype(np.float64)

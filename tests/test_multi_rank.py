@@ -51,7 +51,7 @@ def test_single_rank_needs_no_process_group():
 
 def _grad_worker(rank, world, port, out):
     """Rank r takes envs [r*B/2, (r+1)*B/2) of one recorded batch, computes the checker's gradient on its shard and
-    averages it with the exchange function the replicated driver uses."""
+    sums it with the exchange function the replicated driver uses."""
     sys.path.insert(0, ROOT)
     import numpy as np
 
@@ -74,8 +74,9 @@ def _grad_worker(rank, world, port, out):
         mine, _ = orc.learn(N, H, 0, theta, walls[sl], goal[sl], np.ascontiguousarray(tr.pos[:, sl]),
                             np.ascontiguousarray(tr.action[:, sl]), np.ascontiguousarray(adv[:, sl]), np.ascontiguousarray(ret[:, sl]))
         g = torch.from_numpy(mine.copy())
-        replicas.mean_over_replicas_(g)
-        out[rank] = (g.numpy().copy(), full, mine)
+        n = replicas.sum_over_replicas_(g)
+        assert n == world
+        out[rank] = (g.numpy().copy() / np.float32(n), full, mine)  # the library divides inside its Adam kernel
     finally:
         dist.destroy_process_group()
 

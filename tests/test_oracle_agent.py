@@ -310,6 +310,68 @@ def test_gradient_matches_central_finite_differences_fp64():
     assert not W1g[x.sum(0) == 0].any() and W1g[x.sum(0) > 0].any()
 
 
+def torch_bf16(a):
+    """Round to bf16 and back with torch's cast (the library routine on the other side of the pin)."""
+    return torch.from_numpy(np.ascontiguousarray(a, np.float32)).to(torch.bfloat16).to(torch.float32).numpy()
+
+
+def numpy_backward_bf16(theta, N, H, x, h1, h2, out, act, adv, ret, c_v, c_e, round_at=("dout", "dh2", "dh1")):
+    """The backward pass of the bf16 workload written out with matrix products in fp64: weights rounded to bf16, and the
+    three gradient-side GEMM inputs (output gradients, dh2, dh1) rounded to bf16 where `round_at` names them.  h1, h2
+    (already bf16 values) and the fp32 head outputs come from the forward pass."""
+    d = orc.Dims(N, H)
+    s = d.slices()
+    th = theta.copy()
+    for k in ("W1", "W2", "Wh"):
+        th[s[k]] = torch_bf16(theta[s[k]])
+    W1, b1, W2, b2, Wh, bh = [a.astype(np.float64) for a in unpack(th, N, H)]
+    R = x.shape[0]
+    rnd = lambda a, name: torch_bf16(a.astype(np.float32)).astype(np.float64) if name in round_at else a.astype(np.float32).astype(np.float64)
+    lg = torch.log_softmax(torch.from_numpy(out[:, :4].astype(np.float64)), dim=1).numpy()
+    p = np.exp(lg)
+    ent = -(p * lg).sum(1)
+    onehot = np.eye(4)[act]
+    dz = (-adv[:, None] * (onehot - p) + c_e * p * (lg + ent[:, None])) / R
+    dv = 2.0 * c_v * (out[:, 4].astype(np.float64) - ret) / R
+    dOut = rnd(np.concatenate([dz, dv[:, None]], axis=1), "dout")
+    g = np.zeros(d.P)
+    g[s["Wh"]] = (h2.astype(np.float64).T @ dOut).ravel()
+    g[s["bh"]] = dOut.sum(0)
+    dh2 = rnd((dOut @ Wh.T) * (h2 > 0), "dh2")
+    g[s["W2"]] = (h1.astype(np.float64).T @ dh2).ravel()
+    g[s["b2"]] = dh2.sum(0)
+    dh1 = rnd((dh2 @ W2.T) * (h1 > 0), "dh1")
+    g[s["W1"]] = (x.astype(np.float64).T @ dh1).ravel()
+    g[s["b1"]] = dh1.sum(0)
+    return g
+
+
+def test_bf16_backward_rounds_the_three_gemm_inputs():
+    """bf16 workload: the output gradients, dh2 and dh1 enter their products rounded to bf16 (and the bias gradients
+    sum the same rounded values).  The oracle's gradient equals the restatement with all three roundings, and differs
+    from each restatement that leaves one of them out, so none of the three can be dropped unnoticed."""
+    N, H, B, T = 5, 32, 6, 4
+    d = orc.Dims(N, H)
+    walls, goal, tpos, tact, adv, ret = tiny_batch(4, N=N, H=H, B=B, T=T)
+    adv, ret = adv.astype(np.float32), ret.astype(np.float32)
+    theta = random_params(9, d.P, 0.25)
+    x = np.stack([orc.observe(N, walls[b], int(tpos[t, b]), int(goal[b])) for t in range(T) for b in range(B)])
+    out, h1, h2 = orc.forward(N, H, 1, theta, x, want_hidden=True)
+    grads, _ = orc.learn(N, H, 1, theta, walls, goal, tpos, tact, adv, ret, 0.5, 0.01)
+    args = (theta, N, H, x, h1, h2, out, tact.ravel().astype(int), adv.ravel().astype(np.float64), ret.ravel().astype(np.float64), 0.5, 0.01)
+    want = numpy_backward_bf16(*args)
+    rms = np.sqrt((want**2).mean())
+    # double sums in another order, fp32 storage of the result; a bf16 tie decided the other way would show as 2^-9
+    assert np.abs(grads - want).max() <= 2e-6 * (np.abs(want).max() + rms)
+    sl = d.slices()
+    for left_out, blocks in (("dout", ("Wh", "bh")), ("dh2", ("W2", "b2")), ("dh1", ("W1", "b1"))):
+        kept = tuple(r for r in ("dout", "dh2", "dh1") if r != left_out)
+        other = numpy_backward_bf16(*args, round_at=kept)
+        for blk in blocks:  # the blocks fed directly by the unrounded tensor move by about a bf16 ulp (2^-9 relative)
+            diff = np.abs(grads[sl[blk]] - other[sl[blk]]).max()
+            assert diff > 1e-4 * np.abs(want[sl[blk]]).max(), (left_out, blk, diff)
+
+
 def test_gradient_structure_and_linearity_fp32():
     N, H = 5, 64
     d = orc.Dims(N, H)

@@ -44,6 +44,7 @@ def test_noalloc_rollout_matches_handle_rollout_twice_in_a_row():
                                  out["done"], out["reward"], out["value"], out["logp"])
         assert rc == bnd.OK
         assert n_allocs() == before  # torch's allocator saw nothing from the call
+        assert bnd.noalloc_status() == (bnd.OK, 0)  # the word in the array's tail, which no handle owns
         an.rollout(T)
         torch.cuda.synchronize()
         for name, blob in blobs.items():
@@ -54,6 +55,34 @@ def test_noalloc_rollout_matches_handle_rollout_twice_in_a_row():
             else:
                 assert (got == want).all(), (call, name)
         assert (pos.cpu().numpy() == an.get(bnd.ENV_POS)).all() and (tep.cpu().numpy() == an.get(bnd.ENV_TEP)).all()
+
+
+def test_noalloc_status_reports_a_start_position_on_a_wall():
+    """A caller-supplied env state that is not a legal one (the agent on a wall cell) must not pass silently: the kernels
+    flag it in the status word, and anakin_noalloc_status is the only way a handle-less caller can read that word."""
+    from paper_2104_06272_b200 import binding as bnd
+    from paper_2104_06272_b200.workloads import WORKLOADS, random_params
+
+    w = WORKLOADS["tiny"]
+    cfg = bnd.cfg_from_workload(w)
+    an = bnd.Anakin(cfg)
+    an.reset(5)
+    walls_h = an.get(bnd.ENV_WALLS).reshape(w.B, -1)
+    pos_h = an.get(bnd.ENV_POS).copy()
+    env = next(b for b in range(w.B) if walls_h[b].any())
+    cell = next(c for c in range(w.N * w.N) if (walls_h[env][c // 32] >> (c % 32)) & 1)
+    pos_h[env] = cell  # the agent of one env now stands on a wall
+    dev = lambda a: torch.from_numpy(a.view(np.int32) if a.dtype == np.uint32 else np.ascontiguousarray(a)).cuda()
+    T, B = w.T, w.B
+    u8 = lambda n: torch.empty(n, dtype=torch.uint8, device="cuda")
+    f32 = lambda n: torch.empty(n, dtype=torch.float32, device="cuda")
+    outs = (u8(T * B), torch.empty(T * B, dtype=torch.int8, device="cuda"), u8(T * B), f32(T * B), f32((T + 1) * B), f32(T * B))
+    ins = (dev(random_params(3, w.P, 0.15)), dev(an.get(bnd.ENV_WALLS)), dev(an.get(bnd.ENV_START)), dev(an.get(bnd.ENV_GOAL)))
+    for bad in (True, False):  # a clean call afterwards clears the word again
+        pos = dev(pos_h if bad else an.get(bnd.ENV_POS))
+        assert bnd.rollout_noalloc(cfg, 5, 0, T, *ins, pos, dev(an.get(bnd.ENV_TEP)), *outs) == bnd.OK
+        rc, st = bnd.noalloc_status()
+        assert (rc, st != 0) == ((bnd.E_DEVICE_STATUS, True) if bad else (bnd.OK, False)), (bad, rc, st)
 
 
 def test_noalloc_rollout_refuses_what_does_not_fit():
