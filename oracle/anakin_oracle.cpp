@@ -192,8 +192,10 @@ void observe(const Dims& d, const uint32_t* walls, uint8_t pos, uint8_t goal, S*
 // Parameter init: Xavier-uniform from Philox stream PARAM.  Flat index i draws
 // u = uniform24(word0 of counter (i,0,0)); w = (2u-1)*sqrt(6/(fan_in+fan_out)) evaluated in double and
 // rounded once.  Policy head columns use fan_out 4, the value column fan_out 1.  Biases are zero.
+// With many policies (independent networks trained side by side), policy p draws word 0 of counter (i,p,0): policy 0
+// is the single-policy initialisation.
 template <typename S>
-void param_init(uint64_t seed, const Dims& d, S* theta) {
+void param_init(uint64_t seed, const Dims& d, S* theta, uint32_t policy = 0) {
     for (size_t i = 0; i < d.P; ++i) {
         double bound = 0.0;
         if (i < d.ob1) bound = std::sqrt(6.0 / (double)(d.D + d.H));
@@ -206,7 +208,7 @@ void param_init(uint64_t seed, const Dims& d, S* theta) {
         } else bound = 0.0;
         if (bound == 0.0) { theta[i] = (S)0; continue; }
         uint32_t x[4];
-        philox_at(seed, (uint32_t)i, 0, 0, STREAM_PARAM, x);
+        philox_at(seed, (uint32_t)i, policy, 0, STREAM_PARAM, x);
         const double u = uniform24(x[0]);
         theta[i] = (S)((2.0 * u - 1.0) * bound);
     }
@@ -561,11 +563,13 @@ void orc_sample_from_logits(uint64_t seed, uint32_t gstep0, int T, int B, const 
 // state the action was taken in, the action, reward, done, value and log-probability.  After the last
 // step the value of the current state is stored in value[T][b] (the bootstrap).
 // Env dynamic state (pos, tep) is updated in place; the global step counter advances by T (caller).
-void orc_rollout_kind(int kind, int N, int H, int prec, int B, int T, int cap, const float* theta, const uint32_t* walls,
+// env0: global index of env 0 of this batch (the action uniform of env b is keyed by env0 + b), so that a slice of a
+// larger job (a replica's shard, one policy's envs) draws what the whole job would draw for those envs.
+void orc_rollout_env0(int kind, int N, int H, int prec, int B, int T, int cap, const float* theta, const uint32_t* walls,
                       const uint8_t* start, const uint8_t* goal, uint8_t* pos, uint8_t* tep, uint64_t seed,
                       uint32_t gstep0, const int8_t* forced /*nullable [T][B]*/, uint8_t* tpos, int8_t* tact,
                       uint8_t* tdone, float* trew, float* tval /*[T+1][B]*/, float* tlogp,
-                      float* tlogits /*nullable [T][B][4]*/, uint8_t* tnear /*nullable*/) {
+                      float* tlogits /*nullable [T][B][4]*/, uint8_t* tnear /*nullable*/, uint32_t env0) {
     const Dims d = make_dims(N, H);
     const std::vector<float> cp = compute_params(d, theta, prec);
 #pragma omp parallel
@@ -586,7 +590,7 @@ void orc_rollout_kind(int kind, int N, int H, int prec, int B, int T, int cap, c
                 int a;
                 float lp;
                 uint8_t nr;
-                sample4(out, act_uniform(seed, (uint32_t)b, gstep0 + (uint32_t)t), &a, &lp, &nr);
+                sample4(out, act_uniform(seed, env0 + (uint32_t)b, gstep0 + (uint32_t)t), &a, &lp, &nr);
                 if (forced) {
                     a = (int)forced[i];
                     lp = (float)softmax4(out).logp[a];
@@ -599,6 +603,15 @@ void orc_rollout_kind(int kind, int N, int H, int prec, int B, int T, int cap, c
             }
         }
     }
+}
+
+void orc_rollout_kind(int kind, int N, int H, int prec, int B, int T, int cap, const float* theta, const uint32_t* walls,
+                      const uint8_t* start, const uint8_t* goal, uint8_t* pos, uint8_t* tep, uint64_t seed,
+                      uint32_t gstep0, const int8_t* forced /*nullable [T][B]*/, uint8_t* tpos, int8_t* tact,
+                      uint8_t* tdone, float* trew, float* tval /*[T+1][B]*/, float* tlogp,
+                      float* tlogits /*nullable [T][B][4]*/, uint8_t* tnear /*nullable*/) {
+    orc_rollout_env0(kind, N, H, prec, B, T, cap, theta, walls, start, goal, pos, tep, seed, gstep0, forced, tpos, tact, tdone,
+                     trew, tval, tlogp, tlogits, tnear, 0u);
 }
 
 void orc_rollout(int N, int H, int prec, int B, int T, int cap, const float* theta, const uint32_t* walls,
@@ -684,6 +697,66 @@ void orc_learn_ppo_f64(int N, int H, int B, int T, const double* theta, const ui
                        const double* logp_old, double clip, double c_v, double c_e, double* grads, double* loss4) {
     loss_and_grad<double>(make_dims(N, H), 0, B, T, theta, walls, goal, tpos, tact, adv, ret, c_v, c_e, grads, loss4,
                           nullptr, nullptr, nullptr, logp_old, clip);
+}
+
+// ----------------------------------------------------------------------------------------------
+// Many policies: K independent networks, policy p acting in and learning from its own envs
+// [p*Bp, min(B, (p+1)*Bp)), Bp = ceil(B/K) (the shape of the paper's meta-learning use case, Section 4.1: many
+// small policies trained side by side on one accelerator).  Nothing couples the policies, so every function here
+// is literally a loop of K single-policy calls.  Layout: parameters and gradients [K][P]; per-env arrays [B] in
+// global env order; per-step arrays as K consecutive blocks, block p = [T][B_p] (values [T+1][B_p]) of policy p.
+// ----------------------------------------------------------------------------------------------
+static int policy_envs(int B, int K, int p, int* first) {
+    const int Bp = (B + K - 1) / K;
+    *first = p * Bp;
+    return std::min(Bp, B - p * Bp);
+}
+
+void orc_param_init_policy(uint64_t seed, int N, int H, uint32_t policy, float* theta) {
+    param_init(seed, make_dims(N, H), theta, policy);
+}
+
+void orc_rollout_policies(int kind, int N, int H, int prec, int B, int K, int T, int cap, const float* theta /*[K][P]*/,
+                          const uint32_t* walls, const uint8_t* start, const uint8_t* goal, uint8_t* pos, uint8_t* tep,
+                          uint64_t seed, uint32_t gstep0, uint8_t* tpos, int8_t* tact, uint8_t* tdone, float* trew,
+                          float* tval, float* tlogp, float* tlogits /*nullable*/, uint8_t* tnear /*nullable*/) {
+    const Dims d = make_dims(N, H);
+    for (int p = 0; p < K; ++p) {
+        int e0;
+        const int Bk = policy_envs(B, K, p, &e0);
+        const size_t o = (size_t)T * e0, ov = (size_t)(T + 1) * e0;  // every earlier block is a full one
+        orc_rollout_env0(kind, N, H, prec, Bk, T, cap, theta + (size_t)p * d.P, walls + (size_t)e0 * d.W, start + e0, goal + e0,
+                         pos + e0, tep + e0, seed, gstep0, nullptr, tpos + o, tact + o, tdone + o, trew + o, tval + ov, tlogp + o,
+                         tlogits ? tlogits + 4 * o : nullptr, tnear ? tnear + o : nullptr, (uint32_t)e0);
+    }
+}
+
+void orc_gae_policies(int T, int B, int K, double gamma, double lambda, const float* rew, const float* val,
+                      const uint8_t* done, float* adv, float* ret) {
+    for (int p = 0; p < K; ++p) {
+        int e0;
+        const int Bk = policy_envs(B, K, p, &e0);
+        const size_t o = (size_t)T * e0, ov = (size_t)(T + 1) * e0;
+        orc_gae(T, Bk, gamma, lambda, rew + o, val + ov, done + o, adv + o, ret + o);
+    }
+}
+
+// Each policy's gradient is the mean over ITS OWN B_p*T rows.  gates / gate_info as in orc_learn_f32, per policy:
+// gate bitmaps as K blocks [T*B_p][ceil(H/32)], gate_info [K][6].
+void orc_learn_policies(int N, int H, int prec, int B, int K, int T, const float* theta /*[K][P]*/, const uint32_t* walls,
+                        const uint8_t* goal, const uint8_t* tpos, const int8_t* tact, const float* adv, const float* ret,
+                        double c_v, double c_e, float* grads /*[K][P]*/, double* loss4 /*[K][4]*/,
+                        const uint32_t* gate1 /*nullable*/, const uint32_t* gate2 /*nullable*/, double* gate_info /*nullable*/) {
+    const Dims d = make_dims(N, H);
+    const size_t GW = (size_t)(H + 31) / 32;
+    for (int p = 0; p < K; ++p) {
+        int e0;
+        const int Bk = policy_envs(B, K, p, &e0);
+        const size_t o = (size_t)T * e0;
+        loss_and_grad<float>(d, prec, Bk, T, theta + (size_t)p * d.P, walls + (size_t)e0 * d.W, goal + e0, tpos + o, tact + o,
+                             adv + o, ret + o, c_v, c_e, grads + (size_t)p * d.P, loss4 + 4 * p, gate1 ? gate1 + o * GW : nullptr,
+                             gate2 ? gate2 + o * GW : nullptr, gate_info ? gate_info + 6 * p : nullptr);
+    }
 }
 
 // Adam (Kingma & Ba, Algorithm 1), k = step index AFTER the increment (first call: k = 1):

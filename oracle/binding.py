@@ -206,8 +206,10 @@ class Trajectory:
     near: np.ndarray  # u8 [T][B]  uniform within 1e-5 of a CDF boundary
 
 
-def rollout(N, H, prec, T, cap, theta, walls, start, goal, pos, tep, seed, gstep0, forced=None, kind: int = GRID) -> Trajectory:
-    """Runs T steps for all envs; pos/tep (uint8 arrays) are updated in place."""
+def rollout(N, H, prec, T, cap, theta, walls, start, goal, pos, tep, seed, gstep0, forced=None, kind: int = GRID,
+            env0: int = 0) -> Trajectory:
+    """Runs T steps for all envs; pos/tep (uint8 arrays) are updated in place.  env0 = global index of the batch's first
+    env (the action uniforms are keyed by env0 + b)."""
     B = walls.shape[0]
     tr = Trajectory(
         pos=np.zeros((T, B), np.uint8), action=np.zeros((T, B), np.int8), done=np.zeros((T, B), np.uint8),
@@ -216,11 +218,88 @@ def rollout(N, H, prec, T, cap, theta, walls, start, goal, pos, tep, seed, gstep
     if forced is not None:
         forced = np.ascontiguousarray(forced, dtype=np.int8)
         assert forced.shape == (T, B)
-    lib().orc_rollout_kind(C.c_int(kind), C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), C.c_int(cap), _p(theta),
+    lib().orc_rollout_env0(C.c_int(kind), C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(T), C.c_int(cap), _p(theta),
                            _p(walls), _p(start), _p(goal), _p(pos), _p(tep), C.c_uint64(seed), C.c_uint32(gstep0), _p(forced),
                            _p(tr.pos), _p(tr.action), _p(tr.done), _p(tr.reward), _p(tr.value), _p(tr.logp), _p(tr.logits),
-                           _p(tr.near))
+                           _p(tr.near), C.c_uint32(env0))
     return tr
+
+
+# ---- many policies: K independent networks, policy p on envs [p*Bp, min(B, (p+1)*Bp)), Bp = ceil(B/K) ----
+def policy_envs(B: int, K: int, p: int) -> tuple[int, int]:
+    """(first env, number of envs) of policy p."""
+    Bp = (B + K - 1) // K
+    return p * Bp, min(Bp, B - p * Bp)
+
+
+def param_init_policy(seed: int, N: int, H: int, policy: int) -> np.ndarray:
+    theta = np.zeros(Dims(N, H).P, dtype=np.float32)
+    lib().orc_param_init_policy(C.c_uint64(seed), C.c_int(N), C.c_int(H), C.c_uint32(policy), _p(theta))
+    return theta
+
+
+def block(a: np.ndarray, B: int, K: int, p: int, rows: int, width: int = 1) -> np.ndarray:
+    """Block p of a per-step array stored as K consecutive blocks [rows][B_p][width] (flat input), as [rows][B_p](,width)."""
+    e0, Bk = policy_envs(B, K, p)
+    v = a.reshape(-1)[rows * e0 * width: rows * (e0 + Bk) * width]
+    return v.reshape(rows, Bk, width) if width > 1 else v.reshape(rows, Bk)
+
+
+@dataclass
+class PolicyTrajectories:
+    """Flat arrays of K consecutive per-policy blocks (block p = [T][B_p]; value [T+1][B_p]; logits [T][B_p][4])."""
+    pos: np.ndarray
+    action: np.ndarray
+    done: np.ndarray
+    reward: np.ndarray
+    value: np.ndarray
+    logp: np.ndarray
+    logits: np.ndarray
+    near: np.ndarray
+
+
+def rollout_policies(K, N, H, prec, T, cap, theta, walls, start, goal, pos, tep, seed, gstep0, kind: int = GRID) -> PolicyTrajectories:
+    """K independent single-policy rollouts; theta [K][P]; pos/tep updated in place."""
+    B = walls.shape[0]
+    theta = np.ascontiguousarray(theta, np.float32)
+    assert theta.shape == (K, Dims(N, H).P) and (K - 1) * ((B + K - 1) // K) < B
+    tr = PolicyTrajectories(pos=np.zeros(T * B, np.uint8), action=np.zeros(T * B, np.int8), done=np.zeros(T * B, np.uint8),
+                            reward=np.zeros(T * B, np.float32), value=np.zeros((T + 1) * B, np.float32),
+                            logp=np.zeros(T * B, np.float32), logits=np.zeros(T * B * 4, np.float32), near=np.zeros(T * B, np.uint8))
+    lib().orc_rollout_policies(C.c_int(kind), C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(K), C.c_int(T), C.c_int(cap),
+                               _p(theta), _p(walls), _p(start), _p(goal), _p(pos), _p(tep), C.c_uint64(seed), C.c_uint32(gstep0),
+                               _p(tr.pos), _p(tr.action), _p(tr.done), _p(tr.reward), _p(tr.value), _p(tr.logp), _p(tr.logits), _p(tr.near))
+    return tr
+
+
+def gae_policies(K, B, T, gamma, lam, reward, value, done):
+    adv = np.zeros(T * B, np.float32)
+    ret = np.zeros(T * B, np.float32)
+    lib().orc_gae_policies(C.c_int(T), C.c_int(B), C.c_int(K), C.c_double(gamma), C.c_double(lam), _p(np.ascontiguousarray(reward, np.float32)),
+                           _p(np.ascontiguousarray(value, np.float32)), _p(np.ascontiguousarray(done, np.uint8)), _p(adv), _p(ret))
+    return adv, ret
+
+
+def learn_policies(K, N, H, prec, T, theta, walls, goal, tpos, tact, adv, ret, c_v=0.5, c_e=0.01, gates=None):
+    """K independent single-policy loss/gradient evaluations: (grads [K][P] f32, loss [K][4] f64[, gate reports])."""
+    B = walls.shape[0]
+    theta = np.ascontiguousarray(theta, np.float32)
+    grads = np.zeros((K, Dims(N, H).P), np.float32)
+    loss = np.zeros((K, 4), np.float64)
+    g1 = g2 = info = None
+    if gates is not None:
+        g1, g2 = np.ascontiguousarray(gates[0], np.uint32), np.ascontiguousarray(gates[1], np.uint32)
+        assert g1.size == g2.size == T * B * ((H + 31) // 32)
+        info = np.zeros((K, 6), np.float64)
+    lib().orc_learn_policies(C.c_int(N), C.c_int(H), C.c_int(prec), C.c_int(B), C.c_int(K), C.c_int(T), _p(theta), _p(walls), _p(goal),
+                             _p(np.ascontiguousarray(tpos, np.uint8)), _p(np.ascontiguousarray(tact, np.int8)),
+                             _p(np.ascontiguousarray(adv, np.float32)), _p(np.ascontiguousarray(ret, np.float32)), C.c_double(c_v),
+                             C.c_double(c_e), _p(grads), _p(loss), _p(g1), _p(g2), _p(info))
+    if gates is not None:
+        reports = [{"layer1": dict(mismatched=int(i[0]), max_abs_z=float(i[1]), rms_z=float(i[2])),
+                    "layer2": dict(mismatched=int(i[3]), max_abs_z=float(i[4]), rms_z=float(i[5]))} for i in info]
+        return grads, loss, reports
+    return grads, loss
 
 
 def gae(gamma: float, lam: float, reward: np.ndarray, value: np.ndarray, done: np.ndarray):
