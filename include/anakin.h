@@ -37,6 +37,16 @@
  *   W1[D][H], b1[H], W2[H][H], b2[H], Wh[H][5] (columns 0..3 logits, 4 value), bh[5];
  *   P = D*H + H + H*H + H + 5*H + 5.
  * Trajectory arrays are time-major: element (t, b) at index t*B + b.
+ *
+ * Many policies (anakin_cfg.n_policies = K >= 2).  Every kernel runs with one grid slice per policy on that policy's
+ * own sub-workspace; per policy the arithmetic is exactly the single-policy one (its gradient is the mean over ITS
+ * B_p*T rows, its Adam state is its own; parameter i of policy p is initialised from Philox counter (i, p, 0), so
+ * policy 0 is the single-policy initialisation).  Blobs then hold the K policies one after the other: PARAMS, GRADS,
+ * ADAM_M, ADAM_V as [K][P]; STATS as K anakin_stats; per-env blobs [B] in global env order; per-step blobs as K
+ * consecutive blocks, block p = the single-policy blob of policy p ([T][B_p], values [T+1][B_p]); forced actions
+ * likewise.  Supported: fp32, H in {64, 128, 256}, every policy non-empty ((K-1)*Bp < B), K <= 65535; reset, rollout,
+ * rollout_forced, gae, update, learn, run, grads, apply_grads, get/set, status.  anakin_learn_ppo, anakin_learn_vtrace
+ * and the no-allocation rollout return ANAKIN_E_UNSUPPORTED_CFG.
  */
 #ifndef ANAKIN_H_
 #define ANAKIN_H_
@@ -88,7 +98,10 @@ typedef struct anakin_cfg {
                              that G handles with B/G envs each and offsets 0, B/G, ... hold exactly the envs of one
                              handle with B envs (the replicas of Section 3.1, Figure 2 bottom) */
     int32_t env_kind;     /* ANAKIN_ENV_*: which `step` the envs run (same state, same observation planes) */
-    int32_t reserved;     /* must be 0 */
+    int32_t n_policies;   /* 0 or 1: one policy.  K >= 2: K independent networks trained side by side (the shape of the
+                             paper's meta-learning use case, Section 4.1: many small policies on one accelerator);
+                             policy p acts in and learns from envs [p*Bp, min(B, (p+1)*Bp)), Bp = ceil(B/K), and nothing
+                             couples the policies.  See "Many policies" below. */
 } anakin_cfg;
 
 /* Blob selectors for anakin_get / anakin_set.  Sizes in bytes for the LAST rollout length T (or T_max where noted). */

@@ -29,7 +29,7 @@ class AnakinCfg(C.Structure):
         ("episode_cap", C.c_int32), ("wall_density", C.c_double),
         ("gamma", C.c_float), ("gae_lambda", C.c_float), ("entropy_coef", C.c_float), ("value_coef", C.c_float),
         ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float),
-        ("precision", C.c_int32), ("device", C.c_int32), ("debug_logits", C.c_int32), ("env_offset", C.c_int32), ("env_kind", C.c_int32), ("reserved", C.c_int32),
+        ("precision", C.c_int32), ("device", C.c_int32), ("debug_logits", C.c_int32), ("env_offset", C.c_int32), ("env_kind", C.c_int32), ("n_policies", C.c_int32),
     ]
 
 
@@ -111,21 +111,21 @@ def lib() -> C.CDLL:
 
 def make_cfg(B, N, H, T_max, precision=0, episode_cap=50, wall_density=0.2, gamma=0.99, gae_lambda=0.95,
              entropy_coef=0.01, value_coef=0.5, lr=3e-4, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8, device=0,
-             debug_logits=0, env_offset=0, env_kind=0) -> AnakinCfg:
+             debug_logits=0, env_offset=0, env_kind=0, n_policies=0) -> AnakinCfg:
     c = AnakinCfg()
     c.struct_size = C.sizeof(AnakinCfg)
     c.B, c.N, c.H, c.T_max, c.episode_cap, c.wall_density = B, N, H, T_max, episode_cap, wall_density
     c.gamma, c.gae_lambda, c.entropy_coef, c.value_coef = gamma, gae_lambda, entropy_coef, value_coef
     c.lr, c.adam_b1, c.adam_b2, c.adam_eps = lr, adam_b1, adam_b2, adam_eps
     c.precision, c.device, c.debug_logits, c.env_offset = precision, device, debug_logits, env_offset
-    c.env_kind, c.reserved = env_kind, 0
+    c.env_kind, c.n_policies = env_kind, n_policies
     return c
 
 
 def cfg_from_workload(w, device=0, debug_logits=0, T_max=None, env_offset=0) -> AnakinCfg:
     return make_cfg(w.B, w.N, w.H, w.T if T_max is None else T_max, w.precision, w.episode_cap, w.wall_density, w.gamma,
                     w.gae_lambda, w.entropy_coef, w.value_coef, w.lr, w.adam_b1, w.adam_b2, w.adam_eps, device,
-                    debug_logits, env_offset, getattr(w, "env_kind", 0))
+                    debug_logits, env_offset, getattr(w, "env_kind", 0), getattr(w, "n_policies", 0))
 
 
 def workspace_bytes(cfg: AnakinCfg) -> int:
@@ -175,6 +175,7 @@ class Anakin:
         if rc != OK:
             raise AnakinError(rc)
         self.B, self.N, self.H, self.T_max = cfg.B, cfg.N, cfg.H, cfg.T_max
+        self.K = cfg.n_policies if cfg.n_policies >= 2 else 1  # independent policies; blobs hold them one after the other
         self.P = 3 * cfg.N * cfg.N * cfg.H + cfg.H + cfg.H * cfg.H + cfg.H + 5 * cfg.H + 5
 
     def _ck(self, rc: int):
@@ -238,6 +239,10 @@ class Anakin:
             self._ck(_lib.anakin_get(self._h, which, C.byref(v), 8, 0))
             return np.int64(v.value)
         if which == STATS:
+            if self.K > 1:  # one record per policy
+                arr = (AnakinStats * self.K)()
+                self._ck(_lib.anakin_get(self._h, which, arr, C.sizeof(arr), 0))
+                return list(arr)
             s = AnakinStats()
             self._ck(_lib.anakin_get(self._h, which, C.byref(s), C.sizeof(s), 0))
             return s
@@ -287,8 +292,20 @@ class Anakin:
     def launch_count(self) -> int:
         return int(_lib.anakin_launch_count(self._h))
 
-    def stats(self) -> AnakinStats:
+    def stats(self):
+        """The statistics record (a list of K records with many policies)."""
         return self.get(STATS)
+
+    def policy_envs(self, p: int) -> tuple[int, int]:
+        """(first env, number of envs) of policy p: ceil(B/K) envs each, the last policy takes the rest."""
+        bp = (self.B + self.K - 1) // self.K
+        return p * bp, min(bp, self.B - p * bp)
+
+    def policy_block(self, blob: np.ndarray, p: int, rows: int, width: int = 1) -> np.ndarray:
+        """Policy p's block of a per-step blob read with get() (K consecutive blocks [rows][B_p][width])."""
+        e0, n = self.policy_envs(p)
+        v = blob.reshape(-1)[rows * e0 * width: rows * (e0 + n) * width]
+        return v.reshape(rows, n, width) if width > 1 else v.reshape(rows, n)
 
     def profile_enable(self, on: bool):
         self._ck(_lib.anakin_profile_enable(self._h, 1 if on else 0))

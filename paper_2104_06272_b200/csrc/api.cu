@@ -25,6 +25,8 @@ struct anakin_handle {
     bool acts_valid;  // the saved h1/h2 belong to the pending trajectory and the current parameters
     int last_T;
     int NS;
+    int K;             // policies (>= 1)
+    size_t sub_bytes;  // size of one policy's sub-workspace
     uint64_t seed;
     int64_t gstep;
     int64_t adam_k;
@@ -42,7 +44,7 @@ int validate(const anakin_cfg* c) {
     if (c->B < 1 || c->T_max < 1 || c->episode_cap < 1 || c->episode_cap > 255) return ANAKIN_E_INVALID_ARG;
     if (!(c->wall_density >= 0.0 && c->wall_density < 1.0)) return ANAKIN_E_INVALID_ARG;
     if (c->precision != ANAKIN_PRECISION_FP32 && c->precision != ANAKIN_PRECISION_BF16) return ANAKIN_E_INVALID_ARG;
-    if (c->reserved != 0) return ANAKIN_E_INVALID_ARG;
+    if (c->n_policies < 0) return ANAKIN_E_INVALID_ARG;
     if (c->env_kind != ANAKIN_ENV_GRID && c->env_kind != ANAKIN_ENV_TORUS) return ANAKIN_E_UNSUPPORTED_CFG;
     if (c->env_offset < 0 || (double)c->env_offset + (double)c->B > 2147483647.0) return ANAKIN_E_INVALID_ARG;
     if (c->N < 2 || c->N > 16) return ANAKIN_E_UNSUPPORTED_CFG;
@@ -53,8 +55,16 @@ int validate(const anakin_cfg* c) {
         default: return ANAKIN_E_UNSUPPORTED_CFG;
     }
     if ((double)c->B * (double)c->T_max > 2.0e9) return ANAKIN_E_UNSUPPORTED_CFG;
+    if (c->n_policies >= 2) {  // many policies: fp32 on the warp-level tensor path, every policy with at least one env
+        const int K = c->n_policies, Bp = (c->B + K - 1) / K;
+        if (K > c->B || (long long)(K - 1) * Bp >= c->B) return ANAKIN_E_INVALID_ARG;
+        if (K > 65535 || c->precision != ANAKIN_PRECISION_FP32 || !rollout_mma_supported(c->H)) return ANAKIN_E_UNSUPPORTED_CFG;
+    }
     return ANAKIN_OK;
 }
+
+int policies_of(const anakin_cfg& c) { return c.n_policies >= 2 ? c.n_policies : 1; }
+int envs_per_policy(const anakin_cfg& c) { const int K = policies_of(c); return (c.B + K - 1) / K; }
 
 int choose_splits(const Dims& d) {
     const int tiles = ((d.H + 63) / 64) * ((d.H + 63) / 64);
@@ -142,10 +152,11 @@ struct Blob {
     bool is_traj;
 };
 
-Blob blob_of(anakin_t* h, int which) {
+// The blob of ONE policy with `envs` envs (the handle's Buffers are the first policy's).
+Blob blob_of(anakin_t* h, int which, int envs) {
     const Dims& d = h->d;
     const Buffers& b = h->b;
-    const size_t B = d.B, T = h->last_T > 0 ? h->last_T : d.Tmax, R = B * T, P = d.P;
+    const size_t B = (size_t)envs, T = h->last_T > 0 ? h->last_T : d.Tmax, R = B * T, P = d.P;
     switch (which) {
         case ANAKIN_PARAMS: return {b.theta, P * 4, true, false, false};
         case ANAKIN_GRADS: return {b.grads, P * 4, true, false, false};
@@ -171,6 +182,15 @@ Blob blob_of(anakin_t* h, int which) {
         case ANAKIN_DEBUG_GATES: return {b.dbg_gates, b.dbg_gates ? 2 * R * (size_t)(d.H / 32) * 4 : 0, false, false, false};
         default: return {nullptr, 0, false, false, false};
     }
+}
+
+int envs_of_policy(const anakin_t* h, int p) { return p == h->K - 1 ? h->d.B_last : h->d.B; }
+
+// Size of a blob over all policies (K consecutive single-policy blobs).
+size_t blob_total(anakin_t* h, int which) {
+    const Blob b0 = blob_of(h, which, h->d.B);
+    if (b0.host_only || h->K == 1) return b0.bytes;
+    return b0.bytes * (size_t)(h->K - 1) + blob_of(h, which, h->d.B_last).bytes;
 }
 
 // 16-bit copies of W2 in the layouts the tensor-core kernels read.
@@ -263,8 +283,8 @@ int anakin_workspace_bytes(const anakin_cfg* cfg, size_t* bytes) {
     if (!bytes) return ANAKIN_E_INVALID_ARG;
     const int rc = validate(cfg);
     if (rc != ANAKIN_OK) return rc;
-    const Dims d = make_dims(cfg->B, cfg->N, cfg->H, cfg->T_max);
-    *bytes = carve(*cfg, d, choose_splits(d), nullptr, nullptr);
+    const Dims d = make_dims(envs_per_policy(*cfg), cfg->N, cfg->H, cfg->T_max);
+    *bytes = carve(*cfg, d, choose_splits(d), nullptr, nullptr) * (size_t)policies_of(*cfg);  // one sub-workspace per policy
     return ANAKIN_OK;
 }
 
@@ -274,10 +294,14 @@ int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void
     const int rc = validate(cfg);
     if (rc != ANAKIN_OK) return rc;
     if (!dev_workspace || ((uintptr_t)dev_workspace & 255u)) return ANAKIN_E_INVALID_ARG;
-    Dims d = make_dims(cfg->B, cfg->N, cfg->H, cfg->T_max);
+    const int K = policies_of(*cfg), Bp = envs_per_policy(*cfg);
+    Dims d = make_dims(Bp, cfg->N, cfg->H, cfg->T_max);
     d.env0 = cfg->env_offset;
     const int NS = choose_splits(d);
-    const size_t need = carve(*cfg, d, NS, nullptr, nullptr);
+    const size_t sub = carve(*cfg, d, NS, nullptr, nullptr), need = sub * (size_t)K;
+    d.npol = K;
+    d.B_last = cfg->B - (K - 1) * Bp;
+    d.pstride = sub;
     if (bytes < need) return ANAKIN_E_WORKSPACE_TOO_SMALL;
     anakin_t* h = new (std::nothrow) anakin_t();
     if (!h) return ANAKIN_E_INVALID_ARG;
@@ -290,6 +314,8 @@ int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void
     h->cfg = *cfg;
     h->d = d;
     h->NS = NS;
+    h->K = K;
+    h->sub_bytes = sub;
     h->ws = (unsigned char*)dev_workspace;
     h->ws_bytes = bytes;
     h->stream = (cudaStream_t)cuda_stream;
@@ -422,6 +448,7 @@ int anakin_update(anakin_t* h) {
 
 int anakin_learn_ppo(anakin_t* h, int epochs, float clip_eps) {
     if (!h || epochs < 1 || !(clip_eps > 0.f)) return ANAKIN_E_INVALID_ARG;
+    if (h->K > 1) return ANAKIN_E_UNSUPPORTED_CFG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
     if (!h->adv_valid) {
         const int rc = anakin_gae(h);
@@ -437,7 +464,7 @@ int anakin_learn_ppo(anakin_t* h, int epochs, float clip_eps) {
 int anakin_learn_vtrace(anakin_t* h, int epochs, float rho_bar, float c_bar) {
     if (!h || epochs < 1 || !(rho_bar >= 0.f) || !(c_bar >= 0.f)) return ANAKIN_E_INVALID_ARG;
     if (!h->is_reset || !h->rollout_pending) return ANAKIN_E_BAD_STATE;
-    if (!tensor_path_supported(h->d.H, h->cfg.precision)) return ANAKIN_E_UNSUPPORTED_CFG;  // needs the saved head outputs
+    if (h->K > 1 || !tensor_path_supported(h->d.H, h->cfg.precision)) return ANAKIN_E_UNSUPPORTED_CFG;  // needs the saved head outputs
     for (int ep = 0; ep < epochs; ++ep) {
         cudaError_t e;
         if (!h->base_valid) {
@@ -514,13 +541,13 @@ int anakin_run(anakin_t* h, int iters) {
 
 size_t anakin_blob_bytes(anakin_t* h, int which) {
     if (!h) return 0;
-    return blob_of(h, which).bytes;
+    return blob_total(h, which);
 }
 
 static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is_device, bool to_lib) {
     if (!h || !ptr) return ANAKIN_E_INVALID_ARG;
-    const Blob bl = blob_of(h, which);
-    if (!bl.ptr || bl.bytes == 0 || bytes != bl.bytes) return ANAKIN_E_INVALID_ARG;
+    const Blob bl = blob_of(h, which, h->d.B);
+    if (!bl.ptr || bl.bytes == 0 || bytes != blob_total(h, which)) return ANAKIN_E_INVALID_ARG;
     if (to_lib && !bl.writable) return ANAKIN_E_INVALID_ARG;
     if (bl.host_only) {
         if (ptr_is_device) return ANAKIN_E_INVALID_ARG;
@@ -532,7 +559,16 @@ static int copy_blob(anakin_t* h, int which, void* ptr, size_t bytes, int ptr_is
     const cudaMemcpyKind kind = ptr_is_device == 1 ? cudaMemcpyDeviceToDevice
                               : ptr_is_device == 2 ? cudaMemcpyDefault
                               : (to_lib ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost);
-    cudaError_t e = to_lib ? cudaMemcpyAsync(bl.ptr, ptr, bytes, kind, h->stream) : cudaMemcpyAsync(ptr, bl.ptr, bytes, kind, h->stream);
+    cudaError_t e = cudaSuccess;
+    {   // one copy per policy: its blob sits at the same offset inside its sub-workspace
+        unsigned char* user = static_cast<unsigned char*>(ptr);
+        for (int p = 0; p < h->K && e == cudaSuccess; ++p) {
+            const size_t n = p == h->K - 1 ? blob_of(h, which, h->d.B_last).bytes : bl.bytes;
+            unsigned char* mine = static_cast<unsigned char*>(bl.ptr) + (size_t)p * h->sub_bytes;
+            e = to_lib ? cudaMemcpyAsync(mine, user, n, kind, h->stream) : cudaMemcpyAsync(user, mine, n, kind, h->stream);
+            user += n;
+        }
+    }
     if (e != cudaSuccess) return fail_cuda(h, e);
     if (to_lib) {
         if (which == ANAKIN_PARAMS) {

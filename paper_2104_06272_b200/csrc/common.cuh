@@ -5,6 +5,7 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <type_traits>
 #include <vector>
 
 #include "anakin.h"
@@ -23,11 +24,16 @@ struct Dims {
     int B, N, C, D, H, W, Tmax;  // envs, grid side, cells, obs features, hidden, wall words per env, max T
     int env0;                    // global index of env 0 (Philox counters use env0 + b)
     size_t oW1, ob1, oW2, ob2, oWh, obh, P;
+    // Many policies (independent networks side by side): npol sub-workspaces of identical layout, pstride bytes apart;
+    // policy p owns envs [env0 + p*B, ...): B envs each, B_last for the last policy.  npol <= 1: one policy.
+    int npol, B_last;
+    size_t pstride;
 };
 
 inline Dims make_dims(int B, int N, int H, int Tmax) {
     Dims d;
     d.env0 = 0;
+    d.npol = 1; d.B_last = B; d.pstride = 0;
     d.B = B; d.N = N; d.C = N * N; d.D = 3 * d.C; d.H = H; d.W = (d.C + 31) / 32; d.Tmax = Tmax;
     d.oW1 = 0;
     d.ob1 = d.oW1 + (size_t)d.D * H;
@@ -83,6 +89,30 @@ struct Buffers {
 };
 
 constexpr int LOSS_BLOCKS = 592;
+
+// ---- many policies: a kernel launched with one grid slice per policy moves every workspace pointer to its policy ----
+#ifdef __CUDACC__
+template <class T> __device__ __forceinline__ void shift_ptr(T*& p, size_t off) {
+    if (p) p = reinterpret_cast<T*>(reinterpret_cast<unsigned char*>(const_cast<typename std::remove_const<T>::type*>(p)) + off);
+}
+// All sub-buffers of a policy lie at the same offsets inside its sub-workspace.  The status word stays the first
+// policy's: one sticky word for the whole handle.
+__device__ __forceinline__ void shift_buffers(Buffers& b, size_t off) {
+    shift_ptr(b.theta, off); shift_ptr(b.theta_c, off); shift_ptr(b.grads, off); shift_ptr(b.adam_m, off); shift_ptr(b.adam_v, off);
+    shift_ptr(b.walls, off); shift_ptr(b.start, off); shift_ptr(b.goal, off); shift_ptr(b.pos, off); shift_ptr(b.tep, off);
+    shift_ptr(b.tpos, off); shift_ptr(b.tact, off); shift_ptr(b.tdone, off); shift_ptr(b.trew, off); shift_ptr(b.tval, off);
+    shift_ptr(b.tlogp, off); shift_ptr(b.adv, off); shift_ptr(b.ret, off); shift_ptr(b.dbg_logits, off); shift_ptr(b.dbg_gates, off);
+    shift_ptr(b.base, off); shift_ptr(b.w2f_hi, off); shift_ptr(b.w2f_lo, off); shift_ptr(b.w2tf_hi, off); shift_ptr(b.w2tf_lo, off);
+    shift_ptr(b.w2p_hi, off); shift_ptr(b.w2p_lo, off); shift_ptr(b.h1, off); shift_ptr(b.h2, off); shift_ptr(b.out5, off);
+    shift_ptr(b.vboot, off); shift_ptr(b.dh2, off); shift_ptr(b.dh1, off); shift_ptr(b.dout, off); shift_ptr(b.S, off);
+    shift_ptr(b.part, off); shift_ptr(b.loss_part, off); shift_ptr(b.stats, off);
+}
+__device__ __forceinline__ void select_policy(Dims& d, Buffers& b, int pol) {
+    shift_buffers(b, (size_t)pol * d.pstride);
+    d.env0 += pol * d.B;
+    if (pol == d.npol - 1) d.B = d.B_last;
+}
+#endif
 
 // ---- Philox4x32-10 (Salmon et al., SC'11) ----
 struct U4 { uint32_t x, y, z, w; };
@@ -171,6 +201,36 @@ struct LearnArgs {
     PartRegion reg[NREG];
 };
 
+#ifdef __CUDACC__
+__device__ __forceinline__ void select_policy(RolloutArgs& a, int pol) {
+    if (a.forced) a.forced += (size_t)pol * a.T * a.d.B;  // forced actions come as one [T][B_p] block per policy
+    select_policy(a.d, a.b, pol);
+}
+__device__ __forceinline__ void select_policy(LearnArgs& a, int pol) {
+    const size_t off = (size_t)pol * a.d.pstride;
+    shift_ptr(a.part_small, off);
+#pragma unroll
+    for (int q = 0; q < LearnArgs::NREG; ++q) shift_ptr(a.reg[q].part, off);
+    select_policy(a.d, a.b, pol);
+}
+// What a kernel body works with: the launch parameters themselves (GROUPED = false: nothing is copied), or a copy moved
+// to the policy of this grid slice.
+template <bool GROUPED, class A> struct PolicyArgs;
+template <class A> struct PolicyArgs<false, A> {
+    const A& a;
+    __device__ __forceinline__ PolicyArgs(const A& in, int) : a(in) {}
+};
+template <class A> struct PolicyArgs<true, A> {
+    A a;
+    __device__ __forceinline__ PolicyArgs(const A& in, int pol) : a(in) { select_policy(a, pol); }
+};
+struct DimsBuffers {
+    Dims d;
+    Buffers b;
+};
+__device__ __forceinline__ void select_policy(DimsBuffers& v, int pol) { select_policy(v.d, v.b, pol); }
+#endif
+
 // Split counts and partial-buffer layout of the tensor-pipe learner (a pure function of the sizes).
 struct LearnPlan {
     int ns_w2, ns_agent, ns_env, ns_small, loss_blocks, heads_grid;
@@ -242,7 +302,25 @@ struct GemmTnArgs {
     int M2;
     float* part2;
     size_t stride2;
+    // many policies (npol > 1): grid.z = policy * nsplit + split; every pointer above moves by pstride bytes per policy;
+    // the last policy has K_last rows (period kmod_last)
+    int npol, nsplit, K_last, kmod_last;
+    size_t pstride;
+    size_t alo_off_last, blo_off_last;  // Alo - Ahi and Blo - Bhi (elements) in the last policy's more compact planes
 };
+#ifdef __CUDACC__
+__device__ __forceinline__ void select_policy(GemmTnArgs& g, int pol) {
+    const size_t off = (size_t)pol * g.pstride;
+    shift_ptr(g.Ahi, off); shift_ptr(g.Alo, off); shift_ptr(g.idx, off); shift_ptr(g.walls, off); shift_ptr(g.Bhi, off);
+    shift_ptr(g.Blo, off); shift_ptr(g.part, off); shift_ptr(g.idx2, off); shift_ptr(g.part2, off);
+    if (pol == g.npol - 1) {
+        g.K = g.K_last;
+        g.kmod = g.kmod_last;
+        if (g.Alo) g.Alo = g.Ahi + g.alo_off_last;
+        if (g.Blo) g.Blo = g.Bhi + g.blo_off_last;
+    }
+}
+#endif
 
 // tcgen05 version (tensor memory accumulators, TMA-fed); cudaErrorNotSupported when the shape is not covered.
 cudaError_t launch_gemm_tn_tc(const GemmTnArgs& g, int amode, int apl, int bpl, int prec, int splits, int* status, cudaStream_t s);

@@ -35,8 +35,10 @@ struct HeadsCfg {
     static constexpr size_t smem_bytes = (size_t)NST * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + (size_t)TR * 8 * 4;
 };
 
-template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
-__global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a) {
+template <int H, int NW, int PREC, int HS = H, bool H2BF = false, bool GROUPED = false>
+__global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
+    const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.z);  // many policies: grid.z = policy
+    const LearnArgs& a = pa.a;
     using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
     constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = HS / 2, ESZ = Cfg::ESZ, NST = Cfg::NST;
     static_assert(NTHREADS / HP2 == 4, "four row groups of eight rows");
@@ -482,8 +484,10 @@ struct Dh1Cfg {
     static constexpr size_t smem_bytes = ((size_t)PL * BN * LDW + (size_t)STAGES * A_STAGE) * 2;
 };
 
-template <int H, int BN, int PREC>
-__global__ void __launch_bounds__(Dh1Cfg<H, BN, PREC>::THREADS, 1) k_dh1(LearnArgs a) {
+template <int H, int BN, int PREC, bool GROUPED = false>
+__global__ void __launch_bounds__(Dh1Cfg<H, BN, PREC>::THREADS, 1) k_dh1(LearnArgs a_in) {
+    const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.z);  // many policies: grid.z = policy
+    const LearnArgs& a = pa.a;
     using Cfg = Dh1Cfg<H, BN, PREC>;
     constexpr int NTH = Cfg::THREADS;
     constexpr int BM = Cfg::BM, KC = Cfg::KC, STAGES = Cfg::STAGES, PL = Cfg::PL, LDW = Cfg::LDW, LDA = Cfg::LDA;
@@ -658,8 +662,11 @@ struct GemmTnCfg {
     static constexpr int MT = WM / 16, NT = WN / 8;
 };
 
-template <int BM, int BN, int AMODE, int APL, int BPL, int PREC>
-__global__ void __launch_bounds__(256) k_gemm_tn(GemmTnArgs g) {
+template <int BM, int BN, int AMODE, int APL, int BPL, int PREC, bool GROUPED = false>
+__global__ void __launch_bounds__(256) k_gemm_tn(GemmTnArgs g_in) {
+    // many policies: grid.z = policy * nsplit + split
+    const PolicyArgs<GROUPED, GemmTnArgs> pa(g_in, GROUPED ? (int)blockIdx.z / g_in.nsplit : 0);
+    const GemmTnArgs& g = pa.a;
     using Cfg = GemmTnCfg<BM, BN, AMODE, APL, BPL, PREC>;
     constexpr int BK = Cfg::BK, STAGES = Cfg::STAGES, LDA = Cfg::LDA, LDB = Cfg::LDB, MT = Cfg::MT, NT = Cfg::NT;
     static_assert(NT % 2 == 0, "B fragments are loaded two n-tiles at a time");
@@ -668,7 +675,7 @@ __global__ void __launch_bounds__(256) k_gemm_tn(GemmTnArgs g) {
     __nv_bfloat16* sB = sA + STAGES * Cfg::A_STAGE;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int wm = wid >> 2, wn = wid & 3;
-    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, split = blockIdx.z;
+    const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, split = GROUPED ? (int)blockIdx.z % g.nsplit : (int)blockIdx.z;
     const int kbeg = split * g.klen, kend = min(g.K, kbeg + g.klen);
     const int ntiles = kend > kbeg ? (kend - kbeg + BK - 1) / BK : 0;
 
@@ -801,9 +808,22 @@ __global__ void __launch_bounds__(256) k_gemm_tn(GemmTnArgs g) {
 template <int BM, int BN, int AMODE, int APL, int BPL, int PREC>
 static cudaError_t launch_gemm_tn(const GemmTnArgs& g, int rows_m, int splits, cudaStream_t s) {
     using Cfg = GemmTnCfg<BM, BN, AMODE, APL, BPL, PREC>;
+    dim3 grid((rows_m + BM - 1) / BM, (g.N + BN - 1) / BN, splits);
+    if (g.npol > 1) {  // many policies: grid.z = policy * splits + split
+        if constexpr (PREC == 0) {
+            cudaError_t e = cudaFuncSetAttribute(k_gemm_tn<BM, BN, AMODE, APL, BPL, PREC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
+            if (e != cudaSuccess) return e;
+            if ((size_t)g.npol * splits > 65535) return cudaErrorNotSupported;
+            grid.z = g.npol * splits;
+            GemmTnArgs gg = g;
+            gg.nsplit = splits;
+            k_gemm_tn<BM, BN, AMODE, APL, BPL, PREC, true><<<grid, 256, Cfg::smem_bytes, s>>>(gg);
+            return cudaGetLastError();
+        }
+        return cudaErrorNotSupported;
+    }
     cudaError_t e = cudaFuncSetAttribute(k_gemm_tn<BM, BN, AMODE, APL, BPL, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
     if (e != cudaSuccess) return e;
-    dim3 grid((rows_m + BM - 1) / BM, (g.N + BN - 1) / BN, splits);
     k_gemm_tn<BM, BN, AMODE, APL, BPL, PREC><<<grid, 256, Cfg::smem_bytes, s>>>(g);
     return cudaGetLastError();
 }
@@ -847,8 +867,10 @@ __device__ __forceinline__ void adam_step(const LearnArgs& a, const float* c, si
 }
 
 // Adam from the GRADS blob as it stands (the second half of an update whose gradient was averaged over replicas).
-template <int PREC>
-__global__ void __launch_bounds__(256) k_adam_only(LearnArgs a) {
+template <int PREC, bool GROUPED>
+__global__ void __launch_bounds__(256) k_adam_only(LearnArgs a_in) {
+    const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.y);  // many policies: grid.y = policy
+    const LearnArgs& a = pa.a;
     __shared__ float s_c[2];
     if (threadIdx.x == 0) {
         s_c[0] = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
@@ -869,8 +891,11 @@ __global__ void __launch_bounds__(256) k_adam_only(LearnArgs a) {
 // ----------------------------------------------------------------------------------------------------
 // k_reduce_adam2: fixed-order sums of each parameter region's partials, then Adam (Kingma & Ba, Algorithm 1).
 // ----------------------------------------------------------------------------------------------------
-template <int PREC>
-__global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int loss_blocks) {
+template <int PREC, bool GROUPED>
+__global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_in, int loss_blocks) {
+    const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.y);  // many policies: grid.y = policy
+    const LearnArgs& a = pa.a;
+    const size_t R = GROUPED ? (size_t)a.d.B * a.T : R_in;  // rows of THIS policy
     __shared__ float s_c[2];
     const Dims& d = a.d;
     const Buffers& b = a.b;
@@ -966,7 +991,12 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a, size_t R, int
 }
 
 // Debug record of the ReLU gates from the saved activations (h1 hi plane, h2).
-__global__ void __launch_bounds__(256) k_pack_gates2(Dims d, Buffers b, size_t R, int h2_bf16) {
+template <bool GROUPED>
+__global__ void __launch_bounds__(256) k_pack_gates2(DimsBuffers in, size_t R_in, int h2_bf16) {
+    const PolicyArgs<GROUPED, DimsBuffers> pa(in, blockIdx.y);  // many policies: grid.y = policy
+    const Dims& d = pa.a.d;
+    const Buffers& b = pa.a.b;
+    const size_t R = GROUPED ? R_in / in.d.B * d.B : R_in;  // rows of THIS policy (R_in = B * T of a full one)
     const int lane = threadIdx.x & 31;
     const size_t words = R * (size_t)(d.H / 32);
     const __nv_bfloat16* h1hi = reinterpret_cast<const __nv_bfloat16*>(b.h1);
@@ -1050,6 +1080,14 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
 template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
 static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s) {
     using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
+    if (a.d.npol > 1) {
+        if constexpr (PREC == 0 && HS == H && !H2BF) {
+            CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
+            k_heads_bwd<H, NW, PREC, HS, H2BF, true><<<dim3(grid, 1, a.d.npol), NW * 32, Cfg::smem_bytes, s>>>(a);
+            return cudaGetLastError();
+        }
+        return cudaErrorNotSupported;
+    }
     CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
     k_heads_bwd<H, NW, PREC, HS, H2BF><<<dim3(grid, H / HS), NW * 32, Cfg::smem_bytes, s>>>(a);
     return cudaGetLastError();
@@ -1066,8 +1104,17 @@ static cudaError_t launch_heads_tc_t(const LearnArgs& a, int grid, cudaStream_t 
 template <int H, int BN, int PREC>
 static cudaError_t launch_dh1_t(const LearnArgs& a, cudaStream_t s) {
     using Cfg = Dh1Cfg<H, BN, PREC>;
-    CK(cudaFuncSetAttribute(k_dh1<H, BN, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
     dim3 grid((a.d.B + Cfg::BM - 1) / Cfg::BM, H / BN);
+    if (a.d.npol > 1) {
+        if constexpr (PREC == 0) {
+            CK(cudaFuncSetAttribute(k_dh1<H, BN, PREC, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
+            grid.z = a.d.npol;
+            k_dh1<H, BN, PREC, true><<<grid, Cfg::THREADS, Cfg::smem_bytes, s>>>(a);
+            return cudaGetLastError();
+        }
+        return cudaErrorNotSupported;
+    }
+    CK(cudaFuncSetAttribute(k_dh1<H, BN, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
     k_dh1<H, BN, PREC><<<grid, Cfg::THREADS, Cfg::smem_bytes, s>>>(a);
     return cudaGetLastError();
 }
@@ -1080,6 +1127,9 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     const size_t R = (size_t)B * T, RH = (size_t)B * d.Tmax * H;
     cudaStream_t s = c.s;
     const bool wide = wide_supported(H, PREC);  // bf16 activations in HBM, layer-2 products as large tcgen05 GEMMs
+    // many policies: every kernel gets one grid slice per policy and moves its workspace pointers there; the tcgen05
+    // kernels bake addresses into tensor maps, so this path stays on the warp-level kernels
+    const bool grouped = d.npol > 1;
     LearnPlan pl;
     learn_mma_plan(d, &pl);
     a.part_small = b.part + pl.off_small;
@@ -1117,7 +1167,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     // CTAs covers the SMs.  The mma.sync fall-back keeps one slice.
     a.ts = 1;
     bool fused_agent = false;  // dh1, S and the agent plane of dW1 in one kernel (dh1 stays on chip)
-    if (!wide && dh1_agent_tc_supported(d)) {
+    if (!wide && !grouped && dh1_agent_tc_supported(d)) {
         int gx, ts;
         dh1a_shape(d, T, &gx, &ts);
         a.ts = ts;
@@ -1144,7 +1194,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         CK(launch_dh1_wide(a, c));
     } else {
         Scope sc(c, K_DH1);
-        const cudaError_t etc = launch_dh1_tc(a, PREC, s);  // tcgen05 where covered, else the mma.sync kernel
+        const cudaError_t etc = grouped ? cudaErrorNotSupported : launch_dh1_tc(a, PREC, s);  // tcgen05 where covered, else the mma.sync kernel
         if (etc != cudaErrorNotSupported) CK(etc);
         else switch (H) {
             case 64: CK((launch_dh1_t<64, 64, PREC>(a, s))); break;
@@ -1161,14 +1211,20 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     auto klen_of = [](int K, int ns) { return ((K + ns - 1) / ns + 63) / 64 * 64; };
     GemmTnArgs g;
     memset(&g, 0, sizeof(g));
+    const size_t RH_last = (size_t)d.B_last * d.Tmax * H;  // plane offset inside the last policy's (more compact) buffers
+    if (grouped) { g.npol = d.npol; g.pstride = d.pstride; }
+    auto tc_gemm = [&](int amode, int apl, int bpl, int splits) {
+        return grouped ? cudaErrorNotSupported : launch_gemm_tn_tc(g, amode, apl, bpl, PREC, splits, b.status, s);
+    };
     // dW2 = h1^T dh2
     g.M = H; g.N = H; g.K = (int)R; g.klen = klen_of(g.K, pl.ns_w2);
     g.Ahi = h1hi; g.Alo = h1hi + RH; g.lda = H;
     g.Bhi = dh2hi; g.Blo = dh2hi + RH; g.ldb = H;
     g.part = b.part + pl.off_w2; g.stride = (size_t)H * H; g.off = 0; g.ldc = H; g.ones_row = -1;
+    g.K_last = d.B_last * T; g.kmod_last = 0; g.alo_off_last = g.blo_off_last = RH_last;
     {
         Scope sc(c, K_DW2);
-        cudaError_t e = launch_gemm_tn_tc(g, A_PLANES, PL, PL, PREC, pl.ns_w2, b.status, s);  // tcgen05 where covered
+        cudaError_t e = tc_gemm(A_PLANES, PL, PL, pl.ns_w2);  // tcgen05 where covered
         if (e == cudaErrorNotSupported) {
             if (H >= 128) e = launch_gemm_tn<128, 128, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s);
             else e = launch_gemm_tn<64, 64, A_PLANES, PL, PL, PREC>(g, H, pl.ns_w2, s);
@@ -1182,7 +1238,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     g.part = b.part + pl.off_agent; g.stride = CH; g.off = 0;
     if (!fused_agent) {
         Scope sc(c, K_DW1_AGENT);
-        cudaError_t e = launch_gemm_tn_tc(g, A_ONEHOT, 1, PL, PREC, pl.ns_agent, b.status, s);
+        cudaError_t e = tc_gemm(A_ONEHOT, 1, PL, pl.ns_agent);
         if (e == cudaErrorNotSupported) {
             if (H >= 128) e = launch_gemm_tn<128, 128, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s);
             else e = launch_gemm_tn<64, 64, A_ONEHOT, 1, PL, PREC>(g, C, pl.ns_agent, s);
@@ -1191,6 +1247,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     }
     // dW1, wall plane (+ db1 through the all-ones row) = walls^T S; goal plane = onehot(goal)^T S
     g.K = a.ts * B; g.kmod = B; g.klen = klen_of(g.K, pl.ns_env);
+    g.K_last = a.ts * d.B_last; g.kmod_last = d.B_last; g.blo_off_last = (size_t)a.ts * d.B_last * H;
     g.Bhi = Shi; g.Blo = Shi + (size_t)a.ts * B * H;
     g.walls = b.walls; g.W = d.W; g.ones_row = C; g.M = C + 1;
     g.part = b.part + pl.off_walls; g.stride = (size_t)(C + 1) * H; g.off = 0; g.off_ones = CH;
@@ -1198,14 +1255,14 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     if (PREC == 0) {  // both planes in one launch: row tile 0 = wall bits + ones row, row tile 1 = one-hot of the goal cell
         g.idx2 = b.goal; g.M2 = C; g.part2 = b.part + pl.off_goal; g.stride2 = CH;
         Scope sc(c, K_DW1_WALLS);
-        const cudaError_t e = launch_gemm_tn_tc(g, A_ENV, 1, 2, PREC, pl.ns_env, b.status, s);
+        const cudaError_t e = tc_gemm(A_ENV, 1, 2, pl.ns_env);
         if (e == cudaSuccess) env_planes_done = true;
         else if (e != cudaErrorNotSupported) return e;
     }
     if (!env_planes_done) {
         {
             Scope sc(c, K_DW1_WALLS);
-            cudaError_t e = launch_gemm_tn_tc(g, A_WALLS, 1, 2, PREC, pl.ns_env, b.status, s);
+            cudaError_t e = tc_gemm(A_WALLS, 1, 2, pl.ns_env);
             if (e == cudaErrorNotSupported) {
                 if (H >= 128) e = launch_gemm_tn<128, 128, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
                 else e = launch_gemm_tn<64, 64, A_WALLS, 1, 2, PREC>(g, C + 1, pl.ns_env, s);
@@ -1216,7 +1273,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         g.part = b.part + pl.off_goal; g.stride = CH;
         {
             Scope sc(c, K_DW1_GOAL);
-            cudaError_t e = launch_gemm_tn_tc(g, A_ONEHOT, 1, 2, PREC, pl.ns_env, b.status, s);
+            cudaError_t e = tc_gemm(A_ONEHOT, 1, 2, pl.ns_env);
             if (e == cudaErrorNotSupported) {
                 if (H >= 128) e = launch_gemm_tn<128, 128, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
                 else e = launch_gemm_tn<64, 64, A_ONEHOT, 1, 2, PREC>(g, C, pl.ns_env, s);
@@ -1227,12 +1284,18 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     {
         Scope sc(c, K_REDUCE_ADAM);
         const unsigned nb = (unsigned)((d.ob2 + 255) / 256 + (d.P - d.ob2 + 7) / 8);
-        k_reduce_adam2<PREC><<<nb, 256, 0, s>>>(a, R, pl.loss_blocks);
+        if (d.npol > 1) {
+            if constexpr (PREC == 0) k_reduce_adam2<PREC, true><<<dim3(nb, d.npol), 256, 0, s>>>(a, R, pl.loss_blocks);
+            else return cudaErrorNotSupported;
+        } else {
+            k_reduce_adam2<PREC, false><<<nb, 256, 0, s>>>(a, R, pl.loss_blocks);
+        }
         CK(cudaGetLastError());
     }
     if (b.dbg_gates) {
         Scope sc(c, K_PACK_GATES);
-        k_pack_gates2<<<148 * 8, 256, 0, s>>>(d, b, R, wide ? 1 : 0);
+        if (d.npol > 1) k_pack_gates2<true><<<dim3(64, d.npol), 256, 0, s>>>(DimsBuffers{d, b}, R, 0);
+        else k_pack_gates2<false><<<148 * 8, 256, 0, s>>>(DimsBuffers{d, b}, R, wide ? 1 : 0);
         CK(cudaGetLastError());
     }
     return cudaSuccess;
@@ -1241,8 +1304,11 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
 cudaError_t launch_adam_only(const LearnArgs& a, int prec, const Ctx& c) {
     Scope sc(c, K_REDUCE_ADAM);
     const unsigned nb = (unsigned)((a.d.P + 255) / 256);
-    if (prec == 1) k_adam_only<1><<<nb, 256, 0, c.s>>>(a);
-    else k_adam_only<0><<<nb, 256, 0, c.s>>>(a);
+    if (a.d.npol > 1) {
+        if (prec == 1) return cudaErrorNotSupported;
+        k_adam_only<0, true><<<dim3(nb, a.d.npol), 256, 0, c.s>>>(a);
+    } else if (prec == 1) k_adam_only<1, false><<<nb, 256, 0, c.s>>>(a);
+    else k_adam_only<0, false><<<nb, 256, 0, c.s>>>(a);
     return cudaGetLastError();
 }
 

@@ -57,6 +57,7 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     size_t unused = 0;
     const int rc = anakin_workspace_bytes(cfg, &unused);  // validates cfg; computes sizes only
     if (rc != ANAKIN_OK) return rc;
+    if (cfg->n_policies >= 2) return ANAKIN_E_UNSUPPORTED_CFG;  // one policy only
     if (!dev_params || !dev_walls || !dev_start || !dev_goal || !dev_pos || !dev_tep || !dev_traj_pos || !dev_traj_action ||
         !dev_traj_done || !dev_traj_reward || !dev_traj_value || !dev_traj_logp)
         return ANAKIN_E_INVALID_ARG;

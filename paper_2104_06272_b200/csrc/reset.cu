@@ -7,7 +7,11 @@ namespace anakin {
 
 // One thread per env.  Stream ENV: counter (b,0,0) -> start (word 0) and goal (word 1, among the other C-1
 // cells); counter (b,1+c/4,0) word (c%4) below floor(density*2^32) makes cell c a wall; start and goal stay free.
-__global__ void __launch_bounds__(128) k_reset_env(Dims d, Buffers b, uint32_t k0, uint32_t k1, uint32_t thr) {
+template <bool GROUPED>
+__global__ void __launch_bounds__(128) k_reset_env(DimsBuffers in, uint32_t k0, uint32_t k1, uint32_t thr) {
+    const PolicyArgs<GROUPED, DimsBuffers> pa(in, blockIdx.y);  // many policies: grid.y = policy
+    const Dims& d = pa.a.d;
+    const Buffers& b = pa.a.b;
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= d.B) return;
     const uint32_t ge = (uint32_t)(d.env0 + e);  // global env index
@@ -37,15 +41,20 @@ __global__ void __launch_bounds__(128) k_reset_env(Dims d, Buffers b, uint32_t k
 }
 
 // One thread per parameter.  Stream PARAM: u = uniform24(word 0 of counter (i,0,0));
-// w = (2u-1)*sqrt(6/(fan_in+fan_out)) evaluated in double, rounded once.  Biases are zero.
-__global__ void __launch_bounds__(256) k_reset_params(Dims d, Buffers b, uint32_t k0, uint32_t k1) {
+// w = (2u-1)*sqrt(6/(fan_in+fan_out)) evaluated in double, rounded once.  Biases are zero.  With many policies, policy p
+// draws counter (i,p,0): its own, independent initialisation (policy 0 = the single-policy one).
+template <bool GROUPED>
+__global__ void __launch_bounds__(256) k_reset_params(DimsBuffers in, uint32_t k0, uint32_t k1) {
+    const PolicyArgs<GROUPED, DimsBuffers> pa(in, blockIdx.y);
+    const Dims& d = pa.a.d;
+    const Buffers& b = pa.a.b;
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i == 0) {
         anakin_stats z;
         z.frames = z.episodes = z.goals = z.episode_steps = 0;
         z.loss_total = z.loss_pg = z.loss_value = z.entropy = 0.f;
         *b.stats = z;
-        *b.status = 0;
+        if (blockIdx.y == 0) *b.status = 0;
     }
     if (i >= d.P) return;
     double bound = 0.0;
@@ -56,7 +65,7 @@ __global__ void __launch_bounds__(256) k_reset_params(Dims d, Buffers b, uint32_
     else if (i < d.obh) bound = sqrt(6.0 / (double)(d.H + (((i - d.oWh) % 5) < 4 ? 4 : 1)));
     float w = 0.f;
     if (bound != 0.0) {
-        const U4 x = philox4x32_10((uint32_t)i, 0, 0, STREAM_PARAM, k0, k1);
+        const U4 x = philox4x32_10((uint32_t)i, GROUPED ? blockIdx.y : 0u, 0, STREAM_PARAM, k0, k1);
         const double u = (double)(x.x >> 8) * (1.0 / 16777216.0);
         w = (float)((2.0 * u - 1.0) * bound);
     }
@@ -88,13 +97,16 @@ cudaError_t launch_reset(const Dims& d, const Buffers& b, uint64_t seed, double 
     cudaError_t e;
     {
         Scope sc(c, K_RESET_ENV);
-        k_reset_env<<<(d.B + 127) / 128, 128, 0, c.s>>>(d, b, k0, k1, thr);
+        if (d.npol > 1) k_reset_env<true><<<dim3((d.B + 127) / 128, d.npol), 128, 0, c.s>>>(DimsBuffers{d, b}, k0, k1, thr);
+        else k_reset_env<false><<<(d.B + 127) / 128, 128, 0, c.s>>>(DimsBuffers{d, b}, k0, k1, thr);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return e;
     {
         Scope sc(c, K_RESET_PARAMS);
-        k_reset_params<<<(unsigned)((d.P + 255) / 256), 256, 0, c.s>>>(d, b, k0, k1);
+        const unsigned nb = (unsigned)((d.P + 255) / 256);
+        if (d.npol > 1) k_reset_params<true><<<dim3(nb, d.npol), 256, 0, c.s>>>(DimsBuffers{d, b}, k0, k1);
+        else k_reset_params<false><<<nb, 256, 0, c.s>>>(DimsBuffers{d, b}, k0, k1);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return e;

@@ -10,7 +10,11 @@ namespace anakin {
 // to the first layer is computed once per parameter version instead of once per step.
 // One thread owns four hidden units of one env; the W1 rows are fetched eight at a time (independent loads) and added in
 // ascending cell order, the goal row last.
-__global__ void __launch_bounds__(256) k_env_base(Dims d, Buffers b) {
+template <bool GROUPED>
+__global__ void __launch_bounds__(256) k_env_base(DimsBuffers in) {
+    const PolicyArgs<GROUPED, DimsBuffers> pa(in, blockIdx.y);  // many policies: grid.y = policy
+    const Dims& d = pa.a.d;
+    const Buffers& b = pa.a.b;
     const int H4 = d.H / 4;
     const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (idx >= (size_t)d.B * H4) return;
@@ -49,10 +53,14 @@ __global__ void __launch_bounds__(256) k_env_base(Dims d, Buffers b) {
 }
 
 cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c) {
-    const cudaError_t ew = launch_env_base_wide(d, b, c);  // tensor-core form where it applies
-    if (ew != cudaErrorNotSupported) return ew;
+    if (d.npol <= 1) {
+        const cudaError_t ew = launch_env_base_wide(d, b, c);  // tensor-core form where it applies
+        if (ew != cudaErrorNotSupported) return ew;
+    }
     Scope sc(c, K_ENV_BASE);
-    k_env_base<<<(unsigned)(((size_t)d.B * (d.H / 4) + 255) / 256), 256, 0, c.s>>>(d, b);
+    const unsigned nb = (unsigned)(((size_t)d.B * (d.H / 4) + 255) / 256);
+    if (d.npol > 1) k_env_base<true><<<dim3(nb, d.npol), 256, 0, c.s>>>(DimsBuffers{d, b});
+    else k_env_base<false><<<nb, 256, 0, c.s>>>(DimsBuffers{d, b});
     return cudaGetLastError();
 }
 
@@ -254,15 +262,19 @@ cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c) {
 // GAE reverse scan: lane = env, so every load and store of a warp is one contiguous segment per t.
 //   d_t = 1 - done_t; delta_t = r_t + gamma d_t V_{t+1} - V_t; A_t = delta_t + gamma lambda d_t A_{t+1}; ret = A + V
 // ----------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128) k_gae(Dims d, Buffers b, int T, float gamma, float lambda) {
+template <bool GROUPED>
+__global__ void __launch_bounds__(128) k_gae(DimsBuffers in, int T, float gamma, float lambda) {
+    const PolicyArgs<GROUPED, DimsBuffers> pa(in, blockIdx.y);
+    const Dims& d = pa.a.d;
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= d.B) return;
-    gae_scan_env(b, d.B, T, e, gamma, lambda);
+    gae_scan_env(pa.a.b, d.B, T, e, gamma, lambda);
 }
 
 cudaError_t launch_gae(const Dims& d, const Buffers& b, int T, float gamma, float lambda, const Ctx& c) {
     Scope sc(c, K_GAE);
-    k_gae<<<(d.B + 127) / 128, 128, 0, c.s>>>(d, b, T, gamma, lambda);
+    if (d.npol > 1) k_gae<true><<<dim3((d.B + 127) / 128, d.npol), 128, 0, c.s>>>(DimsBuffers{d, b}, T, gamma, lambda);
+    else k_gae<false><<<(d.B + 127) / 128, 128, 0, c.s>>>(DimsBuffers{d, b}, T, gamma, lambda);
     return cudaGetLastError();
 }
 

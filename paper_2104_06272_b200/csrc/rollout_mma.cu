@@ -16,8 +16,11 @@ namespace anakin {
 
 // B fragments of W2 for mma.m16n8k16 (.col B): entry [(ks*(H/8) + nt)*32 + lane] holds, for g = lane/4, t = lane%4,
 // n = 8*nt + g:  x = {W2[16ks+2t][n], W2[16ks+2t+1][n]},  y = {W2[16ks+2t+8][n], W2[16ks+2t+9][n]}  (low half first).
-template <int PREC>
-__global__ void __launch_bounds__(256) k_pack_w2(Dims d, Buffers b) {
+template <int PREC, bool GROUPED>
+__global__ void __launch_bounds__(256) k_pack_w2(DimsBuffers in) {
+    const PolicyArgs<GROUPED, DimsBuffers> pa(in, blockIdx.y);  // many policies: grid.y = policy
+    const Dims& d = pa.a.d;
+    const Buffers& b = pa.a.b;
     const int H = d.H;
     const int total = H * H / 4;
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -53,8 +56,12 @@ __global__ void __launch_bounds__(256) k_pack_w2(Dims d, Buffers b) {
 cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c) {
     if (!b.w2f_hi) return cudaSuccess;
     Scope sc(c, K_PACK_W2);
-    if (prec == 1) k_pack_w2<1><<<(d.H * d.H / 4 + 255) / 256, 256, 0, c.s>>>(d, b);
-    else k_pack_w2<0><<<(d.H * d.H / 4 + 255) / 256, 256, 0, c.s>>>(d, b);
+    const unsigned nb = (d.H * d.H / 4 + 255) / 256;
+    if (d.npol > 1) {
+        if (prec == 1) return cudaErrorNotSupported;
+        k_pack_w2<0, true><<<dim3(nb, d.npol), 256, 0, c.s>>>(DimsBuffers{d, b});
+    } else if (prec == 1) k_pack_w2<1, false><<<nb, 256, 0, c.s>>>(DimsBuffers{d, b});
+    else k_pack_w2<0, false><<<nb, 256, 0, c.s>>>(DimsBuffers{d, b});
     return cudaGetLastError();
 }
 
@@ -78,8 +85,10 @@ struct RolloutMmaCfg {
     static constexpr size_t gae_bytes(int T) { return (size_t)(T + 1) * ME * 4 + (size_t)T * ME; }
 };
 
-template <int H, int NW, int PREC>
-__global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(RolloutArgs a) {
+template <int H, int NW, int PREC, bool GROUPED>
+__global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(RolloutArgs a_in) {
+    const PolicyArgs<GROUPED, RolloutArgs> pa(a_in, blockIdx.y);  // many policies: grid.y = policy
+    const RolloutArgs& a = pa.a;
     using Cfg = RolloutMmaCfg<H, NW, PREC>;
     constexpr int ME = Cfg::ME, NT = Cfg::NT, KS = Cfg::KS, LD = Cfg::LD, NTHREADS = NW * 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -342,7 +351,7 @@ __global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(Rol
 
 constexpr size_t MAX_DYN_SMEM = 232448;  // 227 KB of dynamic shared memory per CTA
 
-template <int H, int NW, int PREC>
+template <int H, int NW, int PREC, bool GROUPED = false>
 static cudaError_t launch_t(const RolloutArgs& a0, cudaStream_t s) {
     using Cfg = RolloutMmaCfg<H, NW, PREC>;
     RolloutArgs a = a0;
@@ -352,9 +361,10 @@ static cudaError_t launch_t(const RolloutArgs& a0, cudaStream_t s) {
         a.gae_smem = 1;
         smem += Cfg::gae_bytes(a.T);
     }
-    cudaError_t e = cudaFuncSetAttribute(k_rollout_mma<H, NW, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MAX_DYN_SMEM);
+    cudaError_t e = cudaFuncSetAttribute(k_rollout_mma<H, NW, PREC, GROUPED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)MAX_DYN_SMEM);
     if (e != cudaSuccess) return e;
-    k_rollout_mma<H, NW, PREC><<<(a.d.B + Cfg::ME - 1) / Cfg::ME, NW * 32, smem, s>>>(a);
+    const dim3 grid((a.d.B + Cfg::ME - 1) / Cfg::ME, GROUPED ? a.d.npol : 1);
+    k_rollout_mma<H, NW, PREC, GROUPED><<<grid, NW * 32, smem, s>>>(a);
     return cudaGetLastError();
 }
 
@@ -363,6 +373,15 @@ bool rollout_mma_supported(int H) { return H == 64 || H == 128 || H == 256; }
 // Returns cudaErrorNotSupported when the shape is not covered by the tensor-pipe kernel.
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
     if (!a.b.w2f_hi || !rollout_mma_supported(a.d.H)) return cudaErrorNotSupported;
+    if (a.d.npol > 1) {  // many policies: one grid slice per policy, each with its own weights on chip
+        if (prec != 0) return cudaErrorNotSupported;
+        switch (a.d.H) {
+            case 64: return launch_t<64, 4, 0, true>(a, s);
+            case 128: return launch_t<128, 8, 0, true>(a, s);
+            case 256: return launch_t<256, 8, 0, true>(a, s);
+        }
+        return cudaErrorNotSupported;
+    }
     if (prec == 0) {  // the CTA-pair kernel on the 5th-generation tensor cores where it covers the shape
         const cudaError_t e = launch_rollout_pair(a, s);
         if (e != cudaErrorNotSupported) return e;

@@ -33,6 +33,7 @@ class Workload:
     adam_b2: float = 0.999
     adam_eps: float = 1e-8
     env_kind: int = 0  # 0 = gridworld (borders block), 1 = torus (borders wrap around)
+    n_policies: int = 0  # 0 or 1 = one policy; K >= 2 = K independent networks, policy p on envs [p*ceil(B/K), ...)
 
     @property
     def C(self):

@@ -54,7 +54,6 @@ def check_rollout(an, bnd, w, seed, st, T, forced=None, envs=None):
     state.  Transitions are bit-exact; logits/values/logp within tolerance; the GPU's actions equal the
     oracle's samples from the GPU's own logits except where the uniform is within 1e-5 of a CDF
     boundary.  `envs` restricts the oracle's replay to a subset of env indices (full-size workloads)."""
-    rtol = rtol_of(w.precision)
     if forced is None:
         an.rollout(T)
     else:
@@ -63,7 +62,17 @@ def check_rollout(an, bnd, w, seed, st, T, forced=None, envs=None):
         an.rollout_forced(torch.from_numpy(forced).cuda())
     g = gpu_traj(an, bnd, T)
     assert an.status() == 0
-    sel = np.arange(an.B) if envs is None else np.asarray(envs)
+    assert int(an.get(bnd.GLOBAL_STEP)) == st["gstep"] + T
+    counts = compare_rollout(w, seed, st, g, T, an.get(bnd.ENV_POS), an.get(bnd.ENV_TEP), forced=forced, envs=envs)
+    return g, counts
+
+
+def compare_rollout(w, seed, st, g, T, final_pos, final_tep, forced=None, envs=None, env0=0):
+    """The comparisons of check_rollout on arrays already read from the library: st = state before the rollout, g = the
+    recorded trajectory, final_pos / final_tep = env state after it.  env0 = global index of the batch's first env."""
+    rtol = rtol_of(w.precision)
+    B = g["pos"].shape[1]
+    sel = np.arange(B) if envs is None else np.asarray(envs)
     pos, tep = st["pos"][sel].copy(), st["tep"][sel].copy()
     tr = orc.rollout(w.N, w.H, w.precision, T, w.episode_cap, st["theta"], np.ascontiguousarray(st["walls"][sel]),
                      st["start"][sel].copy(), st["goal"][sel].copy(), pos, tep, seed, st["gstep"],
@@ -73,15 +82,14 @@ def check_rollout(an, bnd, w, seed, st, T, forced=None, envs=None):
     assert (g["pos"][:, sel] == tr.pos).all(), "recorded positions differ"
     assert (g["reward"][:, sel] == tr.reward).all(), "rewards differ"
     assert (g["done"][:, sel] == tr.done).all(), "done flags differ"
-    assert (an.get(bnd.ENV_POS)[sel] == pos).all() and (an.get(bnd.ENV_TEP)[sel] == tep).all(), "final env state differs"
-    assert int(an.get(bnd.GLOBAL_STEP)) == st["gstep"] + T
+    assert (final_pos[sel] == pos).all() and (final_tep[sel] == tep).all(), "final env state differs"
     assert_close(g["logits"][:, sel], tr.logits, rtol, "logits")
     assert_close(g["value"][:, sel], tr.value, rtol, "values")
     assert_close(g["logp"][:, sel], tr.logp, rtol, "logp")
     n_near = n_mis = 0
     if forced is None:
         # sample from the GPU's own logits with the same uniforms
-        if envs is None:
+        if envs is None and env0 == 0:
             act, logp, near = orc.sample_from_logits(seed, st["gstep"], g["logits"])
         else:
             act = np.zeros((T, len(sel)), np.int8)
@@ -89,7 +97,7 @@ def check_rollout(an, bnd, w, seed, st, T, forced=None, envs=None):
             near = np.zeros((T, len(sel)), np.uint8)
             for t in range(T):
                 for j, b in enumerate(sel):
-                    a, lp, nr = orc.sample_one(g["logits"][t, b], orc.act_uniform(seed, int(b), st["gstep"] + t))
+                    a, lp, nr = orc.sample_one(g["logits"][t, b], orc.act_uniform(seed, env0 + int(b), st["gstep"] + t))
                     act[t, j], logp[t, j], near[t, j] = a, lp, nr
         mism = act != g["action"][:, sel]
         n_near, n_mis = int(near.sum()), int(mism.sum())
@@ -97,7 +105,7 @@ def check_rollout(an, bnd, w, seed, st, T, forced=None, envs=None):
         assert n_mis <= max(1, int(1e-4 * mism.size)), f"{n_mis} action mismatches in {mism.size} samples"
         ok = ~mism
         assert_close(g["logp"][:, sel][ok], logp[ok], 1e-4 if w.precision == 0 else 1e-4, "logp of sampled action")
-    return g, dict(near=n_near, mismatched=n_mis)
+    return dict(near=n_near, mismatched=n_mis)
 
 
 def check_gae(an, bnd, w, g, T):
@@ -114,12 +122,21 @@ def check_learn(an, bnd, w, st, g, gadv, gret):
     parameters.  Gradients and loss terms are compared directly; Adam is compared on the GPU's own
     gradient (its early steps are close to lr*sign(g), which would otherwise turn a 1e-7 gradient
     difference on a near-zero element into a full-size parameter difference)."""
-    rtol = rtol_of(w.precision)
     an.learn()
+    R = g["pos"].size
+    gates = an.get(bnd.DEBUG_GATES).reshape(2, R, w.H // 32)
+    s = an.stats()
+    new = dict(k=int(an.get(bnd.ADAM_STEP)), m=an.get(bnd.ADAM_M), v=an.get(bnd.ADAM_V), theta=an.get(bnd.PARAMS))
+    return compare_learn(w, st, g, gadv, gret, an.get(bnd.GRADS), gates, [s.loss_total, s.loss_pg, s.loss_value, s.entropy], new)
+
+
+def compare_learn(w, st, g, gadv, gret, ggrads, gates, gloss, new):
+    """The comparisons of check_learn on arrays already read from the library: ggrads = GRADS, gates = the recorded ReLU
+    gates [2][R][H/32], gloss = (total, pg, value, entropy), new = Adam step count, moments and parameters after it."""
+    rtol = rtol_of(w.precision)
     # ReLU gates are floating-point decisions: the oracle's backward pass takes them as the library recorded
     # them (the kernel's precision), and reports where they differ from its own
     R = g["pos"].size
-    gates = an.get(bnd.DEBUG_GATES).reshape(2, R, w.H // 32)
     ograds, oloss, rep = orc.learn(w.N, w.H, w.precision, st["theta"], st["walls"], st["goal"], g["pos"], g["action"], gadv,
                                    gret, np.float32(w.value_coef), np.float32(w.entropy_coef), gates=(gates[0], gates[1]))
     for layer, r in rep.items():
@@ -130,22 +147,20 @@ def check_learn(an, bnd, w, st, g, gadv, gret):
         assert r["mismatched"] <= 10 + 1e-5 * R * w.H, (layer, r)
     print(f"{w.name}: gate decisions differing from the oracle's own: layer1 {rep['layer1']['mismatched']}, "
           f"layer2 {rep['layer2']['mismatched']} of {R * w.H} each")
-    ggrads = an.get(bnd.GRADS)
     d = orc.Dims(w.N, w.H)
     for name, sl in d.slices().items():
         assert_close(ggrads[sl], ograds[sl], rtol, f"grad {name}")
-    s = an.stats()
-    gl = np.array([s.loss_total, s.loss_pg, s.loss_value, s.entropy], dtype=np.float64)
+    gl = np.array(gloss, dtype=np.float64)
     lt = max(rtol, 1e-4)
     scale = np.abs(oloss).max()
     assert (np.abs(gl - oloss) <= lt * (np.abs(oloss) + 1e-3 * scale) + 1e-7).all(), (gl, oloss)
     theta, m, v = st["theta"].copy(), st["m"].copy(), st["v"].copy()
     orc.adam(theta, ggrads, m, v, st["k"] + 1, np.float32(w.lr), np.float32(w.adam_b1), np.float32(w.adam_b2),
              np.float32(w.adam_eps))
-    assert int(an.get(bnd.ADAM_STEP)) == st["k"] + 1
-    assert_close(an.get(bnd.ADAM_M), m, RTOL_FP32, "adam m")
-    assert_close(an.get(bnd.ADAM_V), v, RTOL_FP32, "adam v")
-    gtheta = an.get(bnd.PARAMS)
+    assert new["k"] == st["k"] + 1
+    assert_close(new["m"], m, RTOL_FP32, "adam m")
+    assert_close(new["v"], v, RTOL_FP32, "adam v")
+    gtheta = new["theta"]
     assert_close(gtheta, theta, RTOL_FP32, "updated params")
     # The step is only observable through the fp32 parameter it was added to: one unit in the last place of theta
     # (which can exceed rtol * step for a large weight with a small step) is rounding of the storage format, not error.

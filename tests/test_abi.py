@@ -58,6 +58,22 @@ def test_bad_configs_are_refused(bnd, kw, code):
     assert e.value.code == code
 
 
+def test_many_policies_take_one_sub_workspace_each_and_limits_are_refused(bnd):
+    one = bnd.workspace_bytes(bnd.make_cfg(B=34, N=5, H=64, T_max=4))
+    assert bnd.workspace_bytes(bnd.make_cfg(B=100, N=5, H=64, T_max=4, n_policies=3)) == 3 * one  # ceil(100/3) = 34 envs each
+    assert bnd.workspace_bytes(bnd.make_cfg(B=34, N=5, H=64, T_max=4, n_policies=1)) == one
+    for kw, code in ((dict(precision=1), bnd.E_UNSUPPORTED_CFG), (dict(H=96), bnd.E_UNSUPPORTED_CFG), (dict(B=2), bnd.E_INVALID_ARG),
+                     (dict(B=9, n_policies=4), bnd.E_INVALID_ARG), (dict(n_policies=-1), bnd.E_INVALID_ARG)):
+        args = dict(B=100, N=5, H=64, T_max=4, n_policies=3)
+        args.update(kw)
+        with pytest.raises(bnd.AnakinError) as e:
+            bnd.workspace_bytes(bnd.make_cfg(**args))
+        assert e.value.code == code, kw
+    cfg = bnd.make_cfg(B=100, N=5, H=64, T_max=4, n_policies=3)
+    z = [None] * 12
+    assert bnd.lib().anakin_rollout_noalloc(C.byref(cfg), 1, 0, 4, *z, None) == bnd.E_UNSUPPORTED_CFG
+
+
 def test_workspace_grows_with_the_workload(bnd):
     from paper_2104_06272_b200.workloads import WORKLOADS
 
