@@ -24,7 +24,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2104_06272_b200.workloads import ORDER, WORKLOADS  # noqa: E402
+from paper_2104_06272_b200.workloads import MANY_POLICIES, ORDER, WORKLOADS  # noqa: E402
 
 METRIC = "env_frames_per_sec_act_plus_learn"
 UNIT = "frames/s"
@@ -120,7 +120,8 @@ def ncu_traffic_bytes(workload: str, kernel: str):
 
 
 def workload_label(w):
-    return (f"{w.name}: B={w.B} envs, {w.N}x{w.N} gridworld (obs {w.D}), MLP {w.D}-{w.H}-{w.H}+5, "
+    pol = f"{w.n_policies} independent policies x {(w.B + w.n_policies - 1) // w.n_policies} envs, " if getattr(w, "n_policies", 0) >= 2 else ""
+    return (f"{w.name}: {pol}B={w.B} envs, {w.N}x{w.N} gridworld (obs {w.D}), MLP {w.D}-{w.H}-{w.H}+5, "
             f"{'fp32' if w.precision == 0 else 'bf16'}, T={w.T}")
 
 
@@ -282,7 +283,8 @@ def time_other_workload(bnd, w, stream, flush, local_rank, peaks, seed, K=4, W=3
         an = bnd.Anakin(bnd.cfg_from_workload(w, device=local_rank), stream=stream)
     an.reset(seed)
     value, total_ms, launches, clocks, prof, _ = time_steps(an, an.run, w, K, W, stream, flush, torch.cuda.synchronize, 0, local_rank, 1)
-    ok = an.status() == 0 and bool(np.isfinite(an.stats().loss_total))
+    st = an.stats()
+    ok = an.status() == 0 and bool(np.isfinite([s.loss_total for s in (st if isinstance(st, list) else [st])]).all())
     rl = roofline_of(w, prof, K, peaks, clocks)
     del an
     torch.cuda.empty_cache()
@@ -307,7 +309,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    w = WORKLOADS[args.workload]
+    w = MANY_POLICIES if args.workload == MANY_POLICIES.name else WORKLOADS[args.workload]
     if args.envs:  # reduced batch for profiler captures; such a run is not a bench line of the named workload
         w = w.scaled(name=f"{w.name}[B={args.envs}]", B=args.envs)
     peaks = load_peaks()
@@ -381,6 +383,7 @@ def run_ours(args):
             if name == args.workload:
                 continue
             others[name] = time_other_workload(bnd, WORKLOADS[name], stream, flush, local_rank, peaks, seed)
+        others[MANY_POLICIES.name] = time_other_workload(bnd, MANY_POLICIES, stream, flush, local_rank, peaks, seed)
 
     # ---- the oracle on the host cores, bounded sample of the same workload (about 10-30 s of CPU work)
     if args.no_cpu_baseline or rank != 0:
@@ -467,7 +470,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing (profiler captures only)")
     ap.add_argument("--no-workloads", action="store_true", help="skip the short runs of the other four workloads")
     ap.add_argument("--envs", type=int, default=0, help="override the workload's number of envs (small profiler captures only)")
-    ap.add_argument("--workload", default="throughput", choices=list(WORKLOADS),
+    ap.add_argument("--workload", default="throughput", choices=list(WORKLOADS) + [MANY_POLICIES.name],
                     help="the metric is quoted on 'throughput'; the others are for the per-workload table")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

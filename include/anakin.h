@@ -44,7 +44,7 @@
  * policy 0 is the single-policy initialisation).  Blobs then hold the K policies one after the other: PARAMS, GRADS,
  * ADAM_M, ADAM_V as [K][P]; STATS as K anakin_stats; per-env blobs [B] in global env order; per-step blobs as K
  * consecutive blocks, block p = the single-policy blob of policy p ([T][B_p], values [T+1][B_p]); forced actions
- * likewise.  Supported: fp32, H in {64, 128, 256}, every policy non-empty ((K-1)*Bp < B), K <= 65535; reset, rollout,
+ * likewise.  Supported: fp32, H in {64, 128} (small networks), every policy non-empty ((K-1)*Bp < B), K <= 65535; reset, rollout,
  * rollout_forced, gae, update, learn, run, grads, apply_grads, get/set, status.  anakin_learn_ppo, anakin_learn_vtrace
  * and the no-allocation rollout return ANAKIN_E_UNSUPPORTED_CFG.
  */

@@ -58,7 +58,7 @@ int validate(const anakin_cfg* c) {
     if (c->n_policies >= 2) {  // many policies: fp32 on the warp-level tensor path, every policy with at least one env
         const int K = c->n_policies, Bp = (c->B + K - 1) / K;
         if (K > c->B || (long long)(K - 1) * Bp >= c->B) return ANAKIN_E_INVALID_ARG;
-        if (K > 65535 || c->precision != ANAKIN_PRECISION_FP32 || !rollout_mma_supported(c->H)) return ANAKIN_E_UNSUPPORTED_CFG;
+        if (K > 65535 || c->precision != ANAKIN_PRECISION_FP32 || (c->H != 64 && c->H != 128)) return ANAKIN_E_UNSUPPORTED_CFG;
     }
     return ANAKIN_OK;
 }
@@ -183,8 +183,6 @@ Blob blob_of(anakin_t* h, int which, int envs) {
         default: return {nullptr, 0, false, false, false};
     }
 }
-
-int envs_of_policy(const anakin_t* h, int p) { return p == h->K - 1 ? h->d.B_last : h->d.B; }
 
 // Size of a blob over all policies (K consecutive single-policy blobs).
 size_t blob_total(anakin_t* h, int which) {

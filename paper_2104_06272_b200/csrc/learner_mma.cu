@@ -1182,7 +1182,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
             a.ts = 1;
         }
     }
-    if (!fused_agent && (H == 128 || H == 256)) {
+    if (!fused_agent && !grouped && (H == 128 || H == 256)) {  // (the warp-level dh1 kernel walks all steps itself)
         const int per_slice = ((B + 127) / 128) * (H / 128);
         int ts = 148 / per_slice;
         if (ts > 4) ts = 4;
@@ -1196,7 +1196,8 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         Scope sc(c, K_DH1);
         const cudaError_t etc = grouped ? cudaErrorNotSupported : launch_dh1_tc(a, PREC, s);  // tcgen05 where covered, else the mma.sync kernel
         if (etc != cudaErrorNotSupported) CK(etc);
-        else switch (H) {
+        else a.ts = 1;
+        if (etc == cudaErrorNotSupported) switch (H) {
             case 64: CK((launch_dh1_t<64, 64, PREC>(a, s))); break;
             case 128: CK((launch_dh1_t<128, 128, PREC>(a, s))); break;
             case 256: CK((launch_dh1_t<256, 128, PREC>(a, s))); break;

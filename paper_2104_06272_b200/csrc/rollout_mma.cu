@@ -378,7 +378,6 @@ cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
         switch (a.d.H) {
             case 64: return launch_t<64, 4, 0, true>(a, s);
             case 128: return launch_t<128, 8, 0, true>(a, s);
-            case 256: return launch_t<256, 8, 0, true>(a, s);
         }
         return cudaErrorNotSupported;
     }

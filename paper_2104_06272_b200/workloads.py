@@ -65,6 +65,9 @@ WORKLOADS = {
     "tensor_core": Workload("tensor_core", B=16384, N=16, H=1024, T=32, iters=20, precision=1),
 }
 ORDER = ["tiny", "throughput", "memory_bound", "large_batch", "tensor_core"]
+# The many-policies shape (Section 4.1 of the paper describes a meta-learning run with 1K policies on 60K environments):
+# 1024 independent small networks with 64 envs each.  Not one of the five headline workloads; benchmarked as an extra.
+MANY_POLICIES = Workload("many_policies", B=65536, N=5, H=64, T=16, iters=20, n_policies=1024)
 
 
 def forced_actions(seed: int, T: int, B: int) -> np.ndarray:
