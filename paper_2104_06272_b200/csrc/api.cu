@@ -281,7 +281,8 @@ int anakin_workspace_bytes(const anakin_cfg* cfg, size_t* bytes) {
     if (!bytes) return ANAKIN_E_INVALID_ARG;
     const int rc = validate(cfg);
     if (rc != ANAKIN_OK) return rc;
-    const Dims d = make_dims(envs_per_policy(*cfg), cfg->N, cfg->H, cfg->T_max);
+    Dims d = make_dims(envs_per_policy(*cfg), cfg->N, cfg->H, cfg->T_max);
+    d.npol = policies_of(*cfg);  // (the update's launch plan, and with it the partial buffers, depend on it)
     *bytes = carve(*cfg, d, choose_splits(d), nullptr, nullptr) * (size_t)policies_of(*cfg);  // one sub-workspace per policy
     return ANAKIN_OK;
 }
@@ -295,9 +296,9 @@ int anakin_create(const anakin_cfg* cfg, void* dev_workspace, size_t bytes, void
     const int K = policies_of(*cfg), Bp = envs_per_policy(*cfg);
     Dims d = make_dims(Bp, cfg->N, cfg->H, cfg->T_max);
     d.env0 = cfg->env_offset;
+    d.npol = K;
     const int NS = choose_splits(d);
     const size_t sub = carve(*cfg, d, NS, nullptr, nullptr), need = sub * (size_t)K;
-    d.npol = K;
     d.B_last = cfg->B - (K - 1) * Bp;
     d.pstride = sub;
     if (bytes < need) return ANAKIN_E_WORKSPACE_TOO_SMALL;

@@ -207,10 +207,9 @@ __device__ __forceinline__ void select_policy(RolloutArgs& a, int pol) {
     select_policy(a.d, a.b, pol);
 }
 __device__ __forceinline__ void select_policy(LearnArgs& a, int pol) {
-    const size_t off = (size_t)pol * a.d.pstride;
-    shift_ptr(a.part_small, off);
-#pragma unroll
-    for (int q = 0; q < LearnArgs::NREG; ++q) shift_ptr(a.reg[q].part, off);
+    // (the partial regions reg[] stay as passed: the reduction kernel indexes them dynamically, reads them from the launch
+    // parameters and adds the policy's offset itself)
+    shift_ptr(a.part_small, (size_t)pol * a.d.pstride);
     select_policy(a.d, a.b, pol);
 }
 // What a kernel body works with: the launch parameters themselves (GROUPED = false: nothing is copied), or a copy moved

@@ -13,7 +13,7 @@
 //                      fp32 accumulator; commits free the stage,
 //   warps 2-5          after the last chunk: tcgen05.ld the accumulator and store the partial tile.
 // Long K ranges (plane operands): the tensor core's fp32 accumulation rounds toward zero, which biases a sum of many
-// thousand MMAs by more than the fp32 workloads' 1e-4 bound (measured: -2e-4 after 65,536 rows).  The K range of a CTA
+// thousand MMAs by more than the fp32 workloads' 1e-4 bound (measured: -2e-4 after 65,536 rows; fp32 workloads only).  The K range of a CTA
 // is therefore cut into groups of GROUP chunks; the groups alternate between two accumulators in tensor memory, and
 // while the MMAs of one group run, warps 2-5 add the previous group's accumulator into the partial tile in global
 // memory with ordinary (round-to-nearest) fp32 additions, in group order.
@@ -60,7 +60,7 @@ bool make_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint6
 
 // DEEP: as many stages as fit (plane operands, TMA-latency-bound); otherwise two, so that two CTAs share an SM (the
 // synthesized-A modes are bound by their builder threads, and a second CTA hides them).
-template <int BN, int APL, int BPL, bool DEEP>
+template <int BN, int APL, int BPL, bool DEEP, int PREC = 0>
 struct GemmTcCfg {
     static constexpr int BM = 128, KC = 64, THREADS = 192;
     static constexpr int BOX = 64 * 64 * 2;                  // one 64 x 64 box of 16-bit elements
@@ -71,9 +71,10 @@ struct GemmTcCfg {
     static constexpr int FIT = (232448 - 1024 - 128) / STAGE;
     static constexpr int STAGES = !DEEP ? 2 : (FIT >= 4 ? 4 : (FIT >= 2 ? FIT : 2));
     static constexpr size_t smem_bytes = (size_t)STAGES * STAGE + 1024 /*alignment slack*/ + 128 /*barriers, tmem slot*/;
-    // plane operands: two accumulators, a group of GROUP 64-row chunks (2048 rows, 384 MMAs of an fp32 product) each
-    static constexpr bool FLUSH = DEEP;
-    static constexpr int GROUP = 32;
+    // plane operands of the fp32 workloads: two accumulators, a group of GROUP 64-row chunks (4096 rows, 768 MMAs) each.
+    // The bf16 workload's 2e-2 bound does not need it.
+    static constexpr bool FLUSH = DEEP && PREC == 0;
+    static constexpr int GROUP = 64;
     static constexpr int TMEM_COLS = FLUSH ? 2 * BN : BN;
 };
 
@@ -83,7 +84,7 @@ struct GemmTcMaps {
 
 template <int BN, int AMODE, int APL, int BPL, int PREC>
 __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ GemmTcMaps maps, GemmTnArgs g, int* status) {
-    using Cfg = GemmTcCfg<BN, APL, BPL, AMODE == A_PLANES>;
+    using Cfg = GemmTcCfg<BN, APL, BPL, AMODE == A_PLANES, PREC>;
     constexpr int BM = Cfg::BM, KC = Cfg::KC, STAGES = Cfg::STAGES;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* base = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);  // the swizzle needs 1024-byte alignment
@@ -266,7 +267,7 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
 
 template <int BN, int AMODE, int APL, int BPL, int PREC>
 static cudaError_t launch_t(const GemmTnArgs& g, int splits, int* status, cudaStream_t s) {
-    using Cfg = GemmTcCfg<BN, APL, BPL, AMODE == A_PLANES>;
+    using Cfg = GemmTcCfg<BN, APL, BPL, AMODE == A_PLANES, PREC>;
     GemmTcMaps maps;
     memset(&maps, 0, sizeof(maps));
     const bool bf = PREC == 1;

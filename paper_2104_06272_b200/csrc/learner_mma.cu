@@ -896,6 +896,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
     const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.y);  // many policies: grid.y = policy
     const LearnArgs& a = pa.a;
     const size_t R = GROUPED ? (size_t)a.d.B * a.T : R_in;  // rows of THIS policy
+    const size_t poff = GROUPED ? (size_t)blockIdx.y * a_in.d.pstride : 0;  // byte offset of this policy's partials
     __shared__ float s_c[2];
     const Dims& d = a.d;
     const Buffers& b = a.b;
@@ -914,78 +915,83 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
         int r = 0;
 #pragma unroll
         for (int q = 1; q < LearnArgs::NREG; ++q)
-            if (i >= a.reg[q].start) r = q;
+            if (i >= a_in.reg[q].start) r = q;
         return r;
     };
     // Parameters before b2 (W1, b1, W2) have at most ~128 partials: one thread each, partials added in index order,
     // thirty-two loads in flight.  The tail (b2 | Wh | bh) has two partials per CTA of the heads kernel: one warp per
     // parameter, lane l adds partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
+    // The work is cut into nb_total block-sized pieces; a launch with fewer CTAs per policy (many policies: a handful of
+    // fat CTAs each instead of tens of thousands of tiny ones) walks them in a stride loop.
     const int nb_main = (int)((d.ob2 + 255) / 256);
-    if ((int)blockIdx.x < nb_main) {
-        const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
-        if (i < d.ob2) {
-            const PartRegion& rg = a.reg[region_of(i)];
-            const float* p = rg.part + (i - rg.start);
-            float gsum = 0.f;
-            // thirty-two loads in flight per memory round trip (the ragged last batch is predicated, not split up);
-            // the additions stay in index order
-            for (int s = 0; s < rg.ns; s += 32) {
-                float v[32];
+    const int nb_total = nb_main + (int)((d.P - d.ob2 + 7) / 8);
+    for (int bx = blockIdx.x; bx < nb_total; bx += gridDim.x) {
+        if (bx < nb_main) {
+            const size_t i = (size_t)bx * 256 + threadIdx.x;
+            if (i < d.ob2) {
+                const PartRegion& rg = a_in.reg[region_of(i)];
+                const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(rg.part) + poff) + (i - rg.start);
+                float gsum = 0.f;
+                // thirty-two loads in flight per memory round trip (the ragged last batch is predicated, not split up);
+                // the additions stay in index order
+                for (int s = 0; s < rg.ns; s += 32) {
+                    float v[32];
 #pragma unroll
-                for (int q = 0; q < 32; ++q) v[q] = s + q < rg.ns ? p[(size_t)(s + q) * rg.stride] : 0.f;
+                    for (int q = 0; q < 32; ++q) v[q] = s + q < rg.ns ? p[(size_t)(s + q) * rg.stride] : 0.f;
 #pragma unroll
-                for (int q = 0; q < 32; ++q)
-                    if (s + q < rg.ns) gsum += v[q];
+                    for (int q = 0; q < 32; ++q)
+                        if (s + q < rg.ns) gsum += v[q];
+                }
+                apply(i, gsum);
             }
-            apply(i, gsum);
-        }
-    } else {
-        const int lane = threadIdx.x & 31;
-        const size_t i = d.ob2 + (size_t)(blockIdx.x - nb_main) * 8 + (threadIdx.x >> 5);
-        if (i < d.P) {
-            const PartRegion& rg = a.reg[region_of(i)];
-            const float* p = rg.part + (i - rg.start);
-            float gsum = 0.f;
-            int s = lane;
-            for (; s + 32 * 7 < rg.ns; s += 32 * 8) {  // eight loads in flight per lane
-                float v[8];
+        } else {
+            const int lane = threadIdx.x & 31;
+            const size_t i = d.ob2 + (size_t)(bx - nb_main) * 8 + (threadIdx.x >> 5);
+            if (i < d.P) {
+                const PartRegion& rg = a_in.reg[region_of(i)];
+                const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(rg.part) + poff) + (i - rg.start);
+                float gsum = 0.f;
+                int s = lane;
+                for (; s + 32 * 7 < rg.ns; s += 32 * 8) {  // eight loads in flight per lane
+                    float v[8];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + 32 * q) * rg.stride];
+                    for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + 32 * q) * rg.stride];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) gsum += v[q];
+                    for (int q = 0; q < 8; ++q) gsum += v[q];
+                }
+                for (; s < rg.ns; s += 32) gsum += p[(size_t)s * rg.stride];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, off);
+                if (lane == 0) apply(i, gsum);
             }
-            for (; s < rg.ns; s += 32) gsum += p[(size_t)s * rg.stride];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, off);
-            if (lane == 0) apply(i, gsum);
         }
-    }
-    // Loss statistics: the first warp of the last CTA (the one with the least other work) adds the per-CTA partials of
-    // the heads kernel, lane l taking partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
-    if (blockIdx.x == gridDim.x - 1 && threadIdx.x < 32) {
-        const int lane = threadIdx.x;
-        float l[3];
+        // Loss statistics: the first warp of the last CTA (the one with the least other work) adds the per-CTA partials of
+        // the heads kernel, lane l taking partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
+        if (bx == nb_total - 1 && threadIdx.x < 32) {
+            const int lane = threadIdx.x;
+            float l[3];
 #pragma unroll
-        for (int c = 0; c < 3; ++c) {
-            float s = 0.f;
-            int q = lane;
-            for (; q + 32 * 3 < loss_blocks; q += 32 * 4) {  // four loads in flight per lane
-                float v[4];
+            for (int c = 0; c < 3; ++c) {
+                float s = 0.f;
+                int q = lane;
+                for (; q + 32 * 3 < loss_blocks; q += 32 * 4) {  // four loads in flight per lane
+                    float v[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) v[u] = b.loss_part[(size_t)(q + 32 * u) * 4 + c];
+                    for (int u = 0; u < 4; ++u) v[u] = b.loss_part[(size_t)(q + 32 * u) * 4 + c];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) s += v[u];
+                    for (int u = 0; u < 4; ++u) s += v[u];
+                }
+                for (; q < loss_blocks; q += 32) s += b.loss_part[(size_t)q * 4 + c];
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+                l[c] = s / (float)R;
             }
-            for (; q < loss_blocks; q += 32) s += b.loss_part[(size_t)q * 4 + c];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-            l[c] = s / (float)R;
-        }
-        if (lane == 0) {
-            b.stats->loss_pg = l[0];
-            b.stats->loss_value = l[1];
-            b.stats->entropy = l[2];
-            b.stats->loss_total = l[0] + a.c_v * l[1] - a.c_e * l[2];
+            if (lane == 0) {
+                b.stats->loss_pg = l[0];
+                b.stats->loss_value = l[1];
+                b.stats->entropy = l[2];
+                b.stats->loss_total = l[0] + a.c_v * l[1] - a.c_e * l[2];
+            }
         }
     }
 }
@@ -1062,7 +1068,9 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     }
     p->ns_env = splits_for(d.B, tiles_ch, 128);
     const size_t tiles32 = (R + 31) / 32;
-    p->heads_grid = (int)(tiles32 < (size_t)HEADS_GRID ? tiles32 : (size_t)HEADS_GRID);
+    size_t hg = HEADS_GRID;
+    if (d.npol > 1) hg = (size_t)(2 * HEADS_GRID / d.npol > 0 ? 2 * HEADS_GRID / d.npol : 1);  // many policies: the CTAs of all policies fill the GPU together
+    p->heads_grid = (int)(tiles32 < hg ? tiles32 : hg);
     p->ns_small = 4 * p->heads_grid;
     p->small_stride = (size_t)6 * H + 8;
     size_t off = 0;
@@ -1286,7 +1294,8 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         Scope sc(c, K_REDUCE_ADAM);
         const unsigned nb = (unsigned)((d.ob2 + 255) / 256 + (d.P - d.ob2 + 7) / 8);
         if (d.npol > 1) {
-            if constexpr (PREC == 0) k_reduce_adam2<PREC, true><<<dim3(nb, d.npol), 256, 0, s>>>(a, R, pl.loss_blocks);
+            const unsigned per_policy = d.npol >= 296 ? 2u : (nb < 592u / d.npol ? nb : 592u / d.npol);  // about four CTAs per SM in all
+            if constexpr (PREC == 0) k_reduce_adam2<PREC, true><<<dim3(per_policy, d.npol), 256, 0, s>>>(a, R, pl.loss_blocks);
             else return cudaErrorNotSupported;
         } else {
             k_reduce_adam2<PREC, false><<<nb, 256, 0, s>>>(a, R, pl.loss_blocks);
