@@ -110,10 +110,9 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.dbg_gates = c.debug_logits ? (uint32_t*)take(2 * R * (H / 32) * 4) : nullptr;
     b.base = (float*)take(B * H * 4);
     const bool mma = rollout_mma_supported(d.H), tensor = tensor_path_supported(d.H, c.precision);
-    b.w2f_hi = mma ? (uint2*)take(H * H * 2) : nullptr;
-    b.w2f_lo = mma ? (uint2*)take(H * H * 2) : nullptr;
-    b.w2tf_hi = mma ? (uint2*)take(H * H * 2) : nullptr;
-    b.w2tf_lo = mma ? (uint2*)take(H * H * 2) : nullptr;
+    const bool frags = mma && rollout_uses_fragments(d.H, c.precision);
+    b.w2f_hi = frags ? (uint2*)take(H * H * 2) : nullptr;
+    b.w2f_lo = frags ? (uint2*)take(H * H * 2) : nullptr;
     b.w2p_hi = tensor ? (uint16_t*)take(H * H * 2) : nullptr;
     b.w2p_lo = mma ? (uint16_t*)take(H * H * 2) : nullptr;
     b.h1 = (float*)take(R * H * 4);
@@ -396,6 +395,8 @@ static int learn_after_gae(anakin_t* h, int phase, float ppo_clip = 0.f, bool co
     a.beta2 = h->cfg.adam_b2;
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
+    a.bc1 = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
+    a.bc2 = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
     a.phase = phase;
     a.grad_div = 1.f;
     a.ppo_clip = ppo_clip;
@@ -517,6 +518,8 @@ int anakin_apply_grads_mean(anakin_t* h, int n_replicas) {
     a.beta2 = h->cfg.adam_b2;
     a.eps = h->cfg.adam_eps;
     a.adam_k = (int)(h->adam_k + 1);
+    a.bc1 = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
+    a.bc2 = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
     a.grad_div = (float)n_replicas;
     const cudaError_t e = launch_adam_only(a, h->cfg.precision, h->ctx());
     if (e != cudaSuccess) return fail_cuda(h, e);

@@ -68,10 +68,8 @@ struct Buffers {
     float* dbg_logits;  // [Tmax][B][4] or null
     uint32_t* dbg_gates;  // [2][R][H/32] or null: ReLU gates of the last update
     float* base;     // [B][H]  b1 + sum of W1 rows of the wall cells + W1 row of the goal cell
-    uint2* w2f_hi;   // [H*H/4] W2 as mma B fragments, bf16 high parts (null: tensor-pipe rollout not used)
+    uint2* w2f_hi;   // [H*H/4] W2 as mma.sync B fragments, high parts (null: the warp-level rollout kernel is not used)
     uint2* w2f_lo;   // [H*H/4] bf16 low parts
-    uint2* w2tf_hi;  // the same for W2 transposed (backward pass)
-    uint2* w2tf_lo;
     uint16_t* w2p_hi;  // [H][H] W2 row-major as 16-bit hi / lo planes (B operand of the dh1 kernel)
     uint16_t* w2p_lo;
     float* h1;       // [R][H]
@@ -102,7 +100,7 @@ __device__ __forceinline__ void shift_buffers(Buffers& b, size_t off) {
     shift_ptr(b.walls, off); shift_ptr(b.start, off); shift_ptr(b.goal, off); shift_ptr(b.pos, off); shift_ptr(b.tep, off);
     shift_ptr(b.tpos, off); shift_ptr(b.tact, off); shift_ptr(b.tdone, off); shift_ptr(b.trew, off); shift_ptr(b.tval, off);
     shift_ptr(b.tlogp, off); shift_ptr(b.adv, off); shift_ptr(b.ret, off); shift_ptr(b.dbg_logits, off); shift_ptr(b.dbg_gates, off);
-    shift_ptr(b.base, off); shift_ptr(b.w2f_hi, off); shift_ptr(b.w2f_lo, off); shift_ptr(b.w2tf_hi, off); shift_ptr(b.w2tf_lo, off);
+    shift_ptr(b.base, off); shift_ptr(b.w2f_hi, off); shift_ptr(b.w2f_lo, off);
     shift_ptr(b.w2p_hi, off); shift_ptr(b.w2p_lo, off); shift_ptr(b.h1, off); shift_ptr(b.h2, off); shift_ptr(b.out5, off);
     shift_ptr(b.vboot, off); shift_ptr(b.dh2, off); shift_ptr(b.dh1, off); shift_ptr(b.dout, off); shift_ptr(b.S, off);
     shift_ptr(b.part, off); shift_ptr(b.loss_part, off); shift_ptr(b.stats, off);
@@ -190,6 +188,7 @@ struct LearnArgs {
     float c_v, c_e;
     float lr, beta1, beta2, eps;
     int adam_k;  // step index after the increment
+    float bc1, bc2;  // Adam's bias corrections 1 - beta1^k, 1 - beta2^k (evaluated in double on the host)
     int phase;   // 0: reduce the partials and apply Adam; 1: reduce only (GRADS and loss statistics)
     float grad_div;  // Adam-only launch: > 1 = GRADS holds a sum over this many replicas, divided here into their mean
     float ppo_clip;  // > 0: the policy term is the clipped surrogate over the recorded log-probabilities (TRAJ_LOGP)
@@ -330,6 +329,7 @@ cudaError_t launch_env_base(const Dims& d, const Buffers& b, const Ctx& c);
 cudaError_t launch_rollout(const RolloutArgs& a, int prec, const Ctx& c);
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s);  // cudaErrorNotSupported if not covered
 bool rollout_mma_supported(int H);
+bool rollout_uses_fragments(int H, int prec);  // the warp-level kernel (and with it the fragment copies of W2) serves this shape
 cudaError_t launch_rollout_pair(const RolloutArgs& a, cudaStream_t s);  // CTA-pair tcgen05 rollout (H = 256, fp32); cudaErrorNotSupported otherwise
 bool wide_supported(int H, int prec);         // bf16 workload with a hidden layer too wide for the persistent rollout
 bool tensor_path_supported(int H, int prec);  // either tensor-core path: the update reuses activations the rollout saved

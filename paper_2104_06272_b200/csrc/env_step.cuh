@@ -70,11 +70,16 @@ __device__ __forceinline__ StepPre step_prepare(const EnvLane& s, const RolloutA
     return a.env_kind == ANAKIN_ENV_TORUS ? step_prepare_t<TorusMoves>(s, a, env, t, walls) : step_prepare_t<GridMoves>(s, a, env, t, walls);
 }
 
-// Categorical sampling from the 4 logits (inverse CDF against the prepared uniform), the env transition and the records.
-// Returns bit 0 = the episode ended at this step, bit 1 = it ended at the goal (reward 1).
-__device__ __forceinline__ int act_and_step_pre(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
-                                                float l3, const StepPre& pre) {
-    const Buffers& b = a.b;
+// Categorical sampling from the 4 logits (inverse CDF against the prepared uniform) and the env transition, in two parts
+// so that a kernel can publish the new position before it spends time on the records:
+//   act_decide   softmax terms, the sampled (or forced) action, the transition; updates the env state in `s`
+//   act_record   log-probability and the time-major records of the step
+struct ActOut {
+    float la_mx, Z, rew;  // logit of the action minus the maximum, softmax denominator, reward
+    int act, done, pos0;  // action, episode ended at this step, the state the action was taken in
+};
+__device__ __forceinline__ ActOut act_decide(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2, float l3,
+                                             const StepPre& pre) {
     const size_t i = (size_t)t * a.d.B + env;
     // softmax and inverse CDF: c0 = p0, c1 = c0 + p1, c2 = c1 + p2; a = [u>=c0] + [u>=c1] + [u>=c2]
     const float mx = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
@@ -89,18 +94,18 @@ __device__ __forceinline__ int act_and_step_pre(EnvLane& s, const RolloutArgs& a
         act = a.forced[i];
         if (act < 0 || act > 3) { s.bad |= DEV_E_BAD_ACTION; act &= 3; }
     }
-    const float la = act == 0 ? l0 : act == 1 ? l1 : act == 2 ? l2 : l3;
-    b.tlogp[i] = (la - mx) - logf(Z);
-    b.tpos[i] = (uint8_t)s.pos;
-    b.tact[i] = (int8_t)act;
-    if (b.dbg_logits) reinterpret_cast<float4*>(b.dbg_logits)[i] = make_float4(l0, l1, l2, l3);
+    ActOut o;
+    o.la_mx = (act == 0 ? l0 : act == 1 ? l1 : act == 2 ? l2 : l3) - mx;
+    o.Z = Z;
+    o.act = act;
+    o.pos0 = s.pos;
     const int np = act == 0 ? pre.np[0] : act == 1 ? pre.np[1] : act == 2 ? pre.np[2] : pre.np[3];
     const int te = s.tep + 1;
-    float rew = 0.f;
-    int done = 0;
-    if (np == s.goal) { rew = 1.f; done = 1; }
-    else if (te >= a.cap) { done = 1; }
-    if (done) {
+    o.rew = 0.f;
+    o.done = 0;
+    if (np == s.goal) { o.rew = 1.f; o.done = 1; }
+    else if (te >= a.cap) { o.done = 1; }
+    if (o.done) {
         s.n_episodes += 1;
         s.n_goals += (np == s.goal);
         s.n_epsteps += te;
@@ -110,9 +115,24 @@ __device__ __forceinline__ int act_and_step_pre(EnvLane& s, const RolloutArgs& a
         s.pos = np;
         s.tep = te;
     }
-    b.trew[i] = rew;
-    b.tdone[i] = (uint8_t)done;
-    return done | (rew != 0.f ? 2 : 0);
+    return o;
+}
+__device__ __forceinline__ void act_record(const RolloutArgs& a, int env, int t, float l0, float l1, float l2, float l3, const ActOut& o) {
+    const Buffers& b = a.b;
+    const size_t i = (size_t)t * a.d.B + env;
+    b.tlogp[i] = o.la_mx - logf(o.Z);
+    b.tpos[i] = (uint8_t)o.pos0;
+    b.tact[i] = (int8_t)o.act;
+    if (b.dbg_logits) reinterpret_cast<float4*>(b.dbg_logits)[i] = make_float4(l0, l1, l2, l3);
+    b.trew[i] = o.rew;
+    b.tdone[i] = (uint8_t)o.done;
+}
+// Both parts at once.  Returns bit 0 = the episode ended at this step, bit 1 = it ended at the goal (reward 1).
+__device__ __forceinline__ int act_and_step_pre(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,
+                                                float l3, const StepPre& pre) {
+    const ActOut o = act_decide(s, a, env, t, l0, l1, l2, l3, pre);
+    act_record(a, env, t, l0, l1, l2, l3, o);
+    return o.done | (o.rew != 0.f ? 2 : 0);
 }
 
 __device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, int env, int t, float l0, float l1, float l2,

@@ -278,8 +278,8 @@ __global__ void __launch_bounds__(256) k_reduce_adam(LearnArgs a, size_t R, int 
     const Dims& d = a.d;
     const Buffers& b = a.b;
     if (threadIdx.x == 0) {
-        s_c[0] = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
-        s_c[1] = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
+        s_c[0] = a.bc1;
+        s_c[1] = a.bc2;
     }
     __syncthreads();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;

@@ -855,11 +855,8 @@ __device__ __forceinline__ void adam_step(const LearnArgs& a, const float* c, si
         split1<PREC>(thc, hi, lo);
         if (b.w2f_hi) {
             const size_t ef = ((size_t)((k >> 4) * (H / 8) + (n >> 3)) * 32 + (n & 7) * 4 + ((k & 7) >> 1)) * 4 + ((k & 15) >> 3) * 2 + (k & 1);
-            const size_t et = ((size_t)((n >> 4) * (H / 8) + (k >> 3)) * 32 + (k & 7) * 4 + ((n & 7) >> 1)) * 4 + ((n & 15) >> 3) * 2 + (n & 1);
             reinterpret_cast<uint16_t*>(b.w2f_hi)[ef] = hi;
             reinterpret_cast<uint16_t*>(b.w2f_lo)[ef] = lo;
-            reinterpret_cast<uint16_t*>(b.w2tf_hi)[et] = hi;
-            reinterpret_cast<uint16_t*>(b.w2tf_lo)[et] = lo;
         }
         b.w2p_hi[i - d.oW2] = hi;
         if (b.w2p_lo) b.w2p_lo[i - d.oW2] = lo;
@@ -873,8 +870,8 @@ __global__ void __launch_bounds__(256) k_adam_only(LearnArgs a_in) {
     const LearnArgs& a = pa.a;
     __shared__ float s_c[2];
     if (threadIdx.x == 0) {
-        s_c[0] = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
-        s_c[1] = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
+        s_c[0] = a.bc1;
+        s_c[1] = a.bc2;
     }
     __syncthreads();
     const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
@@ -898,11 +895,12 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
     const size_t R = GROUPED ? (size_t)a.d.B * a.T : R_in;  // rows of THIS policy
     const size_t poff = GROUPED ? (size_t)blockIdx.y * a_in.d.pstride : 0;  // byte offset of this policy's partials
     __shared__ float s_c[2];
+    __shared__ float s_tail[32][8];
     const Dims& d = a.d;
     const Buffers& b = a.b;
     if (threadIdx.x == 0) {
-        s_c[0] = (float)(1.0 - pow((double)a.beta1, (double)a.adam_k));
-        s_c[1] = (float)(1.0 - pow((double)a.beta2, (double)a.adam_k));
+        s_c[0] = a.bc1;
+        s_c[1] = a.bc2;
     }
     __syncthreads();
     // Batch-mean gradient of parameter i, then (phase 0) its Adam step.
@@ -920,7 +918,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
     };
     // Parameters before b2 (W1, b1, W2) have at most ~128 partials: one thread each, partials added in index order,
     // thirty-two loads in flight.  The tail (b2 | Wh | bh) has two partials per CTA of the heads kernel: one warp per
-    // parameter, lane l adds partials l, l+32, ... in order, then a fixed shuffle tree joins the lanes.
+    // parameter group, see below.
     // The work is cut into nb_total block-sized pieces; a launch with fewer CTAs per policy (many policies: a handful of
     // fat CTAs each instead of tens of thousands of tiny ones) walks them in a stride loop.
     const int nb_main = (int)((d.ob2 + 255) / 256);
@@ -945,14 +943,17 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
                 apply(i, gsum);
             }
         } else {
-            const int lane = threadIdx.x & 31;
-            const size_t i = d.ob2 + (size_t)(bx - nb_main) * 8 + (threadIdx.x >> 5);
+            // eight consecutive parameters per CTA: thread = (parameter tid % 8, partial group tid / 8); a group's eight
+            // threads read one 32-byte sector per partial.  Group g adds partials g, g+32, ... in order; then one thread
+            // per parameter adds the 32 group sums in group order (shared memory).
+            const int pi = threadIdx.x & 7, grp = threadIdx.x >> 3;
+            const size_t i = d.ob2 + (size_t)(bx - nb_main) * 8 + pi;
+            float gsum = 0.f;
             if (i < d.P) {
                 const PartRegion& rg = a_in.reg[region_of(i)];
                 const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(rg.part) + poff) + (i - rg.start);
-                float gsum = 0.f;
-                int s = lane;
-                for (; s + 32 * 7 < rg.ns; s += 32 * 8) {  // eight loads in flight per lane
+                int s = grp;
+                for (; s + 32 * 7 < rg.ns; s += 32 * 8) {  // eight loads in flight per thread
                     float v[8];
 #pragma unroll
                     for (int q = 0; q < 8; ++q) v[q] = p[(size_t)(s + 32 * q) * rg.stride];
@@ -960,9 +961,15 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
                     for (int q = 0; q < 8; ++q) gsum += v[q];
                 }
                 for (; s < rg.ns; s += 32) gsum += p[(size_t)s * rg.stride];
+            }
+            __syncthreads();  // (the previous piece's readers of s_tail are done)
+            s_tail[grp][pi] = gsum;
+            __syncthreads();
+            if (grp == 0 && i < d.P) {
+                float tot = 0.f;
 #pragma unroll
-                for (int off = 16; off > 0; off >>= 1) gsum += __shfl_xor_sync(0xFFFFFFFFu, gsum, off);
-                if (lane == 0) apply(i, gsum);
+                for (int g2 = 0; g2 < 32; ++g2) tot += s_tail[g2][pi];
+                apply(i, tot);
             }
         }
         // Loss statistics: the first warp of the last CTA (the one with the least other work) adds the per-CTA partials of

@@ -92,8 +92,10 @@ extern "C" int anakin_rollout_noalloc(const anakin_cfg* cfg, uint64_t seed, int6
     b.base = reinterpret_cast<float*>(scratch);
     unsigned char* frag = scratch + kMaxBaseFloats * sizeof(float);
     if (rollout_mma_supported(cfg->H)) {  // same kernel choice as the handle-based rollout
-        b.w2f_hi = reinterpret_cast<uint2*>(frag);
-        b.w2f_lo = reinterpret_cast<uint2*>(frag + kW2FragBytes / 2);
+        if (rollout_uses_fragments(cfg->H, cfg->precision)) {
+            b.w2f_hi = reinterpret_cast<uint2*>(frag);
+            b.w2f_lo = reinterpret_cast<uint2*>(frag + kW2FragBytes / 2);
+        }
         b.w2p_hi = reinterpret_cast<uint16_t*>(frag + kW2FragBytes);
         b.w2p_lo = reinterpret_cast<uint16_t*>(frag + kW2FragBytes + kW2PlaneBytes / 2);
     }

@@ -29,18 +29,13 @@ __global__ void __launch_bounds__(256) k_pack_w2(DimsBuffers in) {
     const int g = lane >> 2, t = lane & 3;
     const int n = nt * 8 + g, k0 = ks * 16 + 2 * t;
     const float* W2 = b.theta_c + d.oW2;
-    const int ks4[4] = {k0, k0 + 1, k0 + 8, k0 + 9};
-    uint2 hi, lo;
-    split2<PREC>(W2[(size_t)ks4[0] * H + n], W2[(size_t)ks4[1] * H + n], hi.x, lo.x);
-    split2<PREC>(W2[(size_t)ks4[2] * H + n], W2[(size_t)ks4[3] * H + n], hi.y, lo.y);
-    b.w2f_hi[idx] = hi;
-    b.w2f_lo[idx] = lo;
-    // the same for W2^T (the backward pass contracts over W2's second index): B[k][n] = W2[n][k]
-    if (b.w2tf_hi) {
-        split2<PREC>(W2[(size_t)n * H + ks4[0]], W2[(size_t)n * H + ks4[1]], hi.x, lo.x);
-        split2<PREC>(W2[(size_t)n * H + ks4[2]], W2[(size_t)n * H + ks4[3]], hi.y, lo.y);
-        b.w2tf_hi[idx] = hi;
-        b.w2tf_lo[idx] = lo;
+    if (b.w2f_hi) {
+        const int ks4[4] = {k0, k0 + 1, k0 + 8, k0 + 9};
+        uint2 hi, lo;
+        split2<PREC>(W2[(size_t)ks4[0] * H + n], W2[(size_t)ks4[1] * H + n], hi.x, lo.x);
+        split2<PREC>(W2[(size_t)ks4[2] * H + n], W2[(size_t)ks4[3] * H + n], hi.y, lo.y);
+        b.w2f_hi[idx] = hi;
+        b.w2f_lo[idx] = lo;
     }
     // and W2 itself as row-major hi / lo planes: this thread covers elements 4*idx .. 4*idx+3
     if (!b.w2p_hi || !b.w2p_lo) return;
@@ -54,7 +49,7 @@ __global__ void __launch_bounds__(256) k_pack_w2(DimsBuffers in) {
 }
 
 cudaError_t launch_pack_w2(const Dims& d, const Buffers& b, int prec, const Ctx& c) {
-    if (!b.w2f_hi) return cudaSuccess;
+    if (!b.w2f_hi && !b.w2p_hi) return cudaSuccess;
     Scope sc(c, K_PACK_W2);
     const unsigned nb = (d.H * d.H / 4 + 255) / 256;
     if (d.npol > 1) {
@@ -369,10 +364,14 @@ static cudaError_t launch_t(const RolloutArgs& a0, cudaStream_t s) {
 }
 
 bool rollout_mma_supported(int H) { return H == 64 || H == 128 || H == 256; }
+// fp32 at H = 256 runs the CTA-pair tcgen05 kernel, which reads the row-major planes of W2 only.
+bool rollout_uses_fragments(int H, int prec) { return rollout_mma_supported(H) && !(H == 256 && prec == 0); }
 
 // Returns cudaErrorNotSupported when the shape is not covered by the tensor-pipe kernel.
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
-    if (!a.b.w2f_hi || !rollout_mma_supported(a.d.H)) return cudaErrorNotSupported;
+    if (!rollout_mma_supported(a.d.H)) return cudaErrorNotSupported;
+    if (prec == 0 && a.d.npol <= 1 && a.d.H == 256) return launch_rollout_pair(a, s);  // the CTA-pair kernel on the 5th-generation tensor cores
+    if (!a.b.w2f_hi) return cudaErrorNotSupported;
     if (a.d.npol > 1) {  // many policies: one grid slice per policy, each with its own weights on chip
         if (prec != 0) return cudaErrorNotSupported;
         switch (a.d.H) {
@@ -380,10 +379,6 @@ cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
             case 128: return launch_t<128, 8, 0, true>(a, s);
         }
         return cudaErrorNotSupported;
-    }
-    if (prec == 0) {  // the CTA-pair kernel on the 5th-generation tensor cores where it covers the shape
-        const cudaError_t e = launch_rollout_pair(a, s);
-        if (e != cudaErrorNotSupported) return e;
     }
     if (prec == 1) {
         switch (a.d.H) {
@@ -395,7 +390,6 @@ cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
         switch (a.d.H) {
             case 64: return launch_t<64, 4, 0>(a, s);
             case 128: return launch_t<128, 8, 0>(a, s);
-            case 256: return launch_t<256, 8, 0>(a, s);
         }
     }
     return cudaErrorNotSupported;

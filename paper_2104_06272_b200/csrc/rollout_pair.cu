@@ -318,34 +318,51 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg::THREADS, 1)
         }
         // ---- one thread per env: once the eight partials are in, their fixed-order sum, then act and step
         if (!worker && ok) ok = tc::mbar_wait_cluster(pfull, (uint32_t)t & 1u);
-        if (owner) {
+        // The new positions are all the next step's gather needs: the owners publish them and release the workers (named
+        // barrier 1: the workers wait on it, the owner warp only arrives, once and as a whole warp) before they write the
+        // step's records.
+        if (!worker) {
             float o[5];
 #pragma unroll
             for (int c = 0; c < 5; ++c) o[c] = 0.f;
-#pragma unroll
-            for (int blk = 0; blk < 8; ++blk)
-#pragma unroll
-                for (int c = 0; c < 5; ++c) o[c] += s_red[(blk * ME + ow) * 5 + c];
-#pragma unroll
-            for (int c = 0; c < 5; ++c) o[c] += s_bh[c];
+            ActOut ao;
+            ao.la_mx = ao.Z = ao.rew = 0.f;
+            ao.act = ao.done = ao.pos0 = 0;
             const int env = e0 + ow;
-            if (b.out5 && t < a.T) {  // the update reuses the head outputs of every recorded row
-                float4* o5 = reinterpret_cast<float4*>(b.out5 + ((size_t)t * B + env) * 8);
-                o5[0] = make_float4(o[0], o[1], o[2], o[3]);
-                o5[1] = make_float4(o[4], 0.f, 0.f, 0.f);
+            if (owner) {
+#pragma unroll
+                for (int blk = 0; blk < 8; ++blk)
+#pragma unroll
+                    for (int c = 0; c < 5; ++c) o[c] += s_red[(blk * ME + ow) * 5 + c];
+#pragma unroll
+                for (int c = 0; c < 5; ++c) o[c] += s_bh[c];
+                if (acting) {
+                    ao = act_decide(s, a, env, t, o[0], o[1], o[2], o[3], pre);
+                    s_pos[ow] = s.pos;
+                }
             }
-            if (a.replay == 2 && t == a.T) b.vboot[env] = o[4];
-            if (!a.replay) {
-                b.tval[(size_t)t * B + env] = o[4];
-                if (a.gae_smem) s_gv[t * ME + ow] = o[4];
+            __syncwarp();
+            asm volatile("bar.arrive 1, %0;" ::"n"(Cfg::THREADS) : "memory");
+            if (owner) {
+                if (b.out5 && t < a.T) {  // the update reuses the head outputs of every recorded row
+                    float4* o5 = reinterpret_cast<float4*>(b.out5 + ((size_t)t * B + env) * 8);
+                    o5[0] = make_float4(o[0], o[1], o[2], o[3]);
+                    o5[1] = make_float4(o[4], 0.f, 0.f, 0.f);
+                }
+                if (a.replay == 2 && t == a.T) b.vboot[env] = o[4];
+                if (!a.replay) {
+                    b.tval[(size_t)t * B + env] = o[4];
+                    if (a.gae_smem) s_gv[t * ME + ow] = o[4];
+                }
+                if (acting) {
+                    act_record(a, env, t, o[0], o[1], o[2], o[3], ao);
+                    if (a.gae_smem) s_gc[t * ME + ow] = (uint8_t)(ao.done | (ao.rew != 0.f ? 2 : 0));
+                }
             }
-            if (acting) {
-                const int code = act_and_step_pre(s, a, env, t, o[0], o[1], o[2], o[3], pre);
-                if (a.gae_smem) s_gc[t * ME + ow] = (uint8_t)code;
-                s_pos[ow] = s.pos;
-            }
+        } else {
+            // every worker is done with its staging area in the operand tile, and the positions are in place
+            asm volatile("bar.sync 1, %0;" ::"n"(Cfg::THREADS) : "memory");
         }
-        __syncthreads();
     }
     if (owner && !a.replay) {
         b.pos[e0 + ow] = (uint8_t)s.pos;

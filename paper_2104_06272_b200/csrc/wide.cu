@@ -432,7 +432,7 @@ cudaError_t launch_pack_w2_wide(const Dims& d, const Buffers& b, const Ctx& c) {
 // (bf16 workload: the products 1 x w are exact and the accumulation is fp32); cudaErrorNotSupported otherwise.
 // Uses the dh1 buffer, which is dead outside the update, as scratch for the two bf16 operands.
 cudaError_t launch_env_base_wide(const Dims& d, const Buffers& b, const Ctx& c) {
-    const bool wide_buffers = b.w2p_hi && !b.w2f_hi;
+    const bool wide_buffers = b.w2p_hi && d.H >= 512;  // (narrower layers keep fp32-sized activation buffers)
     if (!wide_buffers || d.C % 64 != 0 || d.H % NtCfg::BN != 0 || d.H > NtCfg::MAXN) return cudaErrorNotSupported;
     uint16_t* X = reinterpret_cast<uint16_t*>(b.dh1);
     uint16_t* W1w = X + (size_t)d.B * d.C;
