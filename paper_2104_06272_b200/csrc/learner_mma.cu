@@ -13,7 +13,7 @@
 //   k_reduce_adam2  fixed-order sum of every region's partials (= the batch-mean gradient, the single-device form of
 //                 the paper's cross-core average), Adam, loss statistics.
 // No floating-point atomics: every sum has a fixed order, so runs are bitwise reproducible.
-#include "env_step.cuh"
+#include "tc_common.cuh"
 
 namespace anakin {
 
@@ -31,12 +31,14 @@ template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
 struct HeadsCfg {
     static constexpr int TR = 32;  // rows per tile
     static constexpr int ESZ = H2BF ? 2 : 4;
-    static constexpr int NST = TR * HS * ESZ >= 32768 ? 3 : 4;  // depth of the h2 ring (tiles in flight = NST - 1)
-    static constexpr size_t smem_bytes = (size_t)NST * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + (size_t)TR * 8 * 4;
+    // the widest slab (32 KB tiles, 17 warps) runs one CTA per SM with a deep ring; the narrower ones two CTAs per SM
+    static constexpr int PER_SM = TR * HS * ESZ >= 32768 ? 1 : 2;
+    static constexpr int NST = PER_SM == 1 ? 6 : 4;  // depth of the h2 ring (tiles in flight = NST - 1)
+    static constexpr size_t smem_bytes = (size_t)NST * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + 64 /*barriers*/;
 };
 
 template <int H, int NW, int PREC, int HS = H, bool H2BF = false, bool GROUPED = false>
-__global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
+__global__ void __launch_bounds__(NW * 32 + 32, (HeadsCfg<H, NW, PREC, HS, H2BF>::PER_SM)) k_heads_bwd(LearnArgs a_in) {
     const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.z);  // many policies: grid.z = policy
     const LearnArgs& a = pa.a;
     using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
@@ -45,23 +47,121 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned char* s_h2 = smem_raw;                                                 // [NST][TR][HS] fp32 or bf16
     float* s_dout = reinterpret_cast<float*>(smem_raw + (size_t)NST * TR * HS * ESZ);  // [2][TR][8]
-    float* s_fin = s_dout + 2 * TR * 8;                                           // [TR][8] end-of-kernel reductions
+    uint64_t* bars = reinterpret_cast<uint64_t*>(s_dout + 2 * TR * 8);              // full[2], empty[2]
+    uint64_t* full = bars;
+    uint64_t* empty = bars + 2;
     const int c_base = blockIdx.y * HS;  // first hidden unit of this CTA's slab
     const Dims& d = a.d;
     const Buffers& b = a.b;
     const int tid = threadIdx.x;
     const size_t R = (size_t)d.B * a.T;
     const size_t RH = (size_t)d.B * d.Tmax * H;
+    const int ntiles = (int)((R + TR - 1) / TR);
+    if (tid == 0) {
+        for (int q = 0; q < 2; ++q) { tc::mbar_init(&full[q], 1); tc::mbar_init(&empty[q], NW); }
+        tc::mbar_fence_init();
+    }
+    __syncthreads();
+    bool ok = true;
+
+    if (tid >= NTHREADS) {
+        // ---- the row warp: lane = row of a tile.  It runs ahead of the column warps: the saved head outputs of a row
+        // (and its advantage, return and action) become the five output gradients, written to one of two small buffers
+        // that the column warps consume a tile later; the loads are requested three tiles ahead of their use.
+        const int rr = tid - NTHREADS;
+        const float invR = a.gscale / (float)R;  // output gradients are carried times gscale
+        float a_bh[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
+        float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
+        struct RowIn { float4 o4; float v, adv, ret, lpo; int act; bool ok; };
+        auto row_load = [&](int tile) {
+            RowIn in;
+            const size_t i = (size_t)tile * TR + rr;
+            in.ok = tile < ntiles && i < R;
+            if (in.ok) {
+                in.o4 = *reinterpret_cast<const float4*>(b.out5 + i * 8);
+                in.v = b.out5[i * 8 + 4];
+                in.adv = b.adv[i];
+                in.lpo = a.ppo_clip > 0.f ? b.tlogp[i] : 0.f;
+                in.ret = b.ret[i];
+                in.act = b.tact[i];
+            } else {
+                in.o4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                in.v = in.adv = in.ret = in.lpo = 0.f;
+                in.act = 0;
+            }
+            return in;
+        };
+        struct RowOut { float dO[5]; };
+        auto row_compute = [&](const RowIn& in) {
+            RowOut out;
+#pragma unroll
+            for (int c = 0; c < 5; ++c) out.dO[c] = 0.f;
+            if (in.ok) {
+                const float o[4] = {in.o4.x, in.o4.y, in.o4.z, in.o4.w};
+                const float mx = fmaxf(fmaxf(o[0], o[1]), fmaxf(o[2], o[3]));
+                float ex[4], Z = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { ex[c] = expf(o[c] - mx); Z += ex[c]; }
+                const float logZ = logf(Z);
+                float p[4], lp[4], ent = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
+                const float A = in.adv;
+                const float err = in.v - in.ret;
+                const float pf = policy_term(A, in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3], in.lpo, a.ppo_clip, l_pg);
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    out.dO[c] = rnd<PREC>((-A * pf * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
+                out.dO[4] = rnd<PREC>(2.f * a.c_v * err * invR);
+                l_v += err * err;
+                l_ent += ent;
+#pragma unroll
+                for (int c = 0; c < 5; ++c) a_bh[c] += out.dO[c];
+            }
+            return out;
+        };
+        const int g = (int)gridDim.x;
+        RowIn in0 = row_load(blockIdx.x), in1 = row_load(blockIdx.x + g), in2 = row_load(blockIdx.x + 2 * g);
+        int it = 0;
+        for (int tile = blockIdx.x; tile < ntiles; tile += g, ++it) {
+            const int buf = it & 1;
+            const RowIn in3 = row_load(tile + 3 * g);
+            const RowOut out = row_compute(in0);
+            if (it >= 2 && ok) ok = tc::mbar_wait(&empty[buf], ((it >> 1) - 1) & 1);  // the column warps are done with this buffer
+            float4* o4 = reinterpret_cast<float4*>(s_dout + (buf * TR + rr) * 8);
+            o4[0] = make_float4(out.dO[0], out.dO[1], out.dO[2], out.dO[3]);
+            o4[1] = make_float4(out.dO[4], 0.f, 0.f, 0.f);
+            __syncwarp();
+            if (rr == 0) tc::mbar_arrive(&full[buf]);
+            in0 = in1; in1 = in2; in2 = in3;
+        }
+        // dbh and the loss terms of this CTA: a fixed shuffle tree over the lanes (the first slab's CTAs only)
+        float vals[8] = {a_bh[0], a_bh[1], a_bh[2], a_bh[3], a_bh[4], l_pg, l_v, l_ent};
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) vals[c] += __shfl_xor_sync(0xFFFFFFFFu, vals[c], off);
+        if (blockIdx.y == 0) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                if (rr == c) {
+                    if (c < 5) {
+                        for (int q = 0; q < 4; ++q) a.part_small[(size_t)(4 * blockIdx.x + q) * a.small_stride + (size_t)H * 6 + c] = q == 0 ? vals[c] : 0.f;
+                    } else {
+                        b.loss_part[(size_t)blockIdx.x * 4 + (c - 5)] = vals[c];
+                    }
+                }
+            }
+        }
+        if (!ok && rr == 0) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
+        return;
+    }
+
+    // ---- the column warps: thread = (unit pair cp, row group rg of 8 rows)
     uint32_t* g_dh2hi = reinterpret_cast<uint32_t*>(b.dh2);  // pairs of 16-bit elements
     uint32_t* g_dh2lo = g_dh2hi + RH / 2;
-    const float invR = a.gscale / (float)R;  // output gradients are carried times gscale
-    const int ntiles = (int)((R + TR - 1) / TR);
-
-    // column phase: thread = (unit pair cp, row group rg of 8 rows); row phase: the lanes of ONE warp take the 32 rows of
-    // a tile, and the warps take turns (tile after tile), so that no warp issues the row code for a few active lanes
     const int cp = tid % HP2, rg = tid / HP2;
-    const int wid = tid >> 5;
-    const int rr = tid & 31;
+    const int lane = tid & 31;
     float wh_c[2][5];
 #pragma unroll
     for (int cc = 0; cc < 2; ++cc)
@@ -72,14 +172,12 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
     for (int cc = 0; cc < 2; ++cc)
 #pragma unroll
         for (int c = 0; c < 5; ++c) a_wh[cc][c] = 0.f;
-    float a_bh[5] = {0.f, 0.f, 0.f, 0.f, 0.f};  // row threads: sums of dOut over their rows
-    float l_pg = 0.f, l_v = 0.f, l_ent = 0.f;
 
     // h2 tile loads: 16-byte chunks, zero-filled past the last row; a thread's chunks of one tile differ by a fixed number
     // of rows, so one address is formed per tile and the rest are constant offsets.  Always commits a group.
     constexpr int EPC = 16 / ESZ;             // elements per 16-byte chunk
     constexpr int CPR = HS / EPC;             // chunks per row
-    constexpr int RPP = NTHREADS / CPR;       // rows per pass of the whole CTA
+    constexpr int RPP = NTHREADS / CPR;       // rows per pass of the column warps
     static_assert(NTHREADS % CPR == 0 && TR % RPP == 0, "the tile must split into whole passes");
     const int l_r = tid / CPR, l_k = EPC * (tid % CPR);
     const unsigned char* src_base = reinterpret_cast<const unsigned char*>(b.h2) + (size_t)(c_base + l_k) * ESZ;
@@ -90,86 +188,36 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
             const unsigned char* src = src_base + row0 * H * ESZ;
 #pragma unroll
             for (int j = 0; j < TR / RPP; ++j) {
-                const bool ok = row0 + j * RPP < R;
-                cp_async16(dst + (size_t)j * RPP * HS * ESZ, ok ? src + (size_t)j * RPP * H * ESZ : src_base, ok ? 16 : 0);
+                const bool okr = row0 + j * RPP < R;
+                cp_async16(dst + (size_t)j * RPP * HS * ESZ, okr ? src + (size_t)j * RPP * H * ESZ : src_base, okr ? 16 : 0);
             }
         }
         cp_async_commit();
-    };
-    // Row phase, split in two so that the loads are in flight during the column phase.
-    struct RowIn { float4 o4; float v, adv, ret, lpo; int act; bool ok; };
-    auto row_load = [&](int tile) {
-        RowIn in;
-        const size_t i = (size_t)tile * TR + rr;
-        in.ok = tile < ntiles && i < R;
-        if (in.ok) {
-            in.o4 = *reinterpret_cast<const float4*>(b.out5 + i * 8);
-            in.v = b.out5[i * 8 + 4];
-            in.adv = b.adv[i];
-            in.lpo = a.ppo_clip > 0.f ? b.tlogp[i] : 0.f;
-            in.ret = b.ret[i];
-            in.act = b.tact[i];
-        } else {
-            in.o4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            in.v = in.adv = in.ret = in.lpo = 0.f;
-            in.act = 0;
-        }
-        return in;
-    };
-    auto row_finish = [&](const RowIn& in, int buf) {
-        float dO[5] = {0.f, 0.f, 0.f, 0.f, 0.f};
-        if (in.ok) {
-            const float o[4] = {in.o4.x, in.o4.y, in.o4.z, in.o4.w};
-            const float mx = fmaxf(fmaxf(o[0], o[1]), fmaxf(o[2], o[3]));
-            float ex[4], Z = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) { ex[c] = expf(o[c] - mx); Z += ex[c]; }
-            const float logZ = logf(Z);
-            float p[4], lp[4], ent = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) { p[c] = ex[c] / Z; lp[c] = (o[c] - mx) - logZ; ent -= p[c] * lp[c]; }
-            const float A = in.adv;
-            const float err = in.v - in.ret;
-            const float pf = policy_term(A, in.act == 0 ? lp[0] : in.act == 1 ? lp[1] : in.act == 2 ? lp[2] : lp[3], in.lpo, a.ppo_clip, l_pg);
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                dO[c] = rnd<PREC>((-A * pf * ((c == in.act ? 1.f : 0.f) - p[c]) + a.c_e * p[c] * (lp[c] + ent)) * invR);
-            dO[4] = rnd<PREC>(2.f * a.c_v * err * invR);
-            l_v += err * err;
-            l_ent += ent;
-#pragma unroll
-            for (int c = 0; c < 5; ++c) a_bh[c] += dO[c];
-        }
-        float4* o4 = reinterpret_cast<float4*>(s_dout + (buf * TR + rr) * 8);
-        o4[0] = make_float4(dO[0], dO[1], dO[2], dO[3]);
-        o4[1] = make_float4(dO[4], 0.f, 0.f, 0.f);
     };
 
     int it = 0;
 #pragma unroll
     for (int q = 0; q < NST - 1; ++q) load_tile(blockIdx.x + q * (int)gridDim.x, q);
-    if ((int)blockIdx.x < ntiles && wid == 0) row_finish(row_load(blockIdx.x), 0);
     for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++it) {
         const int buf = it & 1;  // dOut buffer of this tile
-        const int next = tile + (int)gridDim.x;
         cp_async_wait<NST - 2>();
-        __syncthreads();  // this tile's h2 and dOut are in place; everyone is done with the buffers of the tile before
+        // this tile's h2 is in place and every column warp is done with the stage that is refilled next (named barrier
+        // 1: the column warps only); its output gradients come from the row warp
+        asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory");
         load_tile(tile + (NST - 1) * (int)gridDim.x, (it + NST - 1) % NST);
-        const bool row_thread = wid == (it + 1) % NW;  // this warp prepares the next tile's output gradients
-        RowIn nin;
-        if (row_thread) nin = row_load(next);
-        // ---- column phase: dh2 = (dOut Wh^T) gated by h2 > 0, as 16-bit planes; running sums of dWh and db2
+        if (ok) ok = tc::mbar_wait(&full[buf], (it >> 1) & 1);
+        // ---- dh2 = (dOut Wh^T) gated by h2 > 0, as 16-bit planes; running sums of dWh and db2
         const unsigned char* h2t = s_h2 + ((size_t)(it % NST) * TR + rg * 8) * HS * ESZ + (size_t)2 * cp * ESZ;
         const float* dt = s_dout + (buf * TR + rg * 8) * 8;
         const size_t i0 = (size_t)tile * TR + rg * 8;
         const int rows_left = i0 < R ? (int)((R - i0) < 8 ? (R - i0) : 8) : 0;
         uint32_t* o_hi = g_dh2hi + (i0 * H + c_base) / 2 + cp;
         uint32_t* o_lo = g_dh2lo + (i0 * H + c_base) / 2 + cp;
-        const bool full = rows_left == 8;  // all but the last tile: stores without per-row predicates
+        const bool fullt = rows_left == 8;  // all but the last tile: stores without per-row predicates
 #pragma unroll
         for (int r = 0; r < 8; ++r) {
             const float4 d0 = *reinterpret_cast<const float4*>(dt + r * 8);
-            const float d4 = dt[r * 8 + 4];
+            const float d0s[1][5] = {{d0.x, d0.y, d0.z, d0.w, dt[r * 8 + 4]}};
             float hv[2];
             if (H2BF) {
                 const uint32_t pk = *reinterpret_cast<const uint32_t*>(h2t + (size_t)r * HS * 2);
@@ -183,17 +231,17 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
             float dh[2];
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
-                float back = d0.x * wh_c[cc][0];
-                back = fmaf(d0.y, wh_c[cc][1], back);
-                back = fmaf(d0.z, wh_c[cc][2], back);
-                back = fmaf(d0.w, wh_c[cc][3], back);
-                back = fmaf(d4, wh_c[cc][4], back);
+                float back = d0s[0][0] * wh_c[cc][0];
+                back = fmaf(d0s[0][1], wh_c[cc][1], back);
+                back = fmaf(d0s[0][2], wh_c[cc][2], back);
+                back = fmaf(d0s[0][3], wh_c[cc][3], back);
+                back = fmaf(d0s[0][4], wh_c[cc][4], back);
                 dh[cc] = hv[cc] > 0.f ? back : 0.f;
-                a_wh[cc][0] = fmaf(hv[cc], d0.x, a_wh[cc][0]);
-                a_wh[cc][1] = fmaf(hv[cc], d0.y, a_wh[cc][1]);
-                a_wh[cc][2] = fmaf(hv[cc], d0.z, a_wh[cc][2]);
-                a_wh[cc][3] = fmaf(hv[cc], d0.w, a_wh[cc][3]);
-                a_wh[cc][4] = fmaf(hv[cc], d4, a_wh[cc][4]);
+                a_wh[cc][0] = fmaf(hv[cc], d0s[0][0], a_wh[cc][0]);
+                a_wh[cc][1] = fmaf(hv[cc], d0s[0][1], a_wh[cc][1]);
+                a_wh[cc][2] = fmaf(hv[cc], d0s[0][2], a_wh[cc][2]);
+                a_wh[cc][3] = fmaf(hv[cc], d0s[0][3], a_wh[cc][3]);
+                a_wh[cc][4] = fmaf(hv[cc], d0s[0][4], a_wh[cc][4]);
             }
             uint32_t phi, plo;
             split2<PREC>(dh[0], dh[1], phi, plo);
@@ -203,16 +251,16 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
             }
             a_b2[0] += dh[0];
             a_b2[1] += dh[1];
-            if (full || r < rows_left) {
+            if (fullt || r < rows_left) {
                 o_hi[r * (H / 2)] = phi;
                 if (PREC == 0) o_lo[r * (H / 2)] = plo;
             }
         }
-        // ---- row phase of the next tile (its inputs were requested before the column phase)
-        if (row_thread && next < ntiles) row_finish(nin, buf ^ 1);
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&empty[buf]);  // the row warp may refill this buffer of output gradients
     }
     cp_async_wait<0>();
-    // ---- per-CTA results: dWh, db2 partials (split index = 4*CTA + row group); dbh and loss partials
+    // ---- per-CTA results: dWh, db2 partials (split index = 4*CTA + row group)
     {
         float* part = a.part_small + (size_t)(4 * blockIdx.x + rg) * a.small_stride;
 #pragma unroll
@@ -222,28 +270,7 @@ __global__ void __launch_bounds__(NW * 32, 2) k_heads_bwd(LearnArgs a_in) {
             part[(size_t)H * 5 + c_base + 2 * cp + cc] = a_b2[cc];
         }
     }
-    __syncthreads();
-    {   // every warp has taken turns at the row phase: fold its lanes (fixed tree), then the warps in index order
-        float vals[8] = {a_bh[0], a_bh[1], a_bh[2], a_bh[3], a_bh[4], l_pg, l_v, l_ent};
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) vals[c] += __shfl_xor_sync(0xFFFFFFFFu, vals[c], off);
-        if (rr == 0) {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) s_fin[wid * 8 + c] = vals[c];
-        }
-    }
-    __syncthreads();
-    if (tid < 8 && blockIdx.y == 0) {  // rows in index order; dbh and the loss terms come from the first slab only
-        float s = 0.f;
-        for (int e = 0; e < NW; ++e) s += s_fin[e * 8 + tid];
-        if (tid < 5) {
-            for (int q = 0; q < 4; ++q) a.part_small[(size_t)(4 * blockIdx.x + q) * a.small_stride + (size_t)H * 6 + tid] = q == 0 ? s : 0.f;
-        } else {
-            b.loss_part[(size_t)blockIdx.x * 4 + (tid - 5)] = s;
-        }
-    }
+    if (!ok && lane == 0) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
 }
 
 // ----------------------------------------------------------------------------------------------------
@@ -1075,7 +1102,7 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     }
     p->ns_env = splits_for(d.B, tiles_ch, 128);
     const size_t tiles32 = (R + 31) / 32;
-    size_t hg = HEADS_GRID;
+    size_t hg = H == 256 ? HEADS_GRID / 2 : HEADS_GRID;  // (the H = 256 kernel takes a whole SM)
     if (d.npol > 1) hg = (size_t)(2 * HEADS_GRID / d.npol > 0 ? 2 * HEADS_GRID / d.npol : 1);  // many policies: the CTAs of all policies fill the GPU together
     p->heads_grid = (int)(tiles32 < hg ? tiles32 : hg);
     p->ns_small = 4 * p->heads_grid;
@@ -1098,13 +1125,13 @@ static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s) 
     if (a.d.npol > 1) {
         if constexpr (PREC == 0 && HS == H && !H2BF) {
             CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
-            k_heads_bwd<H, NW, PREC, HS, H2BF, true><<<dim3(grid, 1, a.d.npol), NW * 32, Cfg::smem_bytes, s>>>(a);
+            k_heads_bwd<H, NW, PREC, HS, H2BF, true><<<dim3(grid, 1, a.d.npol), NW * 32 + 32, Cfg::smem_bytes, s>>>(a);
             return cudaGetLastError();
         }
         return cudaErrorNotSupported;
     }
     CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
-    k_heads_bwd<H, NW, PREC, HS, H2BF><<<dim3(grid, H / HS), NW * 32, Cfg::smem_bytes, s>>>(a);
+    k_heads_bwd<H, NW, PREC, HS, H2BF><<<dim3(grid, H / HS), NW * 32 + 32, Cfg::smem_bytes, s>>>(a);
     return cudaGetLastError();
 }
 
