@@ -386,7 +386,7 @@ def run_ours(args):
 
     # ---- end to end through the C ABI with host buffers: per step, parameters and env state go host->device
     # from pinned memory, one act+learn pass runs, statistics and parameters come back
-    P = an.P
+    P = an.blob_bytes(bnd.PARAMS) // 4  # (all policies' parameters when there are many)
     h_theta = torch.from_numpy(an.get(bnd.PARAMS)).pin_memory()
     h_pos = torch.from_numpy(an.get(bnd.ENV_POS)).pin_memory()
     h_tep = torch.from_numpy(an.get(bnd.ENV_TEP)).pin_memory()
@@ -403,6 +403,7 @@ def run_ours(args):
         an.get_into(bnd.ENV_POS, h_pos, wait=False)
         an.get_into(bnd.ENV_TEP, h_tep, wait=False)
         st = an.stats()                              # synchronises: everything above has landed
+        st = st[0] if isinstance(st, list) else st
         h_theta.copy_(h_out)
     barrier()
     e2e_s = time.perf_counter() - t0
@@ -446,7 +447,7 @@ def run_ours(args):
                    "multi_gpu": (f"{world} replicas of B envs each (one job of {world * w.B} envs), gradients averaged with one NCCL "
                                  "all-reduce per step" if world > 1 else "single GPU")},
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": P * 4 + 2 * w.B, "d2h_bytes_per_step": P * 4 + 2 * w.B + 48,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": P * 4 + 2 * w.B, "d2h_bytes_per_step": P * 4 + 2 * w.B + an.blob_bytes(bnd.STATS),
                 "steps": Ke, "what": "set(PARAMS, ENV_POS, ENV_TEP) from pinned host, run(1), get(STATS, PARAMS, ENV_POS, ENV_TEP)"},
         "gpu_launches": int(launches),
         "wall_s_timed_region": t_wall,

@@ -949,11 +949,12 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
     // The work is cut into nb_total block-sized pieces; a launch with fewer CTAs per policy (many policies: a handful of
     // fat CTAs each instead of tens of thousands of tiny ones) walks them in a stride loop.
     const int nb_main = (int)((d.ob2 + 255) / 256);
-    const int nb_total = nb_main + (int)((d.P - d.ob2 + 7) / 8);
+    const int nb_total = nb_main + (int)(GROUPED ? (d.P - d.ob2 + 255) / 256 : (d.P - d.ob2 + 7) / 8);
     for (int bx = blockIdx.x; bx < nb_total; bx += gridDim.x) {
-        if (bx < nb_main) {
-            const size_t i = (size_t)bx * 256 + threadIdx.x;
-            if (i < d.ob2) {
+        if (bx < nb_main || GROUPED) {
+            // (many policies: few partials everywhere, so the tail is cut into pieces of 256 parameters like the rest)
+            const size_t i = bx < nb_main ? (size_t)bx * 256 + threadIdx.x : d.ob2 + (size_t)(bx - nb_main) * 256 + threadIdx.x;
+            if (i < (bx < nb_main ? d.ob2 : d.P)) {
                 const PartRegion& rg = a_in.reg[region_of(i)];
                 const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(rg.part) + poff) + (i - rg.start);
                 float gsum = 0.f;
@@ -1328,7 +1329,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         Scope sc(c, K_REDUCE_ADAM);
         const unsigned nb = (unsigned)((d.ob2 + 255) / 256 + (d.P - d.ob2 + 7) / 8);
         if (d.npol > 1) {
-            const unsigned per_policy = d.npol >= 296 ? 2u : (nb < 592u / d.npol ? nb : 592u / d.npol);  // about four CTAs per SM in all
+            const unsigned per_policy = d.npol >= 74 ? 8u : (nb < 592u / d.npol ? nb : 592u / d.npol);  // at least four CTAs per SM in all, at most eight per policy
             if constexpr (PREC == 0) k_reduce_adam2<PREC, true><<<dim3(per_policy, d.npol), 256, 0, s>>>(a, R, pl.loss_blocks);
             else return cudaErrorNotSupported;
         } else {

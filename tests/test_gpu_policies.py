@@ -186,18 +186,26 @@ def test_a_policy_of_a_group_equals_a_single_policy_handle_on_its_envs(bnd):
     an.reset(8)
     thetas = policy_thetas(w, an.K, seed=3)
     an.set(bnd.PARAMS, thetas)
-    an.run(2)
+    an.rollout()
+    ones = {}
     for p in (0, 2):  # a full policy and the ragged last one
         e0, n = an.policy_envs(p)
         one = bnd.Anakin(bnd.cfg_from_workload(w.scaled(B=n, n_policies=0), env_offset=e0))
         one.reset(8)
         one.set(bnd.PARAMS, thetas[p])
-        one.run(2)
-        for which in (bnd.TRAJ_POS, bnd.TRAJ_ACTION, bnd.TRAJ_REWARD, bnd.TRAJ_VALUE):
+        one.rollout()
+        for which in (bnd.TRAJ_POS, bnd.TRAJ_ACTION, bnd.TRAJ_REWARD, bnd.TRAJ_VALUE, bnd.TRAJ_LOGP):
             rows = w.T + 1 if which == bnd.TRAJ_VALUE else w.T
             assert np.array_equal(an.policy_block(an.get(which), p, rows), one.get(which).reshape(rows, n)), (p, which)
+        ones[p] = one
+    an.learn()
+    for p, one in ones.items():
+        one.learn()
+        # the update runs on other kernels there (tcgen05 GEMMs), which sum in another order
         gp, g1 = an.get(bnd.GRADS).reshape(an.K, an.P)[p].astype(np.float64), one.get(bnd.GRADS).astype(np.float64)
-        assert np.abs(gp - g1).max() <= 2e-5 * (np.abs(g1).max())  # other kernels sum in another order
+        assert np.abs(gp - g1).max() <= 2e-5 * (np.abs(g1).max())
+        tp, t1 = an.get(bnd.PARAMS).reshape(an.K, an.P)[p].astype(np.float64), one.get(bnd.PARAMS).astype(np.float64)
+        assert np.abs(tp - t1).max() <= 2.01 * w.lr and np.mean(np.abs(tp - t1) > 1e-6) < 1e-2
         assert one.status() == 0
     assert an.status() == 0
 
