@@ -141,8 +141,9 @@ __device__ __forceinline__ void act_and_step(EnvLane& s, const RolloutArgs& a, i
     act_and_step_pre(s, a, env, t, l0, l1, l2, l3, pre);
 }
 
-// Warp 0 holds every owner thread: fold the per-env counters and add them with integer atomics (order-free totals).
-__device__ __forceinline__ void flush_env_stats(EnvLane& s, const RolloutArgs& a) {
+// An owner warp folds its lanes' per-env counters and adds them with integer atomics (order-free totals); the frame count
+// is added once per launch (by one warp of CTA 0: count_frames).
+__device__ __forceinline__ void flush_env_stats(EnvLane& s, const RolloutArgs& a, bool count_frames = true) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         s.n_episodes += __shfl_xor_sync(0xFFFFFFFFu, s.n_episodes, off);
@@ -155,7 +156,7 @@ __device__ __forceinline__ void flush_env_stats(EnvLane& s, const RolloutArgs& a
         if (s.n_episodes) atomicAdd((unsigned long long*)&b.stats->episodes, s.n_episodes);
         if (s.n_goals) atomicAdd((unsigned long long*)&b.stats->goals, s.n_goals);
         if (s.n_epsteps) atomicAdd((unsigned long long*)&b.stats->episode_steps, s.n_epsteps);
-        if (blockIdx.x == 0) atomicAdd((unsigned long long*)&b.stats->frames, (unsigned long long)a.d.B * a.T);
+        if (blockIdx.x == 0 && count_frames) atomicAdd((unsigned long long*)&b.stats->frames, (unsigned long long)a.d.B * a.T);
         if (s.bad) atomicOr(b.status, s.bad);
     }
 }

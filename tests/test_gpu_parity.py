@@ -48,6 +48,10 @@ SMALL = {
     "torus_tp_256": Workload("torus_tp_256", B=140, N=6, H=256, T=12, iters=1, episode_cap=9, env_kind=1),
     "torus_ffma_96": Workload("torus_ffma_96", B=77, N=5, H=96, T=12, iters=1, episode_cap=9, env_kind=1),
     "torus_wide_512": Workload("torus_wide_512", B=70, N=8, H=512, T=6, iters=1, precision=1, episode_cap=9, env_kind=1),
+    # the two-group tcgen05 rollout (H = 128) takes batches of at least one 128-env CTA per SM: a second, ragged wave of
+    # CTAs whose last one has a full first group and 13 envs in the second
+    "tc128_two_groups": Workload("tc128_two_groups", B=148 * 128 + 77, N=8, H=128, T=5, iters=1, episode_cap=4),
+    "tc128_torus": Workload("tc128_torus", B=148 * 128 + 3, N=6, H=128, T=3, iters=1, episode_cap=3, env_kind=1, wall_density=0.3),
 }
 
 
@@ -404,6 +408,31 @@ def test_update_from_set_trajectory_recomputes_the_forward_pass(bnd):
     c.learn()
     d.learn()
     assert (c.get(bnd.GRADS).view(np.uint32) == d.get(bnd.GRADS).view(np.uint32)).all()
+
+
+def test_two_group_rollout_replays_set_trajectories_bitwise(bnd):
+    """The replay mode of the two-group tcgen05 rollout (H = 128, large batch): an update from a trajectory written with
+    anakin_set recomputes the activations with the same kernel and must equal the update from the rollout's own."""
+    w = SMALL["tc128_two_groups"]
+    a = make(bnd, w, debug=0)
+    b = make(bnd, w, debug=0)
+    for an in (a, b):
+        an.reset(12)
+        an.set(bnd.PARAMS, random_params(2, w.P, 0.15))
+        an.rollout()
+    b.set(bnd.TRAJ_POS, b.get(bnd.TRAJ_POS))  # same data, but it invalidates what the rollout saved
+    a.learn()
+    b.learn()
+    for blob in (bnd.GRADS, bnd.PARAMS):
+        assert (a.get(blob).view(np.uint32) == b.get(blob).view(np.uint32)).all()
+    # and two runs of the kernel give the same bits (its groups meet through mbarriers only)
+    c = make(bnd, w, debug=0)
+    c.reset(12)
+    c.set(bnd.PARAMS, random_params(2, w.P, 0.15))
+    c.rollout()
+    c.learn()
+    assert (a.get(bnd.PARAMS).view(np.uint32) == c.get(bnd.PARAMS).view(np.uint32)).all()
+    assert a.status() == 0 and b.status() == 0
 
 
 def test_torus_env_free_running_and_different_from_the_grid(bnd):
