@@ -192,56 +192,62 @@ __global__ void __launch_bounds__(Tc128Cfg::THREADS, 1) k_rollout_tc128(const __
             }
         }
     } else if (worker) {
-        // ---- layer 1 of group g for step t: 16-byte chunks of eight hidden units; all gathers of the agent's W1 row are
-        // in flight before any is used.  Thread (e, q4) covers the chunks c8 = 2 q4, 2 q4 + 1 of both k blocks of env e:
-        // chunk c8 goes to operand row e (hi) and 64 + e (lo) of its block, at the 16-byte position c8 ^ (e % 8) of the
-        // 128-byte row (the 128-byte swizzle of a K-major operand).  Each finished block is announced to the issuer at once.
+        // ---- layer 1 of group g for step t: 16-byte chunks of eight hidden units; all gathers of the agents' W1 rows are
+        // in flight before any is used.  Thread (e, c8) covers chunk c8 of both k blocks of envs e and e + 32 (eight lanes
+        // read 256 contiguous bytes of one row): chunk c8 goes to operand row (hi) and 64 + row (lo) of its block, at the
+        // 16-byte position c8 ^ (row % 8) of the 128-byte row (the 128-byte swizzle of a K-major operand).  Each finished
+        // block is announced to the issuer at once.
         auto gather = [&](int g, int t) {
-            const int e = tid >> 2, q4 = tid & 3;
-            const int eg = g * NE + e;  // env index within the CTA
+            const int e = tid >> 3, c8 = tid & 7;
             unsigned char* bop = s_bop + g * Cfg::B_BYTES;
-            const float* wrow = W1 + (size_t)(C + s_pos[eg]) * H;
             float4 w[2][2][2];
 #pragma unroll
-            for (int kb = 0; kb < 2; ++kb)
+            for (int p = 0; p < 2; ++p) {
+                const float* wrow = W1 + (size_t)(C + s_pos[g * NE + e + 32 * p]) * H + 8 * c8;
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    const float4* wp = reinterpret_cast<const float4*>(wrow + 64 * kb + 8 * (2 * q4 + cc));
-                    w[kb][cc][0] = __ldg(wp);
-                    w[kb][cc][1] = __ldg(wp + 1);
+                for (int kb = 0; kb < 2; ++kb) {
+                    const float4* wp = reinterpret_cast<const float4*>(wrow + 64 * kb);
+                    w[kb][p][0] = __ldg(wp);
+                    w[kb][p][1] = __ldg(wp + 1);
                 }
+            }
             tc::tc_fence_before();  // this thread's reads of the group's accumulators precede the arrivals below
             uint4 hi[2][2], lo[2][2];
 #pragma unroll
             for (int kb = 0; kb < 2; ++kb) {
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    const int c8 = 2 * q4 + cc, k = 64 * kb + 8 * c8;
-                    const float4 b0 = *reinterpret_cast<const float4*>(s_base + eg * H + k);
-                    const float4 b1 = *reinterpret_cast<const float4*>(s_base + eg * H + k + 4);
-                    const float4 w0 = w[kb][cc][0], w1 = w[kb][cc][1];
-                    split2<0>(fmaxf(b0.x + w0.x, 0.f), fmaxf(b0.y + w0.y, 0.f), hi[kb][cc].x, lo[kb][cc].x);
-                    split2<0>(fmaxf(b0.z + w0.z, 0.f), fmaxf(b0.w + w0.w, 0.f), hi[kb][cc].y, lo[kb][cc].y);
-                    split2<0>(fmaxf(b1.x + w1.x, 0.f), fmaxf(b1.y + w1.y, 0.f), hi[kb][cc].z, lo[kb][cc].z);
-                    split2<0>(fmaxf(b1.z + w1.z, 0.f), fmaxf(b1.w + w1.w, 0.f), hi[kb][cc].w, lo[kb][cc].w);
-                    unsigned char* row = bop + kb * Cfg::B_CHUNK + e * 128 + ((c8 ^ (e & 7)) << 4);
-                    *reinterpret_cast<uint4*>(row) = hi[kb][cc];
-                    *reinterpret_cast<uint4*>(row + NE * 128) = lo[kb][cc];
+                for (int p = 0; p < 2; ++p) {
+                    const int er = e + 32 * p, k = 64 * kb + 8 * c8;  // row within the group
+                    const float* bp = s_base + (g * NE + er) * H + k;
+                    const float4 b0 = *reinterpret_cast<const float4*>(bp);
+                    const float4 b1 = *reinterpret_cast<const float4*>(bp + 4);
+                    const float4 w0 = w[kb][p][0], w1 = w[kb][p][1];
+                    split2<0>(fmaxf(b0.x + w0.x, 0.f), fmaxf(b0.y + w0.y, 0.f), hi[kb][p].x, lo[kb][p].x);
+                    split2<0>(fmaxf(b0.z + w0.z, 0.f), fmaxf(b0.w + w0.w, 0.f), hi[kb][p].y, lo[kb][p].y);
+                    split2<0>(fmaxf(b1.x + w1.x, 0.f), fmaxf(b1.y + w1.y, 0.f), hi[kb][p].z, lo[kb][p].z);
+                    split2<0>(fmaxf(b1.z + w1.z, 0.f), fmaxf(b1.w + w1.w, 0.f), hi[kb][p].w, lo[kb][p].w);
+                    unsigned char* row = bop + kb * Cfg::B_CHUNK + er * 128 + ((c8 ^ (er & 7)) << 4);
+                    *reinterpret_cast<uint4*>(row) = hi[kb][p];
+                    *reinterpret_cast<uint4*>(row + NE * 128) = lo[kb][p];
                 }
                 tc::fence_proxy_async();  // ordinary stores -> visible to the tensor core
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&ready[2 * g + kb]);
             }
             // the copies for the update leave after the arrivals
-            if (b.h1 != nullptr && t < a.T && e0 + eg < B) {
+            if (b.h1 != nullptr && t < a.T) {
 #pragma unroll
-                for (int kb = 0; kb < 2; ++kb)
+                for (int p = 0; p < 2; ++p) {
+                    const int env = e0 + g * NE + e + 32 * p;
+                    if (env < B) {
 #pragma unroll
-                    for (int cc = 0; cc < 2; ++cc) {
-                        const size_t gi = ((size_t)t * B + e0 + eg) * H + 64 * kb + 8 * (2 * q4 + cc);
-                        *reinterpret_cast<uint4*>(g_h1hi + gi) = hi[kb][cc];
-                        *reinterpret_cast<uint4*>(g_h1lo + gi) = lo[kb][cc];
+                        for (int kb = 0; kb < 2; ++kb) {
+                            const size_t gi = ((size_t)t * B + env) * H + 64 * kb + 8 * c8;
+                            *reinterpret_cast<uint4*>(g_h1hi + gi) = hi[kb][p];
+                            *reinterpret_cast<uint4*>(g_h1lo + gi) = lo[kb][p];
+                        }
                     }
+                }
             }
         };
         // ---- heads of group g for step t: thread = hidden unit j, the 32 envs of its half of the group
