@@ -4,7 +4,7 @@
 // Acting half of the Anakin minimal unit (Podracer paper, Section 3.1; Figure 2, top), fp32 workloads.  With many envs per
 // SM the rollout is a throughput problem, but a single env group still walks a strictly serial chain per step (gather the
 // agent's first-layer row -> tensor cores -> heads -> sample -> next gather).  The CTA therefore holds TWO independent
-// groups of 64 envs and the same warps alternate between them, so that one group's tensor-core phase and sampling phase
+// groups of 64 envs, each with eight worker warps of its own, so that one group's tensor-core phase and sampling phase
 // fall into the other group's gather and heads phases.  Per group and step:
 //   layer 1   h1 = relu(base + W1[agent row])       gather-add; the fp16 (hi, lo) terms go straight into the swizzled
 //                                                   K-major operand tile [64 hi rows | 64 lo rows] x 128 k
@@ -29,8 +29,8 @@ namespace anakin {
 namespace {
 
 struct Tc128Cfg {
-    static constexpr int H = 128, NE = 64, NG = 2, NWORK = 8;
-    static constexpr int NWT = NWORK * 32;                      // worker threads
+    static constexpr int H = 128, NE = 64, NG = 2, NWORK = 8;   // NWORK worker warps per group
+    static constexpr int NWT = NG * NWORK * 32;                 // worker threads
     static constexpr int NOWN = NG * NE;                        // owner threads: one per env
     static constexpr int THREADS = NWT + NOWN + 32;             // + the issuer warp
     static constexpr int BOX = 64 * 64 * 2;                     // one 64 x 64 box of 16-bit elements
@@ -111,7 +111,10 @@ __global__ void __launch_bounds__(Tc128Cfg::THREADS, 1) k_rollout_tc128(const __
             }
     }
     // worker constants: hidden unit of this thread in the heads phase (its accumulator lane) and the env half it reads
-    const int q = wid & 3, half = (wid >> 2) & 1;
+    const int wg = worker ? wid / Cfg::NWORK : 0;   // the worker's group
+    const int wl = wid % Cfg::NWORK;                // its warp within the group
+    const int tidg = tid % (Cfg::NWORK * 32);       // its thread index within the group
+    const int q = wl & 3, half = (wl >> 2) & 1;
     const int j = 32 * q + lane;
     float b2j = 0.f;
     uint32_t whf_hi[2][2], whf_lo[2][2];  // Wh rows of this warp's 32 hidden units as mma B fragments (k16 x n8), two k steps
@@ -198,7 +201,7 @@ __global__ void __launch_bounds__(Tc128Cfg::THREADS, 1) k_rollout_tc128(const __
         // 16-byte position c8 ^ (row % 8) of the 128-byte row (the 128-byte swizzle of a K-major operand).  Each finished
         // block is announced to the issuer at once.
         auto gather = [&](int g, int t) {
-            const int e = tid >> 3, c8 = tid & 7;
+            const int e = tidg >> 3, c8 = tidg & 7;
             unsigned char* bop = s_bop + g * Cfg::B_BYTES;
             float4 w[2][2][2];
 #pragma unroll
@@ -254,31 +257,43 @@ __global__ void __launch_bounds__(Tc128Cfg::THREADS, 1) k_rollout_tc128(const __
         auto heads = [&](int g, int t) {
             if (ok) ok = tc::mbar_wait(&tfull[g], (uint32_t)t & 1u);
             tc::tc_fence_after();
-            float v[32];
-            {
-                uint32_t r0[32], r1[32], r2[32];
-                const uint32_t lanes = tmem + (uint32_t)(g * Cfg::ACC) + ((uint32_t)(32 * q) << 16);
-                tc::tmem_ld32_nowait(lanes + (uint32_t)(32 * half), r0);         // W2hi x h1hi
-                tc::tmem_ld32_nowait(lanes + (uint32_t)(NE + 32 * half), r1);    // W2hi x h1lo
-                tc::tmem_ld32_nowait(lanes + 128u + (uint32_t)(32 * half), r2);  // W2lo x h1hi
-                tc::tmem_ld_wait();
+            // sixteen envs at a time (registers): accumulator columns -> bias, ReLU -> the h2 rows for the update -> the
+            // fp16 (hi, lo) terms for the head products.  The group's operand tile is free once the step's MMAs have
+            // finished: warp w keeps [32 units][32 envs] fp16 hi and lo planes in its 4 KB of it, rows of 64 bytes whose
+            // 16-byte chunks are XOR-swizzled by (row / 2) % 4 (conflict-free both ways).
+            unsigned char* wsm = s_bop + g * Cfg::B_BYTES + wl * 4096;
+            const int env0 = e0 + g * NE + 32 * half;  // first env of the block this warp holds
+            const bool save_h2 = b.h2 != nullptr && t < a.T;
+            const uint32_t lanes = tmem + (uint32_t)(g * Cfg::ACC) + ((uint32_t)(32 * q) << 16);
 #pragma unroll
-                for (int e = 0; e < 32; ++e) v[e] = fmaxf(((__uint_as_float(r0[e]) + __uint_as_float(r1[e])) + __uint_as_float(r2[e])) + b2j, 0.f);
-            }
-            // head partials over this warp's 32 hidden units on the warp-level tensor path.  The group's operand tile is
-            // free once the step's MMAs have finished: warp w keeps [32 units][32 envs] fp16 hi and lo planes in its 4 KB of
-            // it, rows of 64 bytes whose 16-byte chunks are XOR-swizzled by (row / 2) % 4 (conflict-free both ways).
-            unsigned char* wsm = s_bop + g * Cfg::B_BYTES + wid * 4096;
+            for (int hf = 0; hf < 2; ++hf) {
+                float v[16];
+                {
+                    uint32_t r0[16], r1[16], r2[16];
+                    tc::tmem_ld16_nowait(lanes + (uint32_t)(32 * half + 16 * hf), r0);         // W2hi x h1hi
+                    tc::tmem_ld16_nowait(lanes + (uint32_t)(NE + 32 * half + 16 * hf), r1);    // W2hi x h1lo
+                    tc::tmem_ld16_nowait(lanes + 128u + (uint32_t)(32 * half + 16 * hf), r2);  // W2lo x h1hi
+                    tc::tmem_ld_wait();
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint4 hi, lo;
-                split2<0>(v[8 * c4 + 0], v[8 * c4 + 1], hi.x, lo.x);
-                split2<0>(v[8 * c4 + 2], v[8 * c4 + 3], hi.y, lo.y);
-                split2<0>(v[8 * c4 + 4], v[8 * c4 + 5], hi.z, lo.z);
-                split2<0>(v[8 * c4 + 6], v[8 * c4 + 7], hi.w, lo.w);
-                const int off = lane * 64 + ((c4 ^ ((lane >> 1) & 3)) << 4);
-                *reinterpret_cast<uint4*>(wsm + off) = hi;
-                *reinterpret_cast<uint4*>(wsm + 2048 + off) = lo;
+                    for (int e = 0; e < 16; ++e) v[e] = fmaxf(((__uint_as_float(r0[e]) + __uint_as_float(r1[e])) + __uint_as_float(r2[e])) + b2j, 0.f);
+                }
+                if (save_h2) {  // one 128-byte line per env and warp
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        if (env0 + 16 * hf + e < B) b.h2[((size_t)t * B + env0 + 16 * hf + e) * H + j] = v[e];
+                }
+#pragma unroll
+                for (int c2 = 0; c2 < 2; ++c2) {
+                    const int c4 = 2 * hf + c2;
+                    uint4 hi, lo;
+                    split2<0>(v[8 * c2 + 0], v[8 * c2 + 1], hi.x, lo.x);
+                    split2<0>(v[8 * c2 + 2], v[8 * c2 + 3], hi.y, lo.y);
+                    split2<0>(v[8 * c2 + 4], v[8 * c2 + 5], hi.z, lo.z);
+                    split2<0>(v[8 * c2 + 6], v[8 * c2 + 7], hi.w, lo.w);
+                    const int off = lane * 64 + ((c4 ^ ((lane >> 1) & 3)) << 4);
+                    *reinterpret_cast<uint4*>(wsm + off) = hi;
+                    *reinterpret_cast<uint4*>(wsm + 2048 + off) = lo;
+                }
             }
             __syncwarp();
             float acc[2][4];
@@ -321,25 +336,15 @@ __global__ void __launch_bounds__(Tc128Cfg::THREADS, 1) k_rollout_tc128(const __
             }
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&pdone[g]);
-            // h2 for the update: one 128-byte line per env
-            const int env0 = e0 + g * NE + 32 * half;  // first env of the block this warp holds
-            if (b.h2 != nullptr && t < a.T) {
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    if (env0 + e < B) b.h2[((size_t)t * B + env0 + e) * H + j] = v[e];
-            }
         };
-        gather(0, 0);
-        gather(1, 0);
+        // a group's eight warps walk its steps on their own; the two groups drift apart by themselves, so that one group's
+        // tensor-core and sampling phases fall into the other's gather and heads phases
+        gather(wg, 0);
         for (int t = 0; t <= t_end; ++t) {
-            heads(0, t);
-            heads(1, t);
+            heads(wg, t);
             if (t < t_end) {
-#pragma unroll
-                for (int g = 0; g < NG; ++g) {
-                    if (ok) ok = tc::mbar_wait(&posrdy[g], (uint32_t)t & 1u);  // the owners have published the positions after step t
-                    gather(g, t + 1);
-                }
+                if (ok) ok = tc::mbar_wait(&posrdy[wg], (uint32_t)t & 1u);  // the owners have published the positions after step t
+                gather(wg, t + 1);
             }
         }
     } else if (ownerw) {
