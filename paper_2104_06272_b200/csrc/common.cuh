@@ -331,6 +331,7 @@ cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s); 
 bool rollout_mma_supported(int H);
 bool rollout_uses_fragments(int H, int prec);  // the warp-level kernel (and with it the fragment copies of W2) serves this shape
 cudaError_t launch_rollout_tc128(const RolloutArgs& a, cudaStream_t s);  // two-group tcgen05 rollout (H = 128, fp32, large batches); cudaErrorNotSupported otherwise
+cudaError_t launch_rollout_pair2(const RolloutArgs& a, cudaStream_t s);  // two env groups per CTA pair (H = 256, fp32, large batches); cudaErrorNotSupported otherwise
 cudaError_t launch_rollout_pair(const RolloutArgs& a, cudaStream_t s);  // CTA-pair tcgen05 rollout (H = 256, fp32); cudaErrorNotSupported otherwise
 bool wide_supported(int H, int prec);         // bf16 workload with a hidden layer too wide for the persistent rollout
 bool tensor_path_supported(int H, int prec);  // either tensor-core path: the update reuses activations the rollout saved

@@ -370,7 +370,11 @@ bool rollout_uses_fragments(int H, int prec) { return rollout_mma_supported(H) &
 // Returns cudaErrorNotSupported when the shape is not covered by the tensor-pipe kernel.
 cudaError_t launch_rollout_mma(const RolloutArgs& a, int prec, cudaStream_t s) {
     if (!rollout_mma_supported(a.d.H)) return cudaErrorNotSupported;
-    if (prec == 0 && a.d.npol <= 1 && a.d.H == 256) return launch_rollout_pair(a, s);  // the CTA-pair kernel on the 5th-generation tensor cores
+    if (prec == 0 && a.d.npol <= 1 && a.d.H == 256) {  // the CTA-pair kernels on the 5th-generation tensor cores
+        const cudaError_t e = launch_rollout_pair2(a, s);  // large batches: two env groups per pair
+        if (e != cudaErrorNotSupported) return e;
+        return launch_rollout_pair(a, s);
+    }
     if (prec == 0 && a.d.npol <= 1 && a.d.H == 128) {  // large batches: two env groups per CTA on the 5th-generation tensor cores
         const cudaError_t e = launch_rollout_tc128(a, s);
         if (e != cudaErrorNotSupported) return e;

@@ -51,6 +51,9 @@ SMALL = {
     # the two-group tcgen05 rollout (H = 128) takes batches of at least one 128-env CTA per SM: a second, ragged wave of
     # CTAs whose last one has a full first group and 13 envs in the second
     "tc128_two_groups": Workload("tc128_two_groups", B=148 * 128 + 77, N=8, H=128, T=5, iters=1, episode_cap=4),
+    # the two-group CTA-pair rollout (H = 256) takes batches of at least 74 clusters of 128 envs: a ragged second wave whose
+    # last cluster has a full first group and 21 envs (all in its first CTA) in the second
+    "pair2_two_groups": Workload("pair2_two_groups", B=74 * 128 + 85, N=10, H=256, T=4, iters=1, episode_cap=3),
     "tc128_torus": Workload("tc128_torus", B=148 * 128 + 3, N=6, H=128, T=6, iters=1, episode_cap=5, env_kind=1, wall_density=0.3),
 }
 
@@ -414,10 +417,11 @@ def test_update_from_set_trajectory_recomputes_the_forward_pass(bnd):
     assert (c.get(bnd.GRADS).view(np.uint32) == d.get(bnd.GRADS).view(np.uint32)).all()
 
 
-def test_two_group_rollout_replays_set_trajectories_bitwise(bnd):
-    """The replay mode of the two-group tcgen05 rollout (H = 128, large batch): an update from a trajectory written with
-    anakin_set recomputes the activations with the same kernel and must equal the update from the rollout's own."""
-    w = SMALL["tc128_two_groups"]
+@pytest.mark.parametrize("name", ["tc128_two_groups", "pair2_two_groups"])
+def test_two_group_rollout_replays_set_trajectories_bitwise(bnd, name):
+    """The replay mode of the two-group tcgen05 rollouts (H = 128 and H = 256, large batch): an update from a trajectory
+    written with anakin_set recomputes the activations with the same kernel and must equal the update from the rollout's own."""
+    w = SMALL[name]
     a = make(bnd, w, debug=0)
     b = make(bnd, w, debug=0)
     for an in (a, b):
