@@ -406,7 +406,7 @@ def run_ours(args):
         an.get_into(bnd.ENV_TEP, h_tep, wait=False)
         st = an.stats()                              # synchronises: everything above has landed
         st = st[0] if isinstance(st, list) else st
-        h_theta.copy_(h_out)
+        h_theta, h_out = h_out, h_theta              # the parameters that came back are the next step's input
     barrier()
     e2e_s = time.perf_counter() - t0
     e2e_s = max_over_ranks(e2e_s, world, "cuda")

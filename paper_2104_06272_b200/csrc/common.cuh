@@ -201,6 +201,19 @@ struct LearnArgs {
 };
 
 #ifdef __CUDACC__
+// One Adam step of one parameter (Kingma & Ba, Algorithm 1):
+//   m = b1 m + (1-b1) g;  v = b2 v + (1-b2) g^2;  theta -= lr (m/(1-b1^k)) / (sqrt(v/(1-b2^k)) + eps)
+// Every product and sum is rounded on its own (no contraction into fused multiply-adds), so that every kernel that
+// takes the step gets the same bits, whatever surrounds the call.
+struct AdamIn { float m, v, theta; };
+__device__ __forceinline__ AdamIn adam_arith(const LearnArgs& a, const AdamIn& in, float g) {
+    AdamIn o;
+    o.m = __fadd_rn(__fmul_rn(a.beta1, in.m), __fmul_rn(1.f - a.beta1, g));
+    o.v = __fadd_rn(__fmul_rn(a.beta2, in.v), __fmul_rn(__fmul_rn(1.f - a.beta2, g), g));
+    const float mhat = __fdiv_rn(o.m, a.bc1), vhat = __fdiv_rn(o.v, a.bc2);
+    o.theta = __fsub_rn(in.theta, __fdiv_rn(__fmul_rn(a.lr, mhat), __fadd_rn(__fsqrt_rn(vhat), a.eps)));
+    return o;
+}
 __device__ __forceinline__ void select_policy(RolloutArgs& a, int pol) {
     if (a.forced) a.forced += (size_t)pol * a.T * a.d.B;  // forced actions come as one [T][B_p] block per policy
     select_policy(a.d, a.b, pol);

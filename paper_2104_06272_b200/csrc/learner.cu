@@ -274,26 +274,18 @@ __global__ void __launch_bounds__(256) k_sum_over_t(Dims d, Buffers b, int T) {
 // Block 0 also folds the loss partials into the statistics.
 template <int PREC>
 __global__ void __launch_bounds__(256) k_reduce_adam(LearnArgs a, size_t R, int loss_blocks) {
-    __shared__ float s_c[2];
     const Dims& d = a.d;
     const Buffers& b = a.b;
-    if (threadIdx.x == 0) {
-        s_c[0] = a.bc1;
-        s_c[1] = a.bc2;
-    }
-    __syncthreads();
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < d.P) {
         float g = 0.f;
         for (int s = 0; s < a.NS; ++s) g += b.part[(size_t)s * d.P + i];
         b.grads[i] = g;
         if (a.phase == 0) {  // phase 1 stops at the gradient
-            const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * g;
-            const float v = a.beta2 * b.adam_v[i] + (1.f - a.beta2) * g * g;
-            b.adam_m[i] = m;
-            b.adam_v[i] = v;
-            const float mhat = m / s_c[0], vhat = v / s_c[1];
-            const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
+            const AdamIn o = adam_arith(a, AdamIn{b.adam_m[i], b.adam_v[i], b.theta[i]}, g);
+            b.adam_m[i] = o.m;
+            b.adam_v[i] = o.v;
+            const float th = o.theta;
             b.theta[i] = th;
             if (PREC == 1) {
                 const bool is_bias = (i >= d.ob1 && i < d.oW2) || (i >= d.ob2 && i < d.oWh) || i >= d.obh;

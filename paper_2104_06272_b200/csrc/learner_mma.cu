@@ -856,17 +856,18 @@ static cudaError_t launch_gemm_tn(const GemmTnArgs& g, int rows_m, int splits, c
 }
 
 // One Adam step of parameter i with gradient g (Kingma & Ba, Algorithm 1), plus the refreshed 16-bit copies.
-// c[0] = 1 - beta1^k, c[1] = 1 - beta2^k.
+// (a parameter's state is loaded ahead of its gradient sum: one memory round trip less)
+__device__ __forceinline__ AdamIn adam_load(const LearnArgs& a, size_t i) {
+    return AdamIn{a.b.adam_m[i], a.b.adam_v[i], a.b.theta[i]};
+}
 template <int PREC>
-__device__ __forceinline__ void adam_step(const LearnArgs& a, const float* c, size_t i, float g) {
+__device__ __forceinline__ void adam_step(const LearnArgs& a, size_t i, float g, const AdamIn& in) {
     const Dims& d = a.d;
     const Buffers& b = a.b;
-    const float m = a.beta1 * b.adam_m[i] + (1.f - a.beta1) * g;
-    const float v = a.beta2 * b.adam_v[i] + (1.f - a.beta2) * g * g;
-    b.adam_m[i] = m;
-    b.adam_v[i] = v;
-    const float mhat = m / c[0], vhat = v / c[1];
-    const float th = b.theta[i] - a.lr * mhat / (sqrtf(vhat) + a.eps);
+    const AdamIn o = adam_arith(a, in, g);
+    b.adam_m[i] = o.m;
+    b.adam_v[i] = o.v;
+    const float th = o.theta;
     b.theta[i] = th;
     float thc = th;
     if (PREC == 1) {
@@ -895,12 +896,6 @@ template <int PREC, bool GROUPED>
 __global__ void __launch_bounds__(256) k_adam_only(LearnArgs a_in) {
     const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.y);  // many policies: grid.y = policy
     const LearnArgs& a = pa.a;
-    __shared__ float s_c[2];
-    if (threadIdx.x == 0) {
-        s_c[0] = a.bc1;
-        s_c[1] = a.bc2;
-    }
-    __syncthreads();
     const size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
     if (i < a.d.P) {
         float g = a.b.grads[i];
@@ -908,7 +903,7 @@ __global__ void __launch_bounds__(256) k_adam_only(LearnArgs a_in) {
             g = g / a.grad_div;
             a.b.grads[i] = g;
         }
-        adam_step<PREC>(a, s_c, i, g);
+        adam_step<PREC>(a, i, g, adam_load(a, i));
     }
 }
 
@@ -921,20 +916,16 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
     const LearnArgs& a = pa.a;
     const size_t R = GROUPED ? (size_t)a.d.B * a.T : R_in;  // rows of THIS policy
     const size_t poff = GROUPED ? (size_t)blockIdx.y * a_in.d.pstride : 0;  // byte offset of this policy's partials
-    __shared__ float s_c[2];
     __shared__ float s_tail[32][8];
     const Dims& d = a.d;
     const Buffers& b = a.b;
-    if (threadIdx.x == 0) {
-        s_c[0] = a.bc1;
-        s_c[1] = a.bc2;
-    }
-    __syncthreads();
     // Batch-mean gradient of parameter i, then (phase 0) its Adam step.
-    auto apply = [&](size_t i, float gsum) {
+    // (the parameter's Adam state is fetched before its partials, so that the two do not queue up behind one another)
+    auto state_of = [&](size_t i) { return a.phase == 0 ? adam_load(a, i) : AdamIn{0.f, 0.f, 0.f}; };
+    auto apply = [&](size_t i, float gsum, const AdamIn& in) {
         gsum *= a.inv_gscale;  // exact: a power of two
         b.grads[i] = gsum;
-        if (a.phase == 0) adam_step<PREC>(a, s_c, i, gsum);
+        if (a.phase == 0) adam_step<PREC>(a, i, gsum, in);
     };
     auto region_of = [&](size_t i) {
         int r = 0;
@@ -957,6 +948,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
             if (i < (bx < nb_main ? d.ob2 : d.P)) {
                 const PartRegion& rg = a_in.reg[region_of(i)];
                 const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(rg.part) + poff) + (i - rg.start);
+                const AdamIn in = state_of(i);
                 float gsum = 0.f;
                 // thirty-two loads in flight per memory round trip (the ragged last batch is predicated, not split up);
                 // the additions stay in index order
@@ -968,7 +960,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
                     for (int q = 0; q < 32; ++q)
                         if (s + q < rg.ns) gsum += v[q];
                 }
-                apply(i, gsum);
+                apply(i, gsum, in);
             }
         } else {
             // eight consecutive parameters per CTA: thread = (parameter tid % 8, partial group tid / 8); a group's eight
@@ -977,7 +969,9 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
             const int pi = threadIdx.x & 7, grp = threadIdx.x >> 3;
             const size_t i = d.ob2 + (size_t)(bx - nb_main) * 8 + pi;
             float gsum = 0.f;
+            AdamIn in{0.f, 0.f, 0.f};
             if (i < d.P) {
+                if (grp == 0) in = state_of(i);
                 const PartRegion& rg = a_in.reg[region_of(i)];
                 const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(rg.part) + poff) + (i - rg.start);
                 int s = grp;
@@ -997,7 +991,7 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
                 float tot = 0.f;
 #pragma unroll
                 for (int g2 = 0; g2 < 32; ++g2) tot += s_tail[g2][pi];
-                apply(i, tot);
+                apply(i, tot, in);
             }
         }
         // Loss statistics: the first warp of the last CTA (the one with the least other work) adds the per-CTA partials of
