@@ -359,6 +359,7 @@ cudaError_t launch_vtrace(const Dims& d, const Buffers& b, int T, float gamma, f
 cudaError_t launch_learn(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_learn_mma(const LearnArgs& a, int prec, const Ctx& c);
 cudaError_t launch_adam_only(const LearnArgs& a, int prec, const Ctx& c);  // Adam from GRADS as they stand
+constexpr int DH1A_UNITS = 128;  // hidden units (columns of dh1) one CTA of the fused dh1 + agent-plane kernel owns
 bool dh1_agent_tc_supported(const Dims& d);
 // dh1, S and the agent plane of dW1 in one tcgen05 kernel; cudaErrorNotSupported if not covered
 cudaError_t launch_dh1_agent_tc(const LearnArgs& a, int prec, int grid_x, float* part_agent, size_t part_stride, cudaStream_t s);

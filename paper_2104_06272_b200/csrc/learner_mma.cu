@@ -1061,7 +1061,7 @@ static int splits_for(int K, int tiles, int min_k) {
 // Launch shape of the fused dh1 + agent-plane kernel: one CTA per SM.  Few env tiles: slice the steps; many: let a CTA
 // walk several tiles, so that the number of agent-plane partials stays at most one per CTA row.
 static void dh1a_shape(const Dims& d, int T, int* grid_x, int* ts) {
-    const int m_tiles = (d.B + 127) / 128, n_tiles = d.H / 64;
+    const int m_tiles = (d.B + 127) / 128, n_tiles = d.H / DH1A_UNITS;
     *grid_x = m_tiles;
     *ts = 1;
     if (m_tiles * n_tiles >= 148) {
