@@ -65,6 +65,8 @@ struct Dh1aCfg {
     static_assert(AGENT_COL + 128 <= TMEM_COLS, "tensor memory: W2 planes + three 128-column accumulators");
     static constexpr int W_BOX = BN * 128;               // W2 lo: 128 unit rows x 64 k (16 KB), K-major
     static constexpr int W_BYTES = W_LO_SMEM ? NCH * W_BOX : 0;
+    // the planes bound for tensor memory are staged by TMA in the (still unused) dh1^T tile where they fit
+    static constexpr bool W_STAGED = WT_PL * NCH * W_BOX <= PL * 2 * BN * 128;
     static constexpr int BARS = 256;
     static constexpr int MAX_SMEM = 232448 - 1024;       // 227 KB per CTA minus alignment slack
     static constexpr int RING = MAX_SMEM - BARS - W_BYTES - D_TILE - O_TILE - G_TILE;
@@ -74,7 +76,7 @@ struct Dh1aCfg {
 };
 
 struct Dh1aMaps {
-    CUtensorMap a_hi, a_lo, gate, w_lo;
+    CUtensorMap a_hi, a_lo, gate, w_hi, w_lo;
 };
 
 template <int H, int PREC>
@@ -101,7 +103,8 @@ __device__ __forceinline__ void dh1a_body(const Dh1aMaps& maps, const LearnArgs&
     uint64_t* tiles_free = tiles_full + 1;  // the agent MMAs that read them have finished
     uint64_t* gfull = tiles_free + 1;       // gate tile landed
     uint64_t* gempty = gfull + 1;           // gate tile read (the epilogue warps arrive)
-    uint32_t* tmem_slot = (uint32_t*)(gempty + 1);
+    uint64_t* wstage = gempty + 1;          // the W2 rows bound for tensor memory have landed in their staging boxes
+    uint32_t* tmem_slot = (uint32_t*)(wstage + 1);
 
     const Dims& d = a.d;
     const Buffers& b = a.b;
@@ -128,6 +131,7 @@ __device__ __forceinline__ void dh1a_body(const Dh1aMaps& maps, const LearnArgs&
         tc::mbar_init(tiles_free, 1);
         tc::mbar_init(gfull, 1);
         tc::mbar_init(gempty, Cfg::EPI_WARPS);
+        tc::mbar_init(wstage, 1);
         tc::mbar_fence_init();
     }
     if (wid == 2) {
@@ -163,7 +167,14 @@ __device__ __forceinline__ void dh1a_body(const Dh1aMaps& maps, const LearnArgs&
     };
 
     if (wid == 0) {
-        if (lane == 0) {  // ---- TMA producer: this CTA's rows of the W2 lo plane once, then the dh2 boxes
+        if (lane == 0) {  // ---- TMA producer: this CTA's rows of W2 once, then the dh2 boxes
+            if (Cfg::W_STAGED) {  // the planes bound for tensor memory: box [plane][k chunk] in the dh1^T tile
+                tc::mbar_expect_tx(wstage, Cfg::WT_PL * NCH * Cfg::W_BOX);
+#pragma unroll
+                for (int pl = 0; pl < Cfg::WT_PL; ++pl)
+#pragma unroll
+                    for (int kc = 0; kc < NCH; ++kc) tc::tma_load_2d(sD + (pl * NCH + kc) * Cfg::W_BOX, pl ? &maps.w_lo : &maps.w_hi, wstage, kc * KC, n0);
+            }
             if (Cfg::W_LO_SMEM) {
                 if (leader) tc::mbar_expect_tx(wfull, NCTA * Cfg::W_BYTES);  // the boxes of both CTAs
                 const uint32_t bar = tc::mapa(tc::smem_u32(wfull), 0);
@@ -292,21 +303,39 @@ __device__ __forceinline__ void dh1a_body(const Dh1aMaps& maps, const LearnArgs&
         const uint32_t lane_base = (uint32_t)(32 * q) << 16;
         {   // This CTA's rows of W2 go into tensor memory once: row n0 + j = lane j, two k per column (they are stored
             // that way), the hi plane in columns [0, H/2), the lo plane behind it.  The two warps of a lane quarter share the columns.
-            // (every load of a plane is in flight before the first store)
+            // The rows come through shared memory (TMA boxes of 64 k, 128-byte swizzle): k chunk kc of row j is the 128
+            // bytes at box kc, row j, its 16-byte pieces permuted by j % 8.
+            if (!Cfg::W_STAGED) {  // (no room to stage them: straight from global memory)
 #pragma unroll 1
-            for (int pl = 0; pl < Cfg::WT_PL; ++pl) {
-                const uint32_t* wrow = reinterpret_cast<const uint32_t*>((pl ? b.w2p_lo : b.w2p_hi) + (size_t)(n0 + j) * H) + half * (H / 4);
-                uint32_t r[H / 128][32];
+                for (int pl = 0; pl < Cfg::WT_PL; ++pl) {
+                    const uint32_t* wrow = reinterpret_cast<const uint32_t*>((pl ? b.w2p_lo : b.w2p_hi) + (size_t)(n0 + j) * H) + half * (H / 4);
+#pragma unroll 1
+                    for (int cc = 0; cc < H / 128; ++cc) {
+                        uint32_t r[32];
 #pragma unroll
-                for (int cc = 0; cc < H / 128; ++cc) {
-#pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
-                        const uint4 v = __ldg(reinterpret_cast<const uint4*>(wrow + 32 * cc + c));
-                        r[cc][c] = v.x; r[cc][c + 1] = v.y; r[cc][c + 2] = v.z; r[cc][c + 3] = v.w;
+                        for (int c = 0; c < 32; c += 4) {
+                            const uint4 v = __ldg(reinterpret_cast<const uint4*>(wrow + 32 * cc + c));
+                            r[c] = v.x; r[c + 1] = v.y; r[c + 2] = v.z; r[c + 3] = v.w;
+                        }
+                        tc::tmem_st32(tmem + lane_base + (uint32_t)(pl * (H / 2) + half * (H / 4) + 32 * cc), r);
                     }
                 }
+            } else if ((ok = tc::mbar_wait(wstage, 0))) {
+#pragma unroll 1
+                for (int pl = 0; pl < Cfg::WT_PL; ++pl) {
 #pragma unroll
-                for (int cc = 0; cc < H / 128; ++cc) tc::tmem_st32(tmem + lane_base + (uint32_t)(pl * (H / 2) + half * (H / 4) + 32 * cc), r[cc]);
+                    for (int cc = 0; cc < H / 128; ++cc) {  // 32 columns = 64 k = one box row
+                        const int kc = half * (H / 128) + cc;
+                        const unsigned char* row = sD + (pl * NCH + kc) * Cfg::W_BOX + j * 128;
+                        uint32_t r[32];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const uint4 v = *reinterpret_cast<const uint4*>(row + ((c ^ (j & 7)) << 4));
+                            r[4 * c] = v.x; r[4 * c + 1] = v.y; r[4 * c + 2] = v.z; r[4 * c + 3] = v.w;
+                        }
+                        tc::tmem_st32(tmem + lane_base + (uint32_t)(pl * (H / 2) + kc * 32), r);
+                    }
+                }
             }
             tc::tmem_st_wait();
             tc::tc_fence_before();
@@ -463,7 +492,8 @@ cudaError_t launch_t(const LearnArgs& a, int grid_x, float* part_agent, size_t p
     if (!make_tensor_map_2d(&maps.a_hi, dh2hi, R, H, Cfg::ROWS, bf)) return cudaErrorNotSupported;
     if (Cfg::PL == 2 && !make_tensor_map_2d(&maps.a_lo, dh2hi + RH, R, H, Cfg::ROWS, bf)) return cudaErrorNotSupported;
     if (!make_tensor_map_2d(&maps.gate, b.h1, R, H, 128, bf)) return cudaErrorNotSupported;  // the hi plane of h1
-    if (Cfg::W_LO_SMEM && !make_tensor_map_2d(&maps.w_lo, b.w2p_lo, H, H, 128, bf)) return cudaErrorNotSupported;
+    if (!make_tensor_map_2d(&maps.w_hi, b.w2p_hi, H, H, 128, bf)) return cudaErrorNotSupported;
+    if (Cfg::PL == 2 && !make_tensor_map_2d(&maps.w_lo, b.w2p_lo, H, H, 128, bf)) return cudaErrorNotSupported;
     if constexpr (Cfg::PAIR) {  // the two CTAs of a pair are neighbours in x; each pair takes all H units
         cudaError_t e = cudaFuncSetAttribute(k_dh1a_pair<H, PREC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes);
         if (e != cudaSuccess) return e;
