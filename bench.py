@@ -135,7 +135,7 @@ class ClockSampler:
 # not reported.
 PROFILE_OF = {
     ("throughput", "rollout"): ("rollout_pair__throughput.md", "rollout_pair.cu"),
-    ("throughput", "dh1"): ("dh1a_tc__throughput.md", "dh1a_tc.cu"),
+    ("throughput", "dh1"): ("dh1a_pair__throughput.md", "dh1a_tc.cu"),
     ("throughput", "dw2"): ("gemm_tn_tc_dw2__throughput.md", "gemm_tc.cu"),
     ("throughput", "heads_bwd"): ("heads_bwd__throughput.md", "learner_mma.cu"),
     ("throughput", "reduce_adam"): ("reduce_adam2__throughput.md", "learner_mma.cu"),
