@@ -950,14 +950,16 @@ __global__ void __launch_bounds__(256) k_reduce_adam2(LearnArgs a_in, size_t R_i
                 const float* p = reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(rg.part) + poff) + (i - rg.start);
                 const AdamIn in = state_of(i);
                 float gsum = 0.f;
-                // thirty-two loads in flight per memory round trip (the ragged last batch is predicated, not split up);
-                // the additions stay in index order
-                for (int s = 0; s < rg.ns; s += 32) {
-                    float v[32];
+                // NF loads in flight per memory round trip (the ragged last batch is predicated, not split up); the
+                // additions stay in index order.  Many policies: a region has a handful of partials, and the registers
+                // a wide batch costs would halve the CTAs per SM.
+                constexpr int NF = GROUPED ? 8 : 32;
+                for (int s = 0; s < rg.ns; s += NF) {
+                    float v[NF];
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) v[q] = s + q < rg.ns ? p[(size_t)(s + q) * rg.stride] : 0.f;
+                    for (int q = 0; q < NF; ++q) v[q] = s + q < rg.ns ? p[(size_t)(s + q) * rg.stride] : 0.f;
 #pragma unroll
-                    for (int q = 0; q < 32; ++q)
+                    for (int q = 0; q < NF; ++q)
                         if (s + q < rg.ns) gsum += v[q];
                 }
                 apply(i, gsum, in);
