@@ -116,6 +116,7 @@ size_t carve(const anakin_cfg& c, const Dims& d, int NS, unsigned char* base, Bu
     b.w2p_hi = tensor ? (uint16_t*)take(H * H * 2) : nullptr;
     b.w2p_lo = mma ? (uint16_t*)take(H * H * 2) : nullptr;
     b.h1 = (float*)take(R * H * 4);
+    b.gate1 = (dh1_agent_tc_supported(d) && policies_of(c) <= 1) ? (uint8_t*)take(R * (H / 8)) : nullptr;  // what the fused dh1 kernel gates with
     b.h2 = (float*)take(R * H * 4);
     b.out5 = tensor ? (float*)take(R * 8 * 4) : nullptr;
     b.vboot = tensor ? (float*)take(B * 4) : nullptr;

@@ -73,6 +73,7 @@ struct Buffers {
     uint16_t* w2p_hi;  // [H][H] W2 row-major as 16-bit hi / lo planes (B operand of the dh1 kernel)
     uint16_t* w2p_lo;
     float* h1;       // [R][H]
+    uint8_t* gate1;  // [R][H/8] layer-1 ReLU gates of every recorded row: bit j%8 of byte j/8 = the 16-bit hi term of h1[j] is not zero (null: not kept)
     float* h2;       // [R][H]
     float* out5;     // [R][8] head outputs (4 logits, value) of every recorded row, saved by the tensor-pipe rollout
     float* vboot;    // [B] value of the state after the last recorded step under the CURRENT parameters (replay mode 2)
@@ -101,7 +102,7 @@ __device__ __forceinline__ void shift_buffers(Buffers& b, size_t off) {
     shift_ptr(b.tpos, off); shift_ptr(b.tact, off); shift_ptr(b.tdone, off); shift_ptr(b.trew, off); shift_ptr(b.tval, off);
     shift_ptr(b.tlogp, off); shift_ptr(b.adv, off); shift_ptr(b.ret, off); shift_ptr(b.dbg_logits, off); shift_ptr(b.dbg_gates, off);
     shift_ptr(b.base, off); shift_ptr(b.w2f_hi, off); shift_ptr(b.w2f_lo, off);
-    shift_ptr(b.w2p_hi, off); shift_ptr(b.w2p_lo, off); shift_ptr(b.h1, off); shift_ptr(b.h2, off); shift_ptr(b.out5, off);
+    shift_ptr(b.w2p_hi, off); shift_ptr(b.w2p_lo, off); shift_ptr(b.h1, off); shift_ptr(b.gate1, off); shift_ptr(b.h2, off); shift_ptr(b.out5, off);
     shift_ptr(b.vboot, off); shift_ptr(b.dh2, off); shift_ptr(b.dh1, off); shift_ptr(b.dout, off); shift_ptr(b.S, off);
     shift_ptr(b.part, off); shift_ptr(b.loss_part, off); shift_ptr(b.stats, off);
 }

@@ -15,8 +15,8 @@
 //                      product  D[unit][cell] += sum over the 128 envs of dh1[env][unit] * onehot[env][cell]  (K = 128,
 //                      operand tiles that the epilogue warps wrote) into a third accumulator that lives for the whole
 //                      kernel
-//   warp 2 (one lane)  TMA loads of the layer-1 gates (the h1 hi plane, 128 envs x 128 units per step) into a box the
-//                      epilogue reads
+//   warp 2 (one lane)  TMA loads of the layer-1 gates (the bit mask the rollout recorded, 128 envs x 16 bytes per step)
+//                      into a box the epilogue reads
 //   warps 3-10         epilogue, thread = (unit, half of the envs): tcgen05.ld, gate, S +=, 16-bit split; writes its
 //                      dh1^T row (hi and lo planes, K-major) and the one-hot elements in the 128-byte-swizzled layout
 // At the end the epilogue warps store S (two 16-bit planes) and the agent accumulator as one split-K partial per
@@ -54,7 +54,7 @@ struct Dh1aCfg {
     static constexpr int D_BOX = BN * 128;               // dh1^T: 128 unit rows x 64 envs (16 KB), K-major
     static constexpr int D_TILE = PL * 2 * D_BOX;        // [plane][env half]
     static constexpr int O_TILE = (2 / NCTA) * BM * 128; // one-hot: 128 k-rows (envs) x this CTA's cells (64-wide boxes), MN-major
-    static constexpr int G_TILE = 2 * BM * 128;          // gates: 128 env rows x 128 units (two 64-wide boxes)
+    static constexpr int G_TILE = BM * (BN / 8);         // gates: 128 env rows x 16 bytes (one bit per unit)
     // W2 rows in tensor memory: two k per 32-bit column, hi plane then lo.  At H = 256 only the hi plane fits beside the
     // accumulators; the lo plane (needed for one of the three fp16 terms) stays in shared memory as K-major boxes.
     static constexpr bool W_LO_SMEM = PL == 2 && H == 256;
@@ -285,15 +285,11 @@ __device__ __forceinline__ void dh1a_body(const Dh1aMaps& maps, const LearnArgs&
     } else if (wid == 2) {
         if (lane == 0) {  // ---- TMA producer of the gate tiles (rows as for dh2, units n0 .. n0+127 of the h1 hi plane)
             for (int g = 0; g < G && ok; ++g) {
-                if (g + 2 < G) {
-                    tc::tma_prefetch_2d(&maps.gate, n0, row_of(g + 2));
-                    tc::tma_prefetch_2d(&maps.gate, n0 + 64, row_of(g + 2));
-                }
+                if (g + 2 < G) tc::tma_prefetch_2d(&maps.gate, n0 / 8, row_of(g + 2));
                 if (g >= 1) ok = tc::mbar_wait(gempty, (uint32_t)(g - 1) & 1u);
                 if (!ok) break;
                 tc::mbar_expect_tx(gfull, Cfg::G_TILE);
-                tc::tma_load_2d(sG, &maps.gate, gfull, n0, row_of(g));
-                tc::tma_load_2d(sG + BM * 128, &maps.gate, gfull, n0 + 64, row_of(g));
+                tc::tma_load_2d(sG, &maps.gate, gfull, n0 / 8, row_of(g));  // (x in bytes: 0 or 16)
             }
             if (!ok) atomicOr(status, DEV_E_WAIT_TIMEOUT);
         }
@@ -342,8 +338,8 @@ __device__ __forceinline__ void dh1a_body(const Dh1aMaps& maps, const LearnArgs&
             __syncwarp();
             if (lane == 0) arrive_leader(wfull);
         }
-        const uint16_t* gcol = reinterpret_cast<const uint16_t*>(sG) + (q >> 1) * (BM * 64);  // the gate box of this unit
-        const int gsub = (j & 63) >> 3, gel = j & 7;  // 16-byte chunk and element of unit j in a row of that box
+        const uint8_t* gcol = sG + (j >> 3);  // the byte of unit j in a row of the gate box; its bit is j % 8
+        const int gbit = j & 7;
         unsigned char* drow = sD + half * Cfg::D_BOX + j * 128;  // this thread's row of the dh1^T hi box of its env half
         int prev_off = -1;  // byte offset of the one-hot element this thread set the step before
         int g = 0;          // running step index of this CTA
@@ -377,15 +373,15 @@ __device__ __forceinline__ void dh1a_body(const Dh1aMaps& maps, const LearnArgs&
                     uint32_t phi[4], plo[4];
 #pragma unroll
                     for (int p2 = 0; p2 < 4; ++p2) {
-                        const int i = 8 * c8 + 2 * p2;  // envs i, i+1 of the half; gate element (env row, unit j) of the swizzled box
+                        const int i = 8 * c8 + 2 * p2;  // envs i, i+1 of the half; gate bit (env row, unit j) of the gate box
                         const int e_a = 64 * half + i, e_b = e_a + 1;
-                        const uint32_t ga = gcol[e_a * 64 + ((gsub ^ (e_a & 7)) << 3) + gel];
-                        const uint32_t gb = gcol[e_b * 64 + ((gsub ^ (e_b & 7)) << 3) + gel];
+                        const uint32_t ga = (uint32_t)gcol[e_a * (BN / 8)] >> gbit;
+                        const uint32_t gb = (uint32_t)gcol[e_b * (BN / 8)] >> gbit;
                         const float x0 = __uint_as_float(i < 32 ? r0[i] : r1[i - 32]);
                         const float x1 = __uint_as_float(i < 32 ? r0[i + 1] : r1[i - 31]);
-                        // h1 >= 0, so "h1 > 0" is "any magnitude bit set"; rows past the batch end are another step's
-                        const float v0 = rnd<PREC>((i < nvalid && (ga & 0x7FFFu)) ? x0 : 0.f);
-                        const float v1 = rnd<PREC>((i + 1 < nvalid && (gb & 0x7FFFu)) ? x1 : 0.f);
+                        // rows past the batch end are another step's
+                        const float v0 = rnd<PREC>((i < nvalid && (ga & 1u)) ? x0 : 0.f);
+                        const float v1 = rnd<PREC>((i + 1 < nvalid && (gb & 1u)) ? x1 : 0.f);
                         s_acc[i] += v0;
                         s_acc[i + 1] += v1;
                         split2<PREC>(v0, v1, phi[p2], plo[p2]);
@@ -491,7 +487,7 @@ cudaError_t launch_t(const LearnArgs& a, int grid_x, float* part_agent, size_t p
     const uint16_t* dh2hi = reinterpret_cast<const uint16_t*>(b.dh2);
     if (!make_tensor_map_2d(&maps.a_hi, dh2hi, R, H, Cfg::ROWS, bf)) return cudaErrorNotSupported;
     if (Cfg::PL == 2 && !make_tensor_map_2d(&maps.a_lo, dh2hi + RH, R, H, Cfg::ROWS, bf)) return cudaErrorNotSupported;
-    if (!make_tensor_map_2d(&maps.gate, b.h1, R, H, 128, bf)) return cudaErrorNotSupported;  // the hi plane of h1
+    if (!b.gate1 || !make_tensor_map_u8(&maps.gate, b.gate1, R, H / 8, 128, Cfg::BN / 8)) return cudaErrorNotSupported;
     if (!make_tensor_map_2d(&maps.w_hi, b.w2p_hi, H, H, 128, bf)) return cudaErrorNotSupported;
     if (Cfg::PL == 2 && !make_tensor_map_2d(&maps.w_lo, b.w2p_lo, H, H, 128, bf)) return cudaErrorNotSupported;
     if constexpr (Cfg::PAIR) {  // the two CTAs of a pair are neighbours in x; each pair takes all H units

@@ -291,6 +291,14 @@ __device__ __forceinline__ void split_bf16(float x, __nv_bfloat16& hi, __nv_bflo
 __device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 lo_elem, __nv_bfloat16 hi_elem) {
     return (uint32_t)__bfloat16_as_ushort(lo_elem) | ((uint32_t)__bfloat16_as_ushort(hi_elem) << 16);
 }
+// One bit per 16-bit element of v that is not a (signed) zero; element 0 = the low half of v.x = bit 0.
+__device__ __forceinline__ uint32_t nonzero_bits16(const uint4& v) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) m |= ((w[i] & 0x00007FFFu) ? 1u : 0u) << (2 * i) | ((w[i] & 0x7FFF0000u) ? 2u : 0u) << (2 * i);
+    return m;
+}
 // 1.0 in the 16-bit operand format
 template <int PREC> __device__ __forceinline__ uint32_t one16() { return PREC == 1 ? 0x3F80u : 0x3C00u; }
 

@@ -58,6 +58,18 @@ bool make_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint6
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same over a row-major byte matrix [rows][cols] (cols a multiple of 16) with a box of box_cols x box_rows bytes, not swizzled.
+bool make_tensor_map_u8(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc || cols % 16 != 0 || box_cols % 16 != 0) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // DEEP: as many stages as fit (plane operands, TMA-latency-bound); otherwise two, so that two CTAs share an SM (the
 // synthesized-A modes are bound by their builder threads, and a second CTA hides them).
 template <int BN, int APL, int BPL, bool DEEP, int PREC = 0>

@@ -189,6 +189,7 @@ __global__ void __launch_bounds__(NW * 32, (H <= 128 ? 2 : 1)) k_rollout_mma(Rol
                     const size_t gi = ((size_t)t * B + e0 + e) * H + k;
                     *reinterpret_cast<uint4*>(g_h1hi + gi) = hi;
                     if (PREC == 0) *reinterpret_cast<uint4*>(g_h1lo + gi) = lo;
+                    if (b.gate1) b.gate1[gi >> 3] = (uint8_t)nonzero_bits16(hi);  // the gates of these eight units
                 }
             }
         }

@@ -251,6 +251,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Pair2Cfg::THREADS, 1
                     const size_t gi = ((size_t)t * B + env) * H + 64 * kb + 8 * c8;
                     *reinterpret_cast<uint4*>(g_h1hi + gi) = hi[kb];
                     *reinterpret_cast<uint4*>(g_h1lo + gi) = lo[kb];
+                    if (b.gate1) b.gate1[gi >> 3] = (uint8_t)nonzero_bits16(hi[kb]);  // the gates of these eight units
                 }
             }
         };

@@ -248,6 +248,7 @@ __global__ void __launch_bounds__(Tc128Cfg::THREADS, 1) k_rollout_tc128(const __
                             const size_t gi = ((size_t)t * B + env) * H + 64 * kb + 8 * c8;
                             *reinterpret_cast<uint4*>(g_h1hi + gi) = hi[kb][p];
                             *reinterpret_cast<uint4*>(g_h1lo + gi) = lo[kb][p];
+                            if (b.gate1) b.gate1[gi >> 3] = (uint8_t)nonzero_bits16(hi[kb][p]);  // the gates of these eight units
                         }
                     }
                 }

@@ -235,5 +235,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mas
 // Host: encodes a 2-D tensor map over a row-major 16-bit matrix [rows][cols] with a box of 64 columns x box_rows rows
 // and the 128-byte swizzle.  Returns false if the driver entry point is missing or the encode fails.
 bool make_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool bf16);
+// Host: the same over a row-major byte matrix [rows][cols] (cols a multiple of 16), box of box_cols x box_rows bytes, no swizzle.
+bool make_tensor_map_u8(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols);
 
 }  // namespace anakin
