@@ -207,20 +207,26 @@ __global__ void __launch_bounds__(192, 1) k_gemm_tn_tc(const __grid_constant__ G
                 } else {  // A_WALLS: thread = (k row, 64-wide box); it writes all eight 16-byte chunks of its row segment
                     const int k = bt >> 1, bx = bt & 1;
                     const int kk = k0 + k;
-                    const uint32_t* wrow = g.walls + (size_t)(g.kmod ? kk % g.kmod : kk) * g.W;
+                    // the 64 cells m = mb .. mb + 63 of this box as one bit mask: wall bits below ones_row, the ones row itself
+                    const int mb = m0 + 64 * bx;  // a multiple of 64: two whole words of the env's wall mask
+                    unsigned long long bits = 0ull;
+                    if (kk < kend) {
+                        const uint32_t* wrow = g.walls + (size_t)(g.kmod ? kk % g.kmod : kk) * g.W;
+                        const int w0 = mb >> 5;
+                        const uint32_t lo32 = w0 < g.W ? wrow[w0] : 0u, hi32 = w0 + 1 < g.W ? wrow[w0 + 1] : 0u;
+                        bits = (unsigned long long)lo32 | ((unsigned long long)hi32 << 32);
+                        const int r1 = g.ones_row - mb;  // position of the ones row in this box
+                        if (r1 <= 0) bits = 0ull;
+                        else if (r1 < 64) bits &= (1ull << r1) - 1ull;
+                        if (r1 >= 0 && r1 < 64) bits |= 1ull << r1;
+                    }
+                    const uint32_t one = one16<PREC>();
 #pragma unroll
                     for (int c8 = 0; c8 < 8; ++c8) {
-                        uint32_t w[4] = {0u, 0u, 0u, 0u};
-                        if (kk < kend) {
+                        const uint32_t by = (uint32_t)(bits >> (8 * c8)) & 0xFFu;
+                        uint32_t w[4];
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const int m = m0 + 64 * bx + 8 * c8 + q;
-                                bool on = false;
-                                if (m < g.ones_row) on = (wrow[m >> 5] >> (m & 31)) & 1u;
-                                else if (m == g.ones_row) on = true;
-                                if (on) w[q >> 1] |= (q & 1) ? (one16<PREC>() << 16) : one16<PREC>();
-                            }
-                        }
+                        for (int q2 = 0; q2 < 4; ++q2) w[q2] = ((by >> (2 * q2)) & 1u) * one | ((by >> (2 * q2 + 1)) & 1u) * (one << 16);
                         *reinterpret_cast<uint4*>(sa + bx * Cfg::BOX + k * 128 + ((c8 ^ (k & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
