@@ -299,6 +299,24 @@ def test_long_runs_of_the_benchmarked_workload_are_bitwise_reproducible(bnd):
     assert np.isfinite(outs[0][0]).all()
 
 
+@pytest.mark.parametrize("name", ["tc128_two_groups", "pair2_two_groups"])
+def test_runs_of_the_large_batch_kernels_are_bitwise_reproducible(bnd, name):
+    """The same for the kernels large batches take: the two-group rollouts, and the fused dh1 kernel walking several
+    env tiles per CTA (one CTA per SM at H = 128, CTA pairs at H = 256) with its accumulators, operand tiles and gate
+    tiles handed over through mbarriers.  20 passes, twice."""
+    w = SMALL[name]
+    outs = []
+    for _ in range(2):
+        an = make(bnd, w, debug=0)
+        an.reset(6)
+        an.run(20)
+        outs.append((an.get(bnd.PARAMS), an.get(bnd.GRADS), an.get(bnd.TRAJ_ACTION), an.get(bnd.ADV)))
+        assert an.status() == 0
+    for a, b in zip(*outs):
+        assert (a.view(np.uint8) == b.view(np.uint8)).all()
+    assert np.isfinite(outs[0][0]).all()
+
+
 def test_checkpoint_resume_is_bitwise(bnd):
     w = SMALL["large_batch_s"].scaled(B=300, T=8)
     a = make(bnd, w, debug=0)
