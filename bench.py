@@ -184,7 +184,11 @@ def kernel_work(w):
     work = {
         # name: (bound, executed flops, bytes)
         "rollout": ("tensor", p3 * 2.0 * B * (T + 1) * H * H, R * (15.0 + pl * H + 4.0 * H) + B * 4),
-        "dh1": ("tensor", p3 * 2.0 * R * H * H, R * H * (2.0 * pl + 2.0)),
+        # fused kernel (H = 128, 256 with at most 128 cells, one policy): also the agent plane of dW1 over 128 padded cells;
+        # reads the dh2 planes and one gate bit per element.  Otherwise: dh2 in, 16-bit h1 gates in, dh1 out.
+        "dh1": (("tensor", p3 * 2.0 * R * H * H + p2 * 2.0 * R * 128 * H, R * H * (pl + 0.125))
+                if H in (128, 256) and C <= 128 and getattr(w, "n_policies", 0) <= 1
+                else ("tensor", p3 * 2.0 * R * H * H, R * H * (2.0 * pl + 2.0))),
         "dw2": ("tensor", p3 * 2.0 * R * H * H, R * H * 2.0 * pl),
         "dw1_agent": ("tensor", p2 * 2.0 * R * C * H, R * H * 1.0 * pl + R),
         "dw1_walls": ("tensor", 2 * 2.0 * B * (C + 1) * H, B * H * 4.0),
