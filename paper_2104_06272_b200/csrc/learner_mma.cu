@@ -4,6 +4,9 @@
 //
 //   k_heads_bwd   flat 32-row tiles: saved head outputs -> softmax / loss terms -> dOut -> dh2 (fp32 FMA, HBM-bound).
 //                 Emits dh2 as 16-bit hi/lo planes and per-CTA partial sums of dWh, dbh, db2 and the loss terms.
+//                 At hidden width 256 (few enough rows per CTA) it also takes dW2 = h1^T dh2 for its rows: the dh2 tile it
+//                 has just computed and the matching h1 tile (TMA) are the operands of tcgen05 MMAs into tensor memory,
+//                 so dh2 is not read back for that product and the stand-alone dW2 GEMM is not launched.
 //   k_dh1         dh1 = (dh2 W2^T) gated by h1 > 0 with mma.sync; a CTA keeps its slice of W2 in shared memory and
 //                 walks t for 64 envs, so S = sum_t dh1 accumulates in registers.  Emits dh1 planes and S planes.
 //   k_gemm_tn     C[m][n] = sum_k A[k][m] B[k][n] with split-K partial outputs, bf16 hi/lo planes as operands and
@@ -27,26 +30,50 @@ namespace anakin {
 // ----------------------------------------------------------------------------------------------------
 // HS = width of the column slab one CTA covers (blockIdx.y picks the slab; HS = H for H <= 256); H2BF: h2 is stored as
 // bf16 (the wide bf16 path) instead of fp32.
-template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
+// FUSE (H = 256 only): the kernel also takes dW2 = h1^T dh2 for its rows on the tcgen05 pipe (see k_heads_bwd).
+template <int H, int NW, int PREC, int HS = H, bool H2BF = false, bool FUSE = false>
 struct HeadsCfg {
     static constexpr int TR = 32;  // rows per tile
     static constexpr int ESZ = H2BF ? 2 : 4;
     // the widest slab (32 KB tiles, 17 warps) runs one CTA per SM with a deep ring; the narrower ones two CTAs per SM
     static constexpr int PER_SM = TR * HS * ESZ >= 32768 ? 1 : 2;
-    static constexpr int NST = PER_SM == 1 ? 6 : 4;  // depth of the h2 ring (tiles in flight = NST - 1)
-    static constexpr size_t smem_bytes = (size_t)NST * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + 64 /*barriers*/;
+    static constexpr int PL = PREC == 1 ? 1 : 2;
+    static constexpr int BOX = TR * 128;                     // 32 rows x 64 16-bit elements, MN-major (4 KB)
+    static constexpr int OP_TILE = PL * (H / 64) * BOX;      // one operand tile: [plane][64-column box]
+    // dh2 and h1 tiles, two each; the shared array is declared 128-byte aligned, so 896 bytes reach the next 1024-byte boundary
+    static constexpr int FUSE_BYTES = FUSE ? 4 * OP_TILE + 896 /*alignment slack*/ + 64 /*barriers, tmem slot*/ : 0;
+    static_assert((size_t)FUSE_BYTES + (size_t)(FUSE ? 3 : 0) * TR * HS * ESZ + 2 * TR * 8 * 4 + 64 <= 232448, "shared memory of the fused kernel");
+    static constexpr int NST = FUSE ? 3 : (PER_SM == 1 ? 6 : 4);  // depth of the h2 ring (tiles in flight = NST - 1)
+    static constexpr int THREADS = NW * 32 + 32 + (FUSE ? 32 : 0);
+    static constexpr size_t smem_bytes = (size_t)FUSE_BYTES + (size_t)NST * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + 64 /*barriers*/;
 };
 
-template <int H, int NW, int PREC, int HS = H, bool H2BF = false, bool GROUPED = false>
-__global__ void __launch_bounds__(NW * 32 + 32, (HeadsCfg<H, NW, PREC, HS, H2BF>::PER_SM)) k_heads_bwd(LearnArgs a_in) {
+struct HeadsMaps {
+    CUtensorMap h1_hi, h1_lo;  // FUSE: the h1 planes [R][H], boxes of 64 columns x 32 rows
+};
+
+template <int H, int NW, int PREC, int HS = H, bool H2BF = false, bool GROUPED = false, bool FUSE = false>
+__global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREADS), (HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::PER_SM))
+    k_heads_bwd(LearnArgs a_in, const __grid_constant__ HeadsMaps maps) {
     const PolicyArgs<GROUPED, LearnArgs> pa(a_in, blockIdx.z);  // many policies: grid.z = policy
     const LearnArgs& a = pa.a;
-    using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
+    using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>;
     constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = HS / 2, ESZ = Cfg::ESZ, NST = Cfg::NST;
     static_assert(NTHREADS / HP2 == 4, "four row groups of eight rows");
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned char* s_h2 = smem_raw;                                                 // [NST][TR][HS] fp32 or bf16
-    float* s_dout = reinterpret_cast<float*>(smem_raw + (size_t)NST * TR * HS * ESZ);  // [2][TR][8]
+    static_assert(!FUSE || (HS == H && H == 256 && !H2BF && !GROUPED), "the fused dW2 product is built for the 256-wide fp32-h2 kernel");
+    extern __shared__ __align__(128) unsigned char heads_smem[];
+    // FUSE: the operand tiles of the dW2 MMAs first (1024-byte aligned for the 128-byte swizzle): dh2 tiles [2], h1 tiles [2]
+    unsigned char* fbase = (unsigned char*)(((uintptr_t)heads_smem + 1023) & ~(uintptr_t)1023);
+    unsigned char* s_t = fbase;                                  // dh2 tile, written by the column warps
+    unsigned char* s_a = s_t + 2 * Cfg::OP_TILE;                 // h1 tile, by TMA
+    uint64_t* fbars = reinterpret_cast<uint64_t*>(s_a + 2 * Cfg::OP_TILE);  // t_ready[2], a_full[2], mma_done[2], epi_done
+    uint64_t* t_ready = fbars;
+    uint64_t* a_full = fbars + 2;
+    uint64_t* mma_done = fbars + 4;
+    uint64_t* epi_done = fbars + 6;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fbars + 7);
+    unsigned char* s_h2 = FUSE ? fbase + 4 * Cfg::OP_TILE + 64 : heads_smem;          // [NST][TR][HS] fp32 or bf16
+    float* s_dout = reinterpret_cast<float*>(s_h2 + (size_t)NST * TR * HS * ESZ);  // [2][TR][8]
     uint64_t* bars = reinterpret_cast<uint64_t*>(s_dout + 2 * TR * 8);              // full[2], empty[2]
     uint64_t* full = bars;
     uint64_t* empty = bars + 2;
@@ -59,11 +86,80 @@ __global__ void __launch_bounds__(NW * 32 + 32, (HeadsCfg<H, NW, PREC, HS, H2BF>
     const int ntiles = (int)((R + TR - 1) / TR);
     if (tid == 0) {
         for (int q = 0; q < 2; ++q) { tc::mbar_init(&full[q], 1); tc::mbar_init(&empty[q], NW); }
+        if (FUSE) {
+            for (int q = 0; q < 2; ++q) { tc::mbar_init(&t_ready[q], NW); tc::mbar_init(&a_full[q], 1); tc::mbar_init(&mma_done[q], 1); }
+            tc::mbar_init(epi_done, NW);
+        }
         tc::mbar_fence_init();
     }
+    if (FUSE && tid >= NTHREADS + 32) tc::tmem_alloc(tmem_slot, 512);  // two 128 x 256 accumulators: dW2 rows 0-127, 128-255
+    if (FUSE) tc::tc_fence_before();
     __syncthreads();
+    if (FUSE) tc::tc_fence_after();
     bool ok = true;
+    const int my_its = (ntiles > (int)blockIdx.x) ? (ntiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;  // tiles of this CTA
 
+    if (FUSE && tid >= NTHREADS + 32) {
+        // ---- the MMA warp (one lane): per tile, dW2[i][j] += sum over the tile's 32 rows of h1[r][i] dh2[r][j] with the h1
+        // tile (TMA, MN-major boxes) as A and the dh2 tile the column warps wrote as B; both are double-buffered.
+        const uint32_t tmem = *tmem_slot;
+        if (tid == NTHREADS + 32) {
+            constexpr int PL = Cfg::PL;
+            const uint32_t idesc = tc::umma_idesc<PREC>(128, H, true, true);
+            auto load_h1 = [&](int it) {
+                const int buf = it & 1, row = ((int)blockIdx.x + it * (int)gridDim.x) * TR;
+                tc::mbar_expect_tx(&a_full[buf], Cfg::OP_TILE);
+#pragma unroll
+                for (int bx = 0; bx < H / 64; ++bx) {
+                    tc::tma_load_2d(s_a + buf * Cfg::OP_TILE + bx * Cfg::BOX, &maps.h1_hi, &a_full[buf], 64 * bx, row);
+                    if (PL == 2) tc::tma_load_2d(s_a + buf * Cfg::OP_TILE + (H / 64 + bx) * Cfg::BOX, &maps.h1_lo, &a_full[buf], 64 * bx, row);
+                }
+            };
+            if (my_its > 0) load_h1(0);
+            if (my_its > 1) load_h1(1);
+            for (int it = 0; it < my_its && ok; ++it) {
+                const int buf = it & 1;
+                const uint32_t ph = (uint32_t)(it >> 1) & 1u;
+                ok = tc::mbar_wait(&a_full[buf], ph);
+                if (ok) ok = tc::mbar_wait(&t_ready[buf], ph);
+                if (!ok) break;
+                tc::tc_fence_after();
+                const unsigned char* ta = s_a + buf * Cfg::OP_TILE;
+                const unsigned char* tb = s_t + buf * Cfg::OP_TILE;
+#pragma unroll
+                for (int k16 = 0; k16 < TR / 16; ++k16) {
+                    // MN-major operands: 16 k rows = 2048 bytes into each box, consecutive 64-wide boxes one box apart
+                    const uint64_t b_hi = tc::umma_desc(tb + k16 * 2048, Cfg::BOX, 1024);
+                    const uint64_t b_lo = tc::umma_desc(tb + (H / 64) * Cfg::BOX + k16 * 2048, Cfg::BOX, 1024);
+#pragma unroll
+                    for (int m = 0; m < 2; ++m) {  // rows (units of h1) 128 m .. +127 of dW2
+                        const uint64_t a_hi = tc::umma_desc(ta + 2 * m * Cfg::BOX + k16 * 2048, Cfg::BOX, 1024);
+                        const uint32_t acc = tmem + (uint32_t)(m * H);
+                        uint32_t accum = (it > 0 || k16 > 0) ? 1u : 0u;
+                        if (PL == 2) {
+                            tc::umma(acc, tc::umma_desc(ta + (H / 64 + 2 * m) * Cfg::BOX + k16 * 2048, Cfg::BOX, 1024), b_hi, idesc, accum);  // lo x hi
+                            tc::umma(acc, a_hi, b_lo, idesc, 1u);                                                                        // hi x lo
+                            accum = 1u;
+                        }
+                        tc::umma(acc, a_hi, b_hi, idesc, accum);
+                    }
+                }
+                tc::umma_commit(&mma_done[buf]);
+                if (it + 2 < my_its) {  // refill this h1 buffer once the MMAs that read it have finished
+                    ok = tc::mbar_wait(&mma_done[buf], ph);
+                    if (ok) load_h1(it + 2);
+                }
+            }
+            if (!ok) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
+        }
+        // tensor memory is freed once every column warp has read its part of the accumulators
+        __syncwarp();
+        const bool got = tc::mbar_wait(epi_done, 0);
+        if (!got && tid == NTHREADS + 32) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
+        tc::tc_fence_after();
+        tc::tmem_dealloc(tmem, 512);
+        return;
+    }
     if (tid >= NTHREADS) {
         // ---- the row warp: lane = row of a tile.  It runs ahead of the column warps: the saved head outputs of a row
         // (and its advantage, return and action) become the five output gradients, written to one of two small buffers
@@ -206,6 +302,8 @@ __global__ void __launch_bounds__(NW * 32 + 32, (HeadsCfg<H, NW, PREC, HS, H2BF>
         asm volatile("bar.sync 1, %0;" ::"n"(NTHREADS) : "memory");
         load_tile(tile + (NST - 1) * (int)gridDim.x, (it + NST - 1) % NST);
         if (ok) ok = tc::mbar_wait(&full[buf], (it >> 1) & 1);
+        // FUSE: this tile's dh2 also goes into operand tile `buf`, free once the MMAs of two tiles ago have read it
+        if (FUSE && ok && it >= 2) ok = tc::mbar_wait(&mma_done[buf], ((it >> 1) - 1) & 1);
         // ---- dh2 = (dOut Wh^T) gated by h2 > 0, as 16-bit planes; running sums of dWh and db2
         const unsigned char* h2t = s_h2 + ((size_t)(it % NST) * TR + rg * 8) * HS * ESZ + (size_t)2 * cp * ESZ;
         const float* dt = s_dout + (buf * TR + rg * 8) * 8;
@@ -255,9 +353,21 @@ __global__ void __launch_bounds__(NW * 32 + 32, (HeadsCfg<H, NW, PREC, HS, H2BF>
                 o_hi[r * (H / 2)] = phi;
                 if (PREC == 0) o_lo[r * (H / 2)] = plo;
             }
+            if (FUSE) {
+                // element (k = tile row, n = unit 2 cp) of the MN-major tile: box n/64, byte k*128 + (((n%64)/8) ^ (k%8))*16 +
+                // (n%8)*2; rows past the end carry zeros (their h2 was zero-filled)
+                const int k = rg * 8 + r;
+                unsigned char* tp = s_t + buf * Cfg::OP_TILE + (cp >> 5) * Cfg::BOX + k * 128 + ((((cp & 31) >> 2) ^ (k & 7)) << 4) + (cp & 3) * 4;
+                *reinterpret_cast<uint32_t*>(tp) = phi;
+                if (PREC == 0) *reinterpret_cast<uint32_t*>(tp + (H / 64) * Cfg::BOX) = plo;
+            }
         }
+        if (FUSE) tc::fence_proxy_async();  // generic-proxy stores -> visible to the tensor core
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&empty[buf]);  // the row warp may refill this buffer of output gradients
+        if (lane == 0) {
+            tc::mbar_arrive(&empty[buf]);  // the row warp may refill this buffer of output gradients
+            if (FUSE) tc::mbar_arrive(&t_ready[buf]);
+        }
     }
     cp_async_wait<0>();
     // ---- per-CTA results: dWh, db2 partials (split index = 4*CTA + row group)
@@ -269,6 +379,37 @@ __global__ void __launch_bounds__(NW * 32 + 32, (HeadsCfg<H, NW, PREC, HS, H2BF>
             for (int c = 0; c < 5; ++c) part[(size_t)(c_base + 2 * cp + cc) * 5 + c] = a_wh[cc][c];
             part[(size_t)H * 5 + c_base + 2 * cp + cc] = a_b2[cc];
         }
+    }
+    if (FUSE) {
+        // ---- this CTA's partial of dW2: accumulator m, lane = row 128 m + lane of dW2, column = column of dW2.  Warp w reads
+        // lane quarter w % 4 and the 64 columns of column group w / 4 (NW = 16: four groups).
+        const int wq = (tid >> 5) & 3, cg = tid >> 7;
+        bool got = ok;
+        if (got && my_its > 0) got = tc::mbar_wait(&mma_done[(my_its - 1) & 1], (uint32_t)((my_its - 1) >> 1) & 1u);
+        if (!got && ok && lane == 0) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
+        tc::tc_fence_after();
+        const uint32_t tmem = *tmem_slot;
+        float* part = const_cast<float*>(a_in.reg[4].part) + (size_t)blockIdx.x * H * H;
+#pragma unroll 1
+        for (int m = 0; m < 2; ++m) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t r[32];
+                if (got && my_its > 0) {
+                    tc::tmem_ld32(tmem + ((uint32_t)(32 * wq) << 16) + (uint32_t)(m * H + 64 * cg + c0), r);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;  // a CTA without tiles contributes zeros
+                }
+                float4* dst = reinterpret_cast<float4*>(part + (size_t)(128 * m + 32 * wq + lane) * H + 64 * cg + c0);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+            }
+        }
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(epi_done);
     }
     if (!ok && lane == 0) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
 }
@@ -1076,6 +1217,17 @@ static void dh1a_shape(const Dims& d, int T, int* grid_x, int* ts) {
     }
 }
 
+// Rows one CTA of the fused heads + dW2 kernel may accumulate in tensor memory (fp32 workloads): the tensor core's own
+// accumulation rounds toward zero, which shows as a bias on longer sums (the stand-alone dW2 kernel drains every 4096 rows).
+constexpr size_t HEADS_FUSE_MAX_ROWS = 4096;
+
+// dW2 inside the heads kernel: hidden width 256, one policy, few enough rows per CTA.
+static bool heads_fuse_dw2(const Dims& d, size_t R, int heads_grid, int prec) {
+    if (d.H != 256 || d.npol > 1 || heads_grid < 1) return false;
+    const size_t tiles = (R + 31) / 32, per_cta = (tiles + heads_grid - 1) / heads_grid * 32;
+    return prec == 1 || per_cta <= HEADS_FUSE_MAX_ROWS;
+}
+
 void learn_mma_plan(const Dims& d, LearnPlan* p) {
     const int H = d.H, C = d.C;
     const size_t R = (size_t)d.B * d.Tmax;
@@ -1102,10 +1254,12 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
     size_t hg = H == 256 ? HEADS_GRID / 2 : HEADS_GRID;  // (the H = 256 kernel takes a whole SM)
     if (d.npol > 1) hg = (size_t)(2 * HEADS_GRID / d.npol > 0 ? 2 * HEADS_GRID / d.npol : 1);  // many policies: the CTAs of all policies fill the GPU together
     p->heads_grid = (int)(tiles32 < hg ? tiles32 : hg);
+    // (the fused heads + dW2 kernel writes one dW2 partial per CTA: room for the larger of the two partial counts)
+    const int w2_slots = heads_fuse_dw2(d, R, p->heads_grid, 1) && p->heads_grid > p->ns_w2 ? p->heads_grid : p->ns_w2;
     p->ns_small = 4 * p->heads_grid;
     p->small_stride = (size_t)6 * H + 8;
     size_t off = 0;
-    p->off_w2 = off; off += (size_t)p->ns_w2 * H * H;
+    p->off_w2 = off; off += (size_t)w2_slots * H * H;
     p->off_agent = off; off += (size_t)p->ns_agent * C * H;
     p->off_walls = off; off += (size_t)p->ns_env * (C + 1) * H;
     p->off_goal = off; off += (size_t)p->ns_env * C * H;
@@ -1117,18 +1271,32 @@ void learn_mma_plan(const Dims& d, LearnPlan* p) {
 #define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) return e_; } while (0)
 
 template <int H, int NW, int PREC, int HS = H, bool H2BF = false>
-static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s) {
+static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s, bool fuse = false) {
     using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF>;
+    HeadsMaps maps;
+    memset(&maps, 0, sizeof(maps));
     if (a.d.npol > 1) {
         if constexpr (PREC == 0 && HS == H && !H2BF) {
             CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
-            k_heads_bwd<H, NW, PREC, HS, H2BF, true><<<dim3(grid, 1, a.d.npol), NW * 32 + 32, Cfg::smem_bytes, s>>>(a);
+            k_heads_bwd<H, NW, PREC, HS, H2BF, true><<<dim3(grid, 1, a.d.npol), Cfg::THREADS, Cfg::smem_bytes, s>>>(a, maps);
             return cudaGetLastError();
         }
         return cudaErrorNotSupported;
     }
+    if constexpr (H == 256 && HS == H && !H2BF) {
+        if (fuse) {  // also dW2 = h1^T dh2 for the CTA's rows (tcgen05; the h1 tiles by TMA)
+            using FCfg = HeadsCfg<H, NW, PREC, HS, H2BF, true>;
+            const size_t R = (size_t)a.d.B * a.T, RH = (size_t)a.d.B * a.d.Tmax * H;
+            const uint16_t* h1hi = reinterpret_cast<const uint16_t*>(a.b.h1);
+            if (!make_tensor_map_2d(&maps.h1_hi, h1hi, R, H, FCfg::TR, PREC == 1)) return cudaErrorNotSupported;
+            if (PREC == 0 && !make_tensor_map_2d(&maps.h1_lo, h1hi + RH, R, H, FCfg::TR, false)) return cudaErrorNotSupported;
+            CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FCfg::smem_bytes));
+            k_heads_bwd<H, NW, PREC, HS, H2BF, false, true><<<dim3(grid, 1), FCfg::THREADS, FCfg::smem_bytes, s>>>(a, maps);
+            return cudaGetLastError();
+        }
+    }
     CK(cudaFuncSetAttribute(k_heads_bwd<H, NW, PREC, HS, H2BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::smem_bytes));
-    k_heads_bwd<H, NW, PREC, HS, H2BF><<<dim3(grid, H / HS), NW * 32 + 32, Cfg::smem_bytes, s>>>(a);
+    k_heads_bwd<H, NW, PREC, HS, H2BF><<<dim3(grid, H / HS), Cfg::THREADS, Cfg::smem_bytes, s>>>(a, maps);
     return cudaGetLastError();
 }
 
@@ -1184,12 +1352,15 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     a.reg[6] = PartRegion{b.part + pl.off_small, pl.ns_small, pl.small_stride, d.oWh};
     a.reg[7] = PartRegion{b.part + pl.off_small + (size_t)6 * H, pl.ns_small, pl.small_stride, d.obh};
 
+    // dW2 = h1^T dh2 rides in the heads kernel where its rows per CTA allow (it then has one partial per heads CTA)
+    const bool fuse_dw2 = !wide && !grouped && b.w2p_hi != nullptr && heads_fuse_dw2(d, R, pl.heads_grid, PREC);
+    if (fuse_dw2) a.reg[4].ns = pl.heads_grid;
     {
         Scope sc(c, K_HEADS_BWD);
         switch (H) {
             case 64: CK((launch_heads_t<64, 4, PREC>(a, pl.heads_grid, s))); break;
             case 128: CK((launch_heads_t<128, 8, PREC>(a, pl.heads_grid, s))); break;
-            case 256: CK((launch_heads_t<256, 16, PREC>(a, pl.heads_grid, s))); break;
+            case 256: CK((launch_heads_t<256, 16, PREC>(a, pl.heads_grid, s, fuse_dw2))); break;
             default:
                 if constexpr (PREC == 1) {
                     if (wide) {  // tensor-pipe version: one partial slot per CTA (slot 4 * CTA of the small region)
@@ -1262,7 +1433,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
     g.Bhi = dh2hi; g.Blo = dh2hi + RH; g.ldb = H;
     g.part = b.part + pl.off_w2; g.stride = (size_t)H * H; g.off = 0; g.ldc = H; g.ones_row = -1;
     g.K_last = d.B_last * T; g.kmod_last = 0; g.alo_off_last = g.blo_off_last = RH_last;
-    {
+    if (!fuse_dw2) {
         Scope sc(c, K_DW2);
         cudaError_t e = tc_gemm(A_PLANES, PL, PL, pl.ns_w2);  // tcgen05 where covered
         if (e == cudaErrorNotSupported) {
