@@ -45,6 +45,9 @@ struct HeadsCfg {
     static_assert((size_t)FUSE_BYTES + (size_t)(FUSE ? 3 : 0) * TR * HS * ESZ + 2 * TR * 8 * 4 + 64 <= 232448, "shared memory of the fused kernel");
     static constexpr int NST = FUSE ? 3 : (PER_SM == 1 ? 6 : 4);  // depth of the h2 ring (tiles in flight = NST - 1)
     static constexpr int THREADS = NW * 32 + 32 + (FUSE ? 32 : 0);
+    // FUSE, fp32 workloads: the accumulators are read out and restarted every GROUP tiles (4096 rows): the tensor core's own
+    // accumulation rounds toward zero, which shows as a bias on longer sums; the groups are added with round-to-nearest
+    static constexpr int GROUP = PREC == 1 ? (1 << 30) : 128;
     static constexpr size_t smem_bytes = (size_t)FUSE_BYTES + (size_t)NST * TR * HS * ESZ + (size_t)2 * TR * 8 * 4 + 64 /*barriers*/;
 };
 
@@ -135,7 +138,7 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
                     for (int m = 0; m < 2; ++m) {  // rows (units of h1) 128 m .. +127 of dW2
                         const uint64_t a_hi = tc::umma_desc(ta + 2 * m * Cfg::BOX + k16 * 2048, Cfg::BOX, 1024);
                         const uint32_t acc = tmem + (uint32_t)(m * H);
-                        uint32_t accum = (it > 0 || k16 > 0) ? 1u : 0u;
+                        uint32_t accum = (it % Cfg::GROUP > 0 || k16 > 0) ? 1u : 0u;  // (a group's first MMA restarts the sum)
                         if (PL == 2) {
                             tc::umma(acc, tc::umma_desc(ta + (H / 64 + 2 * m) * Cfg::BOX + k16 * 2048, Cfg::BOX, 1024), b_hi, idesc, accum);  // lo x hi
                             tc::umma(acc, a_hi, b_lo, idesc, 1u);                                                                        // hi x lo
@@ -291,6 +294,49 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
         cp_async_commit();
     };
 
+    // FUSE: this CTA's partial of dW2.  Accumulator m, lane = row 128 m + lane of dW2, column = column of dW2; warp w reads
+    // lane quarter w % 4 and the 64 columns of column group w / 4 (NW = 16: four groups).  After tile `last` (the last of an
+    // accumulator group): the first group writes the partial, every later one adds to what this same thread wrote.
+    float* const w2part = FUSE ? const_cast<float*>(a_in.reg[4].part) + (size_t)blockIdx.x * H * H : nullptr;
+    const int wq = (tid >> 5) & 3, cg = tid >> 7;
+    auto dw2_out = [&](int last) -> bool {
+        const bool got = tc::mbar_wait(&mma_done[last & 1], (uint32_t)(last >> 1) & 1u);
+        if (!got && lane == 0) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
+        tc::tc_fence_after();
+        const uint32_t tmem = *tmem_slot;
+        const bool first = last / Cfg::GROUP == 0;
+#pragma unroll 1
+        for (int m = 0; m < 2; ++m) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t r[32];
+                if (got) {
+                    tc::tmem_ld32(tmem + ((uint32_t)(32 * wq) << 16) + (uint32_t)(m * H + 64 * cg + c0), r);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;
+                }
+                float4* dst = reinterpret_cast<float4*>(w2part + (size_t)(128 * m + 32 * wq + lane) * H + 64 * cg + c0);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float4 v = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+                    if (!first) {
+                        const float4 o = dst[i];
+                        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                    }
+                    dst[i] = v;
+                }
+            }
+        }
+        tc::tc_fence_before();
+        return got;
+    };
+    auto dw2_zero = [&]() {  // a CTA without tiles contributes zeros
+#pragma unroll 1
+        for (int m = 0; m < 2; ++m)
+            for (int i = 0; i < 16; ++i)
+                reinterpret_cast<float4*>(w2part + (size_t)(128 * m + 32 * wq + lane) * H + 64 * cg)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    };
     int it = 0;
 #pragma unroll
     for (int q = 0; q < NST - 1; ++q) load_tile(blockIdx.x + q * (int)gridDim.x, q);
@@ -368,6 +414,9 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
             tc::mbar_arrive(&empty[buf]);  // the row warp may refill this buffer of output gradients
             if (FUSE) tc::mbar_arrive(&t_ready[buf]);
         }
+        // FUSE: after a group's last tile the accumulators go to this CTA's dW2 partial; the next tile's MMAs (which restart
+        // the sum) are issued only after every column warp has arrived for that tile, i.e. after its part of the read-out
+        if (FUSE && (it + 1) % Cfg::GROUP == 0 && it + 1 < my_its) ok = dw2_out(it) && ok;
     }
     cp_async_wait<0>();
     // ---- per-CTA results: dWh, db2 partials (split index = 4*CTA + row group)
@@ -381,32 +430,8 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
         }
     }
     if (FUSE) {
-        // ---- this CTA's partial of dW2: accumulator m, lane = row 128 m + lane of dW2, column = column of dW2.  Warp w reads
-        // lane quarter w % 4 and the 64 columns of column group w / 4 (NW = 16: four groups).
-        const int wq = (tid >> 5) & 3, cg = tid >> 7;
-        bool got = ok;
-        if (got && my_its > 0) got = tc::mbar_wait(&mma_done[(my_its - 1) & 1], (uint32_t)((my_its - 1) >> 1) & 1u);
-        if (!got && ok && lane == 0) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
-        tc::tc_fence_after();
-        const uint32_t tmem = *tmem_slot;
-        float* part = const_cast<float*>(a_in.reg[4].part) + (size_t)blockIdx.x * H * H;
-#pragma unroll 1
-        for (int m = 0; m < 2; ++m) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t r[32];
-                if (got && my_its > 0) {
-                    tc::tmem_ld32(tmem + ((uint32_t)(32 * wq) << 16) + (uint32_t)(m * H + 64 * cg + c0), r);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = 0u;  // a CTA without tiles contributes zeros
-                }
-                float4* dst = reinterpret_cast<float4*>(part + (size_t)(128 * m + 32 * wq + lane) * H + 64 * cg + c0);
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]), __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
-            }
-        }
+        if (my_its > 0) ok = dw2_out(my_its - 1) && ok;
+        else dw2_zero();
         tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(epi_done);
@@ -1217,15 +1242,10 @@ static void dh1a_shape(const Dims& d, int T, int* grid_x, int* ts) {
     }
 }
 
-// Rows one CTA of the fused heads + dW2 kernel may accumulate in tensor memory (fp32 workloads): the tensor core's own
-// accumulation rounds toward zero, which shows as a bias on longer sums (the stand-alone dW2 kernel drains every 4096 rows).
-constexpr size_t HEADS_FUSE_MAX_ROWS = 4096;
-
-// dW2 inside the heads kernel: hidden width 256, one policy, few enough rows per CTA.
+// dW2 inside the heads kernel: hidden width 256, one policy.
 static bool heads_fuse_dw2(const Dims& d, size_t R, int heads_grid, int prec) {
-    if (d.H != 256 || d.npol > 1 || heads_grid < 1) return false;
-    const size_t tiles = (R + 31) / 32, per_cta = (tiles + heads_grid - 1) / heads_grid * 32;
-    return prec == 1 || per_cta <= HEADS_FUSE_MAX_ROWS;
+    (void)R; (void)prec;
+    return d.H == 256 && d.npol <= 1 && heads_grid >= 1;
 }
 
 void learn_mma_plan(const Dims& d, LearnPlan* p) {
