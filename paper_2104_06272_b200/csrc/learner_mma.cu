@@ -40,9 +40,12 @@ struct HeadsCfg {
     static constexpr int PL = PREC == 1 ? 1 : 2;
     static constexpr int BOX = TR * 128;                     // 32 rows x 64 16-bit elements, MN-major (4 KB)
     static constexpr int OP_TILE = PL * (H / 64) * BOX;      // one operand tile: [plane][64-column box]
-    // dh2 and h1 tiles, two each; the shared array is declared 128-byte aligned, so 896 bytes reach the next 1024-byte boundary
-    static constexpr int FUSE_BYTES = FUSE ? 4 * OP_TILE + 896 /*alignment slack*/ + 64 /*barriers, tmem slot*/ : 0;
-    static_assert((size_t)FUSE_BYTES + (size_t)(FUSE ? 3 : 0) * TR * HS * ESZ + 2 * TR * 8 * 4 + 64 <= 232448, "shared memory of the fused kernel");
+    // two dh2 tiles; two h1 tiles where a CTA has the SM to itself, one where two CTAs share it (H = 128).  The shared
+    // array is declared 128-byte aligned, so 896 bytes reach the next 1024-byte boundary.
+    static constexpr int A_BUFS = PER_SM == 1 ? 2 : 1;
+    static constexpr int TMEM_COLS = (H / 128) * H >= 512 ? 512 : (H / 128) * H;  // H/128 accumulators of 128 lanes x H columns
+    static constexpr int FUSE_BYTES = FUSE ? (2 + A_BUFS) * OP_TILE + 896 /*alignment slack*/ + 64 /*barriers, tmem slot*/ : 0;
+    static_assert(((size_t)FUSE_BYTES + (size_t)(FUSE ? 3 : 0) * TR * HS * ESZ + 2 * TR * 8 * 4 + 64) * PER_SM <= 232448, "shared memory of the fused kernel");
     static constexpr int NST = FUSE ? 3 : (PER_SM == 1 ? 6 : 4);  // depth of the h2 ring (tiles in flight = NST - 1)
     static constexpr int THREADS = NW * 32 + 32 + (FUSE ? 32 : 0);
     // FUSE, fp32 workloads: the accumulators are read out and restarted every GROUP tiles (4096 rows): the tensor core's own
@@ -63,19 +66,19 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
     using Cfg = HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>;
     constexpr int TR = Cfg::TR, NTHREADS = NW * 32, HP2 = HS / 2, ESZ = Cfg::ESZ, NST = Cfg::NST;
     static_assert(NTHREADS / HP2 == 4, "four row groups of eight rows");
-    static_assert(!FUSE || (HS == H && H == 256 && !H2BF && !GROUPED), "the fused dW2 product is built for the 256-wide fp32-h2 kernel");
+    static_assert(!FUSE || (HS == H && (H == 128 || H == 256) && !H2BF && !GROUPED), "the fused dW2 product is built for the 128- and 256-wide fp32-h2 kernels");
     extern __shared__ __align__(128) unsigned char heads_smem[];
     // FUSE: the operand tiles of the dW2 MMAs first (1024-byte aligned for the 128-byte swizzle): dh2 tiles [2], h1 tiles [2]
     unsigned char* fbase = (unsigned char*)(((uintptr_t)heads_smem + 1023) & ~(uintptr_t)1023);
     unsigned char* s_t = fbase;                                  // dh2 tile, written by the column warps
     unsigned char* s_a = s_t + 2 * Cfg::OP_TILE;                 // h1 tile, by TMA
-    uint64_t* fbars = reinterpret_cast<uint64_t*>(s_a + 2 * Cfg::OP_TILE);  // t_ready[2], a_full[2], mma_done[2], epi_done
+    uint64_t* fbars = reinterpret_cast<uint64_t*>(s_a + Cfg::A_BUFS * Cfg::OP_TILE);  // t_ready[2], a_full[2], mma_done[2], epi_done
     uint64_t* t_ready = fbars;
     uint64_t* a_full = fbars + 2;
     uint64_t* mma_done = fbars + 4;
     uint64_t* epi_done = fbars + 6;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(fbars + 7);
-    unsigned char* s_h2 = FUSE ? fbase + 4 * Cfg::OP_TILE + 64 : heads_smem;          // [NST][TR][HS] fp32 or bf16
+    unsigned char* s_h2 = FUSE ? fbase + (2 + Cfg::A_BUFS) * Cfg::OP_TILE + 64 : heads_smem;  // [NST][TR][HS] fp32 or bf16
     float* s_dout = reinterpret_cast<float*>(s_h2 + (size_t)NST * TR * HS * ESZ);  // [2][TR][8]
     uint64_t* bars = reinterpret_cast<uint64_t*>(s_dout + 2 * TR * 8);              // full[2], empty[2]
     uint64_t* full = bars;
@@ -95,7 +98,7 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
         }
         tc::mbar_fence_init();
     }
-    if (FUSE && tid >= NTHREADS + 32) tc::tmem_alloc(tmem_slot, 512);  // two 128 x 256 accumulators: dW2 rows 0-127, 128-255
+    if (FUSE && tid >= NTHREADS + 32) tc::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);  // H/128 accumulators of 128 x H: dW2 rows 128 m .. +127
     if (FUSE) tc::tc_fence_before();
     __syncthreads();
     if (FUSE) tc::tc_fence_after();
@@ -109,8 +112,9 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
         if (tid == NTHREADS + 32) {
             constexpr int PL = Cfg::PL;
             const uint32_t idesc = tc::umma_idesc<PREC>(128, H, true, true);
+            constexpr int AB = Cfg::A_BUFS;
             auto load_h1 = [&](int it) {
-                const int buf = it & 1, row = ((int)blockIdx.x + it * (int)gridDim.x) * TR;
+                const int buf = it % AB, row = ((int)blockIdx.x + it * (int)gridDim.x) * TR;
                 tc::mbar_expect_tx(&a_full[buf], Cfg::OP_TILE);
 #pragma unroll
                 for (int bx = 0; bx < H / 64; ++bx) {
@@ -118,16 +122,16 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
                     if (PL == 2) tc::tma_load_2d(s_a + buf * Cfg::OP_TILE + (H / 64 + bx) * Cfg::BOX, &maps.h1_lo, &a_full[buf], 64 * bx, row);
                 }
             };
-            if (my_its > 0) load_h1(0);
-            if (my_its > 1) load_h1(1);
+            for (int q = 0; q < AB; ++q)
+                if (my_its > q) load_h1(q);
             for (int it = 0; it < my_its && ok; ++it) {
-                const int buf = it & 1;
+                const int buf = it & 1, abuf = it % AB;
                 const uint32_t ph = (uint32_t)(it >> 1) & 1u;
-                ok = tc::mbar_wait(&a_full[buf], ph);
+                ok = tc::mbar_wait(&a_full[abuf], (uint32_t)(it / AB) & 1u);
                 if (ok) ok = tc::mbar_wait(&t_ready[buf], ph);
                 if (!ok) break;
                 tc::tc_fence_after();
-                const unsigned char* ta = s_a + buf * Cfg::OP_TILE;
+                const unsigned char* ta = s_a + abuf * Cfg::OP_TILE;
                 const unsigned char* tb = s_t + buf * Cfg::OP_TILE;
 #pragma unroll
                 for (int k16 = 0; k16 < TR / 16; ++k16) {
@@ -135,7 +139,7 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
                     const uint64_t b_hi = tc::umma_desc(tb + k16 * 2048, Cfg::BOX, 1024);
                     const uint64_t b_lo = tc::umma_desc(tb + (H / 64) * Cfg::BOX + k16 * 2048, Cfg::BOX, 1024);
 #pragma unroll
-                    for (int m = 0; m < 2; ++m) {  // rows (units of h1) 128 m .. +127 of dW2
+                    for (int m = 0; m < H / 128; ++m) {  // rows (units of h1) 128 m .. +127 of dW2
                         const uint64_t a_hi = tc::umma_desc(ta + 2 * m * Cfg::BOX + k16 * 2048, Cfg::BOX, 1024);
                         const uint32_t acc = tmem + (uint32_t)(m * H);
                         uint32_t accum = (it % Cfg::GROUP > 0 || k16 > 0) ? 1u : 0u;  // (a group's first MMA restarts the sum)
@@ -148,9 +152,9 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
                     }
                 }
                 tc::umma_commit(&mma_done[buf]);
-                if (it + 2 < my_its) {  // refill this h1 buffer once the MMAs that read it have finished
+                if (it + AB < my_its) {  // refill this h1 buffer once the MMAs that read it have finished
                     ok = tc::mbar_wait(&mma_done[buf], ph);
-                    if (ok) load_h1(it + 2);
+                    if (ok) load_h1(it + AB);
                 }
             }
             if (!ok) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
@@ -160,7 +164,7 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
         const bool got = tc::mbar_wait(epi_done, 0);
         if (!got && tid == NTHREADS + 32) atomicOr(b.status, DEV_E_WAIT_TIMEOUT);
         tc::tc_fence_after();
-        tc::tmem_dealloc(tmem, 512);
+        tc::tmem_dealloc(tmem, Cfg::TMEM_COLS);
         return;
     }
     if (tid >= NTHREADS) {
@@ -295,7 +299,7 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
     };
 
     // FUSE: this CTA's partial of dW2.  Accumulator m, lane = row 128 m + lane of dW2, column = column of dW2; warp w reads
-    // lane quarter w % 4 and the 64 columns of column group w / 4 (NW = 16: four groups).  After tile `last` (the last of an
+    // lane quarter w % 4 and the 64 columns of column group w / 4 (NW / 4 = H / 64 groups).  After tile `last` (the last of an
     // accumulator group): the first group writes the partial, every later one adds to what this same thread wrote.
     float* const w2part = FUSE ? const_cast<float*>(a_in.reg[4].part) + (size_t)blockIdx.x * H * H : nullptr;
     const int wq = (tid >> 5) & 3, cg = tid >> 7;
@@ -306,7 +310,7 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
         const uint32_t tmem = *tmem_slot;
         const bool first = last / Cfg::GROUP == 0;
 #pragma unroll 1
-        for (int m = 0; m < 2; ++m) {
+        for (int m = 0; m < H / 128; ++m) {
 #pragma unroll 1
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t r[32];
@@ -333,7 +337,7 @@ __global__ void __launch_bounds__((HeadsCfg<H, NW, PREC, HS, H2BF, FUSE>::THREAD
     };
     auto dw2_zero = [&]() {  // a CTA without tiles contributes zeros
 #pragma unroll 1
-        for (int m = 0; m < 2; ++m)
+        for (int m = 0; m < H / 128; ++m)
             for (int i = 0; i < 16; ++i)
                 reinterpret_cast<float4*>(w2part + (size_t)(128 * m + 32 * wq + lane) * H + 64 * cg)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     };
@@ -1242,10 +1246,10 @@ static void dh1a_shape(const Dims& d, int T, int* grid_x, int* ts) {
     }
 }
 
-// dW2 inside the heads kernel: hidden width 256, one policy.
+// dW2 inside the heads kernel: hidden width 128 or 256, one policy.
 static bool heads_fuse_dw2(const Dims& d, size_t R, int heads_grid, int prec) {
     (void)R; (void)prec;
-    return d.H == 256 && d.npol <= 1 && heads_grid >= 1;
+    return (d.H == 128 || d.H == 256) && d.npol <= 1 && heads_grid >= 1;
 }
 
 void learn_mma_plan(const Dims& d, LearnPlan* p) {
@@ -1303,7 +1307,7 @@ static cudaError_t launch_heads_t(const LearnArgs& a, int grid, cudaStream_t s, 
         }
         return cudaErrorNotSupported;
     }
-    if constexpr (H == 256 && HS == H && !H2BF) {
+    if constexpr ((H == 128 || H == 256) && HS == H && !H2BF) {
         if (fuse) {  // also dW2 = h1^T dh2 for the CTA's rows (tcgen05; the h1 tiles by TMA)
             using FCfg = HeadsCfg<H, NW, PREC, HS, H2BF, true>;
             const size_t R = (size_t)a.d.B * a.T, RH = (size_t)a.d.B * a.d.Tmax * H;
@@ -1379,7 +1383,7 @@ static cudaError_t launch_learn_mma_p(LearnArgs a, const Ctx& c) {
         Scope sc(c, K_HEADS_BWD);
         switch (H) {
             case 64: CK((launch_heads_t<64, 4, PREC>(a, pl.heads_grid, s))); break;
-            case 128: CK((launch_heads_t<128, 8, PREC>(a, pl.heads_grid, s))); break;
+            case 128: CK((launch_heads_t<128, 8, PREC>(a, pl.heads_grid, s, fuse_dw2))); break;
             case 256: CK((launch_heads_t<256, 16, PREC>(a, pl.heads_grid, s, fuse_dw2))); break;
             default:
                 if constexpr (PREC == 1) {
