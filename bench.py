@@ -137,7 +137,6 @@ class ClockSampler:
 PROFILE_OF = {
     ("throughput", "rollout"): ("rollout_pair__throughput.md", "rollout_pair.cu"),
     ("throughput", "dh1"): ("dh1a_pair__throughput.md", "dh1a_tc.cu"),
-    ("throughput", "dw2"): ("gemm_tn_tc_dw2__throughput.md", "gemm_tc.cu"),
     ("throughput", "heads_bwd"): ("heads_bwd__throughput.md", "learner_mma.cu"),
     ("throughput", "reduce_adam"): ("reduce_adam2__throughput.md", "learner_mma.cu"),
     ("throughput", "env_base"): ("env_base__throughput.md", "rollout.cu"),
@@ -194,7 +193,10 @@ def kernel_work(w):
         "dw1_agent": ("tensor", p2 * 2.0 * R * C * H, R * H * 1.0 * pl + R),
         "dw1_walls": ("tensor", 2 * 2.0 * B * (C + 1) * H, B * H * 4.0),
         "dw1_goal": ("tensor", 2 * 2.0 * B * C * H, B * H * 4.0),
-        "heads_bwd": ("hbm", R * H * 22.0, R * H * (4.0 + pl) + R * 10.0),
+        # hidden width 128 / 256 (one policy): the kernel also takes dW2 = h1^T dh2 on the tensor pipe and reads the h1 planes
+        "heads_bwd": (("hbm", R * H * 22.0 + p3 * 2.0 * R * H * H, R * H * (4.0 + 2.0 * pl) + R * 10.0)
+                      if H in (128, 256) and getattr(w, "n_policies", 0) <= 1
+                      else ("hbm", R * H * 22.0, R * H * (4.0 + pl) + R * 10.0)),
         "gae": ("hbm", R * 6.0, R * 17.0),
         "env_base": ("hbm", B * H * (0.2 * C + 2), B * H * 4.0),
         "pack_w2": ("hbm", 0.0, H * H * 16.0),
