@@ -107,6 +107,19 @@ def test_one_iteration_stage_by_stage(bnd, name):
         print(name, "worst error / bound (last comparison of each tensor):", {k: round(v, 3) for k, v in par.MARGINS.items()})
 
 
+@pytest.mark.parametrize("name", ["tp_ragged_128", "tp_ragged_256", "large_batch_s", "tp_bf16_256"])
+def test_an_iteration_shorter_than_t_max(bnd, name):
+    """A rollout of fewer steps than the handle was sized for, then the update: the launch plans (partial counts, grids)
+    are made for T_max, so some CTAs of the update kernels find no rows (the fused heads + dW2 kernel then contributes a
+    zero partial) and the t-slices of the dh1 kernel are cut from fewer steps."""
+    w = SMALL[name]
+    an = make(bnd, w)
+    an.reset(13)
+    an.set(bnd.PARAMS, random_params(6, w.P, 0.15))
+    par.check_iteration(an, bnd, w, 13, T=2)
+    par.check_iteration(an, bnd, w, 13, T=1)
+
+
 def free_running_seed(ag, iters, learn=True):
     """First seed for which the ORACLE's own free run draws no uniform within 1e-5 of a CDF boundary (about one sample in
     17,000 does): on such a run the library has no excuse for a different action, so nothing needs to be skipped."""
