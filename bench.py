@@ -140,6 +140,7 @@ PROFILE_OF = {
     ("throughput", "heads_bwd"): ("heads_bwd__throughput.md", "learner_mma.cu"),
     ("throughput", "reduce_adam"): ("reduce_adam2__throughput.md", "learner_mma.cu"),
     ("throughput", "env_base"): ("env_base__throughput.md", "rollout.cu"),
+    ("throughput", "dw1_walls"): ("gemm_tn_tc_env_planes__throughput.md", "gemm_tc.cu"),
 }
 
 
